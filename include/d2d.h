@@ -1,0 +1,203 @@
+/*
+ * d2d.h - C ABI of the B200 (sm_100a) dynamic-k MoE layer library.
+ *
+ * The library runs the inference hot path of one D2DMoE layer
+ * (arXiv 2310.04361): a dense Transformer FFN (plain or gated), or a MoE-fied
+ * attention projection, whose neurons were cut offline into E equal experts
+ * (Sec. 3.2) and that runs, per token, only the experts a small router keeps
+ * (Sec. 3.3, 3.4).  The four steps are
+ *
+ *   router_fwd     R[t,i] = | W_r2 relu(W_r1 x_t + b_r1) + b_r2 |_i      Sec. 3.3
+ *   select_dynk    G[t,i] = ( R[t,i] >= tau * max_i R[t,i] )             Eq. 4
+ *                  + per-token k, per-expert counts, offsets, token lists  Listing 1
+ *   moe_ffn_fwd    y_t = b2 + sum_{i: G[t,i]} W2[:, blk i] A(W1[blk i,:] x_t + b1[blk i])
+ *                                                                         Sec. 3.2, App. G
+ *
+ * General rules
+ *   - Every pointer named "device" is a CUDA device pointer on the current
+ *     device; "host" pointers are ordinary host memory.  All matrices are
+ *     row-major.  Weight matrices use the nn.Linear layout [out, in].
+ *   - The caller owns every buffer it passes, including the workspace.  The
+ *     library allocates device memory only inside d2d_layer_create (packed
+ *     copies of the weights) and frees it in d2d_layer_destroy.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *     stream).  Calls enqueue work and return; none of them synchronises,
+ *     except d2d_layer_create (once, after packing).
+ *   - The return value reports argument and launch errors only.  Conditions
+ *     that depend on the data (a non-finite router score, more selected pairs
+ *     than `perm_capacity`) are written to the device status word
+ *     `d2d_routing.status`, which the caller reads after synchronising.
+ *   - T = 0 is a valid no-op.  There is no CPU fallback: without a CUDA device
+ *     every compute call returns D2D_ERR_CUDA.
+ *   - A handle is not thread-safe; distinct handles may be used concurrently.
+ */
+#ifndef D2D_H_
+#define D2D_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define D2D_API __attribute__((visibility("default")))
+#else
+#define D2D_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    D2D_OK = 0,
+    D2D_ERR_INVALID_ARG = 1, /* null pointer, bad size, tau outside [0,1], misaligned buffer */
+    D2D_ERR_UNSUPPORTED = 2, /* a shape or option the kernels do not cover                  */
+    D2D_ERR_WORKSPACE = 3,   /* workspace smaller than d2d_workspace_bytes reports          */
+    D2D_ERR_CUDA = 4,        /* a CUDA runtime call or a launch failed                      */
+    D2D_ERR_NONFINITE = 5,   /* device status: a router score was NaN or infinite           */
+    D2D_ERR_TIMEOUT = 6,     /* device status: a bounded wait inside a kernel ran out       */
+    D2D_ERR_CAPACITY = 7     /* device status: n_sel exceeded perm_capacity                 */
+} d2d_status;
+
+typedef enum { D2D_F32 = 0, D2D_BF16 = 1 } d2d_dtype;
+
+/* Activation A of the hidden neurons.  The paper evaluates ReLU and GELU models
+ * (Sec. 4, Sec. 5.4) and SiLU-gated FFNs (App. G); it does not say which GELU
+ * form, so both are offered. */
+typedef enum { D2D_ACT_RELU = 0, D2D_ACT_GELU_ERF = 1, D2D_ACT_GELU_TANH = 2, D2D_ACT_SILU = 3 } d2d_act;
+
+/* Shape of one layer.  Expert e owns neurons [e*expert_size, (e+1)*expert_size)
+ * (Sec. 3.2); n_experts * expert_size must equal d_ff.  d and d_h must be
+ * multiples of 8 so that every matrix row starts on a 16-byte boundary. */
+typedef struct {
+    int32_t d;           /* model width (input and output of the layer)           */
+    int32_t d_ff;        /* hidden width of the original FFN                       */
+    int32_t n_experts;   /* E                                                      */
+    int32_t expert_size; /* s = d_ff / E                                           */
+    int32_t d_h;         /* router hidden width (Sec. 3.3; 128 in the paper)       */
+    d2d_dtype dtype;     /* type of x, y and of every weight and bias              */
+    d2d_act act;
+    int32_t gated;       /* 0: y = W2 A(W1 x + b1) + b2                            */
+                         /* 1: y = W2 (A(W_gate x) * (W1 x + b1)) + b2  (App. G)   */
+} d2d_layer_desc;
+
+/* Device pointers to the layer's parameters, element type desc.dtype, read
+ * only during d2d_layer_create (the library keeps packed copies, so the
+ * caller may free these afterwards).  Any bias pointer may be NULL (= zeros). */
+typedef struct {
+    const void *w_r1;   /* [d_h, d]      router layer 1                              */
+    const void *b_r1;   /* [d_h]                                                     */
+    const void *w_r2;   /* [E, d_h]      router layer 2 (absolute value on output)   */
+    const void *b_r2;   /* [E]                                                       */
+    const void *w1;     /* [d_ff, d]     first FFN matrix ("up" when gated)          */
+    const void *b1;     /* [d_ff]                                                    */
+    const void *w_gate; /* [d_ff, d]     gate matrix, required iff desc.gated        */
+    const void *w2;     /* [d, d_ff]     second FFN matrix                           */
+    const void *b2;     /* [d]           shared by all experts, added once per token */
+} d2d_weights;
+
+/* Routing of one batch: the outputs of d2d_select_dynk and the input of
+ * d2d_moe_ffn_fwd.  All pointers are device pointers owned by the caller.
+ * mask, k, counts, offsets, perm, n_sel and status are required; the
+ * token-major dual (tok_off, tok_exp) is optional (both NULL or both set). */
+typedef struct {
+    uint32_t *mask;      /* [T, ceil(E/32)]  expert i of token t = bit i%32 of word i/32       */
+    int32_t *k;          /* [T]              experts kept by token t                           */
+    int32_t *counts;     /* [E]              tokens that keep expert e                         */
+    int32_t *offsets;    /* [E+1]            exclusive prefix sum of counts                    */
+    int32_t *perm;       /* [perm_capacity]  perm[offsets[e]+j] = j-th smallest t keeping e    */
+    int32_t *tok_off;    /* [T+1]            exclusive prefix sum of k            (optional)   */
+    int32_t *tok_exp;    /* [perm_capacity]  experts of token t, ascending        (optional)   */
+    int32_t *n_sel;      /* [1]              total kept (token, expert) pairs = offsets[E]     */
+    int32_t *status;     /* [1]              device status word: 0 or a d2d_status             */
+    int64_t perm_capacity; /* entries available in perm / tok_exp; T*E always suffices         */
+} d2d_routing;
+
+typedef struct d2d_layer d2d_layer;
+
+/* Human-readable name of a status code (host, static storage). */
+D2D_API const char *d2d_status_str(d2d_status s);
+
+/* Number of kernels this library has launched in this process so far (host
+ * counter, all handles and streams); a benchmark takes the difference across
+ * its timed region. */
+D2D_API uint64_t d2d_launch_count(void);
+
+/* Builds a layer handle: validates `desc`, copies and repacks the weights on
+ * the device (W2 is stored transposed so that an expert's slice is
+ * expert_size contiguous rows of d elements) and synchronises `stream` once.
+ * `desc` and `w` are host structs; the pointers inside `w` are device
+ * pointers.  On failure *out is NULL. */
+D2D_API d2d_status d2d_layer_create(const d2d_layer_desc *desc, const d2d_weights *w, void *stream, d2d_layer **out);
+
+/* Frees the handle and its device copies.  NULL is a no-op. */
+D2D_API d2d_status d2d_layer_destroy(d2d_layer *layer);
+
+/* Bytes of device workspace that any call on `layer` with up to max_tokens
+ * tokens needs (256-byte aligned buffer).  Returns 0 for a NULL layer. */
+D2D_API size_t d2d_workspace_bytes(const d2d_layer *layer, int32_t max_tokens);
+
+/* Bytes of device workspace d2d_select_dynk / d2d_routing_from_mask need. */
+D2D_API size_t d2d_select_workspace_bytes(int32_t T, int32_t E);
+
+/* Router forward (Sec. 3.3): R[t,i] = | b_r2[i] + sum_j W_r2[i,j] relu(b_r1[j] + W_r1[j,:] x_t) |.
+ * x: device [T, d] of desc.dtype.  R: device [T, E] float32 (always float32:
+ * the selection rule is evaluated on these values).  Products accumulate in
+ * float32.  ws: device workspace of at least d2d_workspace_bytes(layer, T). */
+D2D_API d2d_status d2d_router_fwd(const d2d_layer *layer, const void *x, int32_t T, float *R,
+                          void *ws, size_t ws_bytes, void *stream);
+
+/* Dynamic-k selection and routing metadata (Eq. 4; Listing 1's per-expert
+ * token lists and counts).  R: device [T, E] float32, expected finite and
+ * non-negative.  For every token: m = max_i R[t,i]; thr = tau*m rounded once to
+ * float32; expert i is kept iff R[t,i] >= thr (ties kept; an all-zero row keeps
+ * every expert).  A token whose row holds a NaN or an infinity keeps every
+ * expert and sets *status = D2D_ERR_NONFINITE.  Inside an expert's list tokens
+ * are in ascending order, which makes every output unique (bit-exact
+ * comparable).  If n_sel > perm_capacity, perm/tok_exp are truncated, the other
+ * outputs are complete and *status = D2D_ERR_CAPACITY.  tau must lie in [0,1]. */
+D2D_API d2d_status d2d_select_dynk(const float *R, int32_t T, int32_t E, float tau, d2d_routing *out,
+                           void *ws, size_t ws_bytes, void *stream);
+
+/* Static top-k selection (the regression router "is still compatible with"
+ * top-k, Sec. 3.3): keeps the kk largest scores of each token, equal scores in
+ * order of the lower expert index, then builds the same metadata. */
+D2D_API d2d_status d2d_select_topk(const float *R, int32_t T, int32_t E, int32_t kk, d2d_routing *out,
+                           void *ws, size_t ws_bytes, void *stream);
+
+/* Routing metadata from a caller-supplied mask (the latency protocol of
+ * Sec. 4.4 overrides the gating decisions with Bernoulli samples).
+ * out->mask is the INPUT here (device, same layout; bits at positions >= E
+ * must be zero); k, counts, offsets, perm, n_sel (and the dual) are written. */
+D2D_API d2d_status d2d_routing_from_mask(int32_t T, int32_t E, d2d_routing *out,
+                                 void *ws, size_t ws_bytes, void *stream);
+
+/* Expert FFN and combine (Sec. 3.2, 3.4; App. G for the gated form):
+ *   y[t,:] = b2 + sum over kept experts e of  W2[:, e-block] * h_e(x_t),
+ *   h_e = A(W1[e-block,:] x_t + b1[e-block])           (gated: A(W_gate x) * (W1 x + b1)).
+ * No router-score weighting (G is binary).  A token that keeps no expert gets
+ * y = b2.  x, y: device [T, d] of desc.dtype; sums accumulate in float32; the
+ * summation order over experts is not fixed, so y matches a reference within a
+ * tolerance, not bit for bit.  `routing` must describe these T tokens. */
+D2D_API d2d_status d2d_moe_ffn_fwd(const d2d_layer *layer, const void *x, int32_t T, const d2d_routing *routing,
+                           void *y, void *ws, size_t ws_bytes, void *stream);
+
+/* The whole layer on one stream with no host synchronisation in between:
+ * router_fwd -> select_dynk -> moe_ffn_fwd.  R_out: optional device [T,E]
+ * float32 copy of the router scores (NULL to keep them in the workspace only).
+ * `routing` supplies the metadata buffers (required; they are outputs). */
+D2D_API d2d_status d2d_layer_fwd(const d2d_layer *layer, const void *x, int32_t T, float tau, void *y,
+                         float *R_out, d2d_routing *routing, void *ws, size_t ws_bytes, void *stream);
+
+/* Host-buffer convenience: the same layer call, but x and y are HOST pointers
+ * ([T,d] of desc.dtype).  The call copies x to the device, runs the layer,
+ * copies y back and synchronises `stream`; all device memory it needs comes
+ * from `ws` (device, at least d2d_layer_fwd_host_workspace_bytes bytes).  For
+ * full copy/compute overlap the host buffers should be page-locked. */
+D2D_API size_t d2d_layer_fwd_host_workspace_bytes(const d2d_layer *layer, int32_t max_tokens);
+D2D_API d2d_status d2d_layer_fwd_host(const d2d_layer *layer, const void *x_host, int32_t T, float tau, void *y_host,
+                              void *ws, size_t ws_bytes, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* D2D_H_ */

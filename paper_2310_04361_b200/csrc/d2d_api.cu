@@ -1,0 +1,300 @@
+// Host side of the C ABI declared in include/d2d.h: argument validation, weight packing,
+// workspace carving and kernel dispatch.  No computation happens on the host.
+#include <math.h>
+#include <new>
+#include <string.h>
+
+#include "d2d_common.cuh"
+
+bool d2d_token_path_supports(const d2d_layer_desc &D);
+d2d_status d2d_launch_moe_ffn_token(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y,
+                                    cudaStream_t st);
+
+unsigned long long d2d_launch_counter = 0;
+
+namespace {
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+bool routing_ok(const d2d_routing *r, bool need_mask_only)
+{
+    if (!r || !r->mask) return false;
+    if (need_mask_only) return true;
+    if (!r->k || !r->counts || !r->offsets || !r->perm || !r->n_sel || !r->status) return false;
+    if ((r->tok_off == nullptr) != (r->tok_exp == nullptr)) return false;
+    return r->perm_capacity >= 0;
+}
+
+// Workspace layout of the layer-level calls: [ u: T*d_h f32 | R: T*E f32 | select scratch | ffn scratch ]
+struct ws_layout {
+    size_t u_off, r_off, sel_off, ffn_off, total;
+};
+
+ws_layout layout_for(const d2d_layer *L, int T)
+{
+    ws_layout w;
+    const size_t Tn = (size_t)(T > 0 ? T : 1);
+    size_t off = 0;
+    w.u_off = off;
+    off += d2d_align_up(Tn * (size_t)L->desc.d_h * sizeof(float), 256);
+    w.r_off = off;
+    off += d2d_align_up(Tn * (size_t)L->desc.n_experts * sizeof(float), 256);
+    w.sel_off = off;
+    off += d2d_select_ws_bytes((int)Tn, L->desc.n_experts);
+    w.ffn_off = off;
+    off += d2d_moe_ffn_ws_bytes(L, (int)Tn);
+    w.total = off;
+    return w;
+}
+
+}  // namespace
+
+size_t d2d_moe_ffn_ws_bytes(const d2d_layer *, int) { return 256; }
+
+d2d_status d2d_launch_moe_ffn(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y,
+                              void *, size_t, cudaStream_t st)
+{
+    return d2d_launch_moe_ffn_token(L, x, T, r, y, st);
+}
+
+extern "C" {
+
+uint64_t d2d_launch_count(void) { return __atomic_load_n(&d2d_launch_counter, __ATOMIC_RELAXED); }
+
+const char *d2d_status_str(d2d_status s)
+{
+    switch (s) {
+    case D2D_OK: return "ok";
+    case D2D_ERR_INVALID_ARG: return "invalid argument";
+    case D2D_ERR_UNSUPPORTED: return "unsupported shape or option";
+    case D2D_ERR_WORKSPACE: return "workspace too small";
+    case D2D_ERR_CUDA: return "CUDA runtime or launch failure";
+    case D2D_ERR_NONFINITE: return "non-finite router score";
+    case D2D_ERR_TIMEOUT: return "bounded wait ran out inside a kernel";
+    case D2D_ERR_CAPACITY: return "more selected pairs than perm_capacity";
+    }
+    return "unknown status";
+}
+
+d2d_status d2d_layer_create(const d2d_layer_desc *desc, const d2d_weights *w, void *stream, d2d_layer **out)
+{
+    if (out) *out = nullptr;
+    if (!desc || !w || !out) return D2D_ERR_INVALID_ARG;
+    const d2d_layer_desc &D = *desc;
+    if (D.d <= 0 || D.d_ff <= 0 || D.n_experts <= 0 || D.expert_size <= 0 || D.d_h <= 0) return D2D_ERR_INVALID_ARG;
+    if ((int64_t)D.n_experts * D.expert_size != D.d_ff) return D2D_ERR_INVALID_ARG;
+    if (D.dtype != D2D_F32 && D.dtype != D2D_BF16) return D2D_ERR_INVALID_ARG;
+    if (D.act < D2D_ACT_RELU || D.act > D2D_ACT_SILU) return D2D_ERR_INVALID_ARG;
+    if (D.d % 8 || D.d_h % 8) return D2D_ERR_INVALID_ARG;
+    if (!w->w_r1 || !w->w_r2 || !w->w1 || !w->w2) return D2D_ERR_INVALID_ARG;
+    if ((D.gated != 0) != (w->w_gate != nullptr)) return D2D_ERR_INVALID_ARG;
+    if (!d2d_token_path_supports(D)) return D2D_ERR_UNSUPPORTED;
+
+    int dev = 0, sms = 0;
+    D2D_CUDA_TRY(cudaGetDevice(&dev));
+    D2D_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+
+    d2d_layer *L = new (std::nothrow) d2d_layer();
+    if (!L) return D2D_ERR_CUDA;
+    memset(L, 0, sizeof(*L));
+    L->desc = D;
+    L->elem = D.dtype == D2D_F32 ? 4 : 2;
+    L->sm_count = sms;
+    const size_t el = L->elem;
+    const size_t n_wr1 = (size_t)D.d_h * D.d, n_wr2 = (size_t)D.n_experts * D.d_h, n_w = (size_t)D.d_ff * D.d;
+
+    struct piece { void **dst; const void *src; size_t n; bool transpose; };
+    piece pieces[] = {
+        {&L->w_r1, w->w_r1, n_wr1, false}, {&L->b_r1, w->b_r1, (size_t)D.d_h, false},
+        {&L->w_r2, w->w_r2, n_wr2, false}, {&L->b_r2, w->b_r2, (size_t)D.n_experts, false},
+        {&L->w1, w->w1, n_w, false},       {&L->b1, w->b1, (size_t)D.d_ff, false},
+        {&L->w_gate, w->w_gate, n_w, false}, {&L->w2t, w->w2, n_w, true},
+        {&L->b2, w->b2, (size_t)D.d, false},
+    };
+    size_t total = 0;
+    for (const piece &p : pieces)
+        if (p.src) total += d2d_align_up(p.n * el, 256);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMalloc(&L->slab, total) != cudaSuccess) {
+        delete L;
+        return D2D_ERR_CUDA;
+    }
+    L->slab_bytes = total;
+    size_t off = 0;
+    d2d_status rc = D2D_OK;
+    for (const piece &p : pieces) {
+        if (!p.src) continue;
+        void *dst = (char *)L->slab + off;
+        off += d2d_align_up(p.n * el, 256);
+        *p.dst = dst;
+        if (p.transpose) {
+            rc = d2d_launch_transpose(p.src, dst, D.d, D.d_ff, el, st);
+        } else if (cudaMemcpyAsync(dst, p.src, p.n * el, cudaMemcpyDeviceToDevice, st) != cudaSuccess) {
+            rc = D2D_ERR_CUDA;
+        }
+        if (rc != D2D_OK) break;
+    }
+    if (rc == D2D_OK && cudaStreamSynchronize(st) != cudaSuccess) rc = D2D_ERR_CUDA;
+    if (rc != D2D_OK) {
+        cudaFree(L->slab);
+        delete L;
+        return rc;
+    }
+    *out = L;
+    return D2D_OK;
+}
+
+d2d_status d2d_layer_destroy(d2d_layer *layer)
+{
+    if (!layer) return D2D_OK;
+    cudaError_t e = cudaFree(layer->slab);
+    delete layer;
+    return e == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
+}
+
+size_t d2d_workspace_bytes(const d2d_layer *layer, int32_t max_tokens)
+{
+    if (!layer || max_tokens < 0) return 0;
+    return layout_for(layer, max_tokens).total;
+}
+
+size_t d2d_select_workspace_bytes(int32_t T, int32_t E)
+{
+    if (T < 0 || E <= 0) return 0;
+    return d2d_select_ws_bytes(T, E);
+}
+
+d2d_status d2d_router_fwd(const d2d_layer *layer, const void *x, int32_t T, float *R,
+                          void *ws, size_t ws_bytes, void *stream)
+{
+    if (!layer || T < 0) return D2D_ERR_INVALID_ARG;
+    if (T == 0) return D2D_OK;
+    if (!x || !R || !ws || !aligned16(x) || !aligned16(R) || !aligned16(ws)) return D2D_ERR_INVALID_ARG;
+    const ws_layout w = layout_for(layer, T);
+    if (ws_bytes < w.total) return D2D_ERR_WORKSPACE;
+    return d2d_launch_router(layer, x, T, R, (float *)((char *)ws + w.u_off), (cudaStream_t)stream);
+}
+
+static d2d_status select_common(const float *R, int32_t T, int32_t E, float tau, int topk, d2d_routing *out,
+                                void *ws, size_t ws_bytes, void *stream, bool mask_is_input)
+{
+    if (T < 0 || E <= 0 || !routing_ok(out, false)) return D2D_ERR_INVALID_ARG;
+    if (!mask_is_input && T > 0 && (!R || !aligned16(R))) return D2D_ERR_INVALID_ARG;
+    if (!mask_is_input && topk == 0 && !(tau >= 0.0f && tau <= 1.0f)) return D2D_ERR_INVALID_ARG;   // also rejects NaN
+    if (topk < 0 || (topk > 0 && E > 2048)) return topk < 0 ? D2D_ERR_INVALID_ARG : D2D_ERR_UNSUPPORTED;
+    if (T > 0 && (!ws || ws_bytes < d2d_select_ws_bytes(T, E))) return D2D_ERR_WORKSPACE;
+    return d2d_launch_select(mask_is_input ? nullptr : R, T, E, tau, topk, out, ws, (cudaStream_t)stream);
+}
+
+d2d_status d2d_select_dynk(const float *R, int32_t T, int32_t E, float tau, d2d_routing *out,
+                           void *ws, size_t ws_bytes, void *stream)
+{
+    return select_common(R, T, E, tau, 0, out, ws, ws_bytes, stream, false);
+}
+
+d2d_status d2d_select_topk(const float *R, int32_t T, int32_t E, int32_t kk, d2d_routing *out,
+                           void *ws, size_t ws_bytes, void *stream)
+{
+    if (kk <= 0) return D2D_ERR_INVALID_ARG;
+    return select_common(R, T, E, 0.0f, kk, out, ws, ws_bytes, stream, false);
+}
+
+d2d_status d2d_routing_from_mask(int32_t T, int32_t E, d2d_routing *out, void *ws, size_t ws_bytes, void *stream)
+{
+    return select_common(nullptr, T, E, 0.0f, 0, out, ws, ws_bytes, stream, true);
+}
+
+d2d_status d2d_moe_ffn_fwd(const d2d_layer *layer, const void *x, int32_t T, const d2d_routing *routing,
+                           void *y, void *ws, size_t ws_bytes, void *stream)
+{
+    if (!layer || T < 0) return D2D_ERR_INVALID_ARG;
+    if (T == 0) return D2D_OK;
+    if (!x || !y || !aligned16(x) || !aligned16(y) || !routing_ok(routing, false)) return D2D_ERR_INVALID_ARG;
+    const ws_layout w = layout_for(layer, T);
+    if (!ws || ws_bytes < w.total) return D2D_ERR_WORKSPACE;
+    return d2d_launch_moe_ffn(layer, x, T, routing, y, (char *)ws + w.ffn_off, w.total - w.ffn_off,
+                              (cudaStream_t)stream);
+}
+
+d2d_status d2d_layer_fwd(const d2d_layer *layer, const void *x, int32_t T, float tau, void *y,
+                         float *R_out, d2d_routing *routing, void *ws, size_t ws_bytes, void *stream)
+{
+    if (!layer || T < 0 || !routing_ok(routing, false)) return D2D_ERR_INVALID_ARG;
+    if (!(tau >= 0.0f && tau <= 1.0f)) return D2D_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int E = layer->desc.n_experts;
+    if (T == 0) return d2d_launch_select(nullptr, 0, E, tau, 0, routing, ws, st);
+    if (!x || !y || !aligned16(x) || !aligned16(y) || (R_out && !aligned16(R_out))) return D2D_ERR_INVALID_ARG;
+    const ws_layout w = layout_for(layer, T);
+    if (!ws || !aligned16(ws) || ws_bytes < w.total) return D2D_ERR_WORKSPACE;
+    char *base = (char *)ws;
+    float *R = R_out ? R_out : (float *)(base + w.r_off);
+    d2d_status rc = d2d_launch_router(layer, x, T, R, (float *)(base + w.u_off), st);
+    if (rc != D2D_OK) return rc;
+    rc = d2d_launch_select(R, T, E, tau, 0, routing, base + w.sel_off, st);
+    if (rc != D2D_OK) return rc;
+    return d2d_launch_moe_ffn(layer, x, T, routing, y, base + w.ffn_off, w.total - w.ffn_off, st);
+}
+
+// Carves routing buffers + x/y staging + the layer workspace out of one device buffer.
+struct host_call_layout {
+    size_t x_off, y_off, mask_off, k_off, counts_off, offsets_off, perm_off, scalars_off, ws_off, total;
+};
+
+static host_call_layout host_layout(const d2d_layer *L, int T)
+{
+    host_call_layout h;
+    const size_t Tn = (size_t)(T > 0 ? T : 1), E = (size_t)L->desc.n_experts, W = (E + 31) / 32;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off += d2d_align_up(bytes, 256); return o; };
+    h.x_off = take(Tn * L->desc.d * L->elem);
+    h.y_off = take(Tn * L->desc.d * L->elem);
+    h.mask_off = take(Tn * W * 4);
+    h.k_off = take(Tn * 4);
+    h.counts_off = take(E * 4);
+    h.offsets_off = take((E + 1) * 4);
+    h.perm_off = take(Tn * E * 4);
+    h.scalars_off = take(2 * 4);
+    h.ws_off = off;
+    off += layout_for(L, (int)Tn).total;
+    h.total = off;
+    return h;
+}
+
+size_t d2d_layer_fwd_host_workspace_bytes(const d2d_layer *layer, int32_t max_tokens)
+{
+    if (!layer || max_tokens < 0) return 0;
+    return host_layout(layer, max_tokens).total;
+}
+
+d2d_status d2d_layer_fwd_host(const d2d_layer *layer, const void *x_host, int32_t T, float tau, void *y_host,
+                              void *ws, size_t ws_bytes, void *stream)
+{
+    if (!layer || T < 0) return D2D_ERR_INVALID_ARG;
+    if (T == 0) return D2D_OK;
+    if (!x_host || !y_host || !ws || !aligned16(ws)) return D2D_ERR_INVALID_ARG;
+    const host_call_layout h = host_layout(layer, T);
+    if (ws_bytes < h.total) return D2D_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    char *base = (char *)ws;
+    const size_t row_bytes = (size_t)T * layer->desc.d * layer->elem;
+    D2D_CUDA_TRY(cudaMemcpyAsync(base + h.x_off, x_host, row_bytes, cudaMemcpyHostToDevice, st));
+    d2d_routing r;
+    memset(&r, 0, sizeof(r));
+    r.mask = (uint32_t *)(base + h.mask_off);
+    r.k = (int32_t *)(base + h.k_off);
+    r.counts = (int32_t *)(base + h.counts_off);
+    r.offsets = (int32_t *)(base + h.offsets_off);
+    r.perm = (int32_t *)(base + h.perm_off);
+    r.n_sel = (int32_t *)(base + h.scalars_off);
+    r.status = r.n_sel + 1;
+    r.perm_capacity = (int64_t)T * layer->desc.n_experts;
+    d2d_status rc = d2d_layer_fwd(layer, base + h.x_off, T, tau, base + h.y_off, nullptr, &r,
+                                  base + h.ws_off, h.total - h.ws_off, st);
+    if (rc != D2D_OK) return rc;
+    D2D_CUDA_TRY(cudaMemcpyAsync(y_host, base + h.y_off, row_bytes, cudaMemcpyDeviceToHost, st));
+    D2D_CUDA_TRY(cudaStreamSynchronize(st));
+    return D2D_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,100 @@
+// Shared declarations of the CUDA translation units behind include/d2d.h.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "d2d.h"
+
+// Packed, library-owned copy of one layer's parameters.
+struct d2d_layer {
+    d2d_layer_desc desc;
+    size_t elem;            // bytes per element of desc.dtype
+    int sm_count;
+    // router
+    void *w_r1, *b_r1, *w_r2, *b_r2;
+    // experts: w1 / w_gate as given ([d_ff, d], an expert = s contiguous rows),
+    // w2t = W2 transposed to [d_ff, d] so that an expert's slice is s contiguous rows too
+    void *w1, *b1, *w_gate, *w2t, *b2;
+    void *slab;             // one allocation backing all of the above
+    size_t slab_bytes;
+};
+
+#define D2D_CUDA_TRY(expr)                                   \
+    do {                                                     \
+        cudaError_t err__ = (expr);                          \
+        if (err__ != cudaSuccess) return D2D_ERR_CUDA;       \
+    } while (0)
+
+// Host-side count of kernel launches (reported by d2d_launch_count()).
+extern unsigned long long d2d_launch_counter;
+#define D2D_LAUNCHED(n) __atomic_fetch_add(&d2d_launch_counter, (unsigned long long)(n), __ATOMIC_RELAXED)
+
+static inline size_t d2d_align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+static inline int d2d_cdiv(int a, int b) { return (a + b - 1) / b; }
+
+// ---- launch wrappers implemented in the kernel files -------------------------------------
+
+d2d_status d2d_launch_router(const d2d_layer *L, const void *x, int T, float *R, float *u_ws, cudaStream_t st);
+
+size_t d2d_select_ws_bytes(int T, int E);
+d2d_status d2d_launch_select(const float *R, int T, int E, float tau, int topk, const d2d_routing *out,
+                             void *ws, cudaStream_t st);   // R == nullptr: mask is an input
+
+d2d_status d2d_launch_moe_ffn(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y,
+                              void *ws, size_t ws_bytes, cudaStream_t st);
+size_t d2d_moe_ffn_ws_bytes(const d2d_layer *L, int T);
+
+d2d_status d2d_launch_transpose(const void *src, void *dst, int rows, int cols, size_t elem, cudaStream_t st);
+
+// ---- device helpers ------------------------------------------------------------------------
+
+#ifdef __CUDACC__
+
+template <typename T> __device__ __forceinline__ float d2d_to_float(T v);
+template <> __device__ __forceinline__ float d2d_to_float<float>(float v) { return v; }
+template <> __device__ __forceinline__ float d2d_to_float<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+template <typename T> __device__ __forceinline__ T d2d_from_float(float v);
+template <> __device__ __forceinline__ float d2d_from_float<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 d2d_from_float<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// Activation of the hidden neurons; evaluated in float32 with the accurate libdevice routines.
+template <int ACT> __device__ __forceinline__ float d2d_activate(float z)
+{
+    if (ACT == D2D_ACT_RELU) return fmaxf(z, 0.0f);
+    if (ACT == D2D_ACT_GELU_ERF) return 0.5f * z * (1.0f + erff(z * 0.70710678118654752f));
+    if (ACT == D2D_ACT_GELU_TANH) {
+        const float c = 0.79788456080286536f;  // sqrt(2/pi)
+        return 0.5f * z * (1.0f + tanhf(c * (z + 0.044715f * z * z * z)));
+    }
+    return z / (1.0f + expf(-z));  // SiLU
+}
+
+__device__ __forceinline__ float d2d_warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// 8 consecutive elements starting at p (16-byte aligned for bf16, 32-byte for float) as floats.
+__device__ __forceinline__ void d2d_load8(const float *p, float (&o)[8])
+{
+    const float4 a = __ldg(reinterpret_cast<const float4 *>(p));
+    const float4 b = __ldg(reinterpret_cast<const float4 *>(p) + 1);
+    o[0] = a.x; o[1] = a.y; o[2] = a.z; o[3] = a.w; o[4] = b.x; o[5] = b.y; o[6] = b.z; o[7] = b.w;
+}
+__device__ __forceinline__ void d2d_load8(const __nv_bfloat16 *p, float (&o)[8])
+{
+    const uint4 raw = __ldg(reinterpret_cast<const uint4 *>(p));
+    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        o[2 * i] = __uint_as_float(w[i] << 16);
+        o[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+}
+
+#endif  // __CUDACC__
