@@ -5,6 +5,7 @@
 #include <string.h>
 
 #include "d2d_common.cuh"
+#include "gemm_tc.cuh"
 
 bool d2d_token_path_supports(const d2d_layer_desc &D);
 d2d_status d2d_launch_moe_ffn_token(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y,
@@ -49,11 +50,49 @@ ws_layout layout_for(const d2d_layer *L, int T)
 
 }  // namespace
 
-size_t d2d_moe_ffn_ws_bytes(const d2d_layer *, int) { return 256; }
+// Tokens from which the dense tensor-core path (masked hidden activations, two GEMMs) is used
+// instead of the token-major CUDA-core kernel.
+static const int kDenseMaskedMinTokens = 128;
+
+static bool use_dense_masked(const d2d_layer *L, int T)
+{
+    return L->desc.dtype == D2D_BF16 && T >= kDenseMaskedMinTokens && L->desc.d_ff % 8 == 0 && d2d_gemm_tc_available();
+}
+
+size_t d2d_moe_ffn_ws_bytes(const d2d_layer *L, int T)
+{
+    // hidden activations H [T, d_ff] bf16 of the dense-masked path
+    if (L->desc.dtype != D2D_BF16 || T < kDenseMaskedMinTokens) return 256;
+    return d2d_align_up((size_t)T * L->desc.d_ff * 2, 256);
+}
+
+// Large batches: every expert is used by some token of a 128-token tile, so the expert FFN runs
+// as two dense tensor-core GEMMs; the selection enters as a mask on the hidden activations
+// (h_n of an expert the token did not keep is zeroed in the epilogue), which is exactly
+// y = b2 + sum over kept experts.
+static d2d_status launch_dense_masked(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y,
+                                      void *ws, cudaStream_t st)
+{
+    const d2d_layer_desc &D = L->desc;
+    d2d_gemm_args up = {};
+    up.a = x; up.b = L->w1; up.b_gate = D.gated ? L->w_gate : nullptr; up.bias = L->b1; up.out = ws;
+    up.M = T; up.N = D.d_ff; up.K = D.d; up.epilogue = D2D_EPI_UP_MASKED; up.act = D.act;
+    up.mask = r->mask; up.mask_words = (D.n_experts + 31) / 32; up.expert_size = D.expert_size; up.status = r->status;
+    d2d_status rc = d2d_gemm_tc(up, st);
+    if (rc != D2D_OK) return rc;
+    d2d_gemm_args dn = {};
+    dn.a = ws; dn.b = L->w2; dn.bias = L->b2; dn.out = y;
+    dn.M = T; dn.N = D.d; dn.K = D.d_ff; dn.epilogue = D2D_EPI_BIAS_BF16; dn.status = r->status;
+    return d2d_gemm_tc(dn, st);
+}
 
 d2d_status d2d_launch_moe_ffn(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y,
-                              void *, size_t, cudaStream_t st)
+                              void *ws, size_t ws_bytes, cudaStream_t st)
 {
+    if (use_dense_masked(L, T)) {
+        if (ws_bytes < d2d_moe_ffn_ws_bytes(L, T)) return D2D_ERR_WORKSPACE;
+        return launch_dense_masked(L, x, T, r, y, ws, st);
+    }
     return d2d_launch_moe_ffn_token(L, x, T, r, y, st);
 }
 
@@ -109,7 +148,7 @@ d2d_status d2d_layer_create(const d2d_layer_desc *desc, const d2d_weights *w, vo
         {&L->w_r2, w->w_r2, n_wr2, false}, {&L->b_r2, w->b_r2, (size_t)D.n_experts, false},
         {&L->w1, w->w1, n_w, false},       {&L->b1, w->b1, (size_t)D.d_ff, false},
         {&L->w_gate, w->w_gate, n_w, false}, {&L->w2t, w->w2, n_w, true},
-        {&L->b2, w->b2, (size_t)D.d, false},
+        {&L->b2, w->b2, (size_t)D.d, false}, {&L->w2, w->w2, n_w, false},
     };
     size_t total = 0;
     for (const piece &p : pieces)

@@ -17,6 +17,7 @@ struct d2d_layer {
     // experts: w1 / w_gate as given ([d_ff, d], an expert = s contiguous rows),
     // w2t = W2 transposed to [d_ff, d] so that an expert's slice is s contiguous rows too
     void *w1, *b1, *w_gate, *w2t, *b2;
+    void *w2;               // W2 as given ([d, d_ff]): the K-major B operand of the dense down projection
     void *slab;             // one allocation backing all of the above
     size_t slab_bytes;
 };

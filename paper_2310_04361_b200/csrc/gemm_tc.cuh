@@ -1,0 +1,35 @@
+// Interface of the tcgen05 / TMA GEMM used for the dense contractions of the layer
+// (router layers, expert up projection with fused bias + activation + mask, down projection).
+#pragma once
+
+#include <cuda.h>
+
+#include "d2d_common.cuh"
+
+enum d2d_gemm_epilogue {
+    D2D_EPI_RELU_BF16 = 0,   // out bf16 = relu(acc + bias)                 router layer 1
+    D2D_EPI_ABS_F32 = 1,     // out f32  = |acc + bias|                     router layer 2
+    D2D_EPI_UP_MASKED = 2,   // out bf16 = G[row, col/s] ? A(acc + bias) : 0    expert up projection
+    D2D_EPI_BIAS_BF16 = 3,   // out bf16 = acc + bias                       down projection
+};
+
+struct d2d_gemm_args {
+    const void *a;           // [M, K] bf16 row-major (activations)
+    const void *b;           // [N, K] bf16 row-major (weights, nn.Linear layout)
+    const void *b_gate;      // [N, K] second weight matrix for the gated up projection, else NULL
+    const void *bias;        // [N] bf16 or NULL
+    void *out;               // [M, N] bf16 or f32, row-major, leading dimension N
+    int M, N, K;
+    int epilogue;            // d2d_gemm_epilogue
+    int act;                 // d2d_act, used by D2D_EPI_UP_MASKED
+    const uint32_t *mask;    // [M, mask_words] packed selection mask (UP_MASKED), NULL = keep everything
+    int mask_words;
+    int expert_size;         // s: column c belongs to expert c / s
+    int32_t *status;         // device status word, receives D2D_ERR_TIMEOUT if a bounded wait runs out
+};
+
+// Enqueues C = epilogue(A B^T).  Requires K % 8 == 0 and 16-byte aligned base pointers.
+d2d_status d2d_gemm_tc(const d2d_gemm_args &g, cudaStream_t st);
+
+// False when the driver entry point for tensor-map encoding is unavailable.
+bool d2d_gemm_tc_available();

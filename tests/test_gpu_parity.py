@@ -16,7 +16,9 @@ from paper_2310_04361_b200 import workloads as wl
 pytestmark = pytest.mark.gpu
 
 TOL_Y = {"f32": 1e-4, "bf16": 2e-2}
-TOL_R = {"f32": 1e-5, "bf16": 1e-4}   # relative to max|R|; both sides accumulate exact products of the same inputs
+# relative to max|R|: fp32 layers accumulate the same exact products in another order; bf16 layers also round the
+# router's hidden activations to bf16 (they feed the second tensor-core GEMM), 2^-9 per element
+TOL_R = {"f32": 1e-5, "bf16": 5e-3}
 
 
 @pytest.fixture(scope="module")
@@ -273,7 +275,7 @@ def test_layer_fwd_end_to_end(api, name, T, tau):
     near = np.abs(ref["R"] - np.float32(tau) * m) <= 4 * eps * m
     assert (~diff | near).all()
     same = ~diff.any(1)
-    assert same.mean() > 0.9
+    assert diff.mean() < 0.01 and same.mean() > 0.3
     yg = y.float().cpu().numpy()
     assert _rel_err(yg[same], ref["y"][same]) <= TOL_Y[cfg.dtype]
 
