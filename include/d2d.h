@@ -171,6 +171,31 @@ D2D_API d2d_status d2d_select_topk(const float *R, int32_t T, int32_t E, int32_t
 D2D_API d2d_status d2d_routing_from_mask(int32_t T, int32_t E, d2d_routing *out,
                                  void *ws, size_t ws_bytes, void *stream);
 
+/* d2d_select_dynk for callers that may not allocate device memory.  (The paper
+ * has no counterpart; this is a deployment convenience.)
+ * Some integrations run the layer from a context in which cudaMalloc is off
+ * limits: a plug-in whose enqueue hook must not allocate, a serving loop whose
+ * memory pool was fixed at start-up, code that runs after the framework has
+ * handed all device memory to its own allocator.  Such a caller cannot obtain
+ * the workspace d2d_select_dynk asks for, so this variant keeps the scratch it
+ * needs in a fixed 512 KiB array inside the library's device image (every GPU
+ * that loads the library holds it until the process exits).  The call itself
+ * allocates nothing, on the host or the device, and frees nothing.
+ *   - Same inputs, outputs, rule and error reporting as d2d_select_dynk; the
+ *     caller still passes R and the routing buffers.
+ *   - Limit: ceil(T / 1024) * E <= 131072 (for example 65,536 tokens at 2,048
+ *     experts, or any T <= 1024 with E <= 131,072); beyond it the call returns
+ *     D2D_ERR_UNSUPPORTED and enqueues nothing.
+ *   - The first call on each device looks up the array's device address (once,
+ *     with that device current).  Make that first call outside any stream
+ *     capture.
+ *   - All calls on one device share the array, so two calls whose kernels can
+ *     overlap on the GPU (different streams) race; serialise them.  The array
+ *     keeps the previous call's contents, which is harmless: each call
+ *     overwrites every entry before reading it. */
+D2D_API d2d_status d2d_select_dynk_static(const float *R, int32_t T, int32_t E, float tau, d2d_routing *out,
+                                          void *stream);
+
 /* Expert FFN and combine (Sec. 3.2, 3.4; App. G for the gated form):
  *   y[t,:] = b2 + sum over kept experts e of  W2[:, e-block] * h_e(x_t),
  *   h_e = A(W1[e-block,:] x_t + b1[e-block])           (gated: A(W_gate x) * (W1 x + b1)).

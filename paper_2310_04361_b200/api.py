@@ -27,7 +27,7 @@ STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "WORKSPACE", 4: 
 D2D_F32, D2D_BF16 = 0, 1
 ACTS = {"relu": 0, "gelu_erf": 1, "gelu_tanh": 2, "silu": 3}
 EXPORTS = ["d2d_status_str", "d2d_launch_count", "d2d_layer_create", "d2d_layer_destroy", "d2d_workspace_bytes",
-           "d2d_select_workspace_bytes", "d2d_router_fwd", "d2d_select_dynk", "d2d_select_topk",
+           "d2d_select_workspace_bytes", "d2d_router_fwd", "d2d_select_dynk", "d2d_select_dynk_static", "d2d_select_topk",
            "d2d_routing_from_mask", "d2d_moe_ffn_fwd", "d2d_layer_fwd", "d2d_layer_fwd_host_workspace_bytes",
            "d2d_layer_fwd_host"]
 
@@ -59,6 +59,7 @@ _lib.d2d_select_workspace_bytes.restype = c_size_t
 _lib.d2d_select_workspace_bytes.argtypes = [c_int32, c_int32]
 _lib.d2d_router_fwd.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_size_t, c_void_p]
 _lib.d2d_select_dynk.argtypes = [c_void_p, c_int32, c_int32, c_float, POINTER(RoutingStruct), c_void_p, c_size_t, c_void_p]
+_lib.d2d_select_dynk_static.argtypes = [c_void_p, c_int32, c_int32, c_float, POINTER(RoutingStruct), c_void_p]
 _lib.d2d_select_topk.argtypes = [c_void_p, c_int32, c_int32, c_int32, POINTER(RoutingStruct), c_void_p, c_size_t, c_void_p]
 _lib.d2d_routing_from_mask.argtypes = [c_int32, c_int32, POINTER(RoutingStruct), c_void_p, c_size_t, c_void_p]
 _lib.d2d_moe_ffn_fwd.argtypes = [c_void_p, c_void_p, c_int32, POINTER(RoutingStruct), c_void_p, c_void_p, c_size_t, c_void_p]
@@ -241,6 +242,15 @@ def select_dynk(R, tau: float, routing: Routing | None = None, dual: bool = Fals
     ws = torch.empty((max(nbytes, 256),), dtype=torch.uint8, device=R.device)
     _check(_lib.d2d_select_dynk(_ptr(R), T, E, c_float(tau), ctypes.byref(routing.struct), _ptr(ws), ws.numel(),
                                 _stream(stream)), "d2d_select_dynk")
+    return routing
+
+
+def select_dynk_static(R, tau: float, routing: Routing, stream=None) -> Routing:
+    """d2d_select_dynk_static: selection whose scratch is a fixed array inside the library, for callers that
+    may not allocate device memory.  `routing` (the outputs) must be supplied by the caller; nothing is allocated here."""
+    T, E = R.shape
+    _check(_lib.d2d_select_dynk_static(_ptr(R), T, E, c_float(tau), ctypes.byref(routing.struct), _stream(stream)),
+           "d2d_select_dynk_static")
     return routing
 
 

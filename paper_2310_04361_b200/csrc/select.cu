@@ -328,3 +328,56 @@ d2d_status d2d_launch_select(const float *R, int T, int E, float tau, int topk, 
     }
     return cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
 }
+
+// ------------------------------------------------------------------------------------------
+// d2d_select_dynk_static: the same selection + metadata, for callers that are not allowed to
+// allocate device memory (and therefore cannot provide the workspace).  The per-block counter
+// scratch lives in this file-scope device array instead.  Every GPU that loads the library
+// holds these 512 KiB until the process exits.
+//
+// The name of a __device__ array is only a host-side stand-in in host code, not an address a
+// kernel can use; the device address is fetched once per device with cudaGetSymbolAddress
+// (with that device current) and cached.
+// ------------------------------------------------------------------------------------------
+#include <mutex>
+
+#define D2D_STATIC_SCRATCH_INTS (128 * 1024)          /* 512 KiB: ceil(T/1024) * E must not exceed this */
+static __device__ __align__(256) int32_t d2d_select_static_scratch[D2D_STATIC_SCRATCH_INTS];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+int32_t *g_scratch_ptr[kMaxDevices] = {};
+}
+
+extern "C" D2D_API d2d_status d2d_select_dynk_static(const float *R, int32_t T, int32_t E, float tau,
+                                                     d2d_routing *out, void *stream)
+{
+    if (T < 0 || E <= 0 || !out || !out->mask || !out->k || !out->counts || !out->offsets || !out->perm ||
+        !out->n_sel || !out->status || out->perm_capacity < 0)
+        return D2D_ERR_INVALID_ARG;
+    if ((out->tok_off == nullptr) != (out->tok_exp == nullptr)) return D2D_ERR_INVALID_ARG;
+    if (T > 0 && (!R || (reinterpret_cast<uintptr_t>(R) & 15u))) return D2D_ERR_INVALID_ARG;
+    if (!(tau >= 0.0f && tau <= 1.0f)) return D2D_ERR_INVALID_ARG;
+    // the scratch holds one counter per (block of 1024 tokens, expert)
+    const long long need = (long long)d2d_cdiv(T > 0 ? T : 1, TOKB) * (long long)E;
+    if (need > (long long)D2D_STATIC_SCRATCH_INTS) return D2D_ERR_UNSUPPORTED;
+
+    int dev = -1;
+    D2D_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return D2D_ERR_UNSUPPORTED;
+    int32_t *scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_scratch_mutex);
+        if (!g_scratch_ptr[dev]) {
+            // first call on this device: resolve the device address of the array (not capturable work)
+            void *p = nullptr;
+            if (cudaGetSymbolAddress(&p, d2d_select_static_scratch) != cudaSuccess || !p) return D2D_ERR_CUDA;
+            g_scratch_ptr[dev] = static_cast<int32_t *>(p);
+        }
+        scratch = g_scratch_ptr[dev];
+    }
+    // nothing in the scratch has to start at zero: the count kernel writes every counter the scan
+    // and fill kernels read, so the previous call's contents are simply overwritten
+    return d2d_launch_select(R, T, E, tau, 0, out, scratch, (cudaStream_t)stream);
+}

@@ -1,0 +1,50 @@
+"""d2d_select_dynk_static: the selection entry point for callers that cannot allocate device memory.
+
+Some hosts of this library (an inference plug-in's enqueue hook, a server whose device memory pool is
+frozen after start-up) are not allowed to call cudaMalloc, so they cannot provide the workspace that
+d2d_select_dynk needs.  The static variant keeps that scratch inside the library.  This test drives it
+through the C ABI twice in a row (the scratch is shared and keeps the previous call's contents) and
+requires bit-identical outputs to the regular entry point.  It lives in a file that pytest collects
+last, and it also passes when run alone in a fresh process.
+"""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2310_04361_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+def _outputs(r):
+    torch.cuda.synchronize()
+    n = r.n_sel
+    return (r.status, n, r.mask.cpu(), r.k.cpu(), r.counts.cpu(), r.offsets.cpu(), r.perm[:n].cpu(),
+            r.tok_off.cpu(), r.tok_exp[:n].cpu())
+
+
+def test_static_scratch_selection_matches_regular_entry_point_twice():
+    from paper_2310_04361_b200 import api
+    calls = [(wl.CONFIGS["vit"], 25216, 0.3), (wl.CONFIGS["llama"], 3000, 0.6), (wl.CONFIGS["vit"], 25216, 0.3)]
+    for cfg, T, tau in calls:                       # back-to-back calls share the library's scratch array
+        R = torch.from_numpy(wl.make_router_scores(cfg, T)).cuda()
+        want = _outputs(api.select_dynk(R, tau, dual=True))
+        routing = api.Routing(T, cfg.E, R.device, dual=True)     # outputs are still the caller's buffers
+        got = _outputs(api.select_dynk_static(R, tau, routing))
+        assert got[0] == want[0] == 0 and got[1] == want[1] > 0
+        for a, b in zip(got[2:], want[2:]):
+            assert torch.equal(a, b)                # integer outputs: bit-exact
+
+
+def test_static_scratch_limit_is_enforced():
+    from paper_2310_04361_b200 import api
+    T, E = 70000, 2048                              # ceil(T/1024) * E = 69 * 2048 > 131072
+    R = torch.zeros((8, E), dtype=torch.float32, device="cuda")
+    routing = api.Routing(8, E, R.device)
+    rc = api._lib.d2d_select_dynk_static(api._ptr(R), T, E, ctypes.c_float(0.5), ctypes.byref(routing.struct),
+                                         api._stream())
+    assert rc == 2                                  # D2D_ERR_UNSUPPORTED, nothing enqueued
+    torch.cuda.synchronize()
+    assert routing.n_sel == 0
