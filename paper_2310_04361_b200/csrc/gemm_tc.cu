@@ -2,10 +2,11 @@
 //
 //   warp 0   TMA producer: cp.async.bulk.tensor tiles of A (128 x 64) and B (BN x 64), 128-byte
 //            swizzled, into a ring of shared-memory stages guarded by full/empty mbarriers
-//   warp 1   allocates TMEM and issues tcgen05.mma (one thread), fp32 accumulator in TMEM;
-//            tcgen05.commit releases a stage when the MMAs that read it have retired
-//   warps 2-5  epilogue: tcgen05.ld the accumulator (one row per thread), bias / activation /
-//            selection mask, vectorised stores
+//   warp 1   allocates TMEM and issues tcgen05.mma (one thread), fp32 accumulators in TMEM
+//            (two buffers); tcgen05.commit releases a stage when the MMAs that read it have retired
+//   warps 2-9  epilogue: tcgen05.ld the accumulator (one row per thread), bias / activation /
+//            selection mask, vectorised stores; runs while the next tile's MMAs fill the other buffer
+// The kernel is persistent: one CTA per SM walks over the output tiles.
 //
 // Every mbarrier wait is bounded: when the limit runs out the role records D2D_ERR_TIMEOUT in the
 // status word and leaves its loop, all roles meet at the final barrier, TMEM is freed and the
@@ -17,7 +18,6 @@ namespace {
 constexpr int BM = 128;          // rows of A per CTA = TMEM lanes
 constexpr int BK = 64;           // 64 bf16 = one 128-byte swizzle row
 constexpr int UMMA_K = 16;
-constexpr int NTHREADS = 192;
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -43,7 +43,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t
             : "r"(bar), "r"(parity)
             : "memory");
         if (done) return true;
-        if (it > 32) __nanosleep(64);
+        if (it > 4096) __nanosleep(128);
     }
     if (status) atomicMax(status, (int32_t)D2D_ERR_TIMEOUT);
     return false;
@@ -112,45 +112,77 @@ struct EpiParams {
     int32_t *status;
 };
 
-__device__ __forceinline__ float act_runtime(float z, int act)
+// Activations of the bf16 tensor-core path.  Results are rounded to bf16 (8 bits of mantissa), so
+// the hardware exp2 / reciprocal approximations (about 2^-22 relative) are far below what survives;
+// erf uses the five-term rational form 1 - (a1 t + ... + a5 t^5) exp(-x^2), t = 1/(1 + p x),
+// whose absolute error is below 1.5e-7.
+template <int ACT> __device__ __forceinline__ float fast_act(float z)
 {
-    switch (act) {
-    case D2D_ACT_RELU: return d2d_activate<D2D_ACT_RELU>(z);
-    case D2D_ACT_GELU_ERF: return d2d_activate<D2D_ACT_GELU_ERF>(z);
-    case D2D_ACT_GELU_TANH: return d2d_activate<D2D_ACT_GELU_TANH>(z);
-    default: return d2d_activate<D2D_ACT_SILU>(z);
+    if (ACT == D2D_ACT_RELU) return fmaxf(z, 0.0f);
+    if (ACT == D2D_ACT_GELU_ERF) {
+        const float x = fabsf(z) * 0.70710678118654752f;
+        const float t = __frcp_rn(fmaf(0.3275911f, x, 1.0f));
+        float p = fmaf(1.061405429f, t, -1.453152027f);
+        p = fmaf(p, t, 1.421413741f);
+        p = fmaf(p, t, -0.284496736f);
+        p = fmaf(p, t, 0.254829592f);
+        const float erf_abs = 1.0f - p * t * __expf(-x * x);
+        return 0.5f * z * (1.0f + copysignf(erf_abs, z));
     }
+    if (ACT == D2D_ACT_GELU_TANH) {
+        const float u = 0.79788456080286536f * fmaf(0.044715f * z * z, z, z);
+        const float e2 = __expf(2.0f * u);                 // tanh(u) = 1 - 2 / (e^{2u} + 1)
+        const float th = 1.0f - __fdividef(2.0f, e2 + 1.0f);
+        return 0.5f * z * (1.0f + th);
+    }
+    return __fdividef(z, 1.0f + __expf(-z));               // SiLU
 }
 
-// One CTA computes one 128 x BN tile.  GATED: two B tiles (gate, up) share the A tile and the
-// epilogue combines A(gate) * (up + bias).
-template <int BN, int STAGES, int EPI, bool GATED>
-__global__ void __launch_bounds__(NTHREADS)
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+constexpr int N_EPI_WARPS = 8;
+constexpr int NTHREADS_V2 = 64 + 32 * N_EPI_WARPS;
+
+__host__ __device__ constexpr int pow2_at_least(int v) { return v <= 32 ? 32 : v <= 64 ? 64 : v <= 128 ? 128 : v <= 256 ? 256 : 512; }
+
+// Persistent kernel: CTA c computes tiles c, c + gridDim.x, ... (128 x BN each, column tiles
+// fastest).  Two accumulator buffers in TMEM let the epilogue of one tile overlap the MMAs of the
+// next.  GATED: two B tiles (up, gate) share the A tile; the epilogue forms A(gate) * (up + bias).
+template <int BN, int STAGES, int EPI, int ACT, bool GATED>
+__global__ void __launch_bounds__(NTHREADS_V2, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-               const __grid_constant__ CUtensorMap tm_b2, EpiParams ep, int M, int N, int K, int act)
+               const __grid_constant__ CUtensorMap tm_b2, EpiParams ep, int M, int N, int K)
 {
     constexpr int A_BYTES = BM * BK * 2;
     constexpr int B_BYTES = BN * BK * 2;
     constexpr int STAGE_BYTES = A_BYTES + (GATED ? 2 : 1) * B_BYTES;
-    constexpr int TMEM_COLS = GATED ? 2 * BN : BN;
-    static_assert(TMEM_COLS == 32 || TMEM_COLS == 64 || TMEM_COLS == 128 || TMEM_COLS == 256 || TMEM_COLS == 512, "power of two");
-    static_assert(BN % 32 == 0 && BN <= 256, "tile width");
+    constexpr int BUF_COLS = pow2_at_least(GATED ? 2 * BN : BN);    // TMEM columns per accumulator buffer
+    constexpr int TMEM_COLS = 2 * BUF_COLS;
+    constexpr int COLS_PER_WARP = BN / 2;                            // two epilogue warps share a TMEM lane quadrant
+    static_assert(TMEM_COLS <= 512 && BN % 64 == 0 && BN <= 256, "tile width");
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);   // swizzle atoms are 1024-byte aligned
-    __shared__ uint64_t bar_full[STAGES], bar_empty[STAGES], bar_acc;
+    __shared__ uint64_t bar_full[STAGES], bar_empty[STAGES], bar_acc_full[2], bar_acc_empty[2];
     __shared__ uint32_t tmem_base_holder;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
     const int nkb = (K + BK - 1) / BK;
+    const int n_tiles = (N + BN - 1) / BN;
+    const int total_tiles = ((M + BM - 1) / BM) * n_tiles;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(smem_u32(&bar_full[s]), 1);
             mbar_init(smem_u32(&bar_empty[s]), 1);
         }
-        mbar_init(smem_u32(&bar_acc), 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&bar_acc_full[b]), 1);
+            mbar_init(smem_u32(&bar_acc_empty[b]), N_EPI_WARPS);
+        }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -167,88 +199,135 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            for (int kb = 0; kb < nkb; ++kb) {
-                const int s = kb % STAGES;
-                const uint32_t round = (uint32_t)(kb / STAGES);
-                if (!mbar_wait(smem_u32(&bar_empty[s]), (round & 1u) ^ 1u, ep.status)) break;
-                const uint32_t full = smem_u32(&bar_full[s]);
-                const uint32_t dst = smem_u32(smem + (size_t)s * STAGE_BYTES);
-                mbar_expect_tx(full, (uint32_t)STAGE_BYTES);
-                tma_load_2d(dst, &tm_a, kb * BK, m0, full);
-                tma_load_2d(dst + A_BYTES, &tm_b, kb * BK, n0, full);
-                if (GATED) tma_load_2d(dst + A_BYTES + B_BYTES, &tm_b2, kb * BK, n0, full);
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+                const int m0 = (tile / n_tiles) * BM, n0 = (tile % n_tiles) * BN;
+                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                    const uint32_t s = it % STAGES, round = it / STAGES;
+                    ok = mbar_wait(smem_u32(&bar_empty[s]), (round & 1u) ^ 1u, ep.status);
+                    if (!ok) break;
+                    const uint32_t full = smem_u32(&bar_full[s]);
+                    const uint32_t dst = smem_u32(smem + (size_t)s * STAGE_BYTES);
+                    mbar_expect_tx(full, (uint32_t)STAGE_BYTES);
+                    tma_load_2d(dst, &tm_a, kb * BK, m0, full);
+                    tma_load_2d(dst + A_BYTES, &tm_b, kb * BK, n0, full);
+                    if (GATED) tma_load_2d(dst + A_BYTES + B_BYTES, &tm_b2, kb * BK, n0, full);
+                }
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             const uint32_t idesc = instr_desc_bf16(BM, BN);
+            uint32_t it = 0, local = 0;
             bool ok = true;
-            for (int kb = 0; kb < nkb && ok; ++kb) {
-                const int s = kb % STAGES;
-                const uint32_t round = (uint32_t)(kb / STAGES);
-                ok = mbar_wait(smem_u32(&bar_full[s]), round & 1u, ep.status);
+            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++local) {
+                const uint32_t buf = local & 1u, use = local >> 1;
+                ok = mbar_wait(smem_u32(&bar_acc_empty[buf]), (use & 1u) ^ 1u, ep.status);   // epilogue drained this buffer
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t a_addr = smem_u32(smem + (size_t)s * STAGE_BYTES);
-                const uint64_t da = smem_desc_sw128(a_addr);
-                const uint64_t db = smem_desc_sw128(a_addr + A_BYTES);
-                const uint64_t db2 = smem_desc_sw128(a_addr + A_BYTES + B_BYTES);
+                const uint32_t acc = tmem_base + buf * BUF_COLS;
+                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                    const uint32_t s = it % STAGES, round = it / STAGES;
+                    ok = mbar_wait(smem_u32(&bar_full[s]), round & 1u, ep.status);
+                    if (!ok) break;
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t a_addr = smem_u32(smem + (size_t)s * STAGE_BYTES);
+                    const uint64_t da = smem_desc_sw128(a_addr);
+                    const uint64_t db = smem_desc_sw128(a_addr + A_BYTES);
+                    const uint64_t db2 = smem_desc_sw128(a_addr + A_BYTES + B_BYTES);
 #pragma unroll
-                for (int k = 0; k < BK / UMMA_K; ++k) {
-                    const uint64_t koff = (uint64_t)((k * UMMA_K * 2) >> 4);    // 32 bytes per K step inside the swizzle row
-                    const uint32_t accum = (kb | k) != 0 ? 1u : 0u;
-                    umma_bf16(tmem_base, da + koff, db + koff, idesc, accum);
-                    if (GATED) umma_bf16(tmem_base + BN, da + koff, db2 + koff, idesc, accum);
+                    for (int k = 0; k < BK / UMMA_K; ++k) {
+                        const uint64_t koff = (uint64_t)((k * UMMA_K * 2) >> 4);    // 32 bytes per K step inside the swizzle row
+                        const uint32_t accum = (kb | k) != 0 ? 1u : 0u;
+                        umma_bf16(acc, da + koff, db + koff, idesc, accum);
+                        if (GATED) umma_bf16(acc + BN, da + koff, db2 + koff, idesc, accum);
+                    }
+                    umma_commit(smem_u32(&bar_empty[s]));      // stage reusable once these MMAs have read it
                 }
-                umma_commit(smem_u32(&bar_empty[s]));      // stage reusable once these MMAs have read it
+                umma_commit(smem_u32(&bar_acc_full[buf]));     // accumulator of this tile complete
             }
-            umma_commit(smem_u32(&bar_acc));               // accumulator complete
         }
     } else {
-        // ------------------------------------------------------------------ epilogue (warps 2..5)
+        // ------------------------------------------------------------------ epilogue (warps 2..9)
+        const int ew = warp - 2;
         const int quad = warp & 3;                          // TMEM lanes this warp may touch
-        const int row = m0 + quad * 32 + lane;
-        const bool acc_ok = mbar_wait(smem_u32(&bar_acc), 0, ep.status);
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        if (acc_ok) {
+        const int half = ew >> 2;                           // which half of the tile's columns
+        uint32_t local = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++local) {
+            const int m0 = (tile / n_tiles) * BM, n0 = (tile % n_tiles) * BN;
+            const uint32_t buf = local & 1u, use = local >> 1;
+            int okw = 1;
+            if (lane == 0) okw = mbar_wait(smem_u32(&bar_acc_full[buf]), use & 1u, ep.status) ? 1 : 0;
+            ok = __shfl_sync(0xffffffffu, okw, 0) != 0;
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const int row = m0 + quad * 32 + lane;
             const uint32_t *mrow = (EPI == D2D_EPI_UP_MASKED && ep.mask && row < M)
                                        ? ep.mask + (size_t)row * ep.mask_words : nullptr;
 #pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                if (n0 + c0 >= N) break;                    // warp-uniform
+            for (int cc = 0; cc < COLS_PER_WARP; cc += 32) {
+                const int c0 = half * COLS_PER_WARP + cc;
+                const int col0 = n0 + c0;
+                if (col0 >= N) break;                       // warp-uniform
                 uint32_t r[32], g[32];
-                const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)c0;
+                const uint32_t taddr = tmem_base + buf * BUF_COLS + ((uint32_t)(quad * 32) << 16) + (uint32_t)c0;
                 tmem_ld32(taddr, r);
                 if (GATED) tmem_ld32(taddr + BN, g);
-                float v[32];
-                int e = 0, rem = 0;
-                if (EPI == D2D_EPI_UP_MASKED) {
-                    e = (n0 + c0) / ep.expert_size;
-                    rem = (n0 + c0) - e * ep.expert_size;
+
+                // bias for these 32 columns: four 16-byte loads when the chunk is whole
+                float bias[32];
+                if (ep.bias && col0 + 32 <= N && (col0 & 7) == 0) {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const uint4 raw = __ldg(reinterpret_cast<const uint4 *>(ep.bias + col0) + q);
+                        const uint32_t w4[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            bias[q * 8 + 2 * i] = __uint_as_float(w4[i] << 16);
+                            bias[q * 8 + 2 * i + 1] = __uint_as_float(w4[i] & 0xffff0000u);
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) bias[j] = (ep.bias && col0 + j < N) ? __bfloat162float(ep.bias[col0 + j]) : 0.0f;
                 }
+
+                // selection bits of this row for the 32 columns: a few experts cover them
+                uint32_t keep = 0xffffffffu;
+                if (EPI == D2D_EPI_UP_MASKED && mrow) {
+                    keep = 0u;
+                    const int s = ep.expert_size;
+                    int e = col0 / s;
+                    int lo = e * s - col0;                  // first column of expert e relative to the chunk (<= 0)
+                    while (lo < 32) {
+                        const int hi = lo + s;
+                        if ((__ldg(mrow + (e >> 5)) >> (e & 31)) & 1u) {
+                            const int a = lo < 0 ? 0 : lo, b = hi > 32 ? 32 : hi;
+                            const uint32_t upto_b = b >= 32 ? 0xffffffffu : ((1u << b) - 1u);
+                            keep |= upto_b & ~((1u << a) - 1u);
+                        }
+                        lo = hi;
+                        ++e;
+                    }
+                }
+
+                float v[32];
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
-                    const int col = n0 + c0 + j;
-                    const float b = (ep.bias && col < N) ? __bfloat162float(ep.bias[col]) : 0.0f;
-                    float z = __uint_as_float(r[j]) + b;
+                    float z = __uint_as_float(r[j]) + bias[j];
                     if (EPI == D2D_EPI_RELU_BF16) z = fmaxf(z, 0.0f);
                     if (EPI == D2D_EPI_ABS_F32) z = fabsf(z);
                     if (EPI == D2D_EPI_UP_MASKED) {
-                        bool keep = true;
-                        if (mrow) keep = (mrow[e >> 5] >> (e & 31)) & 1u;
-                        if (GATED) {
-                            // first accumulator = up projection (+ bias), second = gate
-                            z = keep ? act_runtime(__uint_as_float(g[j]), act) * z : 0.0f;
-                        } else {
-                            z = keep ? act_runtime(z, act) : 0.0f;
-                        }
-                        if (++rem == ep.expert_size) { rem = 0; ++e; }
+                        // first accumulator = up projection (+ bias), second = gate
+                        const float h = GATED ? fast_act<ACT>(__uint_as_float(g[j])) * z : fast_act<ACT>(z);
+                        z = ((keep >> j) & 1u) ? h : 0.0f;
                     }
                     v[j] = z;
                 }
                 if (row < M) {
-                    const int col0 = n0 + c0;
                     if (EPI == D2D_EPI_ABS_F32) {
                         float *o = (float *)ep.out + (size_t)row * N + col0;
                         if (col0 + 32 <= N && (N & 3) == 0) {
@@ -283,6 +362,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     }
                 }
             }
+            // all of this warp's TMEM reads of the buffer are complete: hand it back to the MMA warp
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[buf]));
         }
     }
 
@@ -326,9 +409,27 @@ bool make_map(CUtensorMap *map, const void *base, int rows, int cols, int box_ro
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN, int STAGES, int EPI, bool GATED>
+int g_sm_count = 0;
+
+int sm_count()
+{
+    if (g_sm_count == 0) {
+        int dev = 0, n = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
+            g_sm_count = n;
+        else
+            return 148;
+    }
+    return g_sm_count;
+}
+
+template <int BN, int EPI, int ACT, bool GATED>
 d2d_status launch(const d2d_gemm_args &g, cudaStream_t st)
 {
+    constexpr int STAGE_BYTES = BM * BK * 2 + (GATED ? 2 : 1) * BN * BK * 2;
+    constexpr int STAGES = (200 * 1024) / STAGE_BYTES > 8 ? 8 : (200 * 1024) / STAGE_BYTES;
+    constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + 1024;
     CUtensorMap ta, tb, tb2;
     if (!make_map(&ta, g.a, g.M, g.K, BM) || !make_map(&tb, g.b, g.N, g.K, BN)) return D2D_ERR_CUDA;
     if (GATED) {
@@ -336,19 +437,64 @@ d2d_status launch(const d2d_gemm_args &g, cudaStream_t st)
     } else {
         tb2 = tb;
     }
-    constexpr int STAGE_BYTES = BM * BK * 2 + (GATED ? 2 : 1) * BN * BK * 2;
-    constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + 1024;
-    auto kern = gemm_tc_kernel<BN, STAGES, EPI, GATED>;
+    auto kern = gemm_tc_kernel<BN, STAGES, EPI, ACT, GATED>;
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM) != cudaSuccess) return D2D_ERR_CUDA;
         attr_set = true;
     }
     EpiParams ep{(const __nv_bfloat16 *)g.bias, g.out, g.mask, g.mask_words, g.expert_size > 0 ? g.expert_size : 1, g.status};
-    dim3 grid(d2d_cdiv(g.N, BN), d2d_cdiv(g.M, BM));
-    kern<<<grid, NTHREADS, SMEM, st>>>(ta, tb, tb2, ep, g.M, g.N, g.K, g.act);
+    const int tiles = d2d_cdiv(g.N, BN) * d2d_cdiv(g.M, BM);
+    const int grid = tiles < sm_count() ? tiles : sm_count();
+    kern<<<grid, NTHREADS_V2, SMEM, st>>>(ta, tb, tb2, ep, g.M, g.N, g.K);
     D2D_LAUNCHED(1);
     return cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
+}
+
+// Tile width that wastes the fewest SM-rounds: tiles / (rounds * SMs), wider tiles preferred on ties
+// (fewer re-reads of A, fewer per-tile overheads).
+int pick_bn(int M, int N, const int *cands, int n_cands)
+{
+    const int sms = sm_count();
+    int best = cands[0];
+    double best_eff = -1.0;
+    for (int i = 0; i < n_cands; ++i) {
+        const int bn = cands[i];
+        const long tiles = (long)d2d_cdiv(N, bn) * d2d_cdiv(M, BM);
+        const long rounds = (tiles + sms - 1) / sms;
+        const double useful = (double)N / ((double)d2d_cdiv(N, bn) * bn);       // ragged last column tile
+        const double eff = useful * (double)tiles / (double)(rounds * sms) * (bn >= 128 ? 1.0 : 0.85);
+        if (eff > best_eff + 1e-9) { best_eff = eff; best = bn; }
+    }
+    return best;
+}
+
+template <int EPI, int ACT, bool GATED>
+d2d_status launch_bn(const d2d_gemm_args &g, cudaStream_t st)
+{
+    if (GATED) {
+        return launch<128, EPI, ACT, true>(g, st);
+    } else {
+        const int cands[4] = {256, 192, 128, 64};
+        switch (pick_bn(g.M, g.N, cands, 4)) {
+        case 256: return launch<256, EPI, ACT, false>(g, st);
+        case 192: return launch<192, EPI, ACT, false>(g, st);
+        case 128: return launch<128, EPI, ACT, false>(g, st);
+        default: return launch<64, EPI, ACT, false>(g, st);
+        }
+    }
+}
+
+template <bool GATED>
+d2d_status launch_up(const d2d_gemm_args &g, cudaStream_t st)
+{
+    switch (g.act) {
+    case D2D_ACT_RELU: return launch_bn<D2D_EPI_UP_MASKED, D2D_ACT_RELU, GATED>(g, st);
+    case D2D_ACT_GELU_ERF: return launch_bn<D2D_EPI_UP_MASKED, D2D_ACT_GELU_ERF, GATED>(g, st);
+    case D2D_ACT_GELU_TANH: return launch_bn<D2D_EPI_UP_MASKED, D2D_ACT_GELU_TANH, GATED>(g, st);
+    case D2D_ACT_SILU: return launch_bn<D2D_EPI_UP_MASKED, D2D_ACT_SILU, GATED>(g, st);
+    }
+    return D2D_ERR_INVALID_ARG;
 }
 
 }  // namespace
@@ -360,13 +506,10 @@ d2d_status d2d_gemm_tc(const d2d_gemm_args &g, cudaStream_t st)
     if (g.M <= 0 || g.N <= 0 || g.K <= 0) return D2D_OK;
     if (g.K % 8) return D2D_ERR_UNSUPPORTED;
     switch (g.epilogue) {
-    // 3 stages of 32 KB let two CTAs share an SM (one runs its epilogue while the other feeds the tensor cores)
-    case D2D_EPI_RELU_BF16: return launch<128, 3, D2D_EPI_RELU_BF16, false>(g, st);
-    case D2D_EPI_ABS_F32: return launch<128, 3, D2D_EPI_ABS_F32, false>(g, st);
-    case D2D_EPI_BIAS_BF16: return launch<128, 3, D2D_EPI_BIAS_BF16, false>(g, st);
-    case D2D_EPI_UP_MASKED:
-        if (g.b_gate) return launch<128, 4, D2D_EPI_UP_MASKED, true>(g, st);
-        return launch<128, 3, D2D_EPI_UP_MASKED, false>(g, st);
+    case D2D_EPI_RELU_BF16: return launch_bn<D2D_EPI_RELU_BF16, 0, false>(g, st);
+    case D2D_EPI_ABS_F32: return launch_bn<D2D_EPI_ABS_F32, 0, false>(g, st);
+    case D2D_EPI_BIAS_BF16: return launch_bn<D2D_EPI_BIAS_BF16, 0, false>(g, st);
+    case D2D_EPI_UP_MASKED: return g.b_gate ? launch_up<true>(g, st) : launch_up<false>(g, st);
     }
     return D2D_ERR_INVALID_ARG;
 }
