@@ -183,16 +183,17 @@ D2D_API d2d_status d2d_routing_from_mask(int32_t T, int32_t E, d2d_routing *out,
  * allocates nothing, on the host or the device, and frees nothing.
  *   - Same inputs, outputs, rule and error reporting as d2d_select_dynk; the
  *     caller still passes R and the routing buffers.
- *   - Limit: ceil(T / 1024) * E <= 131072 (for example 65,536 tokens at 2,048
- *     experts, or any T <= 1024 with E <= 131,072); beyond it the call returns
- *     D2D_ERR_UNSUPPORTED and enqueues nothing.
+ *   - Limit: 64 + ceil(T / 256) * E <= 131072 (for example 16,000 tokens at
+ *     2,048 experts, or 87,000 tokens at 384 experts); beyond it the call
+ *     returns D2D_ERR_UNSUPPORTED and enqueues nothing.
  *   - The first call on each device looks up the array's device address (once,
  *     with that device current).  Make that first call outside any stream
  *     capture.
  *   - All calls on one device share the array, so two calls whose kernels can
  *     overlap on the GPU (different streams) race; serialise them.  The array
- *     keeps the previous call's contents, which is harmless: each call
- *     overwrites every entry before reading it. */
+ *     keeps the previous call's contents: the one word that must start at
+ *     zero is cleared by every call, every other entry is overwritten before
+ *     it is read. */
 D2D_API d2d_status d2d_select_dynk_static(const float *R, int32_t T, int32_t E, float tau, d2d_routing *out,
                                           void *stream);
 

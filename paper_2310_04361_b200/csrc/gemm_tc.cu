@@ -89,19 +89,7 @@ __device__ __forceinline__ void umma_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr));
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 struct EpiParams {
     const __nv_bfloat16 *bias;
@@ -116,18 +104,32 @@ struct EpiParams {
 // the hardware exp2 / reciprocal approximations (about 2^-22 relative) are far below what survives;
 // erf uses the five-term rational form 1 - (a1 t + ... + a5 t^5) exp(-x^2), t = 1/(1 + p x),
 // whose absolute error is below 1.5e-7.
+__device__ __forceinline__ float fast_rcp(float x)
+{
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float fast_exp2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 template <int ACT> __device__ __forceinline__ float fast_act(float z)
 {
     if (ACT == D2D_ACT_RELU) return fmaxf(z, 0.0f);
     if (ACT == D2D_ACT_GELU_ERF) {
-        const float x = fabsf(z) * 0.70710678118654752f;
-        const float t = __frcp_rn(fmaf(0.3275911f, x, 1.0f));
+        // gelu(z) = max(z, 0) - 0.5 |z| erfc(|z| / sqrt 2), erfc(x) = (a1 t + ... + a5 t^5) exp(-x^2)
+        const float az = fabsf(z);
+        const float t = fast_rcp(fmaf(0.3275911f * 0.70710678118654752f, az, 1.0f));
         float p = fmaf(1.061405429f, t, -1.453152027f);
         p = fmaf(p, t, 1.421413741f);
         p = fmaf(p, t, -0.284496736f);
         p = fmaf(p, t, 0.254829592f);
-        const float erf_abs = 1.0f - p * t * __expf(-x * x);
-        return 0.5f * z * (1.0f + copysignf(erf_abs, z));
+        const float e = fast_exp2(z * z * -0.72134752044448170f);          // exp(-z^2 / 2)
+        return fmaxf(z, 0.0f) - (0.5f * az) * (p * t) * e;
     }
     if (ACT == D2D_ACT_GELU_TANH) {
         const float u = 0.79788456080286536f * fmaf(0.044715f * z * z, z, z);
@@ -143,7 +145,52 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr));
+}
+
+// 16 accumulator columns -> 16 output values: bias, activation, selection mask.
+template <int EPI, int ACT, bool GATED>
+__device__ __forceinline__ void epilogue_16(const uint32_t (&r)[16], const uint32_t (&g)[16], float *v,
+                                            const float *bias_f, const __nv_bfloat16 *bias_g, bool bias_cached,
+                                            int col0, int N, uint32_t keep)
+{
+    float bias[16];
+    if (bias_g == nullptr) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) bias[j] = 0.0f;
+    } else if (bias_cached && col0 + 16 <= N) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const float4 b4 = *reinterpret_cast<const float4 *>(bias_f + col0 + 4 * q);
+            bias[4 * q] = b4.x; bias[4 * q + 1] = b4.y; bias[4 * q + 2] = b4.z; bias[4 * q + 3] = b4.w;
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) bias[j] = col0 + j < N ? __bfloat162float(bias_g[col0 + j]) : 0.0f;
+    }
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        float z = __uint_as_float(r[j]) + bias[j];
+        if (EPI == D2D_EPI_RELU_BF16) z = fmaxf(z, 0.0f);
+        if (EPI == D2D_EPI_ABS_F32) z = fabsf(z);
+        if (EPI == D2D_EPI_UP_MASKED) {
+            // first accumulator = up projection (+ bias), second = gate
+            const float h = GATED ? fast_act<ACT>(__uint_as_float(g[j])) * z : fast_act<ACT>(z);
+            z = ((keep >> j) & 1u) ? h : 0.0f;
+        }
+        v[j] = z;
+    }
+}
+
 constexpr int N_EPI_WARPS = 8;
+constexpr int BIAS_CACHE_ELEMS = 6144;           // 24 KB of float32 in shared memory behind the operand stages
 constexpr int NTHREADS_V2 = 64 + 32 * N_EPI_WARPS;
 
 __host__ __device__ constexpr int pow2_at_least(int v) { return v <= 32 ? 32 : v <= 64 ? 64 : v <= 128 ? 128 : v <= 256 ? 256 : 512; }
@@ -168,6 +215,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);   // swizzle atoms are 1024-byte aligned
     __shared__ uint64_t bar_full[STAGES], bar_empty[STAGES], bar_acc_full[2], bar_acc_empty[2];
     __shared__ uint32_t tmem_base_holder;
+    constexpr int MASK_REGS = 16;                                    // selection words of a row kept in registers
+    // the whole bias vector is staged once, as float32, behind the operand stages when it fits
+    float *bias_f = reinterpret_cast<float *>(smem + (size_t)STAGES * STAGE_BYTES);
+    const bool bias_cached = ep.bias != nullptr && N <= BIAS_CACHE_ELEMS && (N & 3) == 0;
+    if (bias_cached) {
+        for (int i = threadIdx.x; i < N; i += NTHREADS_V2) bias_f[i] = __bfloat162float(ep.bias[i]);
+    }
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nkb = (K + BK - 1) / BK;
@@ -251,49 +305,45 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         }
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..9)
+        // The chunk loop is deliberately NOT unrolled: the body (32 elements of bias + activation +
+        // mask + pack) is a few KB of code that then stays in the instruction cache; unrolling it over
+        // the chunks made the kernel fetch-bound.  TMEM loads are split in 16-column halves so that the
+        // load of the next half overlaps the math of the current one.
         const int ew = warp - 2;
         const int quad = warp & 3;                          // TMEM lanes this warp may touch
         const int half = ew >> 2;                           // which half of the tile's columns
+        constexpr int N_CHUNKS = COLS_PER_WARP / 32;
         uint32_t local = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++local) {
             const int m0 = (tile / n_tiles) * BM, n0 = (tile % n_tiles) * BN;
             const uint32_t buf = local & 1u, use = local >> 1;
+            const int row = m0 + quad * 32 + lane;
+            // this row's selection words go to registers before the wait, so their latency is hidden
+            uint32_t mw[MASK_REGS];
+            const uint32_t *mrow = nullptr;
+            if (EPI == D2D_EPI_UP_MASKED && ep.mask && row < M) {
+                mrow = ep.mask + (size_t)row * ep.mask_words;
+                if (ep.mask_words <= MASK_REGS) {
+#pragma unroll
+                    for (int i = 0; i < MASK_REGS; ++i) mw[i] = i < ep.mask_words ? __ldg(mrow + i) : 0u;
+                }
+            }
             int okw = 1;
             if (lane == 0) okw = mbar_wait(smem_u32(&bar_acc_full[buf]), use & 1u, ep.status) ? 1 : 0;
             ok = __shfl_sync(0xffffffffu, okw, 0) != 0;
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const int row = m0 + quad * 32 + lane;
-            const uint32_t *mrow = (EPI == D2D_EPI_UP_MASKED && ep.mask && row < M)
-                                       ? ep.mask + (size_t)row * ep.mask_words : nullptr;
-#pragma unroll 1
-            for (int cc = 0; cc < COLS_PER_WARP; cc += 32) {
-                const int c0 = half * COLS_PER_WARP + cc;
-                const int col0 = n0 + c0;
-                if (col0 >= N) break;                       // warp-uniform
-                uint32_t r[32], g[32];
-                const uint32_t taddr = tmem_base + buf * BUF_COLS + ((uint32_t)(quad * 32) << 16) + (uint32_t)c0;
-                tmem_ld32(taddr, r);
-                if (GATED) tmem_ld32(taddr + BN, g);
+            const uint32_t tbase = tmem_base + buf * BUF_COLS + ((uint32_t)(quad * 32) << 16) + (uint32_t)(half * COLS_PER_WARP);
 
-                // bias for these 32 columns: four 16-byte loads when the chunk is whole
-                float bias[32];
-                if (ep.bias && col0 + 32 <= N && (col0 & 7) == 0) {
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const uint4 raw = __ldg(reinterpret_cast<const uint4 *>(ep.bias + col0) + q);
-                        const uint32_t w4[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            bias[q * 8 + 2 * i] = __uint_as_float(w4[i] << 16);
-                            bias[q * 8 + 2 * i + 1] = __uint_as_float(w4[i] & 0xffff0000u);
-                        }
-                    }
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) bias[j] = (ep.bias && col0 + j < N) ? __bfloat162float(ep.bias[col0 + j]) : 0.0f;
-                }
+            uint32_t ra[16], rb[16], ga[16], gb[16];
+            tmem_ld16_issue(tbase, ra);
+            if (GATED) tmem_ld16_issue(tbase + BN, ga);
+#pragma unroll 1
+            for (int ci = 0; ci < N_CHUNKS; ++ci) {
+                const int c0 = half * COLS_PER_WARP + ci * 32;
+                const int col0 = n0 + c0;
+                const bool whole = col0 + 32 <= N;          // warp-uniform; ragged only in the last column tile
 
                 // selection bits of this row for the 32 columns: a few experts cover them
                 uint32_t keep = 0xffffffffu;
@@ -304,9 +354,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     int lo = e * s - col0;                  // first column of expert e relative to the chunk (<= 0)
                     while (lo < 32) {
                         const int hi = lo + s;
-                        if ((__ldg(mrow + (e >> 5)) >> (e & 31)) & 1u) {
-                            const int a = lo < 0 ? 0 : lo, b = hi > 32 ? 32 : hi;
-                            const uint32_t upto_b = b >= 32 ? 0xffffffffu : ((1u << b) - 1u);
+                        uint32_t word;
+                        if (ep.mask_words <= MASK_REGS) {
+                            word = 0u;
+#pragma unroll
+                            for (int i = 0; i < MASK_REGS; ++i) word = (i == (e >> 5)) ? mw[i] : word;
+                        } else {
+                            word = __ldg(mrow + (e >> 5));
+                        }
+                        if ((word >> (e & 31)) & 1u) {
+                            const int a = lo < 0 ? 0 : lo, b2 = hi > 32 ? 32 : hi;
+                            const uint32_t upto_b = b2 >= 32 ? 0xffffffffu : ((1u << b2) - 1u);
                             keep |= upto_b & ~((1u << a) - 1u);
                         }
                         lo = hi;
@@ -315,32 +373,31 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 }
 
                 float v[32];
-#pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    float z = __uint_as_float(r[j]) + bias[j];
-                    if (EPI == D2D_EPI_RELU_BF16) z = fmaxf(z, 0.0f);
-                    if (EPI == D2D_EPI_ABS_F32) z = fabsf(z);
-                    if (EPI == D2D_EPI_UP_MASKED) {
-                        // first accumulator = up projection (+ bias), second = gate
-                        const float h = GATED ? fast_act<ACT>(__uint_as_float(g[j])) * z : fast_act<ACT>(z);
-                        z = ((keep >> j) & 1u) ? h : 0.0f;
-                    }
-                    v[j] = z;
+                tmem_ld_wait();                                                   // ra (and ga) have landed
+                tmem_ld16_issue(tbase + ci * 32 + 16, rb);
+                if (GATED) tmem_ld16_issue(tbase + ci * 32 + 16 + BN, gb);
+                epilogue_16<EPI, ACT, GATED>(ra, ga, v, bias_f, ep.bias, bias_cached, col0, N, keep);
+                tmem_ld_wait();                                                   // rb (and gb) have landed
+                if (ci + 1 < N_CHUNKS) {
+                    tmem_ld16_issue(tbase + (ci + 1) * 32, ra);
+                    if (GATED) tmem_ld16_issue(tbase + (ci + 1) * 32 + BN, ga);
                 }
-                if (row < M) {
+                epilogue_16<EPI, ACT, GATED>(rb, gb, v + 16, bias_f, ep.bias, bias_cached, col0 + 16, N, keep >> 16);
+
+                if (row < M && col0 < N) {
                     if (EPI == D2D_EPI_ABS_F32) {
                         float *o = (float *)ep.out + (size_t)row * N + col0;
-                        if (col0 + 32 <= N && (N & 3) == 0) {
+                        if (whole && (N & 3) == 0) {
 #pragma unroll
                             for (int j = 0; j < 32; j += 4) *reinterpret_cast<float4 *>(o + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-                        } else {
+                        } else {                            // ragged last column tile
 #pragma unroll
                             for (int j = 0; j < 32; ++j)
                                 if (col0 + j < N) o[j] = v[j];
                         }
                     } else {
                         __nv_bfloat16 *o = (__nv_bfloat16 *)ep.out + (size_t)row * N + col0;
-                        if (col0 + 32 <= N && (N & 7) == 0) {
+                        if (whole && (N & 7) == 0) {
 #pragma unroll
                             for (int j = 0; j < 32; j += 8) {
                                 uint4 pk;
@@ -354,7 +411,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                                 pk.w = *reinterpret_cast<uint32_t *>(&t3);
                                 *reinterpret_cast<uint4 *>(o + j) = pk;
                             }
-                        } else {
+                        } else {                            // ragged last column tile
 #pragma unroll
                             for (int j = 0; j < 32; ++j)
                                 if (col0 + j < N) o[j] = __float2bfloat16_rn(v[j]);
@@ -428,8 +485,8 @@ template <int BN, int EPI, int ACT, bool GATED>
 d2d_status launch(const d2d_gemm_args &g, cudaStream_t st)
 {
     constexpr int STAGE_BYTES = BM * BK * 2 + (GATED ? 2 : 1) * BN * BK * 2;
-    constexpr int STAGES = (200 * 1024) / STAGE_BYTES > 8 ? 8 : (200 * 1024) / STAGE_BYTES;
-    constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + 1024;
+    constexpr int STAGES = (196 * 1024) / STAGE_BYTES > 8 ? 8 : (196 * 1024) / STAGE_BYTES;
+    constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + 1024 + (size_t)BIAS_CACHE_ELEMS * 4;
     CUtensorMap ta, tb, tb2;
     if (!make_map(&ta, g.a, g.M, g.K, BM) || !make_map(&tb, g.b, g.N, g.K, BN)) return D2D_ERR_CUDA;
     if (GATED) {

@@ -4,10 +4,10 @@
 //
 //   mask kernel     one warp per token: row max, thr = tau*max (one fp32 RN multiply),
 //                   ballot -> packed mask words, popcount -> k
-//   count kernel    1024 tokens per CTA; each warp turns its 32 tokens x 32 experts bit tile
-//                   into per-expert token bitmaps with 32 ballots (a register transpose)
-//   scan kernel     one CTA: per expert, exclusive scan over the token blocks; then the
-//                   exclusive scan over experts -> counts, offsets, n_sel
+//   count kernel    256 tokens per CTA; each warp turns its 32 tokens x 32 experts bit tile
+//                   into per-expert token bitmaps with 32 ballots (a register transpose);
+//                   the CTA that finishes last scans: per expert over the token blocks, then
+//                   over the experts -> counts, offsets, n_sel
 //   fill kernel     same tiling as the count kernel; rank of a token inside its expert's
 //                   list = block base + popcounts of the warps before it + popcount of the
 //                   lower lanes: tokens come out in ascending order
@@ -16,7 +16,7 @@
 
 namespace {
 
-constexpr int TOKB = 1024;        // tokens per CTA in the count / fill kernels (32 warps x 32 tokens)
+constexpr int TOKB = 256;         // tokens per CTA in the count / fill kernels (8 warps x 32 tokens)
 constexpr unsigned FULL = 0xffffffffu;
 
 __device__ __forceinline__ bool is_finite_f32(float v) { return (__float_as_uint(v) & 0x7f800000u) != 0x7f800000u; }
@@ -133,10 +133,51 @@ __device__ __forceinline__ uint32_t transpose_bits(uint32_t word, int lane)
     return col;
 }
 
-__global__ void __launch_bounds__(TOKB)
-bucket_count_kernel(const uint32_t *__restrict__ mask, int T, int E, int W, int32_t *__restrict__ blockcounts)
+// Exclusive scan of one int per thread over a 256-thread CTA; returns the exclusive prefix and
+// leaves the CTA total in *total_out (shared).
+__device__ __forceinline__ int block_exscan_256(int v, int *warp_sums /*[8]*/, int *total_out)
 {
-    __shared__ int32_t cnt[32][33];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int n = __shfl_up_sync(FULL, inc, o);
+        if (lane >= o) inc += n;
+    }
+    if (lane == 31) warp_sums[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        const int ws = lane < 8 ? warp_sums[lane] : 0;
+        int winc = ws;
+#pragma unroll
+        for (int o = 1; o < 8; o <<= 1) {
+            const int n = __shfl_up_sync(FULL, winc, o);
+            if (lane >= o) winc += n;
+        }
+        if (lane < 8) warp_sums[lane] = winc - ws;
+        if (lane == 7) *total_out = winc;
+    }
+    __syncthreads();
+    const int res = warp_sums[warp] + inc - v;
+    __syncthreads();
+    return res;
+}
+
+// Per-expert token counts of each 256-token block (8 warps x 32 tokens; a warp turns its
+// 32 x 32 bit tile into per-expert bitmaps with 32 ballots).  The CTA that finishes last (ticket
+// counter) then scans: per expert the exclusive prefix over the blocks, and over the experts the
+// exclusive prefix of the totals -> counts, offsets, n_sel.  Integer sums only: the result does
+// not depend on which CTA is last.
+__global__ void __launch_bounds__(TOKB)
+bucket_count_scan_kernel(const uint32_t *__restrict__ mask, int T, int E, int W, int nblk,
+                         int32_t *__restrict__ blockcounts, unsigned int *__restrict__ ticket,
+                         int32_t *__restrict__ counts, int32_t *__restrict__ offsets, int32_t *__restrict__ n_sel,
+                         int32_t *__restrict__ status, long long capacity)
+{
+    __shared__ int32_t cnt[TOKB / 32][33];
+    __shared__ int warp_sums[8];
+    __shared__ int chunk_total;
+    __shared__ unsigned int my_ticket;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int t = blockIdx.x * TOKB + threadIdx.x;
     for (int w = 0; w < W; ++w) {
@@ -146,16 +187,80 @@ bucket_count_kernel(const uint32_t *__restrict__ mask, int T, int E, int W, int3
         if (warp == 0) {
             int total = 0;
 #pragma unroll
-            for (int i = 0; i < 32; ++i) total += cnt[i][lane];
+            for (int i = 0; i < TOKB / 32; ++i) total += cnt[i][lane];
             const int e = w * 32 + lane;
             if (e < E) blockcounts[(size_t)blockIdx.x * E + e] = total;
         }
         __syncthreads();
     }
+    __threadfence();
+    if (threadIdx.x == 0) my_ticket = atomicAdd(ticket, 1u);
+    __syncthreads();
+    if (my_ticket != (unsigned int)(nblk - 1)) return;
+    __threadfence();                         // every other CTA's block counts are visible now
+    if (threadIdx.x == 0) *ticket = 0u;      // ready for the next call
+    int carry = 0;
+    for (int e0 = 0; e0 < E; e0 += TOKB) {
+        const int e = e0 + threadIdx.x;
+        int run = 0;
+        if (e < E) {
+            for (int b = 0; b < nblk; ++b) {
+                const int c = __ldcg(blockcounts + (size_t)b * E + e);
+                blockcounts[(size_t)b * E + e] = run;      // exclusive prefix over the token blocks
+                run += c;
+            }
+            counts[e] = run;
+        }
+        const int ex = block_exscan_256(run, warp_sums, &chunk_total);
+        if (e < E) offsets[e] = carry + ex;
+        carry += chunk_total;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        offsets[E] = carry;
+        *n_sel = carry;
+        if ((long long)carry > capacity) atomicMax(status, (int32_t)D2D_ERR_CAPACITY);
+    }
 }
 
-// Exclusive scan of one int per thread over a 1024-thread CTA; returns the exclusive prefix
-// and leaves the CTA total in *total_out (shared).
+// Writes the per-expert token lists.  Position of token t in expert e's list = offsets[e]
+// + tokens of earlier blocks + tokens of earlier warps of this block + tokens of lower lanes,
+// so lists come out in ascending token order.  For each expert bit the lanes that hold it write
+// consecutive entries (a coalesced store).
+__global__ void __launch_bounds__(TOKB)
+bucket_fill_kernel(const uint32_t *__restrict__ mask, int T, int E, int W,
+                   const int32_t *__restrict__ blockbase, const int32_t *__restrict__ offsets,
+                   int32_t *__restrict__ perm, long long capacity)
+{
+    __shared__ int32_t cnt[TOKB / 32][33];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int t = blockIdx.x * TOKB + threadIdx.x;
+    const uint32_t lower = (1u << lane) - 1u;
+    for (int w = 0; w < W; ++w) {
+        const uint32_t word = (t < T) ? __ldg(mask + (size_t)t * W + w) : 0u;
+        cnt[warp][lane] = __popc(transpose_bits(word, lane));
+        __syncthreads();
+        const int e = w * 32 + lane;
+        long long base = 0;                  // start of this warp's run inside expert e's list (lane = expert)
+        if (e < E) {
+            int before = 0;
+            for (int i = 0; i < warp; ++i) before += cnt[i][lane];
+            base = (long long)offsets[e] + blockbase[(size_t)blockIdx.x * E + e] + before;
+        }
+#pragma unroll 4
+        for (int j = 0; j < 32; ++j) {
+            const uint32_t holders = __ballot_sync(FULL, (word >> j) & 1u);
+            const long long bj = __shfl_sync(FULL, base, j);
+            if ((word >> j) & 1u) {
+                const long long idx = bj + __popc(holders & lower);
+                if (idx < capacity) perm[idx] = t;
+            }
+        }
+        __syncthreads();
+    }
+}
+
+// Exclusive scan of one int per thread over a 1024-thread CTA (used by the token-major dual).
 __device__ __forceinline__ int block_exscan_1024(int v, int *warp_sums /*[32]*/, int *total_out)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -182,67 +287,6 @@ __device__ __forceinline__ int block_exscan_1024(int v, int *warp_sums /*[32]*/,
     const int res = warp_sums[warp] + inc - v;
     __syncthreads();
     return res;
-}
-
-__global__ void __launch_bounds__(1024)
-bucket_scan_kernel(int32_t *__restrict__ blockcounts, int nblk, int E,
-                   int32_t *__restrict__ counts, int32_t *__restrict__ offsets, int32_t *__restrict__ n_sel,
-                   int32_t *__restrict__ status, long long capacity)
-{
-    __shared__ int warp_sums[32];
-    __shared__ int chunk_total;
-    int carry = 0;
-    for (int e0 = 0; e0 < E; e0 += 1024) {
-        const int e = e0 + threadIdx.x;
-        int run = 0;
-        if (e < E) {
-            for (int b = 0; b < nblk; ++b) {
-                const int c = blockcounts[(size_t)b * E + e];
-                blockcounts[(size_t)b * E + e] = run;     // exclusive prefix over the token blocks
-                run += c;
-            }
-            counts[e] = run;
-        }
-        const int ex = block_exscan_1024(run, warp_sums, &chunk_total);
-        if (e < E) offsets[e] = carry + ex;
-        carry += chunk_total;
-        __syncthreads();
-    }
-    if (threadIdx.x == 0) {
-        offsets[E] = carry;
-        *n_sel = carry;
-        if ((long long)carry > capacity) atomicMax(status, (int32_t)D2D_ERR_CAPACITY);
-    }
-}
-
-__global__ void __launch_bounds__(TOKB)
-bucket_fill_kernel(const uint32_t *__restrict__ mask, int T, int E, int W,
-                   const int32_t *__restrict__ blockbase, const int32_t *__restrict__ offsets,
-                   int32_t *__restrict__ perm, long long capacity)
-{
-    __shared__ int32_t cnt[32][33];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int t = blockIdx.x * TOKB + threadIdx.x;
-    const int t_warp0 = blockIdx.x * TOKB + warp * 32;
-    for (int w = 0; w < W; ++w) {
-        const uint32_t word = (t < T) ? __ldg(mask + (size_t)t * W + w) : 0u;
-        uint32_t col = transpose_bits(word, lane);
-        cnt[warp][lane] = __popc(col);
-        __syncthreads();
-        const int e = w * 32 + lane;
-        if (e < E && col) {
-            int before = 0;
-            for (int i = 0; i < warp; ++i) before += cnt[i][lane];
-            long long idx = (long long)offsets[e] + blockbase[(size_t)blockIdx.x * E + e] + before;
-            while (col) {
-                const int b = __ffs(col) - 1;
-                col &= col - 1;
-                if (idx < capacity) perm[idx] = t_warp0 + b;
-                ++idx;
-            }
-        }
-        __syncthreads();
-    }
 }
 
 // ---------------------------------------------------------------------------- token-major dual
@@ -286,8 +330,9 @@ tok_fill_kernel(const uint32_t *__restrict__ mask, int T, int W, const int32_t *
 
 size_t d2d_select_ws_bytes(int T, int E)
 {
+    // [ticket counter, padded to 256 bytes | per-block, per-expert counters]
     const size_t nblk = (size_t)d2d_cdiv(T > 0 ? T : 1, TOKB);
-    return d2d_align_up(nblk * (size_t)E * sizeof(int32_t), 256);
+    return 256 + d2d_align_up(nblk * (size_t)E * sizeof(int32_t), 256);
 }
 
 d2d_status d2d_launch_select(const float *R, int T, int E, float tau, int topk, const d2d_routing *out,
@@ -313,13 +358,15 @@ d2d_status d2d_launch_select(const float *R, int T, int E, float tau, int topk, 
         k_from_mask_kernel<<<d2d_cdiv(T, 256), 256, 0, st>>>(out->mask, T, W, out->k);
     }
     const int nblk = d2d_cdiv(T, TOKB);
-    int32_t *blockcounts = (int32_t *)ws;
-    bucket_count_kernel<<<nblk, TOKB, 0, st>>>(out->mask, T, E, W, blockcounts);
-    bucket_scan_kernel<<<1, 1024, 0, st>>>(blockcounts, nblk, E, out->counts, out->offsets, out->n_sel,
-                                           out->status, (long long)out->perm_capacity);
+    unsigned int *ticket = (unsigned int *)ws;                    // must start at zero: cleared on every call
+    int32_t *blockcounts = (int32_t *)((char *)ws + 256);
+    D2D_CUDA_TRY(cudaMemsetAsync(ticket, 0, sizeof(unsigned int), st));
+    bucket_count_scan_kernel<<<nblk, TOKB, 0, st>>>(out->mask, T, E, W, nblk, blockcounts, ticket, out->counts,
+                                                    out->offsets, out->n_sel, out->status,
+                                                    (long long)out->perm_capacity);
     bucket_fill_kernel<<<nblk, TOKB, 0, st>>>(out->mask, T, E, W, blockcounts, out->offsets, out->perm,
                                               (long long)out->perm_capacity);
-    D2D_LAUNCHED(4);
+    D2D_LAUNCHED(3);
     if (out->tok_off && out->tok_exp) {
         D2D_LAUNCHED(2);
         tok_scan_kernel<<<1, 1024, 0, st>>>(out->k, T, out->tok_off);
@@ -341,7 +388,7 @@ d2d_status d2d_launch_select(const float *R, int T, int E, float tau, int topk, 
 // ------------------------------------------------------------------------------------------
 #include <mutex>
 
-#define D2D_STATIC_SCRATCH_INTS (128 * 1024)          /* 512 KiB: ceil(T/1024) * E must not exceed this */
+#define D2D_STATIC_SCRATCH_INTS (128 * 1024)          /* 512 KiB: 64 + ceil(T/256) * E must not exceed this */
 static __device__ __align__(256) int32_t d2d_select_static_scratch[D2D_STATIC_SCRATCH_INTS];
 
 namespace {
@@ -359,8 +406,8 @@ extern "C" D2D_API d2d_status d2d_select_dynk_static(const float *R, int32_t T, 
     if ((out->tok_off == nullptr) != (out->tok_exp == nullptr)) return D2D_ERR_INVALID_ARG;
     if (T > 0 && (!R || (reinterpret_cast<uintptr_t>(R) & 15u))) return D2D_ERR_INVALID_ARG;
     if (!(tau >= 0.0f && tau <= 1.0f)) return D2D_ERR_INVALID_ARG;
-    // the scratch holds one counter per (block of 1024 tokens, expert)
-    const long long need = (long long)d2d_cdiv(T > 0 ? T : 1, TOKB) * (long long)E;
+    // the scratch holds a ticket counter (64 ints reserved) and one counter per (block of 256 tokens, expert)
+    const long long need = 64 + (long long)d2d_cdiv(T > 0 ? T : 1, TOKB) * (long long)E;
     if (need > (long long)D2D_STATIC_SCRATCH_INTS) return D2D_ERR_UNSUPPORTED;
 
     int dev = -1;
@@ -377,7 +424,7 @@ extern "C" D2D_API d2d_status d2d_select_dynk_static(const float *R, int32_t T, 
         }
         scratch = g_scratch_ptr[dev];
     }
-    // nothing in the scratch has to start at zero: the count kernel writes every counter the scan
-    // and fill kernels read, so the previous call's contents are simply overwritten
+    // the ticket counter at the front must start at zero and is cleared by the launch sequence on
+    // every call; the block counters need no clearing (each is written before it is read)
     return d2d_launch_select(R, T, E, tau, 0, out, scratch, (cudaStream_t)stream);
 }

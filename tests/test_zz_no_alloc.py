@@ -40,7 +40,7 @@ def test_static_scratch_selection_matches_regular_entry_point_twice():
 
 def test_static_scratch_limit_is_enforced():
     from paper_2310_04361_b200 import api
-    T, E = 70000, 2048                              # ceil(T/1024) * E = 69 * 2048 > 131072
+    T, E = 70000, 2048                              # 64 + ceil(T/256) * E = 64 + 274 * 2048 > 131072
     R = torch.zeros((8, E), dtype=torch.float32, device="cuda")
     routing = api.Routing(8, E, R.device)
     rc = api._lib.d2d_select_dynk_static(api._ptr(R), T, E, ctypes.c_float(0.5), ctypes.byref(routing.struct),
