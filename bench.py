@@ -45,6 +45,7 @@ def parse_args():
     p.add_argument("--tau", type=float, default=0.3)
     p.add_argument("--sweep", action="store_true", help="also time the workload's whole tau grid")
     p.add_argument("--no-cpu-baseline", action="store_true")
+    p.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a captured CUDA graph")
     return p.parse_args()
 
 
@@ -144,12 +145,15 @@ def time_cpu_oracle(cfg, weights, x, tau, budget_s=12.0):
     oracle_step_fn(cfg, weights, x[:probe], tau)()
     per_tok = (time.perf_counter() - t0) / probe
     n = int(max(probe, min(x.shape[0], budget_s / max(per_tok, 1e-9))))
+    passes = int(max(1, min(1000, budget_s / max(per_tok * n, 1e-9))))
+    step = oracle_step_fn(cfg, weights, x[:n], tau)
     t0 = time.perf_counter()
-    oracle_step_fn(cfg, weights, x[:n], tau)()
+    for _ in range(passes):
+        step()
     dt = time.perf_counter() - t0
-    return {"value": n / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-            "sample": f"first {n} of {x.shape[0]} tokens of the {cfg.name} workload at tau={tau}, one pass "
-                      f"(router+select+metadata+experts), {dt:.2f} s"}
+    return {"value": n * passes / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"first {n} of {x.shape[0]} tokens of the {cfg.name} workload at tau={tau}, {passes} passes "
+                      f"(router+select+metadata+experts each), {dt:.2f} s"}
 
 
 def run_reference(args):
@@ -244,6 +248,23 @@ def run_ours(args):
         barrier()
         return [a.elapsed_time(b) for a, b in evs]       # ms
 
+    def runner(fn):
+        """The step as it is launched in the timed region: a CUDA-graph replay of the library's launch
+        sequence (the layer is launch-latency bound for small batches), or the eager call with --no-graph."""
+        if args.no_graph:
+            return fn
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for _ in range(3):
+                fn()
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            fn()
+        return g.replay
+
     def max_over_ranks(v):
         if world == 1:
             return v
@@ -254,11 +275,14 @@ def run_ours(args):
     def step():
         layer.layer_fwd(x, args.tau, y=y, routing=routing)
 
+    step()                                   # one eager call: counts the kernels a step launches
+    launches0 = api.launch_count()
+    step()
+    launches_per_step = api.launch_count() - launches0
+    run_step = runner(step)
     sampler = ClockSampler(physical_gpu_index(local_rank))
     sampler.start()
-    launches0 = api.launch_count()
-    times = timed_loop(step, args.steps, args.warmup)
-    launches_per_step = (api.launch_count() - launches0) // (args.steps + args.warmup)
+    times = timed_loop(run_step, args.steps, args.warmup)
     clocks = sampler.stop()
     total_ms = max_over_ranks(sum(times))
     value = world * T * args.steps / (total_ms * 1e-3)
@@ -291,17 +315,31 @@ def run_ours(args):
     if rank == 0:
         # ---- per-stage breakdown (same flush protocol), used for the roofline of the dominant kernel
         R = torch.empty((T, cfg.E), dtype=torch.float32, device=dev)
-        t_router = statistics.mean(timed_loop(lambda: layer.router_fwd(x, R=R), args.steps, 3))
-        t_select = statistics.mean(timed_loop(lambda: api.select_dynk(R, args.tau, routing=routing), args.steps, 3))
-        t_ffn = statistics.mean(timed_loop(lambda: layer.moe_ffn_fwd(x, routing, y=y), args.steps, 3))
+        t_router = statistics.mean(timed_loop(runner(lambda: layer.router_fwd(x, R=R)), args.steps, 3))
+        t_select = statistics.mean(timed_loop(runner(lambda: api.select_dynk(R, args.tau, routing=routing)), args.steps, 3))
+        t_ffn = statistics.mean(timed_loop(runner(lambda: layer.moe_ffn_fwd(x, routing, y=y)), args.steps, 3))
         peaks = measured_peaks()
         f_router, f_experts = flops_algorithmic(cfg, T, n_sel)
-        achieved = f_experts / (t_ffn * 1e-3) / 1e12
-        roofline = {"bound": "tensor", "kernel": "moe_ffn_fwd", "achieved": achieved, "peak": peaks["bf16_tflops"],
-                    "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
-                    "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, args.tau)),
-                    "peak_source": f"{peaks['source']} burst bf16 GEMM", "algorithmic_flops_per_launch": f_experts,
-                    "kernel_ms": t_ffn}
+        elem = 2 if cfg.dtype == "bf16" else 4
+        n_used = int((routing.counts > 0).sum().item())
+        if T <= 64:
+            # decode regime: the expert kernel is bound by HBM traffic on the touched expert slices
+            touched = n_used * (cfg.n_mat * cfg.s * cfg.d + cfg.s) * elem + 2 * T * cfg.d * elem + cfg.d * elem
+            achieved = touched / (t_ffn * 1e-3) / 1e9
+            roofline = {"bound": "hbm", "kernel": "moe_ffn_fwd (small_ffn_kernel)", "achieved": achieved,
+                        "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
+                        "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, T, args.tau)),
+                        "peak_source": f"{peaks['source']} HBM copy", "algorithmic_bytes_per_launch": touched,
+                        "experts_touched": n_used, "kernel_ms": t_ffn}
+        else:
+            achieved = f_experts / (t_ffn * 1e-3) / 1e12
+            roofline = {"bound": "tensor", "kernel": "moe_ffn_fwd (gemm_tc_kernel x2)", "achieved": achieved,
+                        "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
+                        "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, T, args.tau)),
+                        "peak_source": f"{peaks['source']} burst bf16 GEMM", "algorithmic_flops_per_launch": f_experts,
+                        "executed_flops_per_launch": 2.0 * cfg.n_mat * T * cfg.d * cfg.d_ff,
+                        "executed_frac": 2.0 * cfg.n_mat * T * cfg.d * cfg.d_ff / (t_ffn * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                        "kernel_ms": t_ffn}
 
         # ---- dense FFN comparator: torch (cuBLASLt) linear -> act -> linear on the same tensors
         tdt = api.torch_dtype(cfg.dtype)
@@ -318,14 +356,14 @@ def run_ours(args):
             h = actf(F.linear(x, wg)) * up if wg is not None else actf(up)
             return F.linear(h, w2, b2)
 
-        t_dense = statistics.mean(timed_loop(dense, args.steps, 3))
+        t_dense = statistics.mean(timed_loop(runner(dense), args.steps, 3))
         t_layer = sum(times) / len(times)
 
         sweep = None
         if args.sweep:
             sweep = []
             for tau in cfg.taus:
-                ts = timed_loop(lambda: layer.layer_fwd(x, tau, y=y, routing=routing), max(10, args.steps // 2), 3)
+                ts = timed_loop(runner(lambda tau=tau: layer.layer_fwd(x, tau, y=y, routing=routing)), max(10, args.steps // 2), 3)
                 torch.cuda.synchronize()
                 sweep.append({"tau": tau, "rho": routing.n_sel / (T * cfg.E), "ms": statistics.mean(ts),
                               "speedup_vs_dense": t_dense / statistics.mean(ts)})
@@ -342,6 +380,7 @@ def run_ours(args):
                        "expert_size": cfg.s, "d_h": cfg.d_h, "act": cfg.act, "gated": cfg.gated, "tau": args.tau,
                        "rho": n_sel / (T * cfg.E), "pruned_flop_fraction": 1 - n_sel / (T * cfg.E),
                        "l2": f"flushed between steps by writing a {L2_FLUSH_BYTES >> 20} MiB buffer (outside the events)",
+                       "launch": "eager" if args.no_graph else "CUDA graph replay of the library's launch sequence",
                        "parallelism": f"token-sharded replicas x{world}, no collective"},
             "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
             "roofline": roofline, "cpu_baseline": cpu, "clocks": clocks,

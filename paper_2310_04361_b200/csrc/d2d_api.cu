@@ -37,7 +37,7 @@ ws_layout layout_for(const d2d_layer *L, int T)
     const size_t Tn = (size_t)(T > 0 ? T : 1);
     size_t off = 0;
     w.u_off = off;
-    off += d2d_align_up(Tn * (size_t)L->desc.d_h * sizeof(float), 256);
+    off += 256 + d2d_align_up(Tn * (size_t)L->desc.d_h * sizeof(float), 256);   // ticket area + hidden activations
     w.r_off = off;
     off += d2d_align_up(Tn * (size_t)L->desc.n_experts * sizeof(float), 256);
     w.sel_off = off;
@@ -52,18 +52,31 @@ ws_layout layout_for(const d2d_layer *L, int T)
 
 // Tokens from which the dense tensor-core path (masked hidden activations, two GEMMs) is used
 // instead of the token-major CUDA-core kernel.
-static const int kDenseMaskedMinTokens = 128;
+static const int kDenseMaskedMinTokens = 17;
 
 static bool use_dense_masked(const d2d_layer *L, int T)
 {
     return L->desc.dtype == D2D_BF16 && T >= kDenseMaskedMinTokens && L->desc.d_ff % 8 == 0 && d2d_gemm_tc_available();
 }
 
+// Up to this many tokens the expert-per-CTA kernel (each kept expert's slice read once) is used.
+static const int kSmallFfnMaxTokens = 16;
+
+static bool use_small_ffn(const d2d_layer *L, int T)
+{
+    return T <= kSmallFfnMaxTokens && d2d_small_ffn_supports(L->desc);
+}
+
 size_t d2d_moe_ffn_ws_bytes(const d2d_layer *L, int T)
 {
+    size_t need = 256;
+    if (use_small_ffn(L, T)) need = d2d_small_ffn_ws_bytes(L, T);
     // hidden activations H [T, d_ff] bf16 of the dense-masked path
-    if (L->desc.dtype != D2D_BF16 || T < kDenseMaskedMinTokens) return 256;
-    return d2d_align_up((size_t)T * L->desc.d_ff * 2, 256);
+    if (L->desc.dtype == D2D_BF16 && T >= kDenseMaskedMinTokens) {
+        const size_t h = d2d_align_up((size_t)T * L->desc.d_ff * 2, 256);
+        if (h > need) need = h;
+    }
+    return need;
 }
 
 // Large batches: every expert is used by some token of a 128-token tile, so the expert FFN runs
@@ -89,10 +102,9 @@ static d2d_status launch_dense_masked(const d2d_layer *L, const void *x, int T, 
 d2d_status d2d_launch_moe_ffn(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y,
                               void *ws, size_t ws_bytes, cudaStream_t st)
 {
-    if (use_dense_masked(L, T)) {
-        if (ws_bytes < d2d_moe_ffn_ws_bytes(L, T)) return D2D_ERR_WORKSPACE;
-        return launch_dense_masked(L, x, T, r, y, ws, st);
-    }
+    if (ws_bytes < d2d_moe_ffn_ws_bytes(L, T)) return D2D_ERR_WORKSPACE;
+    if (use_small_ffn(L, T)) return d2d_small_ffn(L, x, T, r, y, ws, st);
+    if (use_dense_masked(L, T)) return launch_dense_masked(L, x, T, r, y, ws, st);
     return d2d_launch_moe_ffn_token(L, x, T, r, y, st);
 }
 

@@ -47,6 +47,16 @@ d2d_status d2d_launch_moe_ffn(const d2d_layer *L, const void *x, int T, const d2
                               void *ws, size_t ws_bytes, cudaStream_t st);
 size_t d2d_moe_ffn_ws_bytes(const d2d_layer *L, int T);
 
+// small-batch (T <= 64) kernels
+bool d2d_small_select_supports(int T, int E);
+d2d_status d2d_small_select(const float *R, int T, int E, float tau, const d2d_routing *out, cudaStream_t st);
+bool d2d_small_router_supports(const d2d_layer_desc &D, int T);
+size_t d2d_small_router_ws_bytes(const d2d_layer *L, int T);
+d2d_status d2d_small_router(const d2d_layer *L, const void *x, int T, float *R, void *ws, cudaStream_t st);
+bool d2d_small_ffn_supports(const d2d_layer_desc &D);
+size_t d2d_small_ffn_ws_bytes(const d2d_layer *L, int T);
+d2d_status d2d_small_ffn(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y, void *ws, cudaStream_t st);
+
 d2d_status d2d_launch_transpose(const void *src, void *dst, int rows, int cols, size_t elem, cudaStream_t st);
 
 // ---- device helpers ------------------------------------------------------------------------

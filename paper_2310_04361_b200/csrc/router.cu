@@ -80,20 +80,23 @@ d2d_status run_router(const d2d_layer *L, const void *x, int Tn, float *R, float
 d2d_status d2d_launch_router(const d2d_layer *L, const void *x, int T, float *R, float *u_ws, cudaStream_t st)
 {
     if (T == 0) return D2D_OK;
-    if (L->desc.dtype == D2D_F32) return run_router<float>(L, x, T, R, u_ws, st);
-    if (T >= 32 && d2d_gemm_tc_available()) {
+    // u_ws points at [256-byte ticket area | T*d_h floats]
+    float *u = (float *)((char *)u_ws + 256);
+    if (d2d_small_router_supports(L->desc, T)) return d2d_small_router(L, x, T, R, u_ws, st);
+    if (L->desc.dtype == D2D_F32) return run_router<float>(L, x, T, R, u, st);
+    if (d2d_gemm_tc_available()) {
         // bf16 layers: both router layers are dense contractions on the tensor cores; the hidden
         // activations u are kept in bf16 (they are the A operand of the second GEMM)
         const d2d_layer_desc &D = L->desc;
         d2d_gemm_args l1 = {};
-        l1.a = x; l1.b = L->w_r1; l1.bias = L->b_r1; l1.out = u_ws;
+        l1.a = x; l1.b = L->w_r1; l1.bias = L->b_r1; l1.out = u;
         l1.M = T; l1.N = D.d_h; l1.K = D.d; l1.epilogue = D2D_EPI_RELU_BF16;
         d2d_status rc = d2d_gemm_tc(l1, st);
         if (rc != D2D_OK) return rc;
         d2d_gemm_args l2 = {};
-        l2.a = u_ws; l2.b = L->w_r2; l2.bias = L->b_r2; l2.out = R;
+        l2.a = u; l2.b = L->w_r2; l2.bias = L->b_r2; l2.out = R;
         l2.M = T; l2.N = D.n_experts; l2.K = D.d_h; l2.epilogue = D2D_EPI_ABS_F32;
         return d2d_gemm_tc(l2, st);
     }
-    return run_router<__nv_bfloat16>(L, x, T, R, u_ws, st);
+    return run_router<__nv_bfloat16>(L, x, T, R, u, st);
 }

@@ -180,7 +180,8 @@ bucket_count_scan_kernel(const uint32_t *__restrict__ mask, int T, int E, int W,
     __shared__ unsigned int my_ticket;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int t = blockIdx.x * TOKB + threadIdx.x;
-    for (int w = 0; w < W; ++w) {
+    {
+        const int w = blockIdx.y;                // one 32-expert mask word per CTA
         const uint32_t word = (t < T) ? __ldg(mask + (size_t)t * W + w) : 0u;
         cnt[warp][lane] = __popc(transpose_bits(word, lane));
         __syncthreads();
@@ -196,7 +197,7 @@ bucket_count_scan_kernel(const uint32_t *__restrict__ mask, int T, int E, int W,
     __threadfence();
     if (threadIdx.x == 0) my_ticket = atomicAdd(ticket, 1u);
     __syncthreads();
-    if (my_ticket != (unsigned int)(nblk - 1)) return;
+    if (my_ticket != (unsigned int)(nblk * W - 1)) return;
     __threadfence();                         // every other CTA's block counts are visible now
     if (threadIdx.x == 0) *ticket = 0u;      // ready for the next call
     int carry = 0;
@@ -236,17 +237,17 @@ bucket_fill_kernel(const uint32_t *__restrict__ mask, int T, int E, int W,
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int t = blockIdx.x * TOKB + threadIdx.x;
     const uint32_t lower = (1u << lane) - 1u;
-    for (int w = 0; w < W; ++w) {
+    {
+        const int w = blockIdx.y;                // one 32-expert mask word per CTA
+        const int e = w * 32 + lane;
+        // start of this CTA's run inside expert e's list (lane = expert); issued early to hide the latency
+        const long long cta_base = e < E ? (long long)__ldg(offsets + e) + __ldg(blockbase + (size_t)blockIdx.x * E + e) : 0;
         const uint32_t word = (t < T) ? __ldg(mask + (size_t)t * W + w) : 0u;
         cnt[warp][lane] = __popc(transpose_bits(word, lane));
         __syncthreads();
-        const int e = w * 32 + lane;
-        long long base = 0;                  // start of this warp's run inside expert e's list (lane = expert)
-        if (e < E) {
-            int before = 0;
-            for (int i = 0; i < warp; ++i) before += cnt[i][lane];
-            base = (long long)offsets[e] + blockbase[(size_t)blockIdx.x * E + e] + before;
-        }
+        int before = 0;
+        for (int i = 0; i < warp; ++i) before += cnt[i][lane];
+        const long long base = cta_base + before;
 #pragma unroll 4
         for (int j = 0; j < 32; ++j) {
             const uint32_t holders = __ballot_sync(FULL, (word >> j) & 1u);
@@ -256,7 +257,6 @@ bucket_fill_kernel(const uint32_t *__restrict__ mask, int T, int E, int W,
                 if (idx < capacity) perm[idx] = t;
             }
         }
-        __syncthreads();
     }
 }
 
@@ -347,6 +347,7 @@ d2d_status d2d_launch_select(const float *R, int T, int E, float tau, int topk, 
         if (out->tok_off) D2D_CUDA_TRY(cudaMemsetAsync(out->tok_off, 0, sizeof(int32_t), st));
         return D2D_OK;
     }
+    if (topk == 0 && d2d_small_select_supports(T, E)) return d2d_small_select(R, T, E, tau, out, st);
     const int warps_per_cta = 8;
     const int grid_tok = d2d_cdiv(T, warps_per_cta);
     if (R) {
@@ -361,10 +362,10 @@ d2d_status d2d_launch_select(const float *R, int T, int E, float tau, int topk, 
     unsigned int *ticket = (unsigned int *)ws;                    // must start at zero: cleared on every call
     int32_t *blockcounts = (int32_t *)((char *)ws + 256);
     D2D_CUDA_TRY(cudaMemsetAsync(ticket, 0, sizeof(unsigned int), st));
-    bucket_count_scan_kernel<<<nblk, TOKB, 0, st>>>(out->mask, T, E, W, nblk, blockcounts, ticket, out->counts,
+    bucket_count_scan_kernel<<<dim3(nblk, W), TOKB, 0, st>>>(out->mask, T, E, W, nblk, blockcounts, ticket, out->counts,
                                                     out->offsets, out->n_sel, out->status,
                                                     (long long)out->perm_capacity);
-    bucket_fill_kernel<<<nblk, TOKB, 0, st>>>(out->mask, T, E, W, blockcounts, out->offsets, out->perm,
+    bucket_fill_kernel<<<dim3(nblk, W), TOKB, 0, st>>>(out->mask, T, E, W, blockcounts, out->offsets, out->perm,
                                               (long long)out->perm_capacity);
     D2D_LAUNCHED(3);
     if (out->tok_off && out->tok_exp) {

@@ -1,0 +1,383 @@
+// Small-batch (decode) router and expert kernels: T <= 64 tokens, bound by HBM traffic and latency.
+//
+// Both kernels bring every weight byte they need into shared memory with 16-byte cp.async copies
+// that are all issued before the first use (maximum memory-level parallelism: the copies of a CTA
+// are in flight together instead of one cache line at a time), then compute from shared memory.
+//
+//   small_router_kernel   CTA b owns 8 hidden units: its 8 rows of W_r1 and all token rows go to
+//                         shared memory, one warp per unit forms u[t, j]; every CTA also prefetches
+//                         W_r2, and the CTA that finishes last (ticket) computes layer 2 from it
+//   small_ffn_kernel      one CTA per expert: its W1 / W_gate / W2 slices are read from HBM exactly
+//                         once (only experts some token kept do any work), the expert's tokens are
+//                         handled 8 at a time, partial output rows go to a float32 accumulator with
+//                         16-byte vector reductions; the last CTA adds b2 and writes y
+#include "d2d_common.cuh"
+
+namespace {
+
+constexpr int TBLK = 8;            // tokens processed together
+constexpr int NT = 256;
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void cp_async16(void *dst_smem, const void *src_gmem)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_addr(dst_smem)), "l"(src_gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// Copies `bytes` (multiple of 16, both sides 16-byte aligned) with every thread of the CTA.
+__device__ __forceinline__ void cta_copy_async(void *dst_smem, const void *src_gmem, size_t bytes)
+{
+    for (size_t off = (size_t)threadIdx.x * 16; off < bytes; off += (size_t)NT * 16)
+        cp_async16((char *)dst_smem + off, (const char *)src_gmem + off);
+}
+
+// 8 consecutive elements from shared memory as floats
+__device__ __forceinline__ void lds8(const float *p, float (&o)[8])
+{
+    const float4 a = *reinterpret_cast<const float4 *>(p), b = *(reinterpret_cast<const float4 *>(p) + 1);
+    o[0] = a.x; o[1] = a.y; o[2] = a.z; o[3] = a.w; o[4] = b.x; o[5] = b.y; o[6] = b.z; o[7] = b.w;
+}
+__device__ __forceinline__ void lds8(const __nv_bfloat16 *p, float (&o)[8])
+{
+    const uint4 raw = *reinterpret_cast<const uint4 *>(p);
+    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        o[2 * i] = __uint_as_float(w[i] << 16);
+        o[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+}
+
+// One warp: dot products of a weight row with up to TBLK token rows, all operands in shared memory.
+template <typename TT>
+__device__ __forceinline__ void warp_row_dots(const TT *wrow, const TT *xs, int d, int lane, float (&acc)[TBLK])
+{
+#pragma unroll
+    for (int i = 0; i < TBLK; ++i) acc[i] = 0.0f;
+    for (int c = lane * 8; c < d; c += 256) {
+        float wv[8];
+        lds8(wrow + c, wv);
+#pragma unroll
+        for (int i = 0; i < TBLK; ++i) {
+            float xv[8];
+            lds8(xs + (size_t)i * d + c, xv);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) acc[i] = fmaf(wv[q], xv[q], acc[i]);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < TBLK; ++i) acc[i] = d2d_warp_sum(acc[i]);
+}
+
+// ------------------------------------------------------------------------------------ router
+
+// dynamic shared memory: [ W_r1 rows of this CTA: 8*d | token block: TBLK*d | W_r2: E*d_h (if staged) | u: T*d_h floats ]
+template <typename TT>
+__global__ void __launch_bounds__(NT)
+small_router_kernel(const TT *__restrict__ x, int T, int d, const TT *__restrict__ w_r1, const TT *__restrict__ b_r1,
+                    int d_h, const TT *__restrict__ w_r2, const TT *__restrict__ b_r2, int E, int stage_w2,
+                    float *__restrict__ u, float *__restrict__ R, unsigned int *__restrict__ ticket)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    TT *w1s = reinterpret_cast<TT *>(smem_raw);
+    TT *xs = w1s + (size_t)8 * d;
+    TT *w2s = xs + (size_t)TBLK * d;
+    float *us = reinterpret_cast<float *>(w2s + (stage_w2 ? (size_t)E * d_h : 0));
+    __shared__ unsigned int my_ticket;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int j0 = blockIdx.x * 8;
+    const int rows = d_h - j0 < 8 ? d_h - j0 : 8;
+
+    cta_copy_async(w1s, w_r1 + (size_t)j0 * d, (size_t)rows * d * sizeof(TT));
+    cp_async_commit();
+    if (stage_w2) cta_copy_async(w2s, w_r2, (size_t)E * d_h * sizeof(TT));     // needed only by the last CTA; prefetched by all
+    cp_async_commit();
+
+    for (int t0 = 0; t0 < T; t0 += TBLK) {
+        const int ntok = T - t0 < TBLK ? T - t0 : TBLK;
+        __syncthreads();                                          // previous block's readers of xs are done
+        cta_copy_async(xs, x + (size_t)t0 * d, (size_t)ntok * d * sizeof(TT));
+        if (ntok < TBLK)                                          // unused token slots read zeros
+            for (int i = threadIdx.x; i < (TBLK - ntok) * d; i += NT) xs[(size_t)ntok * d + i] = d2d_from_float<TT>(0.0f);
+        cp_async_commit();
+        cp_async_wait<0>();                                       // everything issued so far has landed
+        __syncthreads();
+        if (warp < rows) {
+            float acc[TBLK];
+            warp_row_dots<TT>(w1s + (size_t)warp * d, xs, d, lane, acc);
+            if (lane == 0) {
+                const float bj = b_r1 ? d2d_to_float<TT>(b_r1[j0 + warp]) : 0.0f;
+#pragma unroll
+                for (int i = 0; i < TBLK; ++i)
+                    if (i < ntok) u[(size_t)(t0 + i) * d_h + j0 + warp] = fmaxf(acc[i] + bj, 0.0f);
+            }
+        }
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) my_ticket = atomicAdd(ticket, 1u);
+    __syncthreads();
+    if (my_ticket != gridDim.x - 1) {
+        cp_async_wait<0>();                                       // no copy may be in flight when the CTA exits
+        return;
+    }
+    __threadfence();
+    if (threadIdx.x == 0) *ticket = 0u;
+    // ---- layer 2 by the last CTA: a thread owns an expert, keeps TBLK accumulators, walks its W_r2 row
+    for (int i = threadIdx.x; i < T * d_h; i += NT) us[i] = __ldcg(u + i);
+    cp_async_wait<0>();
+    __syncthreads();
+    for (int i = threadIdx.x; i < E; i += NT) {
+        const float bi = b_r2 ? d2d_to_float<TT>(b_r2[i]) : 0.0f;
+        for (int t0 = 0; t0 < T; t0 += TBLK) {
+            float acc[TBLK];
+#pragma unroll
+            for (int q = 0; q < TBLK; ++q) acc[q] = 0.0f;
+            for (int c = 0; c < d_h; c += 8) {
+                float wv[8];
+                if (stage_w2) lds8(w2s + (size_t)i * d_h + c, wv);
+                else d2d_load8(w_r2 + (size_t)i * d_h + c, wv);
+#pragma unroll
+                for (int q = 0; q < TBLK; ++q) {
+                    const float *ur = us + (size_t)(t0 + q < T ? t0 + q : t0) * d_h + c;
+#pragma unroll
+                    for (int z = 0; z < 8; ++z) acc[q] = fmaf(wv[z], ur[z], acc[q]);
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < TBLK; ++q)
+                if (t0 + q < T) R[(size_t)(t0 + q) * E + i] = fabsf(acc[q] + bi);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------ expert FFN
+
+__device__ __forceinline__ void red_add_v4(float *addr, float a, float b, float c, float d)
+{
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+
+// dynamic shared memory: [ W1 rows: rc*d | W_gate rows: rc*d (gated) | W2T rows: rc*d | token block: TBLK*d | h: TBLK*rc floats ]
+// rc = neurons handled per pass (the whole expert when its slices fit).
+template <typename TT, int ACT, bool GATED>
+__global__ void __launch_bounds__(NT)
+small_ffn_kernel(const TT *__restrict__ x, int T, int d, int s, int rc, const TT *__restrict__ w1,
+                 const TT *__restrict__ b1, const TT *__restrict__ w_gate, const TT *__restrict__ w2t,
+                 const TT *__restrict__ b2, const int32_t *__restrict__ offsets, const int32_t *__restrict__ perm,
+                 float *__restrict__ y32, unsigned int *__restrict__ ticket, TT *__restrict__ y)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    TT *w1s = reinterpret_cast<TT *>(smem_raw);
+    TT *wgs = w1s + (size_t)rc * d;
+    TT *w2s = wgs + (GATED ? (size_t)rc * d : 0);
+    TT *xs = w2s + (size_t)rc * d;
+    float *hs = reinterpret_cast<float *>(xs + (size_t)TBLK * d);
+    __shared__ unsigned int my_ticket;
+    __shared__ int stok[TBLK];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int e = blockIdx.x;
+    const int beg = offsets[e], end = offsets[e + 1];
+
+    if (beg < end) {
+        for (int r0 = 0; r0 < s; r0 += rc) {
+            const int rows = s - r0 < rc ? s - r0 : rc;
+            const size_t n0 = (size_t)e * s + r0;
+            __syncthreads();                                      // readers of the previous pass are done
+            cta_copy_async(w1s, w1 + n0 * d, (size_t)rows * d * sizeof(TT));
+            if (GATED) cta_copy_async(wgs, w_gate + n0 * d, (size_t)rows * d * sizeof(TT));
+            cta_copy_async(w2s, w2t + n0 * d, (size_t)rows * d * sizeof(TT));
+            cp_async_commit();
+            for (int p0 = beg; p0 < end; p0 += TBLK) {
+                const int ntok = end - p0 < TBLK ? end - p0 : TBLK;
+                __syncthreads();                                  // previous token block fully consumed
+                if (threadIdx.x < TBLK) stok[threadIdx.x] = perm[p0 + (threadIdx.x < ntok ? threadIdx.x : 0)];
+                __syncthreads();
+                for (int i = 0; i < ntok; ++i) cta_copy_async(xs + (size_t)i * d, x + (size_t)stok[i] * d, (size_t)d * sizeof(TT));
+                if (ntok < TBLK)
+                    for (int i = threadIdx.x; i < (TBLK - ntok) * d; i += NT) xs[(size_t)ntok * d + i] = d2d_from_float<TT>(0.0f);
+                cp_async_commit();
+                cp_async_wait<0>();
+                __syncthreads();
+                // ---- up projection + activation: one warp per neuron
+                for (int nl = warp; nl < rows; nl += NT / 32) {
+                    float up[TBLK], gate[TBLK];
+                    warp_row_dots<TT>(w1s + (size_t)nl * d, xs, d, lane, up);
+                    if (GATED) warp_row_dots<TT>(wgs + (size_t)nl * d, xs, d, lane, gate);
+                    if (lane == 0) {
+                        const float bn = b1 ? d2d_to_float<TT>(b1[n0 + nl]) : 0.0f;
+#pragma unroll
+                        for (int i = 0; i < TBLK; ++i) {
+                            const float z = up[i] + bn;
+                            hs[i * rc + nl] = GATED ? d2d_activate<ACT>(gate[i]) * z : d2d_activate<ACT>(z);
+                        }
+                    }
+                }
+                __syncthreads();
+                // ---- down projection: a thread owns 4 adjacent output columns
+                for (int c = threadIdx.x * 4; c < d; c += NT * 4) {
+                    float acc[TBLK][4];
+#pragma unroll
+                    for (int i = 0; i < TBLK; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.0f;
+                    for (int nl = 0; nl < rows; ++nl) {
+                        const TT *wp = w2s + (size_t)nl * d + c;
+                        float w0, w1v, w2v, w3;
+                        if (sizeof(TT) == 2) {
+                            const uint2 raw = *reinterpret_cast<const uint2 *>(wp);
+                            w0 = __uint_as_float(raw.x << 16); w1v = __uint_as_float(raw.x & 0xffff0000u);
+                            w2v = __uint_as_float(raw.y << 16); w3 = __uint_as_float(raw.y & 0xffff0000u);
+                        } else {
+                            const float4 raw = *reinterpret_cast<const float4 *>(wp);
+                            w0 = raw.x; w1v = raw.y; w2v = raw.z; w3 = raw.w;
+                        }
+#pragma unroll
+                        for (int i = 0; i < TBLK; ++i) {
+                            const float h = hs[i * rc + nl];
+                            acc[i][0] = fmaf(h, w0, acc[i][0]);
+                            acc[i][1] = fmaf(h, w1v, acc[i][1]);
+                            acc[i][2] = fmaf(h, w2v, acc[i][2]);
+                            acc[i][3] = fmaf(h, w3, acc[i][3]);
+                        }
+                    }
+#pragma unroll
+                    for (int i = 0; i < TBLK; ++i)
+                        if (i < ntok) red_add_v4(y32 + (size_t)stok[i] * d + c, acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+                }
+            }
+        }
+    }
+    // ---- the CTA that finishes last converts the float32 accumulator (+ b2) to the output dtype
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) my_ticket = atomicAdd(ticket, 1u);
+    __syncthreads();
+    if (my_ticket != gridDim.x - 1) return;
+    __threadfence();
+    if (threadIdx.x == 0) *ticket = 0u;
+    const size_t total = (size_t)T * d;
+    for (size_t i = (size_t)threadIdx.x * 4; i < total; i += (size_t)NT * 4) {
+        const float4 v = __ldcg(reinterpret_cast<const float4 *>(y32 + i));
+        const int c = (int)(i % d);
+        float o[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) y[i + q] = d2d_from_float<TT>(o[q] + (b2 ? d2d_to_float<TT>(b2[c + q]) : 0.0f));
+    }
+}
+
+constexpr size_t kSmemLimit = 200 * 1024;
+
+// neurons per pass so that the slices, one token block and the hidden values fit in shared memory
+int rows_per_pass(const d2d_layer_desc &D, size_t elem)
+{
+    const size_t n_mat = D.gated ? 3 : 2;
+    const size_t fixed = (size_t)TBLK * D.d * elem;
+    for (int rc = D.expert_size; rc >= 1; rc = (rc + 1) / 2) {
+        const size_t need = n_mat * rc * D.d * elem + fixed + (size_t)TBLK * rc * 4;
+        if (need <= kSmemLimit) return rc;
+        if (rc == 1) break;
+    }
+    return 0;
+}
+
+template <typename TT, int ACT, bool GATED>
+d2d_status launch_ffn(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y, float *y32,
+                      unsigned int *ticket, cudaStream_t st)
+{
+    const d2d_layer_desc &D = L->desc;
+    const int rc = rows_per_pass(D, sizeof(TT));
+    if (rc <= 0) return D2D_ERR_UNSUPPORTED;
+    const size_t smem = (size_t)(GATED ? 3 : 2) * rc * D.d * sizeof(TT) + (size_t)TBLK * D.d * sizeof(TT) + (size_t)TBLK * rc * 4;
+    auto kern = small_ffn_kernel<TT, ACT, GATED>;
+    static size_t attr_smem = 0;
+    if (smem > attr_smem) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess) return D2D_ERR_CUDA;
+        attr_smem = kSmemLimit;
+    }
+    kern<<<D.n_experts, NT, smem, st>>>((const TT *)x, T, D.d, D.expert_size, rc, (const TT *)L->w1, (const TT *)L->b1,
+                                        (const TT *)L->w_gate, (const TT *)L->w2t, (const TT *)L->b2, r->offsets, r->perm,
+                                        y32, ticket, (TT *)y);
+    D2D_LAUNCHED(1);
+    return cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
+}
+
+template <typename TT, int ACT>
+d2d_status launch_ffn_gated(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y, float *y32,
+                            unsigned int *ticket, cudaStream_t st)
+{
+    if (L->desc.gated) return launch_ffn<TT, ACT, true>(L, x, T, r, y, y32, ticket, st);
+    return launch_ffn<TT, ACT, false>(L, x, T, r, y, y32, ticket, st);
+}
+
+template <typename TT>
+d2d_status launch_ffn_dtype(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y, float *y32,
+                            unsigned int *ticket, cudaStream_t st)
+{
+    switch (L->desc.act) {
+    case D2D_ACT_RELU: return launch_ffn_gated<TT, D2D_ACT_RELU>(L, x, T, r, y, y32, ticket, st);
+    case D2D_ACT_GELU_ERF: return launch_ffn_gated<TT, D2D_ACT_GELU_ERF>(L, x, T, r, y, y32, ticket, st);
+    case D2D_ACT_GELU_TANH: return launch_ffn_gated<TT, D2D_ACT_GELU_TANH>(L, x, T, r, y, y32, ticket, st);
+    default: return launch_ffn_gated<TT, D2D_ACT_SILU>(L, x, T, r, y, y32, ticket, st);
+    }
+}
+
+template <typename TT>
+d2d_status launch_router(const d2d_layer *L, const void *x, int T, float *R, float *u, unsigned int *ticket, cudaStream_t st)
+{
+    const d2d_layer_desc &D = L->desc;
+    const size_t base = (size_t)(8 + TBLK) * D.d * sizeof(TT) + (size_t)T * D.d_h * 4;
+    const size_t w2_bytes = (size_t)D.n_experts * D.d_h * sizeof(TT);
+    const int stage_w2 = base + w2_bytes <= kSmemLimit ? 1 : 0;
+    const size_t smem = base + (stage_w2 ? w2_bytes : 0);
+    auto kern = small_router_kernel<TT>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess) return D2D_ERR_CUDA;
+        attr_set = true;
+    }
+    kern<<<d2d_cdiv(D.d_h, 8), NT, smem, st>>>((const TT *)x, T, D.d, (const TT *)L->w_r1, (const TT *)L->b_r1, D.d_h,
+                                                (const TT *)L->w_r2, (const TT *)L->b_r2, D.n_experts, stage_w2, u, R, ticket);
+    D2D_LAUNCHED(1);
+    return cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
+}
+
+}  // namespace
+
+// ws: [ticket (256 bytes) | u: T*d_h floats]
+size_t d2d_small_router_ws_bytes(const d2d_layer *L, int T) { return 256 + d2d_align_up((size_t)T * L->desc.d_h * 4, 256); }
+
+bool d2d_small_router_supports(const d2d_layer_desc &D, int T)
+{
+    const size_t elem = D.dtype == D2D_F32 ? 4 : 2;
+    return T >= 1 && T <= 8 && D.d % 8 == 0 && D.d_h % 8 == 0 &&
+           (size_t)(8 + TBLK) * D.d * elem + (size_t)T * D.d_h * 4 <= kSmemLimit;
+}
+
+d2d_status d2d_small_router(const d2d_layer *L, const void *x, int T, float *R, void *ws, cudaStream_t st)
+{
+    unsigned int *ticket = (unsigned int *)ws;
+    float *u = (float *)((char *)ws + 256);
+    D2D_CUDA_TRY(cudaMemsetAsync(ticket, 0, sizeof(unsigned int), st));
+    if (L->desc.dtype == D2D_F32) return launch_router<float>(L, x, T, R, u, ticket, st);
+    return launch_router<__nv_bfloat16>(L, x, T, R, u, ticket, st);
+}
+
+// ws: [ticket (256 bytes) | y32: T*d floats]
+size_t d2d_small_ffn_ws_bytes(const d2d_layer *L, int T) { return 256 + d2d_align_up((size_t)T * L->desc.d * 4, 256); }
+
+bool d2d_small_ffn_supports(const d2d_layer_desc &D)
+{
+    return D.d % 8 == 0 && rows_per_pass(D, D.dtype == D2D_F32 ? 4 : 2) > 0;
+}
+
+d2d_status d2d_small_ffn(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y, void *ws, cudaStream_t st)
+{
+    unsigned int *ticket = (unsigned int *)ws;
+    float *y32 = (float *)((char *)ws + 256);
+    // the ticket and the float32 accumulator must start at zero
+    D2D_CUDA_TRY(cudaMemsetAsync(ws, 0, 256 + (size_t)T * L->desc.d * 4, st));
+    if (L->desc.dtype == D2D_F32) return launch_ffn_dtype<float>(L, x, T, r, y, y32, ticket, st);
+    return launch_ffn_dtype<__nv_bfloat16>(L, x, T, r, y, y32, ticket, st);
+}
