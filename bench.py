@@ -31,7 +31,10 @@ L2_FLUSH_BYTES = 256 << 20
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (None until a capture of that kernel/workload exists).
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    ("bert", 4096): 11.13e6,        # up projection: profiles/bert_gemm_up_down_full.md
+    ("gpt2_ffn", 1, 0.2): 9.884e6,  # decode expert kernel: profiles/gpt2_decode_T1_small_ffn_full.md
+}
 
 
 def parse_args():
@@ -62,7 +65,7 @@ def measured_peaks():
 class ClockSampler(threading.Thread):
     """Polls SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
 
-    def __init__(self, index: int, period_s: float = 0.02):
+    def __init__(self, index: int, period_s: float = 0.001):
         super().__init__(daemon=True)
         self.index, self.period = index, period_s
         self.samples, self.reasons, self.max_mhz = [], set(), None
@@ -332,14 +335,22 @@ def run_ours(args):
                         "peak_source": f"{peaks['source']} HBM copy", "algorithmic_bytes_per_launch": touched,
                         "experts_touched": n_used, "kernel_ms": t_ffn}
         else:
-            achieved = f_experts / (t_ffn * 1e-3) / 1e12
-            roofline = {"bound": "tensor", "kernel": "moe_ffn_fwd (gemm_tc_kernel x2)", "achieved": achieved,
+            # dominant kernel = the expert up projection (one launch of gemm_tc_kernel with the masked
+            # activation epilogue); its algorithmic work is the up half of the kept pairs' FLOP
+            H = torch.empty((T, cfg.d_ff), dtype=torch.bfloat16, device=dev)
+            t_up = statistics.mean(timed_loop(runner(lambda: layer.expert_up_fwd(x, routing, H=H)), args.steps, 3))
+            t_down = statistics.mean(timed_loop(runner(lambda: layer.expert_down_fwd(H, y=y)), args.steps, 3))
+            f_up = 2.0 * (cfg.n_mat - 1) * cfg.d * cfg.s * n_sel
+            f_up_exec = 2.0 * (cfg.n_mat - 1) * T * cfg.d * cfg.d_ff
+            achieved = f_up / (t_up * 1e-3) / 1e12
+            roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel<UP_MASKED> (d2d_expert_up_fwd)", "achieved": achieved,
                         "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
-                        "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, T, args.tau)),
-                        "peak_source": f"{peaks['source']} burst bf16 GEMM", "algorithmic_flops_per_launch": f_experts,
-                        "executed_flops_per_launch": 2.0 * cfg.n_mat * T * cfg.d * cfg.d_ff,
-                        "executed_frac": 2.0 * cfg.n_mat * T * cfg.d * cfg.d_ff / (t_ffn * 1e-3) / 1e12 / peaks["bf16_tflops"],
-                        "kernel_ms": t_ffn}
+                        "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, T)),
+                        "peak_source": f"{peaks['source']} burst bf16 GEMM", "algorithmic_flops_per_launch": f_up,
+                        "executed_flops_per_launch": f_up_exec,
+                        "executed_frac": f_up_exec / (t_up * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                        "kernel_ms": t_up, "down_kernel_ms": t_down,
+                        "expert_step_frac": f_experts / (t_ffn * 1e-3) / 1e12 / peaks["bf16_tflops"]}
 
         # ---- dense FFN comparator: torch (cuBLASLt) linear -> act -> linear on the same tensors
         tdt = api.torch_dtype(cfg.dtype)

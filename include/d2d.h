@@ -207,6 +207,22 @@ D2D_API d2d_status d2d_select_dynk_static(const float *R, int32_t T, int32_t E, 
 D2D_API d2d_status d2d_moe_ffn_fwd(const d2d_layer *layer, const void *x, int32_t T, const d2d_routing *routing,
                            void *y, void *ws, size_t ws_bytes, void *stream);
 
+/* The two halves of the tensor-core expert step, exposed so that each can be
+ * called, checked and timed on its own (bf16 layers only; other layers return
+ * D2D_ERR_UNSUPPORTED).
+ * d2d_expert_up_fwd (Sec. 3.2; gated form App. G):
+ *   H[t, n] = G[t, n / s] ? A(W1[n,:] x_t + b1[n]) : 0        (gated: A(W_gate x)_n * (W1 x + b1)_n)
+ * for every neuron n of the original FFN: the expert up projections of all
+ * kept (token, expert) pairs as one dense contraction with the selection
+ * applied as a mask.  x: device [T, d]; H: device [T, d_ff] bf16 (caller's).
+ * d2d_expert_down_fwd (Sec. 3.2, 3.4): y = H W2^T + b2, which is
+ * b2 + sum over kept experts of W2[:, blk] h_blk.  y: device [T, d] bf16;
+ * status: device status word (receives D2D_ERR_TIMEOUT), may be NULL. */
+D2D_API d2d_status d2d_expert_up_fwd(const d2d_layer *layer, const void *x, int32_t T, const d2d_routing *routing,
+                                     void *H, void *stream);
+D2D_API d2d_status d2d_expert_down_fwd(const d2d_layer *layer, const void *H, int32_t T, void *y, int32_t *status,
+                                       void *stream);
+
 /* The whole layer on one stream with no host synchronisation in between:
  * router_fwd -> select_dynk -> moe_ffn_fwd.  R_out: optional device [T,E]
  * float32 copy of the router scores (NULL to keep them in the workspace only).

@@ -28,7 +28,7 @@ D2D_F32, D2D_BF16 = 0, 1
 ACTS = {"relu": 0, "gelu_erf": 1, "gelu_tanh": 2, "silu": 3}
 EXPORTS = ["d2d_status_str", "d2d_launch_count", "d2d_layer_create", "d2d_layer_destroy", "d2d_workspace_bytes",
            "d2d_select_workspace_bytes", "d2d_router_fwd", "d2d_select_dynk", "d2d_select_dynk_static", "d2d_select_topk",
-           "d2d_routing_from_mask", "d2d_moe_ffn_fwd", "d2d_layer_fwd", "d2d_layer_fwd_host_workspace_bytes",
+           "d2d_routing_from_mask", "d2d_moe_ffn_fwd", "d2d_expert_up_fwd", "d2d_expert_down_fwd", "d2d_layer_fwd", "d2d_layer_fwd_host_workspace_bytes",
            "d2d_layer_fwd_host"]
 
 
@@ -63,6 +63,8 @@ _lib.d2d_select_dynk_static.argtypes = [c_void_p, c_int32, c_int32, c_float, POI
 _lib.d2d_select_topk.argtypes = [c_void_p, c_int32, c_int32, c_int32, POINTER(RoutingStruct), c_void_p, c_size_t, c_void_p]
 _lib.d2d_routing_from_mask.argtypes = [c_int32, c_int32, POINTER(RoutingStruct), c_void_p, c_size_t, c_void_p]
 _lib.d2d_moe_ffn_fwd.argtypes = [c_void_p, c_void_p, c_int32, POINTER(RoutingStruct), c_void_p, c_void_p, c_size_t, c_void_p]
+_lib.d2d_expert_up_fwd.argtypes = [c_void_p, c_void_p, c_int32, POINTER(RoutingStruct), c_void_p, c_void_p]
+_lib.d2d_expert_down_fwd.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p]
 _lib.d2d_layer_fwd.argtypes = [c_void_p, c_void_p, c_int32, c_float, c_void_p, c_void_p, POINTER(RoutingStruct),
                                c_void_p, c_size_t, c_void_p]
 _lib.d2d_layer_fwd_host_workspace_bytes.restype = c_size_t
@@ -206,6 +208,23 @@ class Layer:
         ws = self.workspace(T)
         _check(_lib.d2d_moe_ffn_fwd(self.handle, _ptr(x), T, ctypes.byref(routing.struct), _ptr(y), _ptr(ws),
                                     ws.numel(), _stream(stream)), "d2d_moe_ffn_fwd")
+        return y
+
+    def expert_up_fwd(self, x, routing: Routing, H=None, stream=None):
+        """H = mask * A(x W1^T + b1), bf16 [T, d_ff] (the tensor-core up projection on its own)."""
+        T = x.shape[0]
+        if H is None:
+            H = torch.empty((T, self.d_ff), dtype=torch.bfloat16, device=self.device)
+        _check(_lib.d2d_expert_up_fwd(self.handle, _ptr(x), T, ctypes.byref(routing.struct), _ptr(H), _stream(stream)),
+               "d2d_expert_up_fwd")
+        return H
+
+    def expert_down_fwd(self, H, y=None, stream=None):
+        """y = H W2^T + b2, bf16 [T, d] (the tensor-core down projection on its own)."""
+        T = H.shape[0]
+        if y is None:
+            y = torch.empty((T, self.d), dtype=torch.bfloat16, device=self.device)
+        _check(_lib.d2d_expert_down_fwd(self.handle, _ptr(H), T, _ptr(y), None, _stream(stream)), "d2d_expert_down_fwd")
         return y
 
     def layer_fwd(self, x, tau: float, y=None, routing: Routing | None = None, R_out=None, stream=None):

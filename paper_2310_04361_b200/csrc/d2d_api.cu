@@ -267,6 +267,35 @@ d2d_status d2d_moe_ffn_fwd(const d2d_layer *layer, const void *x, int32_t T, con
                               (cudaStream_t)stream);
 }
 
+d2d_status d2d_expert_up_fwd(const d2d_layer *layer, const void *x, int32_t T, const d2d_routing *routing,
+                             void *H, void *stream)
+{
+    if (!layer || T < 0) return D2D_ERR_INVALID_ARG;
+    if (T == 0) return D2D_OK;
+    if (!x || !H || !aligned16(x) || !aligned16(H) || !routing_ok(routing, false)) return D2D_ERR_INVALID_ARG;
+    if (layer->desc.dtype != D2D_BF16 || layer->desc.d_ff % 8 || !d2d_gemm_tc_available()) return D2D_ERR_UNSUPPORTED;
+    const d2d_layer_desc &D = layer->desc;
+    d2d_gemm_args up = {};
+    up.a = x; up.b = layer->w1; up.b_gate = D.gated ? layer->w_gate : nullptr; up.bias = layer->b1; up.out = H;
+    up.M = T; up.N = D.d_ff; up.K = D.d; up.epilogue = D2D_EPI_UP_MASKED; up.act = D.act;
+    up.mask = routing->mask; up.mask_words = (D.n_experts + 31) / 32; up.expert_size = D.expert_size;
+    up.status = routing->status;
+    return d2d_gemm_tc(up, (cudaStream_t)stream);
+}
+
+d2d_status d2d_expert_down_fwd(const d2d_layer *layer, const void *H, int32_t T, void *y, int32_t *status, void *stream)
+{
+    if (!layer || T < 0) return D2D_ERR_INVALID_ARG;
+    if (T == 0) return D2D_OK;
+    if (!H || !y || !aligned16(H) || !aligned16(y)) return D2D_ERR_INVALID_ARG;
+    if (layer->desc.dtype != D2D_BF16 || layer->desc.d_ff % 8 || !d2d_gemm_tc_available()) return D2D_ERR_UNSUPPORTED;
+    const d2d_layer_desc &D = layer->desc;
+    d2d_gemm_args dn = {};
+    dn.a = H; dn.b = layer->w2; dn.bias = layer->b2; dn.out = y;
+    dn.M = T; dn.N = D.d; dn.K = D.d_ff; dn.epilogue = D2D_EPI_BIAS_BF16; dn.status = status;
+    return d2d_gemm_tc(dn, (cudaStream_t)stream);
+}
+
 d2d_status d2d_layer_fwd(const d2d_layer *layer, const void *x, int32_t T, float tau, void *y,
                          float *R_out, d2d_routing *routing, void *ws, size_t ws_bytes, void *stream)
 {

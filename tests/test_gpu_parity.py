@@ -321,6 +321,24 @@ def test_layer_fwd_host_buffers(api):
     assert torch.equal(yh, y_dev.cpu())
 
 
+@pytest.mark.parametrize("name,T,tau", [("bert", 333, 0.3), ("llama", 150, 0.4)])
+def test_expert_up_then_down_matches_oracle(api, name, T, tau):
+    """The two halves of the tensor-core expert step, called on their own: H is zero exactly where the token
+    did not keep the expert, and down(up(x)) is the oracle's y on the same routing."""
+    cfg, w, x, layer = _setup(api, name, T)
+    R = oracle.router(x, w["w_r1"], w["b_r1"], w["w_r2"], w["b_r2"])
+    G, _, _ = oracle.select(R, tau)
+    r = api.routing_from_mask(torch.from_numpy(oracle.pack_mask(G).view(np.int32)).cuda(), cfg.E)
+    xd = api.to_device(x, cfg.dtype)
+    H = layer.expert_up_fwd(xd, r)
+    y = layer.expert_down_fwd(H).float().cpu().numpy()
+    Hn = H.float().cpu().numpy().reshape(T, cfg.E, cfg.s)
+    assert not Hn[G == 0].any()
+    assert np.abs(Hn[G == 1]).max() > 0
+    y_ref = oracle.moe_ffn(x, w["w1"], w["b1"], w["w_gate"], w["w2"], w["b2"], oracle.ACT_BY_NAME[cfg.act], G)
+    assert _rel_err(y, y_ref) <= TOL_Y[cfg.dtype]
+
+
 # ------------------------------------------------------------------------------------ argument errors
 
 def test_argument_errors(api):
