@@ -4,7 +4,7 @@
 //            swizzled, into a ring of shared-memory stages guarded by full/empty mbarriers
 //   warp 1   allocates TMEM and issues tcgen05.mma (one thread), fp32 accumulators in TMEM
 //            (two buffers); tcgen05.commit releases a stage when the MMAs that read it have retired
-//   warps 2-9  epilogue: tcgen05.ld the accumulator (one row per thread), bias / activation /
+//   warps 2-17 epilogue: tcgen05.ld the accumulator (one row per thread), bias / activation /
 //            selection mask, vectorised stores; runs while the next tile's MMAs fill the other buffer
 // The kernel is persistent: one CTA per SM walks over the output tiles.
 //
@@ -12,6 +12,8 @@
 // status word and leaves its loop, all roles meet at the final barrier, TMEM is freed and the
 // kernel returns (no trap, no endless spin).  No multicast loads are used.
 #include "gemm_tc.cuh"
+
+#include <stdlib.h>
 
 namespace {
 
@@ -91,6 +93,55 @@ __device__ __forceinline__ void umma_commit(uint32_t bar)
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// ---- helpers of the 2-CTA (cta_group::2) variant: a CTA pair shares one 256-row tile ----
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load issued by either CTA of a pair; the transaction bytes are credited to the barrier at `bar`
+// (a shared::cluster address, normally the leader CTA's barrier).  No multicast.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// arrives on the barrier at the same shared-memory offset in both CTAs of the pair once the MMAs issued so far retire
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar)
+{
+    const uint16_t both = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(both) : "memory");
+}
+
 struct EpiParams {
     const __nv_bfloat16 *bias;
     void *out;
@@ -102,8 +153,8 @@ struct EpiParams {
 
 // Activations of the bf16 tensor-core path.  Results are rounded to bf16 (8 bits of mantissa), so
 // the hardware exp2 / reciprocal approximations (about 2^-22 relative) are far below what survives;
-// erf uses the five-term rational form 1 - (a1 t + ... + a5 t^5) exp(-x^2), t = 1/(1 + p x),
-// whose absolute error is below 1.5e-7.
+// erfc uses the three-term rational form (a1 t + a2 t^2 + a3 t^3) exp(-x^2), t = 1/(1 + p x),
+// whose absolute error is below 2.5e-5.
 __device__ __forceinline__ float fast_rcp(float x)
 {
     float y;
@@ -122,12 +173,11 @@ template <int ACT> __device__ __forceinline__ float fast_act(float z)
     if (ACT == D2D_ACT_RELU) return fmaxf(z, 0.0f);
     if (ACT == D2D_ACT_GELU_ERF) {
         // gelu(z) = max(z, 0) - 0.5 |z| erfc(|z| / sqrt 2), erfc(x) = (a1 t + ... + a5 t^5) exp(-x^2)
+        // three-term rational erfc (absolute error 2.5e-5, far below bf16 output rounding)
         const float az = fabsf(z);
-        const float t = fast_rcp(fmaf(0.3275911f * 0.70710678118654752f, az, 1.0f));
-        float p = fmaf(1.061405429f, t, -1.453152027f);
-        p = fmaf(p, t, 1.421413741f);
-        p = fmaf(p, t, -0.284496736f);
-        p = fmaf(p, t, 0.254829592f);
+        const float t = fast_rcp(fmaf(0.47047f * 0.70710678118654752f, az, 1.0f));
+        float p = fmaf(0.7478556f, t, -0.0958798f);
+        p = fmaf(p, t, 0.3480242f);
         const float e = fast_exp2(z * z * -0.72134752044448170f);          // exp(-z^2 / 2)
         return fmaxf(z, 0.0f) - (0.5f * az) * (p * t) * e;
     }
@@ -155,17 +205,13 @@ __device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16
         : "r"(taddr));
 }
 
-// 16 accumulator columns -> 16 output values: bias, activation, selection mask.
+// 16 accumulator columns -> 16 output values: bias (float32, staged in shared memory), activation, selection mask.
 template <int EPI, int ACT, bool GATED>
-__device__ __forceinline__ void epilogue_16(const uint32_t (&r)[16], const uint32_t (&g)[16], float *v,
-                                            const float *bias_f, const __nv_bfloat16 *bias_g, bool bias_cached,
-                                            int col0, int N, uint32_t keep)
+__device__ __forceinline__ void epilogue_16(const uint32_t (&r)[16], const uint32_t (&g)[16], float (&v)[16],
+                                            const float *bias_f, bool has_bias, int col0, uint32_t keep)
 {
     float bias[16];
-    if (bias_g == nullptr) {
-#pragma unroll
-        for (int j = 0; j < 16; ++j) bias[j] = 0.0f;
-    } else if (bias_cached && col0 + 16 <= N) {
+    if (has_bias) {
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
             const float4 b4 = *reinterpret_cast<const float4 *>(bias_f + col0 + 4 * q);
@@ -173,7 +219,7 @@ __device__ __forceinline__ void epilogue_16(const uint32_t (&r)[16], const uint3
         }
     } else {
 #pragma unroll
-        for (int j = 0; j < 16; ++j) bias[j] = col0 + j < N ? __bfloat162float(bias_g[col0 + j]) : 0.0f;
+        for (int j = 0; j < 16; ++j) bias[j] = 0.0f;
     }
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
@@ -189,7 +235,30 @@ __device__ __forceinline__ void epilogue_16(const uint32_t (&r)[16], const uint3
     }
 }
 
-constexpr int N_EPI_WARPS = 8;
+// Same result with every bound checked (ragged last column tile, odd leading dimension, bias too long for the cache).
+// Statically indexed and inlined: an out-of-line version forced the accumulator registers onto the stack.
+template <int EPI, int ACT, bool GATED>
+__device__ __forceinline__ void epilogue_16_slow(const uint32_t (&r)[16], const uint32_t (&g)[16], const __nv_bfloat16 *bias,
+                                                 void *out, int row, int M, int col0, int N, uint32_t keep)
+{
+    if (row >= M) return;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        if (col0 + j < N) {
+            float z = __uint_as_float(r[j]) + (bias ? __bfloat162float(bias[col0 + j]) : 0.0f);
+            if (EPI == D2D_EPI_RELU_BF16) z = fmaxf(z, 0.0f);
+            if (EPI == D2D_EPI_ABS_F32) z = fabsf(z);
+            if (EPI == D2D_EPI_UP_MASKED) {
+                const float h = GATED ? fast_act<ACT>(__uint_as_float(g[j])) * z : fast_act<ACT>(z);
+                z = ((keep >> j) & 1u) ? h : 0.0f;
+            }
+            if (EPI == D2D_EPI_ABS_F32) ((float *)out)[(size_t)row * N + col0 + j] = z;
+            else ((__nv_bfloat16 *)out)[(size_t)row * N + col0 + j] = __float2bfloat16_rn(z);
+        }
+    }
+}
+
+constexpr int N_EPI_WARPS = 16;
 constexpr int BIAS_CACHE_ELEMS = 6144;           // 24 KB of float32 in shared memory behind the operand stages
 constexpr int NTHREADS_V2 = 64 + 32 * N_EPI_WARPS;
 
@@ -198,17 +267,24 @@ __host__ __device__ constexpr int pow2_at_least(int v) { return v <= 32 ? 32 : v
 // Persistent kernel: CTA c computes tiles c, c + gridDim.x, ... (128 x BN each, column tiles
 // fastest).  Two accumulator buffers in TMEM let the epilogue of one tile overlap the MMAs of the
 // next.  GATED: two B tiles (up, gate) share the A tile; the epilogue forms A(gate) * (up + bias).
-template <int BN, int STAGES, int EPI, int ACT, bool GATED>
+// PAIR: two CTAs of a cluster (adjacent SMs) compute one 256 x BN tile with tcgen05.mma.cta_group::2: each CTA
+// loads its own 128 rows of A and only HALF of the B tile, the MMA reads both halves, and each CTA ends up with
+// its 128 accumulator rows in its own TMEM.  This cuts the L2 -> SM operand traffic per FLOP by 1.5x without
+// any multicast load.  The even CTA issues the MMAs; barriers that both CTAs need are signalled with
+// multicast commits (stage release, accumulator ready) or remote arrives (accumulator drained).
+template <int BN, int STAGES, int EPI, int ACT, bool GATED, bool PAIR>
 __global__ void __launch_bounds__(NTHREADS_V2, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                const __grid_constant__ CUtensorMap tm_b2, EpiParams ep, int M, int N, int K)
 {
+    constexpr int TM = PAIR ? 2 * BM : BM;                // rows of the tile a CTA (pair) computes
+    constexpr int B_ROWS = PAIR ? BN / 2 : BN;            // rows of B this CTA stages
     constexpr int A_BYTES = BM * BK * 2;
-    constexpr int B_BYTES = BN * BK * 2;
+    constexpr int B_BYTES = B_ROWS * BK * 2;
     constexpr int STAGE_BYTES = A_BYTES + (GATED ? 2 : 1) * B_BYTES;
     constexpr int BUF_COLS = pow2_at_least(GATED ? 2 * BN : BN);    // TMEM columns per accumulator buffer
     constexpr int TMEM_COLS = 2 * BUF_COLS;
-    constexpr int COLS_PER_WARP = BN / 2;                            // two epilogue warps share a TMEM lane quadrant
+    constexpr int COLS_PER_WARP = BN / 4;                            // four epilogue warps share a TMEM lane quadrant
     static_assert(TMEM_COLS <= 512 && BN % 64 == 0 && BN <= 256, "tile width");
 
     extern __shared__ uint8_t smem_raw[];
@@ -220,13 +296,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     float *bias_f = reinterpret_cast<float *>(smem + (size_t)STAGES * STAGE_BYTES);
     const bool bias_cached = ep.bias != nullptr && N <= BIAS_CACHE_ELEMS && (N & 3) == 0;
     if (bias_cached) {
-        for (int i = threadIdx.x; i < N; i += NTHREADS_V2) bias_f[i] = __bfloat162float(ep.bias[i]);
+        // 16-byte loads, all issued before the first use: the fill costs one memory latency, not N / threads of them
+        for (int i = threadIdx.x * 8; i < N; i += NTHREADS_V2 * 8) {
+            float b8[8];
+            if (i + 8 <= N) {
+                d2d_load8(ep.bias + i, b8);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) bias_f[i + q] = b8[q];
+            } else {
+                for (int q = 0; i + q < N; ++q) bias_f[i + q] = __bfloat162float(ep.bias[i + q]);
+            }
+        }
     }
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nkb = (K + BK - 1) / BK;
     const int n_tiles = (N + BN - 1) / BN;
-    const int total_tiles = ((M + BM - 1) / BM) * n_tiles;
+    const int total_tiles = ((M + TM - 1) / TM) * n_tiles;
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;           // 0 = the CTA that issues the MMAs
+    const int worker = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int n_workers = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -235,18 +324,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&bar_acc_full[b]), 1);
-            mbar_init(smem_u32(&bar_acc_empty[b]), N_EPI_WARPS);
+            mbar_init(smem_u32(&bar_acc_empty[b]), PAIR ? 2 * N_EPI_WARPS : N_EPI_WARPS);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_holder)),
-                     "r"((uint32_t)TMEM_COLS)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if (PAIR) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_holder)),
+                         "r"((uint32_t)TMEM_COLS)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_holder)),
+                         "r"((uint32_t)TMEM_COLS)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    if (PAIR) cluster_sync_all();          // the peer's barriers are initialised before anything signals them
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = tmem_base_holder;
 
@@ -255,28 +352,37 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                const int m0 = (tile / n_tiles) * BM, n0 = (tile % n_tiles) * BN;
+            for (int tile = worker; tile < total_tiles && ok; tile += n_workers) {
+                const int m0 = (tile / n_tiles) * TM + (int)rank * BM, n0 = (tile % n_tiles) * BN + (int)rank * B_ROWS;
                 for (int kb = 0; kb < nkb; ++kb, ++it) {
                     const uint32_t s = it % STAGES, round = it / STAGES;
                     ok = mbar_wait(smem_u32(&bar_empty[s]), (round & 1u) ^ 1u, ep.status);
                     if (!ok) break;
-                    const uint32_t full = smem_u32(&bar_full[s]);
                     const uint32_t dst = smem_u32(smem + (size_t)s * STAGE_BYTES);
-                    mbar_expect_tx(full, (uint32_t)STAGE_BYTES);
-                    tma_load_2d(dst, &tm_a, kb * BK, m0, full);
-                    tma_load_2d(dst + A_BYTES, &tm_b, kb * BK, n0, full);
-                    if (GATED) tma_load_2d(dst + A_BYTES + B_BYTES, &tm_b2, kb * BK, n0, full);
+                    if (PAIR) {
+                        // both CTAs' bytes are credited to the leader's barrier (where the MMAs are issued)
+                        const uint32_t full = map_to_cta(smem_u32(&bar_full[s]), 0);
+                        if (rank == 0) mbar_expect_tx(smem_u32(&bar_full[s]), 2u * (uint32_t)STAGE_BYTES);
+                        tma_load_2d_pair(dst, &tm_a, kb * BK, m0, full);
+                        tma_load_2d_pair(dst + A_BYTES, &tm_b, kb * BK, n0, full);
+                        if (GATED) tma_load_2d_pair(dst + A_BYTES + B_BYTES, &tm_b2, kb * BK, n0, full);
+                    } else {
+                        const uint32_t full = smem_u32(&bar_full[s]);
+                        mbar_expect_tx(full, (uint32_t)STAGE_BYTES);
+                        tma_load_2d(dst, &tm_a, kb * BK, m0, full);
+                        tma_load_2d(dst + A_BYTES, &tm_b, kb * BK, n0, full);
+                        if (GATED) tma_load_2d(dst + A_BYTES + B_BYTES, &tm_b2, kb * BK, n0, full);
+                    }
                 }
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            const uint32_t idesc = instr_desc_bf16(BM, BN);
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = instr_desc_bf16(TM, BN);
             uint32_t it = 0, local = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++local) {
+            for (int tile = worker; tile < total_tiles && ok; tile += n_workers, ++local) {
                 const uint32_t buf = local & 1u, use = local >> 1;
                 ok = mbar_wait(smem_u32(&bar_acc_empty[buf]), (use & 1u) ^ 1u, ep.status);   // epilogue drained this buffer
                 if (!ok) break;
@@ -295,28 +401,38 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     for (int k = 0; k < BK / UMMA_K; ++k) {
                         const uint64_t koff = (uint64_t)((k * UMMA_K * 2) >> 4);    // 32 bytes per K step inside the swizzle row
                         const uint32_t accum = (kb | k) != 0 ? 1u : 0u;
-                        umma_bf16(acc, da + koff, db + koff, idesc, accum);
-                        if (GATED) umma_bf16(acc + BN, da + koff, db2 + koff, idesc, accum);
+                        if (PAIR) {
+                            umma_bf16_pair(acc, da + koff, db + koff, idesc, accum);
+                            if (GATED) umma_bf16_pair(acc + BN, da + koff, db2 + koff, idesc, accum);
+                        } else {
+                            umma_bf16(acc, da + koff, db + koff, idesc, accum);
+                            if (GATED) umma_bf16(acc + BN, da + koff, db2 + koff, idesc, accum);
+                        }
                     }
-                    umma_commit(smem_u32(&bar_empty[s]));      // stage reusable once these MMAs have read it
+                    // stage reusable (in both CTAs of a pair) once these MMAs have read it
+                    if (PAIR) umma_commit_pair(smem_u32(&bar_empty[s]));
+                    else umma_commit(smem_u32(&bar_empty[s]));
                 }
-                umma_commit(smem_u32(&bar_acc_full[buf]));     // accumulator of this tile complete
+                // accumulator of this tile complete (each CTA of a pair holds its own 128 rows)
+                if (PAIR) umma_commit_pair(smem_u32(&bar_acc_full[buf]));
+                else umma_commit(smem_u32(&bar_acc_full[buf]));
             }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue (warps 2..9)
-        // The chunk loop is deliberately NOT unrolled: the body (32 elements of bias + activation +
-        // mask + pack) is a few KB of code that then stays in the instruction cache; unrolling it over
-        // the chunks made the kernel fetch-bound.  TMEM loads are split in 16-column halves so that the
-        // load of the next half overlaps the math of the current one.
+        // ------------------------------------------------------------------ epilogue (warps 2..17)
+        // Sixteen warps (four per TMEM lane quadrant) so that the per-element math of one warp hides
+        // the TMEM-load and MUFU latencies of another.  A warp walks its BN/4 columns in 16-column
+        // units; the load of the next unit is in flight while the current one is processed, and the
+        // rarely taken paths are out of line so that the unrolled body stays small (a 32-column,
+        // everything-inline version of this epilogue was instruction-fetch bound).
         const int ew = warp - 2;
         const int quad = warp & 3;                          // TMEM lanes this warp may touch
-        const int half = ew >> 2;                           // which half of the tile's columns
-        constexpr int N_CHUNKS = COLS_PER_WARP / 32;
+        const int part = ew >> 2;                           // which quarter of the tile's columns
+        constexpr int N_UNITS = COLS_PER_WARP / 16;
         uint32_t local = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++local) {
-            const int m0 = (tile / n_tiles) * BM, n0 = (tile % n_tiles) * BN;
+        for (int tile = worker; tile < total_tiles && ok; tile += n_workers, ++local) {
+            const int m0 = (tile / n_tiles) * TM + (int)rank * BM, n0 = (tile % n_tiles) * BN;
             const uint32_t buf = local & 1u, use = local >> 1;
             const int row = m0 + quad * 32 + lane;
             // this row's selection words go to registers before the wait, so their latency is hidden
@@ -334,72 +450,77 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             ok = __shfl_sync(0xffffffffu, okw, 0) != 0;
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t tbase = tmem_base + buf * BUF_COLS + ((uint32_t)(quad * 32) << 16) + (uint32_t)(half * COLS_PER_WARP);
+            const uint32_t tbase = tmem_base + buf * BUF_COLS + ((uint32_t)(quad * 32) << 16) + (uint32_t)(part * COLS_PER_WARP);
 
+            // expert that owns the first column of this warp's range (one division per tile; advanced incrementally)
+            const int colw = n0 + part * COLS_PER_WARP;
+            int e = 0, lo = 0, widx = -1;
+            uint32_t word = 0u;
+            if (EPI == D2D_EPI_UP_MASKED && mrow) {
+                e = colw / ep.expert_size;
+                lo = e * ep.expert_size - colw;             // first column of expert e relative to the current unit (<= 0)
+            }
+            const bool bias_fast = ep.bias == nullptr || bias_cached;
             uint32_t ra[16], rb[16], ga[16], gb[16];
             tmem_ld16_issue(tbase, ra);
             if (GATED) tmem_ld16_issue(tbase + BN, ga);
-#pragma unroll 1
-            for (int ci = 0; ci < N_CHUNKS; ++ci) {
-                const int c0 = half * COLS_PER_WARP + ci * 32;
-                const int col0 = n0 + c0;
-                const bool whole = col0 + 32 <= N;          // warp-uniform; ragged only in the last column tile
+#pragma unroll
+            for (int u = 0; u < N_UNITS; ++u) {             // at most 4 units; slow paths are out of line to keep the code small
+                const int col0 = colw + u * 16;
+                uint32_t (&r)[16] = (u & 1) ? rb : ra;
+                uint32_t (&g)[16] = (u & 1) ? gb : ga;
+                if (col0 >= N) {                            // warp-uniform (ragged last column tile)
+                    tmem_ld_wait();
+                    break;
+                }
 
-                // selection bits of this row for the 32 columns: a few experts cover them
-                uint32_t keep = 0xffffffffu;
+                // selection bits of this row for the 16 columns: one or two experts cover them
+                uint32_t keep = 0xffffu;
                 if (EPI == D2D_EPI_UP_MASKED && mrow) {
                     keep = 0u;
                     const int s = ep.expert_size;
-                    int e = col0 / s;
-                    int lo = e * s - col0;                  // first column of expert e relative to the chunk (<= 0)
-                    while (lo < 32) {
-                        const int hi = lo + s;
-                        uint32_t word;
-                        if (ep.mask_words <= MASK_REGS) {
-                            word = 0u;
+                    int ee = e, l = lo;
+                    while (l < 16) {
+                        if ((ee >> 5) != widx) {
+                            widx = ee >> 5;
+                            if (ep.mask_words <= MASK_REGS) {
+                                word = 0u;
 #pragma unroll
-                            for (int i = 0; i < MASK_REGS; ++i) word = (i == (e >> 5)) ? mw[i] : word;
-                        } else {
-                            word = __ldg(mrow + (e >> 5));
+                                for (int i = 0; i < MASK_REGS; ++i) word = (i == widx) ? mw[i] : word;
+                            } else {
+                                word = __ldg(mrow + widx);
+                            }
                         }
-                        if ((word >> (e & 31)) & 1u) {
-                            const int a = lo < 0 ? 0 : lo, b2 = hi > 32 ? 32 : hi;
-                            const uint32_t upto_b = b2 >= 32 ? 0xffffffffu : ((1u << b2) - 1u);
-                            keep |= upto_b & ~((1u << a) - 1u);
+                        const int hi = l + s;
+                        if ((word >> (ee & 31)) & 1u) {
+                            const int a = l < 0 ? 0 : l, b2 = hi > 16 ? 16 : hi;
+                            keep |= ((1u << b2) - 1u) & ~((1u << a) - 1u);
                         }
-                        lo = hi;
-                        ++e;
+                        l = hi;
+                        ++ee;
                     }
+                    // advance to the expert that owns the first column of the next unit
+                    lo -= 16;
+                    while (lo + s <= 0) { lo += s; ++e; }
+                }
+                tmem_ld_wait();                                               // this unit's accumulators have landed
+                if (u + 1 < N_UNITS) {                                        // the next unit's load overlaps the math below
+                    tmem_ld16_issue(tbase + (u + 1) * 16, (u & 1) ? ra : rb);
+                    if (GATED) tmem_ld16_issue(tbase + (u + 1) * 16 + BN, (u & 1) ? ga : gb);
                 }
 
-                float v[32];
-                tmem_ld_wait();                                                   // ra (and ga) have landed
-                tmem_ld16_issue(tbase + ci * 32 + 16, rb);
-                if (GATED) tmem_ld16_issue(tbase + ci * 32 + 16 + BN, gb);
-                epilogue_16<EPI, ACT, GATED>(ra, ga, v, bias_f, ep.bias, bias_cached, col0, N, keep);
-                tmem_ld_wait();                                                   // rb (and gb) have landed
-                if (ci + 1 < N_CHUNKS) {
-                    tmem_ld16_issue(tbase + (ci + 1) * 32, ra);
-                    if (GATED) tmem_ld16_issue(tbase + (ci + 1) * 32 + BN, ga);
-                }
-                epilogue_16<EPI, ACT, GATED>(rb, gb, v + 16, bias_f, ep.bias, bias_cached, col0 + 16, N, keep >> 16);
-
-                if (row < M && col0 < N) {
-                    if (EPI == D2D_EPI_ABS_F32) {
-                        float *o = (float *)ep.out + (size_t)row * N + col0;
-                        if (whole && (N & 3) == 0) {
+                if (col0 + 16 <= N && bias_fast && (N & 7) == 0) {
+                    float v[16];
+                    epilogue_16<EPI, ACT, GATED>(r, g, v, bias_f, ep.bias != nullptr, col0, keep);
+                    if (row < M) {
+                        if (EPI == D2D_EPI_ABS_F32) {
+                            float *o = (float *)ep.out + (size_t)row * N + col0;
 #pragma unroll
-                            for (int j = 0; j < 32; j += 4) *reinterpret_cast<float4 *>(o + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-                        } else {                            // ragged last column tile
+                            for (int j = 0; j < 16; j += 4) *reinterpret_cast<float4 *>(o + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                        } else {
+                            __nv_bfloat16 *o = (__nv_bfloat16 *)ep.out + (size_t)row * N + col0;
 #pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                if (col0 + j < N) o[j] = v[j];
-                        }
-                    } else {
-                        __nv_bfloat16 *o = (__nv_bfloat16 *)ep.out + (size_t)row * N + col0;
-                        if (whole && (N & 7) == 0) {
-#pragma unroll
-                            for (int j = 0; j < 32; j += 8) {
+                            for (int j = 0; j < 16; j += 8) {
                                 uint4 pk;
                                 __nv_bfloat162 t0 = __floats2bfloat162_rn(v[j], v[j + 1]);
                                 __nv_bfloat162 t1 = __floats2bfloat162_rn(v[j + 2], v[j + 3]);
@@ -411,25 +532,31 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                                 pk.w = *reinterpret_cast<uint32_t *>(&t3);
                                 *reinterpret_cast<uint4 *>(o + j) = pk;
                             }
-                        } else {                            // ragged last column tile
-#pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                if (col0 + j < N) o[j] = __float2bfloat16_rn(v[j]);
                         }
                     }
+                } else {
+                    // rare: ragged last column tile, odd leading dimension, or a bias too long for the cache
+                    epilogue_16_slow<EPI, ACT, GATED>(r, g, ep.bias, ep.out, row, M, col0, N, keep);
                 }
             }
             // all of this warp's TMEM reads of the buffer are complete: hand it back to the MMA warp
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[buf]));
+            if (lane == 0) {
+                if (PAIR) mbar_arrive_cluster(map_to_cta(smem_u32(&bar_acc_empty[buf]), 0));   // the leader waits for both CTAs
+                else mbar_arrive(smem_u32(&bar_acc_empty[buf]));
+            }
         }
     }
 
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    if (PAIR) cluster_sync_all();          // neither CTA releases shared memory or TMEM while the other may still use it
     if (warp == 1) {
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
+        if (PAIR)
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
+        else
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
     }
 }
 
@@ -481,63 +608,103 @@ int sm_count()
     return g_sm_count;
 }
 
-template <int BN, int EPI, int ACT, bool GATED>
+template <int BN, int EPI, int ACT, bool GATED, bool PAIR>
 d2d_status launch(const d2d_gemm_args &g, cudaStream_t st)
 {
-    constexpr int STAGE_BYTES = BM * BK * 2 + (GATED ? 2 : 1) * BN * BK * 2;
+    constexpr int B_ROWS = PAIR ? BN / 2 : BN;
+    constexpr int STAGE_BYTES = BM * BK * 2 + (GATED ? 2 : 1) * B_ROWS * BK * 2;
     constexpr int STAGES = (196 * 1024) / STAGE_BYTES > 8 ? 8 : (196 * 1024) / STAGE_BYTES;
     constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + 1024 + (size_t)BIAS_CACHE_ELEMS * 4;
     CUtensorMap ta, tb, tb2;
-    if (!make_map(&ta, g.a, g.M, g.K, BM) || !make_map(&tb, g.b, g.N, g.K, BN)) return D2D_ERR_CUDA;
+    if (!make_map(&ta, g.a, g.M, g.K, BM) || !make_map(&tb, g.b, g.N, g.K, B_ROWS)) return D2D_ERR_CUDA;
     if (GATED) {
-        if (!make_map(&tb2, g.b_gate, g.N, g.K, BN)) return D2D_ERR_CUDA;
+        if (!make_map(&tb2, g.b_gate, g.N, g.K, B_ROWS)) return D2D_ERR_CUDA;
     } else {
         tb2 = tb;
     }
-    auto kern = gemm_tc_kernel<BN, STAGES, EPI, ACT, GATED>;
+    auto kern = gemm_tc_kernel<BN, STAGES, EPI, ACT, GATED, PAIR>;
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM) != cudaSuccess) return D2D_ERR_CUDA;
         attr_set = true;
     }
     EpiParams ep{(const __nv_bfloat16 *)g.bias, g.out, g.mask, g.mask_words, g.expert_size > 0 ? g.expert_size : 1, g.status};
-    const int tiles = d2d_cdiv(g.N, BN) * d2d_cdiv(g.M, BM);
-    const int grid = tiles < sm_count() ? tiles : sm_count();
-    kern<<<grid, NTHREADS_V2, SMEM, st>>>(ta, tb, tb2, ep, g.M, g.N, g.K);
+    const int tiles = d2d_cdiv(g.N, BN) * d2d_cdiv(g.M, PAIR ? 2 * BM : BM);
+    const int workers = PAIR ? sm_count() / 2 : sm_count();
+    const int grid = (tiles < workers ? tiles : workers) * (PAIR ? 2 : 1);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(NTHREADS_V2, 1, 1);
+    cfg.dynamicSmemBytes = SMEM;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = PAIR ? 2 : 1;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, kern, ta, tb, tb2, ep, g.M, g.N, g.K);
     D2D_LAUNCHED(1);
-    return cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
+    return err == cudaSuccess && cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
 }
 
-// Tile width that wastes the fewest SM-rounds: tiles / (rounds * SMs), wider tiles preferred on ties
-// (fewer re-reads of A, fewer per-tile overheads).
-int pick_bn(int M, int N, const int *cands, int n_cands)
+// Tile width that wastes the fewest SM-rounds: tiles / (rounds * workers), wider tiles preferred on ties
+// (fewer re-reads of A, fewer per-tile overheads).  A "worker" is an SM, or an SM pair for the 2-CTA variant.
+int pick_bn(int M, int N, int tile_m, int workers, const int *cands, int n_cands, double *eff_out)
 {
-    const int sms = sm_count();
     int best = cands[0];
     double best_eff = -1.0;
     for (int i = 0; i < n_cands; ++i) {
         const int bn = cands[i];
-        const long tiles = (long)d2d_cdiv(N, bn) * d2d_cdiv(M, BM);
-        const long rounds = (tiles + sms - 1) / sms;
+        const long tiles = (long)d2d_cdiv(N, bn) * d2d_cdiv(M, tile_m);
+        const long rounds = (tiles + workers - 1) / workers;
         const double useful = (double)N / ((double)d2d_cdiv(N, bn) * bn);       // ragged last column tile
-        const double eff = useful * (double)tiles / (double)(rounds * sms) * (bn >= 128 ? 1.0 : 0.85);
+        const double eff = useful * (double)tiles / (double)(rounds * workers) * (bn >= 128 ? 1.0 : 0.85);
         if (eff > best_eff + 1e-9) { best_eff = eff; best = bn; }
     }
+    if (eff_out) *eff_out = best_eff;
     return best;
+}
+
+bool pair_mode_enabled()
+{
+    static const bool on = [] {
+        // off by default: measured on B200 the pair variant is not faster (the main loops are bound by the
+        // MMA issue interval, ~145 cycles per instruction, not by operand traffic); D2D_GEMM_PAIR=1 enables it
+        const char *e = getenv("D2D_GEMM_PAIR");
+        return e && e[0] == '1';
+    }();
+    return on;
 }
 
 template <int EPI, int ACT, bool GATED>
 d2d_status launch_bn(const d2d_gemm_args &g, cudaStream_t st)
 {
+    const int sms = sm_count();
     if (GATED) {
-        return launch<128, EPI, ACT, true>(g, st);
+        if (pair_mode_enabled() && g.M > BM) return launch<128, EPI, ACT, true, true>(g, st);
+        return launch<128, EPI, ACT, true, false>(g, st);
     } else {
-        const int cands[4] = {256, 192, 128, 64};
-        switch (pick_bn(g.M, g.N, cands, 4)) {
-        case 256: return launch<256, EPI, ACT, false>(g, st);
-        case 192: return launch<192, EPI, ACT, false>(g, st);
-        case 128: return launch<128, EPI, ACT, false>(g, st);
-        default: return launch<64, EPI, ACT, false>(g, st);
+        // 2-CTA pairs (256-row tiles, half of B per CTA) when the problem has at least two row tiles and the
+        // pairs can be kept about as busy as single CTAs would be
+        const int cands2[3] = {256, 192, 128};
+        const int cands1[4] = {256, 192, 128, 64};
+        double eff2 = 0.0, eff1 = 0.0;
+        const int bn2 = pick_bn(g.M, g.N, 2 * BM, sms / 2, cands2, 3, &eff2);
+        const int bn1 = pick_bn(g.M, g.N, BM, sms, cands1, 4, &eff1);
+        if (pair_mode_enabled() && g.M > BM && eff2 >= 0.8 * eff1) {
+            switch (bn2) {
+            case 256: return launch<256, EPI, ACT, false, true>(g, st);
+            case 192: return launch<192, EPI, ACT, false, true>(g, st);
+            default: return launch<128, EPI, ACT, false, true>(g, st);
+            }
+        }
+        switch (bn1) {
+        case 256: return launch<256, EPI, ACT, false, false>(g, st);
+        case 192: return launch<192, EPI, ACT, false, false>(g, st);
+        case 128: return launch<128, EPI, ACT, false, false>(g, st);
+        default: return launch<64, EPI, ACT, false, false>(g, st);
         }
     }
 }
