@@ -309,9 +309,18 @@ d2d_status d2d_layer_fwd(const d2d_layer *layer, const void *x, int32_t T, float
     if (!ws || !aligned16(ws) || ws_bytes < w.total) return D2D_ERR_WORKSPACE;
     char *base = (char *)ws;
     float *R = R_out ? R_out : (float *)(base + w.r_off);
-    d2d_status rc = d2d_launch_router(layer, x, T, R, (float *)(base + w.u_off), st);
-    if (rc != D2D_OK) return rc;
-    rc = d2d_launch_select(R, T, E, tau, 0, routing, base + w.sel_off, st);
+    d2d_status rc;
+    if (d2d_router_fused_supports(layer->desc, T)) {
+        // router and dynamic-k mask in one kernel; the selection step then only builds the per-expert metadata
+        if (cudaMemsetAsync(routing->status, 0, sizeof(int32_t), st) != cudaSuccess) return D2D_ERR_CUDA;
+        rc = d2d_router_fused(layer, x, T, tau, 1, R, routing->mask, routing->k, routing->status, st);
+        if (rc != D2D_OK) return rc;
+        rc = d2d_launch_select(nullptr, T, E, tau, 0, routing, base + w.sel_off, st, 1);
+    } else {
+        rc = d2d_launch_router(layer, x, T, R, (float *)(base + w.u_off), st);
+        if (rc != D2D_OK) return rc;
+        rc = d2d_launch_select(R, T, E, tau, 0, routing, base + w.sel_off, st);
+    }
     if (rc != D2D_OK) return rc;
     return d2d_launch_moe_ffn(layer, x, T, routing, y, base + w.ffn_off, w.total - w.ffn_off, st);
 }

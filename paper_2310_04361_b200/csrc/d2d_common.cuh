@@ -40,8 +40,10 @@ static inline int d2d_cdiv(int a, int b) { return (a + b - 1) / b; }
 d2d_status d2d_launch_router(const d2d_layer *L, const void *x, int T, float *R, float *u_ws, cudaStream_t st);
 
 size_t d2d_select_ws_bytes(int T, int E);
+// R == nullptr: the mask is an input.  mask_ready != 0: mask, k and the status word were already written
+// (fused router), only the per-expert metadata is built.
 d2d_status d2d_launch_select(const float *R, int T, int E, float tau, int topk, const d2d_routing *out,
-                             void *ws, cudaStream_t st);   // R == nullptr: mask is an input
+                             void *ws, cudaStream_t st, int mask_ready = 0);
 
 d2d_status d2d_launch_moe_ffn(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y,
                               void *ws, size_t ws_bytes, cudaStream_t st);
@@ -49,7 +51,11 @@ size_t d2d_moe_ffn_ws_bytes(const d2d_layer *L, int T);
 
 // small-batch (T <= 64) kernels
 bool d2d_small_select_supports(int T, int E);
-d2d_status d2d_small_select(const float *R, int T, int E, float tau, const d2d_routing *out, cudaStream_t st);
+d2d_status d2d_small_select(const float *R, int T, int E, float tau, const d2d_routing *out, cudaStream_t st,
+                            int mask_ready = 0);
+bool d2d_router_fused_supports(const d2d_layer_desc &D, int T);
+d2d_status d2d_router_fused(const d2d_layer *L, const void *x, int T, float tau, int do_mask, float *R, uint32_t *mask,
+                            int32_t *k, int32_t *status, cudaStream_t st);
 bool d2d_small_router_supports(const d2d_layer_desc &D, int T);
 size_t d2d_small_router_ws_bytes(const d2d_layer *L, int T);
 d2d_status d2d_small_router(const d2d_layer *L, const void *x, int T, float *R, void *ws, cudaStream_t st);

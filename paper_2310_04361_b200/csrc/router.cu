@@ -83,6 +83,7 @@ d2d_status d2d_launch_router(const d2d_layer *L, const void *x, int T, float *R,
     // u_ws points at [256-byte ticket area | T*d_h floats]
     float *u = (float *)((char *)u_ws + 256);
     if (d2d_small_router_supports(L->desc, T)) return d2d_small_router(L, x, T, R, u_ws, st);
+    if (d2d_router_fused_supports(L->desc, T)) return d2d_router_fused(L, x, T, 0.0f, 0, R, nullptr, nullptr, nullptr, st);
     if (L->desc.dtype == D2D_F32) return run_router<float>(L, x, T, R, u, st);
     if (d2d_gemm_tc_available()) {
         // bf16 layers: both router layers are dense contractions on the tensor cores; the hidden

@@ -1,0 +1,417 @@
+// Fused router + dynamic-k mask for bf16 layers (Sec. 3.3 and Eq. 4): one kernel computes
+//   u = relu(x W_r1^T + b_r1)            tcgen05 GEMM, 128 tokens x d_h, accumulator in TMEM
+//   R = | u W_r2^T + b_r2 |              second tcgen05 GEMM whose A operand is u, written by the first
+//                                        epilogue straight into shared memory in the swizzled K-major layout
+//   m = max_i R[t,i], thr = tau * m (one fp32 RN multiply), mask words, k[t]     per-row epilogue on TMEM
+// so the hidden activations never touch HBM, R is written once (the caller may want it) and the
+// mask kernel's extra pass over R disappears.  One CTA per 128 tokens; 18 warps: TMA producer,
+// MMA issuer, 16 epilogue warps (four per TMEM lane quadrant, each a quarter of the columns).
+// All mbarrier waits are bounded (status D2D_ERR_TIMEOUT); no multicast.
+#include <cuda.h>
+
+#include "d2d_common.cuh"
+#include "gemm_tc.cuh"
+
+namespace {
+
+constexpr int BM = 128, BK = 64, UMMA_K = 16;
+constexpr int STAGES = 3;
+constexpr uint32_t WAIT_LIMIT = 1u << 22;
+constexpr int NTHREADS = 64 + 512;       // TMA warp, MMA warp, 16 epilogue warps
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t *status)
+{
+    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (done) return true;
+        if (it > 4096) __nanosleep(128);
+    }
+    if (status) atomicMax(status, (int32_t)D2D_ERR_TIMEOUT);
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3fffu);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+__device__ __forceinline__ uint32_t instr_desc_bf16(int m, int n)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared memory (dynamic, 1024-byte aligned):
+//   [ STAGES x (x tile 128x64 | W_r1 tile DH x 64) ]        first GEMM operand ring
+//   [ u: DH/64 k-blocks x (128 rows x 128 B) ]              A operand of the second GEMM (written by epilogue 1)
+//   [ W_r2: NT2 column tiles x DH/64 k-blocks x (256 rows x 128 B) ]   B operand of the second GEMM (TMA)
+// TMEM: columns [0, DH) accumulator of u, columns [256, 256 + E_pad) accumulator of R (E <= 256).
+template <int DH>
+__global__ void __launch_bounds__(NTHREADS, 1)
+router_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w1,
+                    const __grid_constant__ CUtensorMap tm_w2, const __nv_bfloat16 *__restrict__ b_r1,
+                    const __nv_bfloat16 *__restrict__ b_r2, int T, int d, int E, int EN /* E rounded up to 16 */,
+                    float tau, int do_mask, float *__restrict__ R, uint32_t *__restrict__ mask, int32_t *__restrict__ k,
+                    int32_t *__restrict__ status)
+{
+    constexpr int KB2 = DH / BK;                          // k-blocks of the second GEMM
+    constexpr int A_BYTES = BM * BK * 2, B1_BYTES = DH * BK * 2;
+    constexpr int STAGE_BYTES = A_BYTES + B1_BYTES;
+    constexpr int U_BYTES = KB2 * BM * 128;
+    constexpr int W2_KB_BYTES = 256 * 128;                // one k-block of W_r2 rows (box of 256 rows, zero filled past E)
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t *u_s = smem + (size_t)STAGES * STAGE_BYTES;
+    uint8_t *w2_s = u_s + U_BYTES;
+    __shared__ uint64_t bar_full[STAGES], bar_empty[STAGES], bar_w2, bar_acc1, bar_u_ready, bar_acc2;
+    __shared__ uint32_t tmem_base_holder;
+    __shared__ float b1_s[DH], b2_s[256];                  // biases as float32
+    __shared__ float pmax_s[4 * BM];                       // per column-part row maxima
+    __shared__ int pbad_s[4 * BM], pk_s[4 * BM];
+    for (int i = threadIdx.x; i < DH; i += NTHREADS) b1_s[i] = b_r1 ? __bfloat162float(b_r1[i]) : 0.0f;
+    for (int i = threadIdx.x; i < 256; i += NTHREADS) b2_s[i] = (b_r2 && i < E) ? __bfloat162float(b_r2[i]) : 0.0f;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m0 = blockIdx.x * BM;
+    const int nkb = (d + BK - 1) / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(smem_u32(&bar_full[s]), 1);
+            mbar_init(smem_u32(&bar_empty[s]), 1);
+        }
+        mbar_init(smem_u32(&bar_w2), 1);
+        mbar_init(smem_u32(&bar_acc1), 1);
+        mbar_init(smem_u32(&bar_u_ready), 16);            // one arrival per epilogue warp
+        mbar_init(smem_u32(&bar_acc2), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_holder)),
+                     "r"(512u)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = tmem_base_holder;
+    const uint32_t tmem_r = tmem_base + 256;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            // W_r2 first (small, needed last): all its k-blocks land on one barrier
+            mbar_expect_tx(smem_u32(&bar_w2), (uint32_t)(KB2 * W2_KB_BYTES));
+            for (int kb = 0; kb < KB2; ++kb)
+                tma_load_2d(smem_u32(w2_s + (size_t)kb * W2_KB_BYTES), &tm_w2, kb * BK, 0, smem_u32(&bar_w2));
+            for (int kb = 0; kb < nkb; ++kb) {
+                const uint32_t s = kb % STAGES, round = kb / STAGES;
+                if (!mbar_wait(smem_u32(&bar_empty[s]), (round & 1u) ^ 1u, status)) break;
+                const uint32_t full = smem_u32(&bar_full[s]);
+                const uint32_t dst = smem_u32(smem + (size_t)s * STAGE_BYTES);
+                mbar_expect_tx(full, (uint32_t)STAGE_BYTES);
+                tma_load_2d(dst, &tm_x, kb * BK, m0, full);
+                tma_load_2d(dst + A_BYTES, &tm_w1, kb * BK, 0, full);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            bool ok = true;
+            const uint32_t idesc1 = instr_desc_bf16(BM, DH);
+            for (int kb = 0; kb < nkb && ok; ++kb) {
+                const uint32_t s = kb % STAGES, round = kb / STAGES;
+                ok = mbar_wait(smem_u32(&bar_full[s]), round & 1u, status);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t a_addr = smem_u32(smem + (size_t)s * STAGE_BYTES);
+                const uint64_t da = smem_desc_sw128(a_addr), db = smem_desc_sw128(a_addr + A_BYTES);
+#pragma unroll
+                for (int q = 0; q < BK / UMMA_K; ++q) {
+                    const uint64_t koff = (uint64_t)((q * UMMA_K * 2) >> 4);
+                    umma_bf16(tmem_base, da + koff, db + koff, idesc1, (kb | q) != 0 ? 1u : 0u);
+                }
+                umma_commit(smem_u32(&bar_empty[s]));
+            }
+            umma_commit(smem_u32(&bar_acc1));              // u accumulator complete
+            // second GEMM: wait for u (written to shared memory by the epilogue warps) and for W_r2
+            ok = ok && mbar_wait(smem_u32(&bar_u_ready), 0, status) && mbar_wait(smem_u32(&bar_w2), 0, status);
+            if (ok) {
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t idesc2 = instr_desc_bf16(BM, EN);
+                for (int kb = 0; kb < KB2; ++kb) {
+                    const uint64_t da = smem_desc_sw128(smem_u32(u_s + (size_t)kb * BM * 128));
+                    const uint64_t db = smem_desc_sw128(smem_u32(w2_s + (size_t)kb * W2_KB_BYTES));
+#pragma unroll
+                    for (int q = 0; q < BK / UMMA_K; ++q) {
+                        const uint64_t koff = (uint64_t)((q * UMMA_K * 2) >> 4);
+                        umma_bf16(tmem_r, da + koff, db + koff, idesc2, (kb | q) != 0 ? 1u : 0u);
+                    }
+                }
+            }
+            umma_commit(smem_u32(&bar_acc2));
+        }
+    } else {
+        // ------------------------------------------------------------------ 16 epilogue warps
+        // warp -> TMEM lane quadrant (warp & 3) and one of four column parts; a thread owns one token row
+        const int quad = warp & 3, part = (warp - 2) >> 2;
+        const int r_local = quad * 32 + lane;
+        const int row = m0 + r_local;
+        const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+        int okw = 1;
+        if (lane == 0) okw = mbar_wait(smem_u32(&bar_acc1), 0, status) ? 1 : 0;
+        bool ok = __shfl_sync(0xffffffffu, okw, 0) != 0;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (ok) {
+            // ---- epilogue 1: u = relu(acc + b_r1) -> bf16 -> swizzled K-major tile in shared memory
+            constexpr int C1 = DH / 4;                     // columns of u per part
+#pragma unroll
+            for (int cc = 0; cc < C1; cc += 16) {
+                const int c0 = part * C1 + cc;
+                uint32_t acc[16];
+                tmem_ld16(tmem_base + lane_base + (uint32_t)c0, acc);
+                uint32_t pk[8];
+#pragma unroll
+                for (int j = 0; j < 16; j += 2) {
+                    const __nv_bfloat162 v = __floats2bfloat162_rn(fmaxf(__uint_as_float(acc[j]) + b1_s[c0 + j], 0.0f),
+                                                                   fmaxf(__uint_as_float(acc[j + 1]) + b1_s[c0 + j + 1], 0.0f));
+                    pk[j >> 1] = *reinterpret_cast<const uint32_t *>(&v);
+                }
+                // 16 columns = two 16-byte chunks of this row inside k-block c0/64; chunk index XOR (row % 8)
+                const int kb = c0 >> 6, chunk = (c0 & 63) >> 3;
+                uint8_t *rowp = u_s + (size_t)kb * BM * 128 + (size_t)r_local * 128;
+                *reinterpret_cast<uint4 *>(rowp + (((chunk) ^ (r_local & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                *reinterpret_cast<uint4 *>(rowp + (((chunk + 1) ^ (r_local & 7)) << 4)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+            }
+            // make the generic-proxy writes visible to the tensor-core (async) proxy, then signal the MMA warp
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bar_u_ready));
+
+            // ---- epilogue 2: R = |acc + b_r2|; part p owns mask words p and p + 4 (columns 32w .. 32w+31)
+            if (lane == 0) okw = mbar_wait(smem_u32(&bar_acc2), 0, status) ? 1 : 0;
+            ok = __shfl_sync(0xffffffffu, okw, 0) != 0;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const int W = (E + 31) / 32;
+            float v[2][32];
+            float m = -INFINITY;
+            bool bad = false;
+            if (ok) {
+#pragma unroll
+                for (int q = 0; q < 2; ++q) {
+                    const int w = part + 4 * q;
+                    if (w < W) {
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const int c0 = w * 32 + h * 16;
+                            if (c0 < EN) {
+                                uint32_t acc[16];
+                                tmem_ld16(tmem_r + lane_base + (uint32_t)c0, acc);
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) {
+                                    const int i = c0 + j;
+                                    const float val = fabsf(__uint_as_float(acc[j]) + b2_s[i]);
+                                    v[q][h * 16 + j] = val;
+                                    if (i < E) {
+                                        bad |= (__float_as_uint(val) & 0x7f800000u) == 0x7f800000u;
+                                        m = val > m ? val : m;
+                                    }
+                                }
+                                if (R && row < T) {
+                                    float *o = R + (size_t)row * E + c0;
+                                    if (c0 + 16 <= E && (E & 3) == 0) {
+#pragma unroll
+                                        for (int j = 0; j < 16; j += 4)
+                                            *reinterpret_cast<float4 *>(o + j) = make_float4(v[q][h * 16 + j], v[q][h * 16 + j + 1],
+                                                                                             v[q][h * 16 + j + 2], v[q][h * 16 + j + 3]);
+                                    } else {
+#pragma unroll
+                                        for (int j = 0; j < 16; ++j)
+                                            if (c0 + j < E) o[j] = v[q][h * 16 + j];
+                                    }
+                                }
+                            } else {
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) v[q][h * 16 + j] = 0.0f;
+                            }
+                        }
+                    }
+                }
+            }
+            if (do_mask) {
+                // row maximum across the four column parts (and the non-finite flag), through shared memory
+                pmax_s[part * BM + r_local] = m;
+                pbad_s[part * BM + r_local] = bad ? 1 : 0;
+                asm volatile("bar.sync 1, 512;" ::: "memory");           // the 16 epilogue warps only
+                float mm = pmax_s[r_local];
+                int anybad = pbad_s[r_local];
+#pragma unroll
+                for (int p = 1; p < 4; ++p) {
+                    const float o = pmax_s[p * BM + r_local];
+                    mm = o > mm ? o : mm;
+                    anybad |= pbad_s[p * BM + r_local];
+                }
+                const float thr = __fmul_rn(tau, mm);
+                int kt = 0;
+                if (ok) {
+#pragma unroll
+                    for (int q = 0; q < 2; ++q) {
+                        const int w = part + 4 * q;
+                        if (w < W) {
+                            uint32_t word = 0u;
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) {
+                                const int i = w * 32 + j;
+                                if (i < E && (anybad || v[q][j] >= thr)) word |= 1u << j;
+                            }
+                            if (row < T) mask[(size_t)row * W + w] = word;
+                            kt += __popc(word);
+                        }
+                    }
+                }
+                pk_s[part * BM + r_local] = kt;
+                asm volatile("bar.sync 1, 512;" ::: "memory");
+                if (part == 0 && row < T) {
+                    k[row] = pk_s[r_local] + pk_s[BM + r_local] + pk_s[2 * BM + r_local] + pk_s[3 * BM + r_local];
+                    if (anybad) atomicMax(status, (int32_t)D2D_ERR_NONFINITE);
+                }
+            }
+        } else if (do_mask) {
+            // keep the named barrier balanced when a bounded wait ran out
+            asm volatile("bar.sync 1, 512;" ::: "memory");
+            asm volatile("bar.sync 1, 512;" ::: "memory");
+        }
+    }
+
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    }
+}
+
+typedef CUresult (*encode_tiled_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                    const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+encode_tiled_fn get_encode()
+{
+    static encode_tiled_fn fn = [] {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return (encode_tiled_fn)p;
+    }();
+    return fn;
+}
+
+bool make_map(CUtensorMap *map, const void *base, int rows, int cols, int box_rows)
+{
+    encode_tiled_fn enc = get_encode();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int DH>
+d2d_status launch(const d2d_layer *L, const void *x, int T, float tau, int do_mask, float *R, uint32_t *mask, int32_t *k,
+                  int32_t *status, cudaStream_t st)
+{
+    const d2d_layer_desc &D = L->desc;
+    constexpr int STAGE_BYTES = BM * BK * 2 + DH * BK * 2;
+    constexpr int KB2 = DH / BK;
+    constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + (size_t)KB2 * BM * 128 + (size_t)KB2 * 256 * 128 + 1024;
+    CUtensorMap tx, tw1, tw2;
+    if (!make_map(&tx, x, T, D.d, BM) || !make_map(&tw1, L->w_r1, D.d_h, D.d, DH) ||
+        !make_map(&tw2, L->w_r2, D.n_experts, D.d_h, 256))
+        return D2D_ERR_CUDA;
+    auto kern = router_fused_kernel<DH>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM) != cudaSuccess) return D2D_ERR_CUDA;
+        attr_set = true;
+    }
+    const int EN = (D.n_experts + 15) / 16 * 16;
+    kern<<<d2d_cdiv(T, BM), NTHREADS, SMEM, st>>>(tx, tw1, tw2, (const __nv_bfloat16 *)L->b_r1, (const __nv_bfloat16 *)L->b_r2,
+                                                 T, D.d, D.n_experts, EN, tau, do_mask, R, mask, k, status);
+    D2D_LAUNCHED(1);
+    return cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
+}
+
+}  // namespace
+
+bool d2d_router_fused_supports(const d2d_layer_desc &D, int T)
+{
+    // d_h = 128 (the paper's router width) and E <= 256: operand ring, u and W_r2 then fit in shared memory together
+    return D.dtype == D2D_BF16 && T >= 9 && D.d_h == 128 && D.n_experts <= 256 && D.d % 8 == 0 && get_encode() != nullptr;
+}
+
+// R may be NULL when only the mask is wanted; mask / k / status are used when do_mask != 0.
+d2d_status d2d_router_fused(const d2d_layer *L, const void *x, int T, float tau, int do_mask, float *R, uint32_t *mask,
+                            int32_t *k, int32_t *status, cudaStream_t st)
+{
+    return launch<128>(L, x, T, tau, do_mask, R, mask, k, status, st);
+}

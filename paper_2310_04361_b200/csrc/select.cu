@@ -336,10 +336,10 @@ size_t d2d_select_ws_bytes(int T, int E)
 }
 
 d2d_status d2d_launch_select(const float *R, int T, int E, float tau, int topk, const d2d_routing *out,
-                             void *ws, cudaStream_t st)
+                             void *ws, cudaStream_t st, int mask_ready)
 {
     const int W = (E + 31) / 32;
-    D2D_CUDA_TRY(cudaMemsetAsync(out->status, 0, sizeof(int32_t), st));
+    if (!mask_ready) D2D_CUDA_TRY(cudaMemsetAsync(out->status, 0, sizeof(int32_t), st));
     if (T == 0) {
         D2D_CUDA_TRY(cudaMemsetAsync(out->counts, 0, sizeof(int32_t) * (size_t)E, st));
         D2D_CUDA_TRY(cudaMemsetAsync(out->offsets, 0, sizeof(int32_t) * (size_t)(E + 1), st));
@@ -347,7 +347,7 @@ d2d_status d2d_launch_select(const float *R, int T, int E, float tau, int topk, 
         if (out->tok_off) D2D_CUDA_TRY(cudaMemsetAsync(out->tok_off, 0, sizeof(int32_t), st));
         return D2D_OK;
     }
-    if (topk == 0 && d2d_small_select_supports(T, E)) return d2d_small_select(R, T, E, tau, out, st);
+    if (topk == 0 && d2d_small_select_supports(T, E)) return d2d_small_select(R, T, E, tau, out, st, mask_ready);
     const int warps_per_cta = 8;
     const int grid_tok = d2d_cdiv(T, warps_per_cta);
     if (R) {
@@ -355,7 +355,7 @@ d2d_status d2d_launch_select(const float *R, int T, int E, float tau, int topk, 
             topk_mask_kernel<<<grid_tok, 256, 0, st>>>(R, T, E, W, topk, out->mask, out->k, out->status);
         else
             dynk_mask_kernel<<<grid_tok, 256, 0, st>>>(R, T, E, W, tau, out->mask, out->k, out->status);
-    } else {
+    } else if (!mask_ready) {
         k_from_mask_kernel<<<d2d_cdiv(T, 256), 256, 0, st>>>(out->mask, T, W, out->k);
     }
     const int nblk = d2d_cdiv(T, TOKB);
@@ -367,7 +367,7 @@ d2d_status d2d_launch_select(const float *R, int T, int E, float tau, int topk, 
                                                     (long long)out->perm_capacity);
     bucket_fill_kernel<<<dim3(nblk, W), TOKB, 0, st>>>(out->mask, T, E, W, blockcounts, out->offsets, out->perm,
                                               (long long)out->perm_capacity);
-    D2D_LAUNCHED(3);
+    D2D_LAUNCHED(mask_ready ? 2 : 3);
     if (out->tok_off && out->tok_exp) {
         D2D_LAUNCHED(2);
         tok_scan_kernel<<<1, 1024, 0, st>>>(out->k, T, out->tok_off);

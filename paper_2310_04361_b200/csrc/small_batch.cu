@@ -21,14 +21,14 @@ small_select_kernel(const float *__restrict__ R, int T, int E, int W, float tau,
                     uint32_t *__restrict__ mask, int32_t *__restrict__ k, int32_t *__restrict__ counts,
                     int32_t *__restrict__ offsets, int32_t *__restrict__ perm, int32_t *__restrict__ tok_off,
                     int32_t *__restrict__ tok_exp, int32_t *__restrict__ n_sel, int32_t *__restrict__ status,
-                    long long capacity)
+                    long long capacity, int keep_status)
 {
     extern __shared__ uint32_t smask[];          // [T][W]
     __shared__ int warp_sums[32];
     __shared__ int chunk_total;
     __shared__ int sk[64];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (threadIdx.x == 0) *status = 0;
+    if (threadIdx.x == 0 && !keep_status) *status = 0;
     __syncthreads();
 
     for (int t = warp; t < T; t += 32) {
@@ -140,7 +140,8 @@ small_select_kernel(const float *__restrict__ R, int T, int E, int W, float tau,
 
 bool d2d_small_select_supports(int T, int E) { return T >= 1 && T <= 64 && (size_t)T * ((E + 31) / 32) * 4 <= 96 * 1024; }
 
-d2d_status d2d_small_select(const float *R, int T, int E, float tau, const d2d_routing *out, cudaStream_t st)
+d2d_status d2d_small_select(const float *R, int T, int E, float tau, const d2d_routing *out, cudaStream_t st,
+                            int mask_ready)
 {
     const int W = (E + 31) / 32;
     const size_t smem = (size_t)T * W * sizeof(uint32_t);
@@ -152,7 +153,7 @@ d2d_status d2d_small_select(const float *R, int T, int E, float tau, const d2d_r
     }
     small_select_kernel<<<1, 1024, smem, st>>>(R, T, E, W, tau, out->mask, out->k, out->counts, out->offsets, out->perm,
                                                out->tok_off, out->tok_exp, out->n_sel, out->status,
-                                               (long long)out->perm_capacity);
+                                               (long long)out->perm_capacity, mask_ready);
     D2D_LAUNCHED(1);
     return cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
 }
