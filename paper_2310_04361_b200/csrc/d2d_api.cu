@@ -186,7 +186,14 @@ d2d_status d2d_layer_create(const d2d_layer_desc *desc, const d2d_weights *w, vo
         if (rc != D2D_OK) break;
     }
     if (rc == D2D_OK && cudaStreamSynchronize(st) != cudaSuccess) rc = D2D_ERR_CUDA;
+    if (rc == D2D_OK && (cudaStreamCreateWithFlags(&L->side_stream, cudaStreamNonBlocking) != cudaSuccess ||
+                         cudaEventCreateWithFlags(&L->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+                         cudaEventCreateWithFlags(&L->ev_join, cudaEventDisableTiming) != cudaSuccess))
+        rc = D2D_ERR_CUDA;
     if (rc != D2D_OK) {
+        if (L->ev_join) cudaEventDestroy(L->ev_join);
+        if (L->ev_fork) cudaEventDestroy(L->ev_fork);
+        if (L->side_stream) cudaStreamDestroy(L->side_stream);
         cudaFree(L->slab);
         delete L;
         return rc;
@@ -198,6 +205,9 @@ d2d_status d2d_layer_create(const d2d_layer_desc *desc, const d2d_weights *w, vo
 d2d_status d2d_layer_destroy(d2d_layer *layer)
 {
     if (!layer) return D2D_OK;
+    if (layer->ev_join) cudaEventDestroy(layer->ev_join);
+    if (layer->ev_fork) cudaEventDestroy(layer->ev_fork);
+    if (layer->side_stream) cudaStreamDestroy(layer->side_stream);
     cudaError_t e = cudaFree(layer->slab);
     delete layer;
     return e == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
@@ -315,6 +325,20 @@ d2d_status d2d_layer_fwd(const d2d_layer *layer, const void *x, int32_t T, float
         if (cudaMemsetAsync(routing->status, 0, sizeof(int32_t), st) != cudaSuccess) return D2D_ERR_CUDA;
         rc = d2d_router_fused(layer, x, T, tau, 1, R, routing->mask, routing->k, routing->status, st);
         if (rc != D2D_OK) return rc;
+        if (use_dense_masked(layer, T) && !use_small_ffn(layer, T)) {
+            // The dense-masked expert GEMMs read only the mask: build counts / offsets / token lists on the side
+            // stream while they run (the small metadata CTAs fit beside the persistent GEMM CTAs), join at the end.
+            if (cudaEventRecord(layer->ev_fork, st) != cudaSuccess ||
+                cudaStreamWaitEvent(layer->side_stream, layer->ev_fork, 0) != cudaSuccess)
+                return D2D_ERR_CUDA;
+            rc = d2d_launch_select(nullptr, T, E, tau, 0, routing, base + w.sel_off, layer->side_stream, 1);
+            if (rc != D2D_OK) return rc;
+            rc = d2d_launch_moe_ffn(layer, x, T, routing, y, base + w.ffn_off, w.total - w.ffn_off, st);
+            if (cudaEventRecord(layer->ev_join, layer->side_stream) != cudaSuccess ||
+                cudaStreamWaitEvent(st, layer->ev_join, 0) != cudaSuccess)
+                return D2D_ERR_CUDA;
+            return rc;
+        }
         rc = d2d_launch_select(nullptr, T, E, tau, 0, routing, base + w.sel_off, st, 1);
     } else {
         rc = d2d_launch_router(layer, x, T, R, (float *)(base + w.u_off), st);

@@ -20,6 +20,10 @@ struct d2d_layer {
     void *w2;               // W2 as given ([d, d_ff]): the K-major B operand of the dense down projection
     void *slab;             // one allocation backing all of the above
     size_t slab_bytes;
+    // side stream + events: the per-expert metadata (counts, offsets, token lists) is built beside the
+    // expert GEMMs, which do not read it
+    cudaStream_t side_stream;
+    cudaEvent_t ev_fork, ev_join;
 };
 
 #define D2D_CUDA_TRY(expr)                                   \
