@@ -45,7 +45,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t
             : "r"(bar), "r"(parity)
             : "memory");
         if (done) return true;
-        if (it > 4096) __nanosleep(128);
+        if (it > 64) __nanosleep(32);
     }
     if (status) atomicMax(status, (int32_t)D2D_ERR_TIMEOUT);
     return false;
@@ -149,22 +149,22 @@ struct EpiParams {
     int mask_words;
     int expert_size;
     int32_t *status;
+    uint32_t inv_expert_size;        // ceil(2^32 / expert_size): column / expert_size = umulhi(column, inv) for columns < 2^16
 };
 
-// Activations of the bf16 tensor-core path.  Results are rounded to bf16 (8 bits of mantissa), so
-// the hardware exp2 / reciprocal approximations (about 2^-22 relative) are far below what survives;
-// erfc uses the three-term rational form (a1 t + a2 t^2 + a3 t^3) exp(-x^2), t = 1/(1 + p x),
-// whose absolute error is below 2.5e-5.
-__device__ __forceinline__ float fast_rcp(float x)
+// Activations of the bf16 tensor-core path.  Results are rounded to bf16 (8 bits of mantissa,
+// 2^-9 relative), and the epilogue of the up projection is issue-bound (K = d is short compared
+// with the 128 x BN outputs of a tile), so every activation is built on ONE special-function
+// instruction, the hardware tanh (relative error about 2^-11):
+//   SiLU       z * sigmoid(z)            = z * (0.5 + 0.5 tanh(z / 2))
+//   GELU tanh  0.5 z (1 + tanh(c (z + 0.044715 z^3)))
+//   GELU erf   0.5 z (1 + erf(z / sqrt 2)),  erf(z / sqrt 2) ~= tanh(z (a + b z^2 + c z^4)), a quintic
+//              argument fitted to erf with maximum error 3.7e-5 (GELU: 5.4e-5 absolute before the tanh
+//              instruction's own error) -- well below what a bf16 result can represent.
+__device__ __forceinline__ float fast_tanh(float x)
 {
     float y;
-    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-__device__ __forceinline__ float fast_exp2(float x)
-{
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
 
@@ -172,22 +172,19 @@ template <int ACT> __device__ __forceinline__ float fast_act(float z)
 {
     if (ACT == D2D_ACT_RELU) return fmaxf(z, 0.0f);
     if (ACT == D2D_ACT_GELU_ERF) {
-        // gelu(z) = max(z, 0) - 0.5 |z| erfc(|z| / sqrt 2), erfc(x) = (a1 t + ... + a5 t^5) exp(-x^2)
-        // three-term rational erfc (absolute error 2.5e-5, far below bf16 output rounding)
-        const float az = fabsf(z);
-        const float t = fast_rcp(fmaf(0.47047f * 0.70710678118654752f, az, 1.0f));
-        float p = fmaf(0.7478556f, t, -0.0958798f);
-        p = fmaf(p, t, 0.3480242f);
-        const float e = fast_exp2(z * z * -0.72134752044448170f);          // exp(-z^2 / 2)
-        return fmaxf(z, 0.0f) - (0.5f * az) * (p * t) * e;
+        // the quintic was fitted on |z| <= 8 and turns over beyond |z| ~ 11: clamp z^2 inside it (tanh is 1 there anyway)
+        const float z2 = fminf(z * z, 64.0f);
+        const float q = fmaf(fmaf(-3.15807042e-4f, z2, 3.67982560e-2f), z2, 7.97717834e-1f);
+        const float t = fast_tanh(z * q);
+        return z * fmaf(0.5f, t, 0.5f);
     }
     if (ACT == D2D_ACT_GELU_TANH) {
-        const float u = 0.79788456080286536f * fmaf(0.044715f * z * z, z, z);
-        const float e2 = __expf(2.0f * u);                 // tanh(u) = 1 - 2 / (e^{2u} + 1)
-        const float th = 1.0f - __fdividef(2.0f, e2 + 1.0f);
-        return 0.5f * z * (1.0f + th);
+        const float q = fmaf(0.79788456080286536f * 0.044715f, z * z, 0.79788456080286536f);
+        const float t = fast_tanh(z * q);
+        return z * fmaf(0.5f, t, 0.5f);
     }
-    return __fdividef(z, 1.0f + __expf(-z));               // SiLU
+    const float t = fast_tanh(0.5f * z);                   // SiLU
+    return z * fmaf(0.5f, t, 0.5f);
 }
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar)
@@ -208,7 +205,7 @@ __device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16
 // 16 accumulator columns -> 16 output values: bias (float32, staged in shared memory), activation, selection mask.
 template <int EPI, int ACT, bool GATED>
 __device__ __forceinline__ void epilogue_16(const uint32_t (&r)[16], const uint32_t (&g)[16], float (&v)[16],
-                                            const float *bias_f, bool has_bias, int col0, uint32_t keep)
+                                            const float *bias_f, bool has_bias, int col0, uint32_t keep, bool halves)
 {
     float bias[16];
     if (has_bias) {
@@ -221,13 +218,24 @@ __device__ __forceinline__ void epilogue_16(const uint32_t (&r)[16], const uint3
 #pragma unroll
         for (int j = 0; j < 16; ++j) bias[j] = 0.0f;
     }
+    if (EPI == D2D_EPI_UP_MASKED && halves) {
+        // each 8-column half belongs to one expert: one predicate per half, one select per element
+        const bool k0 = (keep & 1u) != 0, k1 = (keep & 0x100u) != 0;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const float z = __uint_as_float(r[j]) + bias[j];
+            // first accumulator = up projection (+ bias), second = gate
+            const float h = GATED ? fast_act<ACT>(__uint_as_float(g[j])) * z : fast_act<ACT>(z);
+            v[j] = (j < 8 ? k0 : k1) ? h : 0.0f;
+        }
+        return;
+    }
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
         float z = __uint_as_float(r[j]) + bias[j];
         if (EPI == D2D_EPI_RELU_BF16) z = fmaxf(z, 0.0f);
         if (EPI == D2D_EPI_ABS_F32) z = fabsf(z);
         if (EPI == D2D_EPI_UP_MASKED) {
-            // first accumulator = up projection (+ bias), second = gate
             const float h = GATED ? fast_act<ACT>(__uint_as_float(g[j])) * z : fast_act<ACT>(z);
             z = ((keep >> j) & 1u) ? h : 0.0f;
         }
@@ -461,6 +469,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 lo = e * ep.expert_size - colw;             // first column of expert e relative to the current unit (<= 0)
             }
             const bool bias_fast = ep.bias == nullptr || bias_cached;
+            const bool gran8 = EPI == D2D_EPI_UP_MASKED && mrow != nullptr && (ep.expert_size & 7) == 0;
             uint32_t ra[16], rb[16], ga[16], gb[16];
             tmem_ld16_issue(tbase, ra);
             if (GATED) tmem_ld16_issue(tbase + BN, ga);
@@ -474,34 +483,55 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     break;
                 }
 
-                // selection bits of this row for the 16 columns: one or two experts cover them
+                // selection bits of this row for the 16 columns
                 uint32_t keep = 0xffffu;
                 if (EPI == D2D_EPI_UP_MASKED && mrow) {
                     keep = 0u;
-                    const int s = ep.expert_size;
-                    int ee = e, l = lo;
-                    while (l < 16) {
-                        if ((ee >> 5) != widx) {
-                            widx = ee >> 5;
-                            if (ep.mask_words <= MASK_REGS) {
-                                word = 0u;
+                    if (gran8) {
+                        // expert sizes that are multiples of 8: each 8-column half of the unit belongs to one
+                        // expert; e = col / s by a multiply-high with the precomputed reciprocal
 #pragma unroll
-                                for (int i = 0; i < MASK_REGS; ++i) word = (i == widx) ? mw[i] : word;
+                        for (int h = 0; h < 2; ++h) {
+                            const uint32_t ee = __umulhi((uint32_t)(col0 + 8 * h), ep.inv_expert_size);
+                            const int wi = (int)(ee >> 5);
+                            uint32_t wd;
+                            if (ep.mask_words <= 4) {
+                                wd = wi == 0 ? mw[0] : wi == 1 ? mw[1] : wi == 2 ? mw[2] : mw[3];
+                            } else if (ep.mask_words <= MASK_REGS) {
+                                wd = mw[0];
+#pragma unroll
+                                for (int i = 1; i < MASK_REGS; ++i) wd = (i == wi) ? mw[i] : wd;
                             } else {
-                                word = __ldg(mrow + widx);
+                                wd = __ldg(mrow + wi);
                             }
+                            if ((wd >> (ee & 31)) & 1u) keep |= 0xffu << (8 * h);
                         }
-                        const int hi = l + s;
-                        if ((word >> (ee & 31)) & 1u) {
-                            const int a = l < 0 ? 0 : l, b2 = hi > 16 ? 16 : hi;
-                            keep |= ((1u << b2) - 1u) & ~((1u << a) - 1u);
+                    } else {
+                        const int s = ep.expert_size;
+                        int ee = e, l = lo;
+                        while (l < 16) {
+                            if ((ee >> 5) != widx) {
+                                widx = ee >> 5;
+                                if (ep.mask_words <= MASK_REGS) {
+                                    word = 0u;
+#pragma unroll
+                                    for (int i = 0; i < MASK_REGS; ++i) word = (i == widx) ? mw[i] : word;
+                                } else {
+                                    word = __ldg(mrow + widx);
+                                }
+                            }
+                            const int hi = l + s;
+                            if ((word >> (ee & 31)) & 1u) {
+                                const int a = l < 0 ? 0 : l, b2 = hi > 16 ? 16 : hi;
+                                keep |= ((1u << b2) - 1u) & ~((1u << a) - 1u);
+                            }
+                            l = hi;
+                            ++ee;
                         }
-                        l = hi;
-                        ++ee;
+                        // advance to the expert that owns the first column of the next unit
+                        lo -= 16;
+                        while (lo + s <= 0) { lo += s; ++e; }
                     }
-                    // advance to the expert that owns the first column of the next unit
-                    lo -= 16;
-                    while (lo + s <= 0) { lo += s; ++e; }
                 }
                 tmem_ld_wait();                                               // this unit's accumulators have landed
                 if (u + 1 < N_UNITS) {                                        // the next unit's load overlaps the math below
@@ -511,7 +541,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 
                 if (col0 + 16 <= N && bias_fast && (N & 7) == 0) {
                     float v[16];
-                    epilogue_16<EPI, ACT, GATED>(r, g, v, bias_f, ep.bias != nullptr, col0, keep);
+                    epilogue_16<EPI, ACT, GATED>(r, g, v, bias_f, ep.bias != nullptr, col0, keep, gran8);
                     if (row < M) {
                         if (EPI == D2D_EPI_ABS_F32) {
                             float *o = (float *)ep.out + (size_t)row * N + col0;
@@ -628,7 +658,9 @@ d2d_status launch(const d2d_gemm_args &g, cudaStream_t st)
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM) != cudaSuccess) return D2D_ERR_CUDA;
         attr_set = true;
     }
-    EpiParams ep{(const __nv_bfloat16 *)g.bias, g.out, g.mask, g.mask_words, g.expert_size > 0 ? g.expert_size : 1, g.status};
+    const int es = g.expert_size > 0 ? g.expert_size : 1;
+    EpiParams ep{(const __nv_bfloat16 *)g.bias, g.out, g.mask, g.mask_words, es, g.status,
+                 (uint32_t)((0x100000000ull + (unsigned long long)es - 1) / (unsigned long long)es)};
     const int tiles = d2d_cdiv(g.N, BN) * d2d_cdiv(g.M, PAIR ? 2 * BM : BM);
     const int workers = PAIR ? sm_count() / 2 : sm_count();
     const int grid = (tiles < workers ? tiles : workers) * (PAIR ? 2 : 1);
