@@ -15,7 +15,7 @@
 
 namespace {
 
-constexpr int TBLK = 8;            // tokens processed together
+constexpr int MAX_TBLK = 8;        // at most this many tokens are processed together (template parameter TBLK)
 constexpr int NT = 256;
 
 __device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -52,7 +52,7 @@ __device__ __forceinline__ void lds8(const __nv_bfloat16 *p, float (&o)[8])
 }
 
 // One warp: dot products of a weight row with up to TBLK token rows, all operands in shared memory.
-template <typename TT>
+template <typename TT, int TBLK>
 __device__ __forceinline__ void warp_row_dots(const TT *wrow, const TT *xs, int d, int lane, float (&acc)[TBLK])
 {
 #pragma unroll
@@ -75,7 +75,7 @@ __device__ __forceinline__ void warp_row_dots(const TT *wrow, const TT *xs, int 
 // ------------------------------------------------------------------------------------ router
 
 // dynamic shared memory: [ W_r1 rows of this CTA: 8*d | token block: TBLK*d | W_r2: E*d_h (if staged) | u: T*d_h floats ]
-template <typename TT>
+template <typename TT, int TBLK>
 __global__ void __launch_bounds__(NT)
 small_router_kernel(const TT *__restrict__ x, int T, int d, const TT *__restrict__ w_r1, const TT *__restrict__ b_r1,
                     int d_h, const TT *__restrict__ w_r2, const TT *__restrict__ b_r2, int E, int stage_w2,
@@ -107,7 +107,7 @@ small_router_kernel(const TT *__restrict__ x, int T, int d, const TT *__restrict
         __syncthreads();
         if (warp < rows) {
             float acc[TBLK];
-            warp_row_dots<TT>(w1s + (size_t)warp * d, xs, d, lane, acc);
+            warp_row_dots<TT, TBLK>(w1s + (size_t)warp * d, xs, d, lane, acc);
             if (lane == 0) {
                 const float bj = b_r1 ? d2d_to_float<TT>(b_r1[j0 + warp]) : 0.0f;
 #pragma unroll
@@ -163,7 +163,7 @@ __device__ __forceinline__ void red_add_v4(float *addr, float a, float b, float 
 
 // dynamic shared memory: [ W1 rows: rc*d | W_gate rows: rc*d (gated) | W2T rows: rc*d | token block: TBLK*d | h: TBLK*rc floats ]
 // rc = neurons handled per pass (the whole expert when its slices fit).
-template <typename TT, int ACT, bool GATED>
+template <typename TT, int ACT, bool GATED, int TBLK>
 __global__ void __launch_bounds__(NT)
 small_ffn_kernel(const TT *__restrict__ x, int T, int d, int s, int rc, const TT *__restrict__ w1,
                  const TT *__restrict__ b1, const TT *__restrict__ w_gate, const TT *__restrict__ w2t,
@@ -205,8 +205,8 @@ small_ffn_kernel(const TT *__restrict__ x, int T, int d, int s, int rc, const TT
                 // ---- up projection + activation: one warp per neuron
                 for (int nl = warp; nl < rows; nl += NT / 32) {
                     float up[TBLK], gate[TBLK];
-                    warp_row_dots<TT>(w1s + (size_t)nl * d, xs, d, lane, up);
-                    if (GATED) warp_row_dots<TT>(wgs + (size_t)nl * d, xs, d, lane, gate);
+                    warp_row_dots<TT, TBLK>(w1s + (size_t)nl * d, xs, d, lane, up);
+                    if (GATED) warp_row_dots<TT, TBLK>(wgs + (size_t)nl * d, xs, d, lane, gate);
                     if (lane == 0) {
                         const float bn = b1 ? d2d_to_float<TT>(b1[n0 + nl]) : 0.0f;
 #pragma unroll
@@ -270,27 +270,31 @@ small_ffn_kernel(const TT *__restrict__ x, int T, int d, int s, int rc, const TT
 constexpr size_t kSmemLimit = 200 * 1024;
 
 // neurons per pass so that the slices, one token block and the hidden values fit in shared memory
-int rows_per_pass(const d2d_layer_desc &D, size_t elem)
+int rows_per_pass(const d2d_layer_desc &D, size_t elem, int tb = MAX_TBLK)
 {
     const size_t n_mat = D.gated ? 3 : 2;
-    const size_t fixed = (size_t)TBLK * D.d * elem;
+    const size_t fixed = (size_t)tb * D.d * elem;
     for (int rc = D.expert_size; rc >= 1; rc = (rc + 1) / 2) {
-        const size_t need = n_mat * rc * D.d * elem + fixed + (size_t)TBLK * rc * 4;
+        const size_t need = n_mat * rc * D.d * elem + fixed + (size_t)tb * rc * 4;
         if (need <= kSmemLimit) return rc;
         if (rc == 1) break;
     }
     return 0;
 }
 
-template <typename TT, int ACT, bool GATED>
-d2d_status launch_ffn(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y, float *y32,
-                      unsigned int *ticket, cudaStream_t st)
+// tokens handled together: the smallest of 1, 2, 4, 8 that covers the batch (a token slot that stays empty
+// still costs its share of the dot products)
+int token_block(int T) { return T <= 1 ? 1 : T <= 2 ? 2 : T <= 4 ? 4 : 8; }
+
+template <typename TT, int ACT, bool GATED, int TBLK>
+d2d_status launch_ffn_tb(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y, float *y32,
+                         unsigned int *ticket, cudaStream_t st)
 {
     const d2d_layer_desc &D = L->desc;
-    const int rc = rows_per_pass(D, sizeof(TT));
+    const int rc = rows_per_pass(D, sizeof(TT), TBLK);
     if (rc <= 0) return D2D_ERR_UNSUPPORTED;
     const size_t smem = (size_t)(GATED ? 3 : 2) * rc * D.d * sizeof(TT) + (size_t)TBLK * D.d * sizeof(TT) + (size_t)TBLK * rc * 4;
-    auto kern = small_ffn_kernel<TT, ACT, GATED>;
+    auto kern = small_ffn_kernel<TT, ACT, GATED, TBLK>;
     static size_t attr_smem = 0;
     if (smem > attr_smem) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess) return D2D_ERR_CUDA;
@@ -301,6 +305,18 @@ d2d_status launch_ffn(const d2d_layer *L, const void *x, int T, const d2d_routin
                                         y32, ticket, (TT *)y);
     D2D_LAUNCHED(1);
     return cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
+}
+
+template <typename TT, int ACT, bool GATED>
+d2d_status launch_ffn(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y, float *y32,
+                      unsigned int *ticket, cudaStream_t st)
+{
+    switch (token_block(T)) {
+    case 1: return launch_ffn_tb<TT, ACT, GATED, 1>(L, x, T, r, y, y32, ticket, st);
+    case 2: return launch_ffn_tb<TT, ACT, GATED, 2>(L, x, T, r, y, y32, ticket, st);
+    case 4: return launch_ffn_tb<TT, ACT, GATED, 4>(L, x, T, r, y, y32, ticket, st);
+    default: return launch_ffn_tb<TT, ACT, GATED, 8>(L, x, T, r, y, y32, ticket, st);
+    }
 }
 
 template <typename TT, int ACT>
@@ -323,15 +339,15 @@ d2d_status launch_ffn_dtype(const d2d_layer *L, const void *x, int T, const d2d_
     }
 }
 
-template <typename TT>
-d2d_status launch_router(const d2d_layer *L, const void *x, int T, float *R, float *u, unsigned int *ticket, cudaStream_t st)
+template <typename TT, int TBLK>
+d2d_status launch_router_tb(const d2d_layer *L, const void *x, int T, float *R, float *u, unsigned int *ticket, cudaStream_t st)
 {
     const d2d_layer_desc &D = L->desc;
     const size_t base = (size_t)(8 + TBLK) * D.d * sizeof(TT) + (size_t)T * D.d_h * 4;
     const size_t w2_bytes = (size_t)D.n_experts * D.d_h * sizeof(TT);
     const int stage_w2 = base + w2_bytes <= kSmemLimit ? 1 : 0;
     const size_t smem = base + (stage_w2 ? w2_bytes : 0);
-    auto kern = small_router_kernel<TT>;
+    auto kern = small_router_kernel<TT, TBLK>;
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess) return D2D_ERR_CUDA;
@@ -343,6 +359,17 @@ d2d_status launch_router(const d2d_layer *L, const void *x, int T, float *R, flo
     return cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
 }
 
+template <typename TT>
+d2d_status launch_router(const d2d_layer *L, const void *x, int T, float *R, float *u, unsigned int *ticket, cudaStream_t st)
+{
+    switch (token_block(T)) {
+    case 1: return launch_router_tb<TT, 1>(L, x, T, R, u, ticket, st);
+    case 2: return launch_router_tb<TT, 2>(L, x, T, R, u, ticket, st);
+    case 4: return launch_router_tb<TT, 4>(L, x, T, R, u, ticket, st);
+    default: return launch_router_tb<TT, 8>(L, x, T, R, u, ticket, st);
+    }
+}
+
 }  // namespace
 
 // ws: [ticket (256 bytes) | u: T*d_h floats]
@@ -352,7 +379,7 @@ bool d2d_small_router_supports(const d2d_layer_desc &D, int T)
 {
     const size_t elem = D.dtype == D2D_F32 ? 4 : 2;
     return T >= 1 && T <= 8 && D.d % 8 == 0 && D.d_h % 8 == 0 &&
-           (size_t)(8 + TBLK) * D.d * elem + (size_t)T * D.d_h * 4 <= kSmemLimit;
+           (size_t)(8 + MAX_TBLK) * D.d * elem + (size_t)T * D.d_h * 4 <= kSmemLimit;
 }
 
 d2d_status d2d_small_router(const d2d_layer *L, const void *x, int T, float *R, void *ws, cudaStream_t st)
