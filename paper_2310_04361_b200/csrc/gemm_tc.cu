@@ -387,7 +387,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0 && rank == 0) {
-            const uint32_t idesc = instr_desc_bf16(TM, BN);
+            // Gated (single CTA): the up and gate tiles sit back to back in shared memory, so they are ONE K-major
+            // B operand of 2*BN rows and one MMA fills both accumulators (columns [0,BN) up, [BN,2BN) gate).
+            // Two N=BN instructions would each pay the full A-operand read and run at half the rate.
+            const uint32_t idesc = instr_desc_bf16(TM, (GATED && !PAIR) ? 2 * BN : BN);
             uint32_t it = 0, local = 0;
             bool ok = true;
             for (int tile = worker; tile < total_tiles && ok; tile += n_workers, ++local) {
@@ -414,7 +417,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                             if (GATED) umma_bf16_pair(acc + BN, da + koff, db2 + koff, idesc, accum);
                         } else {
                             umma_bf16(acc, da + koff, db + koff, idesc, accum);
-                            if (GATED) umma_bf16(acc + BN, da + koff, db2 + koff, idesc, accum);
                         }
                     }
                     // stage reusable (in both CTAs of a pair) once these MMAs have read it
@@ -470,17 +472,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             }
             const bool bias_fast = ep.bias == nullptr || bias_cached;
             const bool gran8 = EPI == D2D_EPI_UP_MASKED && mrow != nullptr && (ep.expert_size & 7) == 0;
-            uint32_t ra[16], rb[16], ga[16], gb[16];
-            tmem_ld16_issue(tbase, ra);
-            if (GATED) tmem_ld16_issue(tbase + BN, ga);
+            // Non-gated: the next unit's accumulators are prefetched into a second register set.  Gated tiles need
+            // two accumulators per column; a second set would spill, so each unit is loaded when it is needed and
+            // the other epilogue warps of the SM sub-partition cover the latency.
+            uint32_t ra[16], rb[GATED ? 1 : 16], ga[GATED ? 16 : 1];
+            if (!GATED) tmem_ld16_issue(tbase, ra);
 #pragma unroll
-            for (int u = 0; u < N_UNITS; ++u) {             // at most 4 units; slow paths are out of line to keep the code small
+            for (int u = 0; u < N_UNITS; ++u) {             // at most 4 units
                 const int col0 = colw + u * 16;
-                uint32_t (&r)[16] = (u & 1) ? rb : ra;
-                uint32_t (&g)[16] = (u & 1) ? gb : ga;
+                uint32_t (&r)[16] = GATED ? ra : ((u & 1) ? reinterpret_cast<uint32_t (&)[16]>(rb) : ra);
+                uint32_t (&g)[16] = reinterpret_cast<uint32_t (&)[16]>(ga);
                 if (col0 >= N) {                            // warp-uniform (ragged last column tile)
-                    tmem_ld_wait();
+                    if (!GATED) tmem_ld_wait();
                     break;
+                }
+                if (GATED) {
+                    tmem_ld16_issue(tbase + u * 16, ra);
+                    tmem_ld16_issue(tbase + u * 16 + BN, reinterpret_cast<uint32_t (&)[16]>(ga));
                 }
 
                 // selection bits of this row for the 16 columns
@@ -534,10 +542,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     }
                 }
                 tmem_ld_wait();                                               // this unit's accumulators have landed
-                if (u + 1 < N_UNITS) {                                        // the next unit's load overlaps the math below
-                    tmem_ld16_issue(tbase + (u + 1) * 16, (u & 1) ? ra : rb);
-                    if (GATED) tmem_ld16_issue(tbase + (u + 1) * 16 + BN, (u & 1) ? ga : gb);
-                }
+                if (!GATED && u + 1 < N_UNITS)                                // the next unit's load overlaps the math below
+                    tmem_ld16_issue(tbase + (u + 1) * 16, (u & 1) ? ra : reinterpret_cast<uint32_t (&)[16]>(rb));
 
                 if (col0 + 16 <= N && bias_fast && (N & 7) == 0) {
                     float v[16];
