@@ -73,7 +73,8 @@ size_t d2d_moe_ffn_ws_bytes(const d2d_layer *L, int T)
     if (use_small_ffn(L, T)) need = d2d_small_ffn_ws_bytes(L, T);
     // hidden activations H [T, d_ff] bf16 of the dense-masked path
     if (L->desc.dtype == D2D_BF16 && T >= kDenseMaskedMinTokens) {
-        const size_t h = d2d_align_up((size_t)T * L->desc.d_ff * 2, 256);
+        size_t h = d2d_align_up((size_t)T * L->desc.d_ff * 2, 256);
+        if (d2d_gemm_tc_splits(T, L->desc.d, L->desc.d_ff) > 1) h += d2d_align_up((size_t)T * L->desc.d * 4, 256);   // split-K partial sums
         if (h > need) need = h;
     }
     return need;
@@ -96,6 +97,9 @@ static d2d_status launch_dense_masked(const d2d_layer *L, const void *x, int T, 
     d2d_gemm_args dn = {};
     dn.a = ws; dn.b = L->w2; dn.bias = L->b2; dn.out = y;
     dn.M = T; dn.N = D.d; dn.K = D.d_ff; dn.epilogue = D2D_EPI_BIAS_BF16; dn.status = r->status;
+    // decode-sized batches: split K over the SMs, partial sums in the float32 scratch behind H
+    dn.k_splits = d2d_gemm_tc_splits(T, D.d, D.d_ff);
+    dn.partial = dn.k_splits > 1 ? (float *)((char *)ws + d2d_align_up((size_t)T * D.d_ff * 2, 256)) : nullptr;
     return d2d_gemm_tc(dn, st);
 }
 

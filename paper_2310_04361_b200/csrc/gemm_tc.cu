@@ -260,7 +260,8 @@ __device__ __forceinline__ void epilogue_16_slow(const uint32_t (&r)[16], const 
                 const float h = GATED ? fast_act<ACT>(__uint_as_float(g[j])) * z : fast_act<ACT>(z);
                 z = ((keep >> j) & 1u) ? h : 0.0f;
             }
-            if (EPI == D2D_EPI_ABS_F32) ((float *)out)[(size_t)row * N + col0 + j] = z;
+            if (EPI == D2D_EPI_PARTIAL_F32) atomicAdd((float *)out + (size_t)row * N + col0 + j, z);
+            else if (EPI == D2D_EPI_ABS_F32) ((float *)out)[(size_t)row * N + col0 + j] = z;
             else ((__nv_bfloat16 *)out)[(size_t)row * N + col0 + j] = __float2bfloat16_rn(z);
         }
     }
@@ -283,7 +284,7 @@ __host__ __device__ constexpr int pow2_at_least(int v) { return v <= 32 ? 32 : v
 template <int BN, int STAGES, int EPI, int ACT, bool GATED, bool PAIR>
 __global__ void __launch_bounds__(NTHREADS_V2, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-               const __grid_constant__ CUtensorMap tm_b2, EpiParams ep, int M, int N, int K)
+               const __grid_constant__ CUtensorMap tm_b2, EpiParams ep, int M, int N, int K, int k_splits)
 {
     constexpr int TM = PAIR ? 2 * BM : BM;                // rows of the tile a CTA (pair) computes
     constexpr int B_ROWS = PAIR ? BN / 2 : BN;            // rows of B this CTA stages
@@ -320,7 +321,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nkb = (K + BK - 1) / BK;
     const int n_tiles = (N + BN - 1) / BN;
-    const int total_tiles = ((M + TM - 1) / TM) * n_tiles;
+    // work item = (output tile, K split); with k_splits > 1 every item accumulates a slice of K and the
+    // epilogue adds its partial sums to a float32 buffer (small-M problems that would leave most SMs idle)
+    const int total_tiles = ((M + TM - 1) / TM) * n_tiles * k_splits;
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;           // 0 = the CTA that issues the MMAs
     const int worker = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
     const int n_workers = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
@@ -360,9 +363,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (int tile = worker; tile < total_tiles && ok; tile += n_workers) {
+            for (int item = worker; item < total_tiles && ok; item += n_workers) {
+                const int tile = item / k_splits, sp = item - tile * k_splits;
+                const int kb0 = (int)((long long)sp * nkb / k_splits), kb1 = (int)((long long)(sp + 1) * nkb / k_splits);
                 const int m0 = (tile / n_tiles) * TM + (int)rank * BM, n0 = (tile % n_tiles) * BN + (int)rank * B_ROWS;
-                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                for (int kb = kb0; kb < kb1; ++kb, ++it) {
                     const uint32_t s = it % STAGES, round = it / STAGES;
                     ok = mbar_wait(smem_u32(&bar_empty[s]), (round & 1u) ^ 1u, ep.status);
                     if (!ok) break;
@@ -393,13 +398,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             const uint32_t idesc = instr_desc_bf16(TM, (GATED && !PAIR) ? 2 * BN : BN);
             uint32_t it = 0, local = 0;
             bool ok = true;
-            for (int tile = worker; tile < total_tiles && ok; tile += n_workers, ++local) {
+            for (int item = worker; item < total_tiles && ok; item += n_workers, ++local) {
+                const int sp = item % k_splits;
+                const int kb0 = (int)((long long)sp * nkb / k_splits), kb1 = (int)((long long)(sp + 1) * nkb / k_splits);
                 const uint32_t buf = local & 1u, use = local >> 1;
                 ok = mbar_wait(smem_u32(&bar_acc_empty[buf]), (use & 1u) ^ 1u, ep.status);   // epilogue drained this buffer
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t acc = tmem_base + buf * BUF_COLS;
-                for (int kb = 0; kb < nkb; ++kb, ++it) {
+                for (int kb = kb0; kb < kb1; ++kb, ++it) {
                     const uint32_t s = it % STAGES, round = it / STAGES;
                     ok = mbar_wait(smem_u32(&bar_full[s]), round & 1u, ep.status);
                     if (!ok) break;
@@ -411,7 +418,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
 #pragma unroll
                     for (int k = 0; k < BK / UMMA_K; ++k) {
                         const uint64_t koff = (uint64_t)((k * UMMA_K * 2) >> 4);    // 32 bytes per K step inside the swizzle row
-                        const uint32_t accum = (kb | k) != 0 ? 1u : 0u;
+                        const uint32_t accum = (kb > kb0 || k != 0) ? 1u : 0u;
                         if (PAIR) {
                             umma_bf16_pair(acc, da + koff, db + koff, idesc, accum);
                             if (GATED) umma_bf16_pair(acc + BN, da + koff, db2 + koff, idesc, accum);
@@ -441,7 +448,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         constexpr int N_UNITS = COLS_PER_WARP / 16;
         uint32_t local = 0;
         bool ok = true;
-        for (int tile = worker; tile < total_tiles && ok; tile += n_workers, ++local) {
+        for (int item = worker; item < total_tiles && ok; item += n_workers, ++local) {
+            const int tile = item / k_splits;
             const int m0 = (tile / n_tiles) * TM + (int)rank * BM, n0 = (tile % n_tiles) * BN;
             const uint32_t buf = local & 1u, use = local >> 1;
             const int row = m0 + quad * 32 + lane;
@@ -545,11 +553,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 if (!GATED && u + 1 < N_UNITS)                                // the next unit's load overlaps the math below
                     tmem_ld16_issue(tbase + (u + 1) * 16, (u & 1) ? ra : reinterpret_cast<uint32_t (&)[16]>(rb));
 
-                if (col0 + 16 <= N && bias_fast && (N & 7) == 0) {
+                if (col0 + 16 <= N && bias_fast && (N & 7) == 0) {   // (N % 8 also keeps the 16-byte vector accesses aligned)
                     float v[16];
                     epilogue_16<EPI, ACT, GATED>(r, g, v, bias_f, ep.bias != nullptr, col0, keep, gran8);
                     if (row < M) {
-                        if (EPI == D2D_EPI_ABS_F32) {
+                        if (EPI == D2D_EPI_PARTIAL_F32) {
+                            float *o = (float *)ep.out + (size_t)row * N + col0;
+#pragma unroll
+                            for (int j = 0; j < 16; j += 4)
+                                asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(o + j), "f"(v[j]), "f"(v[j + 1]),
+                                             "f"(v[j + 2]), "f"(v[j + 3]) : "memory");
+                        } else if (EPI == D2D_EPI_ABS_F32) {
                             float *o = (float *)ep.out + (size_t)row * N + col0;
 #pragma unroll
                             for (int j = 0; j < 16; j += 4) *reinterpret_cast<float4 *>(o + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
@@ -667,7 +681,8 @@ d2d_status launch(const d2d_gemm_args &g, cudaStream_t st)
     const int es = g.expert_size > 0 ? g.expert_size : 1;
     EpiParams ep{(const __nv_bfloat16 *)g.bias, g.out, g.mask, g.mask_words, es, g.status,
                  (uint32_t)((0x100000000ull + (unsigned long long)es - 1) / (unsigned long long)es)};
-    const int tiles = d2d_cdiv(g.N, BN) * d2d_cdiv(g.M, PAIR ? 2 * BM : BM);
+    const int k_splits = g.k_splits > 1 ? g.k_splits : 1;
+    const int tiles = d2d_cdiv(g.N, BN) * d2d_cdiv(g.M, PAIR ? 2 * BM : BM) * k_splits;
     const int workers = PAIR ? sm_count() / 2 : sm_count();
     const int grid = (tiles < workers ? tiles : workers) * (PAIR ? 2 : 1);
     cudaLaunchConfig_t cfg = {};
@@ -682,7 +697,7 @@ d2d_status launch(const d2d_gemm_args &g, cudaStream_t st)
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    const cudaError_t err = cudaLaunchKernelEx(&cfg, kern, ta, tb, tb2, ep, g.M, g.N, g.K);
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, kern, ta, tb, tb2, ep, g.M, g.N, g.K, k_splits);
     D2D_LAUNCHED(1);
     return err == cudaSuccess && cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
 }
@@ -761,7 +776,33 @@ d2d_status launch_up(const d2d_gemm_args &g, cudaStream_t st)
 
 }  // namespace
 
+// y = bf16(partial + bias) after a split-K GEMM
+__global__ void __launch_bounds__(256)
+splitk_finalize_kernel(const float *__restrict__ partial, const __nv_bfloat16 *__restrict__ bias, __nv_bfloat16 *__restrict__ out,
+                       int M, int N)
+{
+    const size_t total = (size_t)M * N;
+    for (size_t i = ((size_t)blockIdx.x * 256 + threadIdx.x) * 4; i < total; i += (size_t)gridDim.x * 1024) {
+        const float4 v = __ldcg(reinterpret_cast<const float4 *>(partial + i));
+        const int c = (int)(i % N);
+        const float o[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) out[i + q] = __float2bfloat16_rn(o[q] + (bias ? __bfloat162float(bias[c + q]) : 0.0f));
+    }
+}
+
 bool d2d_gemm_tc_available() { return get_encode() != nullptr; }
+
+int d2d_gemm_tc_splits(int M, int N, int K)
+{
+    // only single-row-tile problems whose column tiles would occupy less than half of the SMs
+    if (M > BM || (N & 3)) return 1;
+    const int tiles = d2d_cdiv(N, 64);
+    const int nkb = d2d_cdiv(K, BK);
+    int splits = sm_count() / (tiles > 0 ? tiles : 1);
+    if (splits > nkb / 2) splits = nkb / 2;          // at least two k-blocks per slice
+    return splits >= 2 ? splits : 1;
+}
 
 d2d_status d2d_gemm_tc(const d2d_gemm_args &g, cudaStream_t st)
 {
@@ -770,7 +811,22 @@ d2d_status d2d_gemm_tc(const d2d_gemm_args &g, cudaStream_t st)
     switch (g.epilogue) {
     case D2D_EPI_RELU_BF16: return launch_bn<D2D_EPI_RELU_BF16, 0, false>(g, st);
     case D2D_EPI_ABS_F32: return launch_bn<D2D_EPI_ABS_F32, 0, false>(g, st);
-    case D2D_EPI_BIAS_BF16: return launch_bn<D2D_EPI_BIAS_BF16, 0, false>(g, st);
+    case D2D_EPI_BIAS_BF16:
+        if (g.k_splits > 1 && g.partial) {
+            if (cudaMemsetAsync(g.partial, 0, (size_t)g.M * g.N * sizeof(float), st) != cudaSuccess) return D2D_ERR_CUDA;
+            d2d_gemm_args p = g;
+            p.epilogue = D2D_EPI_PARTIAL_F32;
+            p.bias = nullptr;
+            p.out = g.partial;
+            const d2d_status rc = launch<64, D2D_EPI_PARTIAL_F32, 0, false, false>(p, st);
+            if (rc != D2D_OK) return rc;
+            const int blocks = d2d_cdiv(g.M * g.N, 1024);
+            splitk_finalize_kernel<<<blocks < 148 ? blocks : 148, 256, 0, st>>>(g.partial, (const __nv_bfloat16 *)g.bias,
+                                                                                 (__nv_bfloat16 *)g.out, g.M, g.N);
+            D2D_LAUNCHED(1);
+            return cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
+        }
+        return launch_bn<D2D_EPI_BIAS_BF16, 0, false>(g, st);
     case D2D_EPI_UP_MASKED: return g.b_gate ? launch_up<true>(g, st) : launch_up<false>(g, st);
     }
     return D2D_ERR_INVALID_ARG;

@@ -11,6 +11,7 @@ enum d2d_gemm_epilogue {
     D2D_EPI_ABS_F32 = 1,     // out f32  = |acc + bias|                     router layer 2
     D2D_EPI_UP_MASKED = 2,   // out bf16 = G[row, col/s] ? A(acc + bias) : 0    expert up projection
     D2D_EPI_BIAS_BF16 = 3,   // out bf16 = acc + bias                       down projection
+    D2D_EPI_PARTIAL_F32 = 4, // out f32 += acc (vector reductions)          one K slice of a split-K GEMM (internal)
 };
 
 struct d2d_gemm_args {
@@ -26,7 +27,15 @@ struct d2d_gemm_args {
     int mask_words;
     int expert_size;         // s: column c belongs to expert c / s
     int32_t *status;         // device status word, receives D2D_ERR_TIMEOUT if a bounded wait runs out
+    // Split-K (D2D_EPI_BIAS_BF16 only): with k_splits > 1 the K range is cut into slices that run as separate work
+    // items, partial sums meet in `partial` (float32 [M, N], cleared by the call), a small kernel adds the bias and
+    // converts.  For problems with so few output tiles that most SMs would idle (decode batches).
+    int k_splits;
+    float *partial;
 };
+
+// Number of K slices d2d_gemm_tc would use for a [M,N,K] down projection (1 = no split) and the float32 scratch it needs.
+int d2d_gemm_tc_splits(int M, int N, int K);
 
 // Enqueues C = epilogue(A B^T).  Requires K % 8 == 0 and 16-byte aligned base pointers.
 d2d_status d2d_gemm_tc(const d2d_gemm_args &g, cudaStream_t st);
