@@ -300,6 +300,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);   // swizzle atoms are 1024-byte aligned
     __shared__ uint64_t bar_full[STAGES], bar_empty[STAGES], bar_acc_full[2], bar_acc_empty[2];
     __shared__ uint32_t tmem_base_holder;
+    __shared__ volatile int epi_ok[2];                               // outcome of the epilogue's accumulator wait (per buffer parity)
     constexpr int MASK_REGS = 16;                                    // selection words of a row kept in registers
     // the whole bias vector is staged once, as float32, behind the operand stages when it fits
     float *bias_f = reinterpret_cast<float *>(smem + (size_t)STAGES * STAGE_BYTES);
@@ -463,9 +464,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     for (int i = 0; i < MASK_REGS; ++i) mw[i] = i < ep.mask_words ? __ldg(mrow + i) : 0u;
                 }
             }
-            int okw = 1;
-            if (lane == 0) okw = mbar_wait(smem_u32(&bar_acc_full[buf]), use & 1u, ep.status) ? 1 : 0;
-            ok = __shfl_sync(0xffffffffu, okw, 0) != 0;
+            // ONE thread polls the accumulator barrier and the other epilogue warps sleep on a hardware barrier: sixteen
+            // pollers measurably slow the producer and MMA threads, whose own barrier tests share the same unit
+            if (ew == 0 && lane == 0) epi_ok[local & 1u] = mbar_wait(smem_u32(&bar_acc_full[buf]), use & 1u, ep.status) ? 1 : 0;
+            asm volatile("bar.sync 1, %0;" ::"r"(N_EPI_WARPS * 32) : "memory");
+            ok = epi_ok[local & 1u] != 0;
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const uint32_t tbase = tmem_base + buf * BUF_COLS + ((uint32_t)(quad * 32) << 16) + (uint32_t)(part * COLS_PER_WARP);
