@@ -84,11 +84,16 @@ size_t d2d_moe_ffn_ws_bytes(const d2d_layer *L, int T)
 // as two dense tensor-core GEMMs; the selection enters as a mask on the hidden activations
 // (h_n of an expert the token did not keep is zeroed in the epilogue), which is exactly
 // y = b2 + sum over kept experts.
+// up_counter (optional): a zeroed device counter; its presence also states that the kernel launched just before
+// on this stream is the router, which writes only the mask (and R, k), so that the up projection's main loops may
+// overlap it and draw their tiles dynamically.
 static d2d_status launch_dense_masked(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y,
-                                      void *ws, cudaStream_t st)
+                                      void *ws, cudaStream_t st, int *up_counter)
 {
     const d2d_layer_desc &D = L->desc;
     d2d_gemm_args up = {};
+    up.tile_counter = up_counter;
+    up.pdl_late_wait = up_counter != nullptr;
     up.a = x; up.b = L->w1; up.b_gate = D.gated ? L->w_gate : nullptr; up.bias = L->b1; up.out = ws;
     up.M = T; up.N = D.d_ff; up.K = D.d; up.epilogue = D2D_EPI_UP_MASKED; up.act = D.act;
     up.mask = r->mask; up.mask_words = (D.n_experts + 31) / 32; up.expert_size = D.expert_size; up.status = r->status;
@@ -104,11 +109,11 @@ static d2d_status launch_dense_masked(const d2d_layer *L, const void *x, int T, 
 }
 
 d2d_status d2d_launch_moe_ffn(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y,
-                              void *ws, size_t ws_bytes, cudaStream_t st)
+                              void *ws, size_t ws_bytes, cudaStream_t st, int *up_counter)
 {
     if (ws_bytes < d2d_moe_ffn_ws_bytes(L, T)) return D2D_ERR_WORKSPACE;
     if (use_small_ffn(L, T)) return d2d_small_ffn(L, x, T, r, y, ws, st);
-    if (use_dense_masked(L, T)) return launch_dense_masked(L, x, T, r, y, ws, st);
+    if (use_dense_masked(L, T)) return launch_dense_masked(L, x, T, r, y, ws, st, up_counter);
     return d2d_launch_moe_ffn_token(L, x, T, r, y, st);
 }
 
@@ -327,9 +332,14 @@ d2d_status d2d_layer_fwd(const d2d_layer *layer, const void *x, int32_t T, float
     if (d2d_router_fused_supports(layer->desc, T)) {
         // router and dynamic-k mask in one kernel; the selection step then only builds the per-expert metadata
         if (cudaMemsetAsync(routing->status, 0, sizeof(int32_t), st) != cudaSuccess) return D2D_ERR_CUDA;
+        const bool dense = use_dense_masked(layer, T) && !use_small_ffn(layer, T);
+        // tile counter of the up projection (the ticket area in front of u is unused on this path), cleared before
+        // the router starts because the up projection may begin while the router is still running
+        int *up_counter = dense ? (int *)(base + w.u_off) : nullptr;
+        if (up_counter && cudaMemsetAsync(up_counter, 0, sizeof(int), st) != cudaSuccess) return D2D_ERR_CUDA;
         rc = d2d_router_fused(layer, x, T, tau, 1, R, routing->mask, routing->k, routing->status, st);
         if (rc != D2D_OK) return rc;
-        if (use_dense_masked(layer, T) && !use_small_ffn(layer, T)) {
+        if (dense) {
             // The dense-masked expert GEMMs read only the mask: build counts / offsets / token lists on the side
             // stream while they run (the small metadata CTAs fit beside the persistent GEMM CTAs), join at the end.
             if (cudaEventRecord(layer->ev_fork, st) != cudaSuccess ||
@@ -337,7 +347,7 @@ d2d_status d2d_layer_fwd(const d2d_layer *layer, const void *x, int32_t T, float
                 return D2D_ERR_CUDA;
             rc = d2d_launch_select(nullptr, T, E, tau, 0, routing, base + w.sel_off, layer->side_stream, 1);
             if (rc != D2D_OK) return rc;
-            rc = d2d_launch_moe_ffn(layer, x, T, routing, y, base + w.ffn_off, w.total - w.ffn_off, st);
+            rc = d2d_launch_moe_ffn(layer, x, T, routing, y, base + w.ffn_off, w.total - w.ffn_off, st, up_counter);
             if (cudaEventRecord(layer->ev_join, layer->side_stream) != cudaSuccess ||
                 cudaStreamWaitEvent(st, layer->ev_join, 0) != cudaSuccess)
                 return D2D_ERR_CUDA;

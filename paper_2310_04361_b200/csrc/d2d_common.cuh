@@ -49,8 +49,9 @@ size_t d2d_select_ws_bytes(int T, int E);
 d2d_status d2d_launch_select(const float *R, int T, int E, float tau, int topk, const d2d_routing *out,
                              void *ws, cudaStream_t st, int mask_ready = 0);
 
+// up_counter: see launch_dense_masked (NULL unless the fused router was launched just before on `st`)
 d2d_status d2d_launch_moe_ffn(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y,
-                              void *ws, size_t ws_bytes, cudaStream_t st);
+                              void *ws, size_t ws_bytes, cudaStream_t st, int *up_counter = nullptr);
 size_t d2d_moe_ffn_ws_bytes(const d2d_layer *L, int T);
 
 // small-batch (T <= 64) kernels

@@ -150,6 +150,8 @@ struct EpiParams {
     int expert_size;
     int32_t *status;
     uint32_t inv_expert_size;        // ceil(2^32 / expert_size): column / expert_size = umulhi(column, inv) for columns < 2^16
+    int *tile_counter;               // device counter (zero at launch) for dynamic tile scheduling, NULL = static round-robin
+    int late_wait;                   // 1: only the epilogue waits for the previous kernel of the stream (see below)
 };
 
 // Activations of the bf16 tensor-core path.  Results are rounded to bf16 (8 bits of mantissa,
@@ -301,6 +303,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     __shared__ uint64_t bar_full[STAGES], bar_empty[STAGES], bar_acc_full[2], bar_acc_empty[2];
     __shared__ uint32_t tmem_base_holder;
     __shared__ volatile int epi_ok[2];                               // outcome of the epilogue's accumulator wait (per buffer parity)
+    // dynamic scheduling: the producer draws work items from a global counter and hands them to the MMA thread and
+    // to the epilogue through a two-slot ring (a CTA that starts late, or gets slow tiles, simply draws fewer)
+    __shared__ uint64_t sched_full[2], sched_empty[2];
+    __shared__ volatile int sched_item[2], epi_item[2];
     constexpr int MASK_REGS = 16;                                    // selection words of a row kept in registers
     // the whole bias vector is staged once, as float32, behind the operand stages when it fits
     float *bias_f = reinterpret_cast<float *>(smem + (size_t)STAGES * STAGE_BYTES);
@@ -337,6 +343,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&bar_acc_full[b]), 1);
             mbar_init(smem_u32(&bar_acc_empty[b]), PAIR ? 2 * N_EPI_WARPS : N_EPI_WARPS);
+            mbar_init(smem_u32(&sched_full[b]), 1);
+            mbar_init(smem_u32(&sched_empty[b]), 2);          // read by the MMA thread and by the epilogue's leader
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -358,13 +366,31 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     if (PAIR) cluster_sync_all();          // the peer's barriers are initialised before anything signals them
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = tmem_base_holder;
+    // Programmatic dependent launch: everything above (barriers, TMEM, the bias vector: parameters, not activations)
+    // may run while the previous kernel of the stream drains; nothing below starts before that kernel has completed
+    // and its writes are visible.  The next kernel of the stream may be scheduled onto SMs as this grid frees them.
+    // With late_wait only the epilogue depends on that kernel (the selection mask written by the router): the
+    // operand loads and the MMAs of the first tiles then overlap it, and only the epilogue warps wait.
+    const bool dyn = !PAIR && ep.tile_counter != nullptr;
+    if (!ep.late_wait || warp >= 2) asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            for (int item = worker; item < total_tiles && ok; item += n_workers) {
+            for (uint32_t local = 0; ok; ++local) {
+                int item = worker + (int)local * n_workers;
+                if (dyn) {
+                    const uint32_t sl = local & 1u, use = local >> 1;
+                    ok = mbar_wait(smem_u32(&sched_empty[sl]), (use & 1u) ^ 1u, ep.status);
+                    if (!ok) break;
+                    item = atomicAdd(ep.tile_counter, 1);
+                    sched_item[sl] = item < total_tiles ? item : -1;
+                    mbar_arrive(smem_u32(&sched_full[sl]));       // release: the slot's content is visible to whoever sees the phase
+                }
+                if (item >= total_tiles) break;
                 const int tile = item / k_splits, sp = item - tile * k_splits;
                 const int kb0 = (int)((long long)sp * nkb / k_splits), kb1 = (int)((long long)(sp + 1) * nkb / k_splits);
                 const int m0 = (tile / n_tiles) * TM + (int)rank * BM, n0 = (tile % n_tiles) * BN + (int)rank * B_ROWS;
@@ -399,7 +425,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             const uint32_t idesc = instr_desc_bf16(TM, (GATED && !PAIR) ? 2 * BN : BN);
             uint32_t it = 0, local = 0;
             bool ok = true;
-            for (int item = worker; item < total_tiles && ok; item += n_workers, ++local) {
+            for (;; ++local) {
+                int item = worker + (int)local * n_workers;
+                if (dyn) {
+                    const uint32_t sl = local & 1u, su = local >> 1;
+                    ok = mbar_wait(smem_u32(&sched_full[sl]), su & 1u, ep.status);
+                    if (!ok) break;
+                    item = sched_item[sl];
+                    mbar_arrive(smem_u32(&sched_empty[sl]));
+                    if (item < 0) break;
+                }
+                if (item >= total_tiles) break;
                 const int sp = item % k_splits;
                 const int kb0 = (int)((long long)sp * nkb / k_splits), kb1 = (int)((long long)(sp + 1) * nkb / k_splits);
                 const uint32_t buf = local & 1u, use = local >> 1;
@@ -431,6 +467,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     if (PAIR) umma_commit_pair(smem_u32(&bar_empty[s]));
                     else umma_commit(smem_u32(&bar_empty[s]));
                 }
+                if (!ok) break;
                 // accumulator of this tile complete (each CTA of a pair holds its own 128 rows)
                 if (PAIR) umma_commit_pair(smem_u32(&bar_acc_full[buf]));
                 else umma_commit(smem_u32(&bar_acc_full[buf]));
@@ -449,10 +486,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         constexpr int N_UNITS = COLS_PER_WARP / 16;
         uint32_t local = 0;
         bool ok = true;
-        for (int item = worker; item < total_tiles && ok; item += n_workers, ++local) {
+        for (;; ++local) {
+            const uint32_t buf = local & 1u, use = local >> 1;
+            int item = worker + (int)local * n_workers;
+            if (dyn) {
+                // the leader takes the item from the ring and publishes it to the sixteen warps
+                if (ew == 0 && lane == 0) {
+                    int got = -2;                            // -2: the wait ran out
+                    if (mbar_wait(smem_u32(&sched_full[buf]), use & 1u, ep.status)) {
+                        got = sched_item[buf];
+                        mbar_arrive(smem_u32(&sched_empty[buf]));
+                    }
+                    epi_item[buf] = got;
+                }
+                asm volatile("bar.sync 1, %0;" ::"r"(N_EPI_WARPS * 32) : "memory");
+                item = epi_item[buf];
+                if (item < 0) break;
+            }
+            if (item >= total_tiles) break;
             const int tile = item / k_splits;
             const int m0 = (tile / n_tiles) * TM + (int)rank * BM, n0 = (tile % n_tiles) * BN;
-            const uint32_t buf = local & 1u, use = local >> 1;
             const int row = m0 + quad * 32 + lane;
             // this row's selection words go to registers before the wait, so their latency is hidden
             uint32_t mw[MASK_REGS];
@@ -599,6 +652,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 if (PAIR) mbar_arrive_cluster(map_to_cta(smem_u32(&bar_acc_empty[buf]), 0));   // the leader waits for both CTAs
                 else mbar_arrive(smem_u32(&bar_acc_empty[buf]));
             }
+
         }
     }
 
@@ -661,6 +715,8 @@ int sm_count()
     return g_sm_count;
 }
 
+bool pdl_enabled();
+
 template <int BN, int EPI, int ACT, bool GATED, bool PAIR>
 d2d_status launch(const d2d_gemm_args &g, cudaStream_t st)
 {
@@ -683,7 +739,8 @@ d2d_status launch(const d2d_gemm_args &g, cudaStream_t st)
     }
     const int es = g.expert_size > 0 ? g.expert_size : 1;
     EpiParams ep{(const __nv_bfloat16 *)g.bias, g.out, g.mask, g.mask_words, es, g.status,
-                 (uint32_t)((0x100000000ull + (unsigned long long)es - 1) / (unsigned long long)es)};
+                 (uint32_t)((0x100000000ull + (unsigned long long)es - 1) / (unsigned long long)es),
+                 PAIR ? nullptr : g.tile_counter, (g.pdl_late_wait && pdl_enabled()) ? 1 : 0};
     const int k_splits = g.k_splits > 1 ? g.k_splits : 1;
     const int tiles = d2d_cdiv(g.N, BN) * d2d_cdiv(g.M, PAIR ? 2 * BM : BM) * k_splits;
     const int workers = PAIR ? sm_count() / 2 : sm_count();
@@ -693,13 +750,16 @@ d2d_status launch(const d2d_gemm_args &g, cudaStream_t st)
     cfg.blockDim = dim3(NTHREADS_V2, 1, 1);
     cfg.dynamicSmemBytes = SMEM;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = PAIR ? 2 : 1;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    // the kernel's prologue may overlap the tail of the previous kernel in the stream (see griddepcontrol.wait in the kernel)
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = pdl_enabled() ? 2 : 1;
     const cudaError_t err = cudaLaunchKernelEx(&cfg, kern, ta, tb, tb2, ep, g.M, g.N, g.K, k_splits);
     D2D_LAUNCHED(1);
     return err == cudaSuccess && cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
@@ -721,6 +781,15 @@ int pick_bn(int M, int N, int tile_m, int workers, const int *cands, int n_cands
     }
     if (eff_out) *eff_out = best_eff;
     return best;
+}
+
+bool pdl_enabled()
+{
+    static const bool on = [] {
+        const char *e = getenv("D2D_GEMM_PDL");            // D2D_GEMM_PDL=0 launches every GEMM fully serialised
+        return !(e && e[0] == '0');
+    }();
+    return on;
 }
 
 bool pair_mode_enabled()

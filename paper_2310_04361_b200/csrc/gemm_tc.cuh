@@ -32,6 +32,13 @@ struct d2d_gemm_args {
     // converts.  For problems with so few output tiles that most SMs would idle (decode batches).
     int k_splits;
     float *partial;
+    // Dynamic tile scheduling: a device counter that is ZERO when the kernel starts (the caller clears it); CTAs draw
+    // work items from it instead of walking a fixed round-robin list.  NULL = static schedule.
+    int *tile_counter;
+    // 1: A, B and the bias do NOT depend on the previous kernel of the stream, only the epilogue inputs (the selection
+    // mask) do.  With programmatic dependent launch the main loops then start while that kernel still runs and only the
+    // epilogue waits for it.  Never set this when A may be written by the preceding kernel.
+    int pdl_late_wait;
 };
 
 // Number of K slices d2d_gemm_tc would use for a [M,N,K] down projection (1 = no split) and the float32 scratch it needs.

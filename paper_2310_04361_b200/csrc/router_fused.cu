@@ -151,6 +151,9 @@ router_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_const
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = tmem_base_holder;
     const uint32_t tmem_r = tmem_base + 256;
+    // the expert up projection that follows on the stream may start its operand loads and MMAs on the SMs this
+    // grid leaves idle (T / 128 CTAs); its epilogue waits for this kernel to complete before it reads the mask
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
