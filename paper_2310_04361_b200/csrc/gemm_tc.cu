@@ -535,6 +535,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 lo = e * ep.expert_size - colw;             // first column of expert e relative to the current unit (<= 0)
             }
             const bool bias_fast = ep.bias == nullptr || bias_cached;
+            const bool wide_store = (N & 15) == 0 && (reinterpret_cast<uintptr_t>(ep.out) & 31) == 0;   // 32-byte aligned rows
             const bool gran8 = EPI == D2D_EPI_UP_MASKED && mrow != nullptr && (ep.expert_size & 7) == 0;
             // Non-gated: the next unit's accumulators are prefetched into a second register set.  Gated tiles need
             // two accumulators per column; a second set would spill, so each unit is loaded when it is needed and
@@ -625,18 +626,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                             for (int j = 0; j < 16; j += 4) *reinterpret_cast<float4 *>(o + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
                         } else {
                             __nv_bfloat16 *o = (__nv_bfloat16 *)ep.out + (size_t)row * N + col0;
+                            uint32_t pk[8];
 #pragma unroll
-                            for (int j = 0; j < 16; j += 8) {
-                                uint4 pk;
-                                __nv_bfloat162 t0 = __floats2bfloat162_rn(v[j], v[j + 1]);
-                                __nv_bfloat162 t1 = __floats2bfloat162_rn(v[j + 2], v[j + 3]);
-                                __nv_bfloat162 t2 = __floats2bfloat162_rn(v[j + 4], v[j + 5]);
-                                __nv_bfloat162 t3 = __floats2bfloat162_rn(v[j + 6], v[j + 7]);
-                                pk.x = *reinterpret_cast<uint32_t *>(&t0);
-                                pk.y = *reinterpret_cast<uint32_t *>(&t1);
-                                pk.z = *reinterpret_cast<uint32_t *>(&t2);
-                                pk.w = *reinterpret_cast<uint32_t *>(&t3);
-                                *reinterpret_cast<uint4 *>(o + j) = pk;
+                            for (int j = 0; j < 8; ++j) {
+                                __nv_bfloat162 t = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+                                pk[j] = *reinterpret_cast<uint32_t *>(&t);
+                            }
+                            if (wide_store) {
+                                // one 32-byte store per row and unit: a whole sector per lane, half as many store instructions
+                                asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(o), "r"(pk[0]), "r"(pk[1]),
+                                             "r"(pk[2]), "r"(pk[3]), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]), "r"(pk[7]) : "memory");
+                            } else {
+                                *reinterpret_cast<uint4 *>(o) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                                *reinterpret_cast<uint4 *>(o + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
                             }
                         }
                     }
