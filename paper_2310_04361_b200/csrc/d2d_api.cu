@@ -52,7 +52,7 @@ ws_layout layout_for(const d2d_layer *L, int T)
 
 // Tokens from which the dense tensor-core path (masked hidden activations, two GEMMs) is used
 // instead of the token-major CUDA-core kernel.
-static const int kDenseMaskedMinTokens = 17;
+static const int kDenseMaskedMinTokens = 9;
 
 static bool use_dense_masked(const d2d_layer *L, int T)
 {
@@ -60,7 +60,7 @@ static bool use_dense_masked(const d2d_layer *L, int T)
 }
 
 // Up to this many tokens the expert-per-CTA kernel (each kept expert's slice read once) is used.
-static const int kSmallFfnMaxTokens = 16;
+static const int kSmallFfnMaxTokens = 8;
 
 static bool use_small_ffn(const d2d_layer *L, int T)
 {
@@ -109,10 +109,10 @@ static d2d_status launch_dense_masked(const d2d_layer *L, const void *x, int T, 
 }
 
 d2d_status d2d_launch_moe_ffn(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y,
-                              void *ws, size_t ws_bytes, cudaStream_t st, int *up_counter)
+                              void *ws, size_t ws_bytes, cudaStream_t st, int *up_counter, int small_fused)
 {
     if (ws_bytes < d2d_moe_ffn_ws_bytes(L, T)) return D2D_ERR_WORKSPACE;
-    if (use_small_ffn(L, T)) return d2d_small_ffn(L, x, T, r, y, ws, st);
+    if (use_small_ffn(L, T)) return d2d_small_ffn(L, x, T, r, y, ws, st, small_fused);
     if (use_dense_masked(L, T)) return launch_dense_masked(L, x, T, r, y, ws, st, up_counter);
     return d2d_launch_moe_ffn_token(L, x, T, r, y, st);
 }
@@ -171,7 +171,7 @@ d2d_status d2d_layer_create(const d2d_layer_desc *desc, const d2d_weights *w, vo
         {&L->w_gate, w->w_gate, n_w, false}, {&L->w2t, w->w2, n_w, true},
         {&L->b2, w->b2, (size_t)D.d, false}, {&L->w2, w->w2, n_w, false},
     };
-    size_t total = 0;
+    size_t total = 256;                                   // the ticket words (see d2d_layer::tickets)
     for (const piece &p : pieces)
         if (p.src) total += d2d_align_up(p.n * el, 256);
     cudaStream_t st = (cudaStream_t)stream;
@@ -180,10 +180,11 @@ d2d_status d2d_layer_create(const d2d_layer_desc *desc, const d2d_weights *w, vo
         return D2D_ERR_CUDA;
     }
     L->slab_bytes = total;
-    size_t off = 0;
-    d2d_status rc = D2D_OK;
+    L->tickets = (unsigned int *)L->slab;
+    size_t off = 256;
+    d2d_status rc = cudaMemsetAsync(L->tickets, 0, 256, st) == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
     for (const piece &p : pieces) {
-        if (!p.src) continue;
+        if (!p.src || rc != D2D_OK) continue;
         void *dst = (char *)L->slab + off;
         off += d2d_align_up(p.n * el, 256);
         *p.dst = dst;
@@ -354,6 +355,14 @@ d2d_status d2d_layer_fwd(const d2d_layer *layer, const void *x, int32_t T, float
             return rc;
         }
         rc = d2d_launch_select(nullptr, T, E, tau, 0, routing, base + w.sel_off, st, 1);
+    } else if (d2d_small_router_supports(layer->desc, T)) {
+        // decode batches: the router kernel's last CTA selects as well (one launch for router + selection)
+        const bool small = use_small_ffn(layer, T);
+        float *y32 = (float *)(base + w.ffn_off + 256);
+        rc = d2d_small_router(layer, x, T, R, base + w.u_off, st, routing, tau, 1, small ? y32 : nullptr,
+                              small ? T * layer->desc.d : 0);
+        if (rc != D2D_OK) return rc;
+        return d2d_launch_moe_ffn(layer, x, T, routing, y, base + w.ffn_off, w.total - w.ffn_off, st, nullptr, small ? 1 : 0);
     } else {
         rc = d2d_launch_router(layer, x, T, R, (float *)(base + w.u_off), st);
         if (rc != D2D_OK) return rc;

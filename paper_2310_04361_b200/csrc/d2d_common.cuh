@@ -24,6 +24,10 @@ struct d2d_layer {
     // expert GEMMs, which do not read it
     cudaStream_t side_stream;
     cudaEvent_t ev_fork, ev_join;
+    // layer-owned "last CTA" tickets of the decode kernels used by d2d_layer_fwd (zero at creation, reset by the kernel
+    // that used them): word 0 router, word 16 experts.  Like the side stream, they make concurrent d2d_layer_fwd calls on
+    // ONE layer object from several streams unsafe; use one layer object per stream for that.
+    unsigned int *tickets;
 };
 
 #define D2D_CUDA_TRY(expr)                                   \
@@ -51,7 +55,7 @@ d2d_status d2d_launch_select(const float *R, int T, int E, float tau, int topk, 
 
 // up_counter: see launch_dense_masked (NULL unless the fused router was launched just before on `st`)
 d2d_status d2d_launch_moe_ffn(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y,
-                              void *ws, size_t ws_bytes, cudaStream_t st, int *up_counter = nullptr);
+                              void *ws, size_t ws_bytes, cudaStream_t st, int *up_counter = nullptr, int small_fused = 0);
 size_t d2d_moe_ffn_ws_bytes(const d2d_layer *L, int T);
 
 // small-batch (T <= 64) kernels
@@ -63,10 +67,17 @@ d2d_status d2d_router_fused(const d2d_layer *L, const void *x, int T, float tau,
                             int32_t *k, int32_t *status, cudaStream_t st);
 bool d2d_small_router_supports(const d2d_layer_desc &D, int T);
 size_t d2d_small_router_ws_bytes(const d2d_layer *L, int T);
-d2d_status d2d_small_router(const d2d_layer *L, const void *x, int T, float *R, void *ws, cudaStream_t st);
+// select_into != NULL: the kernel's last CTA also performs the dynamic-k selection (threshold tau) and writes the routing
+// fused != 0 (d2d_layer_fwd): the layer-owned ticket is used (no memset node) and the kernel also clears `zero_words`
+// floats at `zero` (the experts' float32 accumulator), so that the expert kernel needs no memset either
+d2d_status d2d_small_router(const d2d_layer *L, const void *x, int T, float *R, void *ws, cudaStream_t st,
+                            const d2d_routing *select_into = nullptr, float tau = 0.0f, int fused = 0,
+                            float *zero = nullptr, int zero_words = 0);
 bool d2d_small_ffn_supports(const d2d_layer_desc &D);
 size_t d2d_small_ffn_ws_bytes(const d2d_layer *L, int T);
-d2d_status d2d_small_ffn(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y, void *ws, cudaStream_t st);
+// fused != 0: the accumulator in ws was cleared by the router kernel and the layer-owned ticket is used
+d2d_status d2d_small_ffn(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y, void *ws, cudaStream_t st,
+                         int fused = 0);
 
 d2d_status d2d_launch_transpose(const void *src, void *dst, int rows, int cols, size_t elem, cudaStream_t st);
 

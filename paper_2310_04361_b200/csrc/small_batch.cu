@@ -6,16 +6,12 @@
 //                         per-expert counts, offsets, token lists (and the token-major dual)
 // The router and expert kernels of this path are in small_batch_ffn.cu.
 #include "d2d_common.cuh"
+#include "small_select.cuh"
 
 namespace {
 
-constexpr unsigned FULL = 0xffffffffu;
-
-__device__ __forceinline__ bool finite_f32(float v) { return (__float_as_uint(v) & 0x7f800000u) != 0x7f800000u; }
-
 // ------------------------------------------------------------------------------------ selection
 
-// R == nullptr: the mask words are an input (override protocol), otherwise they are computed.
 __global__ void __launch_bounds__(1024)
 small_select_kernel(const float *__restrict__ R, int T, int E, int W, float tau,
                     uint32_t *__restrict__ mask, int32_t *__restrict__ k, int32_t *__restrict__ counts,
@@ -24,116 +20,8 @@ small_select_kernel(const float *__restrict__ R, int T, int E, int W, float tau,
                     long long capacity, int keep_status)
 {
     extern __shared__ uint32_t smask[];          // [T][W]
-    __shared__ int warp_sums[32];
-    __shared__ int chunk_total;
-    __shared__ int sk[64];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (threadIdx.x == 0 && !keep_status) *status = 0;
-    __syncthreads();
-
-    for (int t = warp; t < T; t += 32) {
-        int kt = 0;
-        if (R) {
-            const float *row = R + (size_t)t * E;
-            float m = -INFINITY;
-            bool bad = false;
-            for (int i = lane; i < E; i += 32) {
-                const float v = __ldg(row + i);
-                bad |= !finite_f32(v);
-                m = v > m ? v : m;
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                const float other = __shfl_xor_sync(FULL, m, o);
-                m = other > m ? other : m;
-            }
-            bad = __any_sync(FULL, bad);
-            const float thr = __fmul_rn(tau, m);
-            for (int w = 0; w < W; ++w) {
-                const int i = w * 32 + lane;
-                const bool keep = (i < E) && (bad || __ldg(row + i) >= thr);
-                const uint32_t word = __ballot_sync(FULL, keep);
-                if (lane == 0) { mask[(size_t)t * W + w] = word; smask[t * W + w] = word; }
-                kt += __popc(word);
-            }
-            if (lane == 0 && bad) atomicMax(status, (int32_t)D2D_ERR_NONFINITE);
-        } else {
-            for (int w = lane; w < W; w += 32) {
-                const uint32_t word = mask[(size_t)t * W + w];
-                smask[t * W + w] = word;
-                kt += __popc(word);
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) kt += __shfl_xor_sync(FULL, kt, o);
-        }
-        if (lane == 0) { k[t] = kt; sk[t] = kt; }
-    }
-    __syncthreads();
-
-    // per-expert counts and the exclusive scan over experts (chunks of 1024 experts)
-    int carry = 0;
-    for (int e0 = 0; e0 < E; e0 += 1024) {
-        const int e = e0 + threadIdx.x;
-        int c = 0;
-        if (e < E)
-            for (int t = 0; t < T; ++t) c += (smask[t * W + (e >> 5)] >> (e & 31)) & 1u;
-        // block-wide exclusive scan of c
-        int inc = c;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int n = __shfl_up_sync(FULL, inc, o);
-            if (lane >= o) inc += n;
-        }
-        if (lane == 31) warp_sums[warp] = inc;
-        __syncthreads();
-        if (warp == 0) {
-            const int ws = warp_sums[lane];
-            int winc = ws;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int n = __shfl_up_sync(FULL, winc, o);
-                if (lane >= o) winc += n;
-            }
-            warp_sums[lane] = winc - ws;
-            if (lane == 31) chunk_total = winc;
-        }
-        __syncthreads();
-        const int off = carry + warp_sums[warp] + inc - c;
-        if (e < E) {
-            counts[e] = c;
-            offsets[e] = off;
-            long long idx = off;
-            for (int t = 0; t < T; ++t)
-                if ((smask[t * W + (e >> 5)] >> (e & 31)) & 1u) {
-                    if (idx < capacity) perm[idx] = t;
-                    ++idx;
-                }
-        }
-        carry += chunk_total;
-        __syncthreads();
-    }
-    if (threadIdx.x == 0) {
-        offsets[E] = carry;
-        *n_sel = carry;
-        if ((long long)carry > capacity) atomicMax(status, (int32_t)D2D_ERR_CAPACITY);
-    }
-    // token-major dual: T <= 64, one thread per token
-    if (tok_off && tok_exp && threadIdx.x < T) {
-        const int t = threadIdx.x;
-        long long base = 0;
-        for (int u = 0; u < t; ++u) base += sk[u];
-        tok_off[t] = (int32_t)base;
-        if (t == T - 1) tok_off[T] = (int32_t)(base + sk[t]);
-        for (int w = 0; w < W; ++w) {
-            uint32_t word = smask[t * W + w];
-            while (word) {
-                const int b = __ffs(word) - 1;
-                word &= word - 1;
-                if (base < capacity) tok_exp[base] = w * 32 + b;
-                ++base;
-            }
-        }
-    }
+    d2d_small::select_cta(R, T, E, W, tau, mask, k, counts, offsets, perm, tok_off, tok_exp, n_sel, status, capacity,
+                          keep_status, smask);
 }
 
 }  // namespace

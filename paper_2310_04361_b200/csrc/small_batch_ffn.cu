@@ -6,12 +6,14 @@
 //
 //   small_router_kernel   CTA b owns 8 hidden units: its 8 rows of W_r1 and all token rows go to
 //                         shared memory, one warp per unit forms u[t, j]; every CTA also prefetches
-//                         W_r2, and the CTA that finishes last (ticket) computes layer 2 from it
+//                         W_r2, and the CTA that finishes last (ticket) computes layer 2 from it and,
+//                         when asked to, the dynamic-k selection and its metadata as well (no second launch)
 //   small_ffn_kernel      one CTA per expert: its W1 / W_gate / W2 slices are read from HBM exactly
 //                         once (only experts some token kept do any work), the expert's tokens are
 //                         handled 8 at a time, partial output rows go to a float32 accumulator with
 //                         16-byte vector reductions; the last CTA adds b2 and writes y
 #include "d2d_common.cuh"
+#include "small_select.cuh"
 
 namespace {
 
@@ -74,13 +76,26 @@ __device__ __forceinline__ void warp_row_dots(const TT *wrow, const TT *xs, int 
 
 // ------------------------------------------------------------------------------------ router
 
-// dynamic shared memory: [ W_r1 rows of this CTA: 8*d | token block: TBLK*d | W_r2: E*d_h (if staged) | u: T*d_h floats ]
+// Outputs of the selection the router's last CTA may perform (enabled == 0: scores only).
+struct SmallSel {
+    int enabled;
+    float tau;
+    uint32_t *mask;
+    int32_t *k, *counts, *offsets, *perm, *tok_off, *tok_exp, *n_sel, *status;
+    long long capacity;
+};
+
+// dynamic shared memory: [ W_r1 rows of this CTA: 8*d | token block: TBLK*d | W_r2: E*d_h (if staged) | u: T*d_h floats |
+//                          selection words: T*ceil(E/32) ]
 template <typename TT, int TBLK>
 __global__ void __launch_bounds__(NT)
 small_router_kernel(const TT *__restrict__ x, int T, int d, const TT *__restrict__ w_r1, const TT *__restrict__ b_r1,
                     int d_h, const TT *__restrict__ w_r2, const TT *__restrict__ b_r2, int E, int stage_w2,
-                    float *__restrict__ u, float *__restrict__ R, unsigned int *__restrict__ ticket)
+                    float *__restrict__ u, float *R, unsigned int *__restrict__ ticket, SmallSel sel, float *__restrict__ zero,
+                    int zero_words)
 {
+    // clear the float32 accumulator of the expert kernel that follows on the stream (saves a memset node)
+    for (int i = blockIdx.x * NT + threadIdx.x; i < zero_words; i += gridDim.x * NT) zero[i] = 0.0f;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     TT *w1s = reinterpret_cast<TT *>(smem_raw);
     TT *xs = w1s + (size_t)8 * d;
@@ -151,6 +166,13 @@ small_router_kernel(const TT *__restrict__ x, int T, int d, const TT *__restrict
             for (int q = 0; q < TBLK; ++q)
                 if (t0 + q < T) R[(size_t)(t0 + q) * E + i] = fabsf(acc[q] + bi);
         }
+    }
+    if (sel.enabled) {
+        // the scores of all T <= 8 tokens were written by this CTA: select from them right here
+        __syncthreads();
+        uint32_t *smask = reinterpret_cast<uint32_t *>(us + (size_t)T * d_h);
+        d2d_small::select_cta(R, T, E, (E + 31) / 32, sel.tau, sel.mask, sel.k, sel.counts, sel.offsets, sel.perm, sel.tok_off,
+                              sel.tok_exp, sel.n_sel, sel.status, sel.capacity, 0, smask);
     }
 }
 
@@ -340,10 +362,11 @@ d2d_status launch_ffn_dtype(const d2d_layer *L, const void *x, int T, const d2d_
 }
 
 template <typename TT, int TBLK>
-d2d_status launch_router_tb(const d2d_layer *L, const void *x, int T, float *R, float *u, unsigned int *ticket, cudaStream_t st)
+d2d_status launch_router_tb(const d2d_layer *L, const void *x, int T, float *R, float *u, unsigned int *ticket, cudaStream_t st,
+                            const SmallSel &sel, float *zero, int zero_words)
 {
     const d2d_layer_desc &D = L->desc;
-    const size_t base = (size_t)(8 + TBLK) * D.d * sizeof(TT) + (size_t)T * D.d_h * 4;
+    const size_t base = (size_t)(8 + TBLK) * D.d * sizeof(TT) + (size_t)T * D.d_h * 4 + (size_t)T * ((D.n_experts + 31) / 32) * 4;
     const size_t w2_bytes = (size_t)D.n_experts * D.d_h * sizeof(TT);
     const int stage_w2 = base + w2_bytes <= kSmemLimit ? 1 : 0;
     const size_t smem = base + (stage_w2 ? w2_bytes : 0);
@@ -354,19 +377,20 @@ d2d_status launch_router_tb(const d2d_layer *L, const void *x, int T, float *R, 
         attr_set = true;
     }
     kern<<<d2d_cdiv(D.d_h, 8), NT, smem, st>>>((const TT *)x, T, D.d, (const TT *)L->w_r1, (const TT *)L->b_r1, D.d_h,
-                                                (const TT *)L->w_r2, (const TT *)L->b_r2, D.n_experts, stage_w2, u, R, ticket);
+                                                (const TT *)L->w_r2, (const TT *)L->b_r2, D.n_experts, stage_w2, u, R, ticket, sel, zero, zero_words);
     D2D_LAUNCHED(1);
     return cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
 }
 
 template <typename TT>
-d2d_status launch_router(const d2d_layer *L, const void *x, int T, float *R, float *u, unsigned int *ticket, cudaStream_t st)
+d2d_status launch_router(const d2d_layer *L, const void *x, int T, float *R, float *u, unsigned int *ticket, cudaStream_t st,
+                         const SmallSel &sel, float *zero, int zero_words)
 {
     switch (token_block(T)) {
-    case 1: return launch_router_tb<TT, 1>(L, x, T, R, u, ticket, st);
-    case 2: return launch_router_tb<TT, 2>(L, x, T, R, u, ticket, st);
-    case 4: return launch_router_tb<TT, 4>(L, x, T, R, u, ticket, st);
-    default: return launch_router_tb<TT, 8>(L, x, T, R, u, ticket, st);
+    case 1: return launch_router_tb<TT, 1>(L, x, T, R, u, ticket, st, sel, zero, zero_words);
+    case 2: return launch_router_tb<TT, 2>(L, x, T, R, u, ticket, st, sel, zero, zero_words);
+    case 4: return launch_router_tb<TT, 4>(L, x, T, R, u, ticket, st, sel, zero, zero_words);
+    default: return launch_router_tb<TT, 8>(L, x, T, R, u, ticket, st, sel, zero, zero_words);
     }
 }
 
@@ -379,16 +403,26 @@ bool d2d_small_router_supports(const d2d_layer_desc &D, int T)
 {
     const size_t elem = D.dtype == D2D_F32 ? 4 : 2;
     return T >= 1 && T <= 8 && D.d % 8 == 0 && D.d_h % 8 == 0 &&
-           (size_t)(8 + MAX_TBLK) * D.d * elem + (size_t)T * D.d_h * 4 <= kSmemLimit;
+           (size_t)(8 + MAX_TBLK) * D.d * elem + (size_t)T * D.d_h * 4 + (size_t)T * ((D.n_experts + 31) / 32) * 4 <= kSmemLimit;
 }
 
-d2d_status d2d_small_router(const d2d_layer *L, const void *x, int T, float *R, void *ws, cudaStream_t st)
+d2d_status d2d_small_router(const d2d_layer *L, const void *x, int T, float *R, void *ws, cudaStream_t st,
+                            const d2d_routing *select_into, float tau, int fused, float *zero, int zero_words)
 {
-    unsigned int *ticket = (unsigned int *)ws;
+    unsigned int *ticket = fused ? L->tickets : (unsigned int *)ws;
     float *u = (float *)((char *)ws + 256);
-    D2D_CUDA_TRY(cudaMemsetAsync(ticket, 0, sizeof(unsigned int), st));
-    if (L->desc.dtype == D2D_F32) return launch_router<float>(L, x, T, R, u, ticket, st);
-    return launch_router<__nv_bfloat16>(L, x, T, R, u, ticket, st);
+    if (!fused) D2D_CUDA_TRY(cudaMemsetAsync(ticket, 0, sizeof(unsigned int), st));
+    SmallSel sel = {};
+    if (select_into) {
+        sel.enabled = 1;
+        sel.tau = tau;
+        sel.mask = select_into->mask; sel.k = select_into->k; sel.counts = select_into->counts;
+        sel.offsets = select_into->offsets; sel.perm = select_into->perm; sel.tok_off = select_into->tok_off;
+        sel.tok_exp = select_into->tok_exp; sel.n_sel = select_into->n_sel; sel.status = select_into->status;
+        sel.capacity = (long long)select_into->perm_capacity;
+    }
+    if (L->desc.dtype == D2D_F32) return launch_router<float>(L, x, T, R, u, ticket, st, sel, zero, zero_words);
+    return launch_router<__nv_bfloat16>(L, x, T, R, u, ticket, st, sel, zero, zero_words);
 }
 
 // ws: [ticket (256 bytes) | y32: T*d floats]
@@ -399,12 +433,13 @@ bool d2d_small_ffn_supports(const d2d_layer_desc &D)
     return D.d % 8 == 0 && rows_per_pass(D, D.dtype == D2D_F32 ? 4 : 2) > 0;
 }
 
-d2d_status d2d_small_ffn(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y, void *ws, cudaStream_t st)
+d2d_status d2d_small_ffn(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y, void *ws, cudaStream_t st,
+                         int fused)
 {
-    unsigned int *ticket = (unsigned int *)ws;
+    unsigned int *ticket = fused ? L->tickets + 16 : (unsigned int *)ws;
     float *y32 = (float *)((char *)ws + 256);
     // the ticket and the float32 accumulator must start at zero
-    D2D_CUDA_TRY(cudaMemsetAsync(ws, 0, 256 + (size_t)T * L->desc.d * 4, st));
+    if (!fused) D2D_CUDA_TRY(cudaMemsetAsync(ws, 0, 256 + (size_t)T * L->desc.d * 4, st));
     if (L->desc.dtype == D2D_F32) return launch_ffn_dtype<float>(L, x, T, r, y, y32, ticket, st);
     return launch_ffn_dtype<__nv_bfloat16>(L, x, T, r, y, y32, ticket, st);
 }
