@@ -5,6 +5,7 @@
 #include <string.h>
 
 #include "d2d_common.cuh"
+#include <stdlib.h>
 #include "gemm_tc.cuh"
 
 bool d2d_token_path_supports(const d2d_layer_desc &D);

@@ -278,7 +278,15 @@ router_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_const
                                 }
                                 if (R && row < T) {
                                     float *o = R + (size_t)row * E + c0;
-                                    if (c0 + 16 <= E && (E & 3) == 0) {
+                                    if (c0 + 16 <= E && (E & 7) == 0 && (reinterpret_cast<uintptr_t>(R) & 31) == 0) {
+                                        // 32-byte stores: a whole sector per lane and instruction
+#pragma unroll
+                                        for (int j = 0; j < 16; j += 8)
+                                            asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(o + j),
+                                                         "f"(v[q][h * 16 + j]), "f"(v[q][h * 16 + j + 1]), "f"(v[q][h * 16 + j + 2]),
+                                                         "f"(v[q][h * 16 + j + 3]), "f"(v[q][h * 16 + j + 4]), "f"(v[q][h * 16 + j + 5]),
+                                                         "f"(v[q][h * 16 + j + 6]), "f"(v[q][h * 16 + j + 7]) : "memory");
+                                    } else if (c0 + 16 <= E && (E & 3) == 0) {
 #pragma unroll
                                         for (int j = 0; j < 16; j += 4)
                                             *reinterpret_cast<float4 *>(o + j) = make_float4(v[q][h * 16 + j], v[q][h * 16 + j + 1],
