@@ -32,8 +32,8 @@ L2_FLUSH_BYTES = 256 << 20
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (None until a capture of that kernel/workload exists).
 NCU_TRAFFIC_BYTES = {
-    ("bert", 4096): 11.13e6,        # up projection: profiles/bert_gemm_up_down_full.md
-    ("gpt2_ffn", 1, 0.2): 9.884e6,  # decode expert kernel: profiles/gpt2_decode_T1_small_ffn_full.md
+    ("bert", 4096): 11.20e6,        # up projection: profiles/bert_gemm_up_down_full.md
+    ("gpt2_ffn", 1, 0.2): 9.868e6,  # decode expert kernel: profiles/gpt2_decode_T1_small_kernels_full.md
 }
 
 
@@ -329,7 +329,7 @@ def run_ours(args):
             # decode regime: the expert kernel is bound by HBM traffic on the touched expert slices
             touched = n_used * (cfg.n_mat * cfg.s * cfg.d + cfg.s) * elem + 2 * T * cfg.d * elem + cfg.d * elem
             achieved = touched / (t_ffn * 1e-3) / 1e9
-            roofline = {"bound": "hbm", "kernel": "moe_ffn_fwd (small_ffn_kernel)" if T <= 16 else "moe_ffn_fwd", "achieved": achieved,
+            roofline = {"bound": "hbm", "kernel": "moe_ffn_fwd (small_ffn_kernel)" if T <= 8 else "moe_ffn_fwd", "achieved": achieved,
                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
                         "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, T, args.tau)),
                         "peak_source": f"{peaks['source']} HBM copy", "algorithmic_bytes_per_launch": touched,

@@ -339,7 +339,8 @@ d2d_status d2d_layer_fwd(const d2d_layer *layer, const void *x, int32_t T, float
         // the router starts because the up projection may begin while the router is still running
         int *up_counter = dense ? (int *)(base + w.u_off) : nullptr;
         if (up_counter && cudaMemsetAsync(up_counter, 0, sizeof(int), st) != cudaSuccess) return D2D_ERR_CUDA;
-        rc = d2d_router_fused(layer, x, T, tau, 1, R, routing->mask, routing->k, routing->status, st);
+        // the scores themselves are written only when the caller asked for them: mask and k come out of the same kernel
+        rc = d2d_router_fused(layer, x, T, tau, 1, R_out, routing->mask, routing->k, routing->status, st);
         if (rc != D2D_OK) return rc;
         if (dense) {
             // The dense-masked expert GEMMs read only the mask: build counts / offsets / token lists on the side
