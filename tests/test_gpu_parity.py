@@ -250,7 +250,11 @@ def test_other_activations_and_odd_expert_size(api, act):
 
 # ------------------------------------------------------------------------------------ whole layer
 
-LAYER_CASES = [("tiny", None, 0.5), ("bert", 1000, 0.3), ("vit", 900, 0.3), ("gpt2_ffn", 8, 0.2), ("llama", 64, 0.4)]
+# token counts on both sides of every dispatch boundary: decode kernels (T <= 8), tensor-core path with the split-K
+# down projection (9 <= T <= 128), one and several row tiles, ragged last tile
+LAYER_CASES = [("tiny", None, 0.5), ("bert", 1000, 0.3), ("vit", 900, 0.3), ("gpt2_ffn", 8, 0.2), ("llama", 64, 0.4),
+               ("gpt2_ffn", 1, 0.2), ("gpt2_ffn", 9, 0.2), ("gpt2_ffn", 16, 0.5), ("gpt2_attn", 100, 0.2),
+               ("gpt2_attn", 128, 0.5), ("bert", 129, 0.3), ("llama", 300, 0.4)]
 
 
 @pytest.mark.parametrize("name,T,tau", LAYER_CASES)
@@ -278,6 +282,27 @@ def test_layer_fwd_end_to_end(api, name, T, tau):
     assert diff.mean() < 0.01 and same.mean() > 0.3
     yg = y.float().cpu().numpy()
     assert _rel_err(yg[same], ref["y"][same]) <= TOL_Y[cfg.dtype]
+
+
+@pytest.mark.parametrize("name,T,tau", [("bert", 700, 0.3), ("gpt2_ffn", 5, 0.2), ("gpt2_ffn", 40, 0.2)])
+def test_layer_fwd_without_scores_output_matches_the_run_with_it(api, name, T, tau):
+    """R is an optional output: asking for it must not change the routing or y (tile-to-CTA assignment is dynamic,
+    results must not depend on it)."""
+    cfg, w, x, layer = _setup(api, name, T)
+    xd = api.to_device(x, cfg.dtype)
+    R_out = torch.empty((x.shape[0], cfg.E), dtype=torch.float32, device="cuda")
+    y1, r1 = layer.layer_fwd(xd, tau, R_out=R_out)
+    torch.cuda.synchronize()
+    m1, k1, p1, n1 = r1.mask_u32().copy(), r1.k.cpu().numpy().copy(), r1.perm.cpu().numpy().copy(), r1.n_sel
+    y1 = y1.float().cpu().numpy()
+    for _ in range(2):
+        y2, r2 = layer.layer_fwd(xd, tau)
+        torch.cuda.synchronize()
+        assert r2.status == 0 and r2.n_sel == n1
+        assert np.array_equal(r2.mask_u32(), m1) and np.array_equal(r2.k.cpu().numpy(), k1)
+        assert np.array_equal(r2.perm.cpu().numpy()[:n1], p1[:n1])
+        # float32 reductions of the decode and split-K paths may be reordered between runs
+        assert _rel_err(y2.float().cpu().numpy(), y1) <= (0 if (T > 128) else 1e-2)
 
 
 # ------------------------------------------------------------------------------------ full-size sampled checks
