@@ -307,7 +307,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     // to the epilogue through a two-slot ring (a CTA that starts late, or gets slow tiles, simply draws fewer)
     __shared__ uint64_t sched_full[2], sched_empty[2];
     __shared__ volatile int sched_item[2], epi_item[2];
-    constexpr int MASK_REGS = 16;                                    // selection words of a row kept in registers
+    constexpr int MASK_REGS = 8;                                     // selection words of a row kept in registers (E <= 256; wider masks are read through L1)
     // the whole bias vector is staged once, as float32, behind the operand stages when it fits
     float *bias_f = reinterpret_cast<float *>(smem + (size_t)STAGES * STAGE_BYTES);
     const bool bias_cached = ep.bias != nullptr && N <= BIAS_CACHE_ELEMS && (N & 3) == 0;
