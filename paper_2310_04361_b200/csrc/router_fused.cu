@@ -15,7 +15,7 @@
 namespace {
 
 constexpr int BM = 128, BK = 64, UMMA_K = 16;
-constexpr int STAGES = 3;
+constexpr int STAGES = 5;          // 5 x 32 KB of operands in flight: the first GEMM's main loop is bound by load latency
 constexpr uint32_t WAIT_LIMIT = 1u << 22;
 constexpr int NTHREADS = 64 + 512;       // TMA warp, MMA warp, 16 epilogue warps
 
@@ -97,7 +97,8 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
 // Shared memory (dynamic, 1024-byte aligned):
 //   [ STAGES x (x tile 128x64 | W_r1 tile DH x 64) ]        first GEMM operand ring
 //   [ u: DH/64 k-blocks x (128 rows x 128 B) ]              A operand of the second GEMM (written by epilogue 1)
-//   [ W_r2: NT2 column tiles x DH/64 k-blocks x (256 rows x 128 B) ]   B operand of the second GEMM (TMA)
+//   W_r2 (DH/64 k-blocks x 256 rows x 128 B, the B operand of the second GEMM) reuses the first stages of the ring:
+//   it is loaded as soon as the last k-blocks that used those stages have been consumed, under epilogue 1.
 // TMEM: columns [0, DH) accumulator of u, columns [256, 256 + E_pad) accumulator of R (E <= 256).
 template <int DH>
 __global__ void __launch_bounds__(NTHREADS, 1)
@@ -116,7 +117,9 @@ router_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_const
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t *u_s = smem + (size_t)STAGES * STAGE_BYTES;
-    uint8_t *w2_s = u_s + U_BYTES;
+    uint8_t *w2_s = smem;                                  // aliases the first stages (see above)
+    static_assert((size_t)KB2 * W2_KB_BYTES <= (size_t)STAGES * STAGE_BYTES, "W_r2 must fit in the operand ring");
+    constexpr int W2_STAGES = (KB2 * W2_KB_BYTES + STAGE_BYTES - 1) / STAGE_BYTES;      // stages W_r2 overwrites
     __shared__ uint64_t bar_full[STAGES], bar_empty[STAGES], bar_w2, bar_acc1, bar_u_ready, bar_acc2;
     __shared__ uint32_t tmem_base_holder;
     __shared__ float b1_s[DH], b2_s[256];                  // biases as float32
@@ -158,18 +161,28 @@ router_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_const
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            // W_r2 first (small, needed last): all its k-blocks land on one barrier
-            mbar_expect_tx(smem_u32(&bar_w2), (uint32_t)(KB2 * W2_KB_BYTES));
-            for (int kb = 0; kb < KB2; ++kb)
-                tma_load_2d(smem_u32(w2_s + (size_t)kb * W2_KB_BYTES), &tm_w2, kb * BK, 0, smem_u32(&bar_w2));
-            for (int kb = 0; kb < nkb; ++kb) {
+            bool ok = true;
+            for (int kb = 0; kb < nkb && ok; ++kb) {
                 const uint32_t s = kb % STAGES, round = kb / STAGES;
-                if (!mbar_wait(smem_u32(&bar_empty[s]), (round & 1u) ^ 1u, status)) break;
+                ok = mbar_wait(smem_u32(&bar_empty[s]), (round & 1u) ^ 1u, status);
+                if (!ok) break;
                 const uint32_t full = smem_u32(&bar_full[s]);
                 const uint32_t dst = smem_u32(smem + (size_t)s * STAGE_BYTES);
                 mbar_expect_tx(full, (uint32_t)STAGE_BYTES);
                 tma_load_2d(dst, &tm_x, kb * BK, m0, full);
                 tma_load_2d(dst + A_BYTES, &tm_w1, kb * BK, 0, full);
+            }
+            // W_r2 goes into stages 0 .. W2_STAGES-1 once the MMAs of the last k-block that used each of them have retired
+            for (int s = 0; s < W2_STAGES && ok; ++s) {
+                if (s < nkb) {
+                    const int last = s + ((nkb - 1 - s) / STAGES) * STAGES;      // last k-block held by stage s
+                    ok = mbar_wait(smem_u32(&bar_empty[s]), (uint32_t)(last / STAGES) & 1u, status);
+                }
+            }
+            if (ok) {
+                mbar_expect_tx(smem_u32(&bar_w2), (uint32_t)(KB2 * W2_KB_BYTES));
+                for (int kb = 0; kb < KB2; ++kb)
+                    tma_load_2d(smem_u32(w2_s + (size_t)kb * W2_KB_BYTES), &tm_w2, kb * BK, 0, smem_u32(&bar_w2));
             }
         }
     } else if (warp == 1) {
@@ -394,7 +407,7 @@ d2d_status launch(const d2d_layer *L, const void *x, int T, float tau, int do_ma
     const d2d_layer_desc &D = L->desc;
     constexpr int STAGE_BYTES = BM * BK * 2 + DH * BK * 2;
     constexpr int KB2 = DH / BK;
-    constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + (size_t)KB2 * BM * 128 + (size_t)KB2 * 256 * 128 + 1024;
+    constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + (size_t)KB2 * BM * 128 + 1024;
     CUtensorMap tx, tw1, tw2;
     if (!make_map(&tx, x, T, D.d, BM) || !make_map(&tw1, L->w_r1, D.d_h, D.d, DH) ||
         !make_map(&tw2, L->w_r2, D.n_experts, D.d_h, 256))
