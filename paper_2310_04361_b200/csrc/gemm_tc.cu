@@ -724,7 +724,7 @@ d2d_status launch(const d2d_gemm_args &g, cudaStream_t st)
 {
     constexpr int B_ROWS = PAIR ? BN / 2 : BN;
     constexpr int STAGE_BYTES = BM * BK * 2 + (GATED ? 2 : 1) * B_ROWS * BK * 2;
-    constexpr int STAGES = (196 * 1024) / STAGE_BYTES > 8 ? 8 : (196 * 1024) / STAGE_BYTES;
+    constexpr int STAGES = (200 * 1024) / STAGE_BYTES > 8 ? 8 : (200 * 1024) / STAGE_BYTES;   // 200 KB of operand stages (+ 24 KB bias cache)
     constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + 1024 + (size_t)BIAS_CACHE_ELEMS * 4;
     CUtensorMap ta, tb, tb2;
     if (!make_map(&ta, g.a, g.M, g.K, BM) || !make_map(&tb, g.b, g.N, g.K, B_ROWS)) return D2D_ERR_CUDA;
