@@ -223,10 +223,20 @@ D2D_API d2d_status d2d_expert_up_fwd(const d2d_layer *layer, const void *x, int3
 D2D_API d2d_status d2d_expert_down_fwd(const d2d_layer *layer, const void *H, int32_t T, void *y, int32_t *status,
                                        void *stream);
 
-/* The whole layer on one stream with no host synchronisation in between:
- * router_fwd -> select_dynk -> moe_ffn_fwd.  R_out: optional device [T,E]
- * float32 copy of the router scores (NULL to keep them in the workspace only).
- * `routing` supplies the metadata buffers (required; they are outputs). */
+/* The whole layer with no host synchronisation in between:
+ * router_fwd -> select_dynk -> moe_ffn_fwd (Sec. 3.2-3.4).  R_out: optional
+ * device [T,E] float32 output of the router scores; with NULL the scores may
+ * never reach memory (for bf16 batches of 9 or more tokens the router kernel
+ * thresholds them on chip).  `routing` supplies the metadata buffers
+ * (required; they are outputs).  Work is enqueued on `stream`; the per-expert
+ * metadata may be built on a stream the layer owns, joined back into `stream`
+ * before the call's last operation, so everything the call writes is ordered
+ * before whatever the caller enqueues on `stream` next.  The layer object
+ * holds that side stream, two events and the self-resetting tickets of the
+ * decode kernels: calls on ONE layer object must not overlap in time (use one
+ * layer object per stream for concurrent streams).  On `stream` the up
+ * projection may start before the router has finished (programmatic dependent
+ * launch); it reads only x and the weights until the router has completed. */
 D2D_API d2d_status d2d_layer_fwd(const d2d_layer *layer, const void *x, int32_t T, float tau, void *y,
                          float *R_out, d2d_routing *routing, void *ws, size_t ws_bytes, void *stream);
 
