@@ -335,10 +335,9 @@ d2d_status d2d_layer_fwd(const d2d_layer *layer, const void *x, int32_t T, float
         // router and dynamic-k mask in one kernel; the selection step then only builds the per-expert metadata
         if (cudaMemsetAsync(routing->status, 0, sizeof(int32_t), st) != cudaSuccess) return D2D_ERR_CUDA;
         const bool dense = use_dense_masked(layer, T) && !use_small_ffn(layer, T);
-        // tile counter of the up projection (the ticket area in front of u is unused on this path), cleared before
-        // the router starts because the up projection may begin while the router is still running
-        int *up_counter = dense ? (int *)(base + w.u_off) : nullptr;
-        if (up_counter && cudaMemsetAsync(up_counter, 0, sizeof(int), st) != cudaSuccess) return D2D_ERR_CUDA;
+        // tile counter of the up projection: layer-owned, zero at creation and reset by the kernel that used it, so no
+        // memset node sits in front of the router (the up projection may begin while the router is still running)
+        int *up_counter = dense ? (int *)(layer->tickets + 32) : nullptr;
         // the scores themselves are written only when the caller asked for them: mask and k come out of the same kernel
         rc = d2d_router_fused(layer, x, T, tau, 1, R_out, routing->mask, routing->k, routing->status, st);
         if (rc != D2D_OK) return rc;

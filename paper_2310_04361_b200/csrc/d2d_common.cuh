@@ -25,8 +25,9 @@ struct d2d_layer {
     cudaStream_t side_stream;
     cudaEvent_t ev_fork, ev_join;
     // layer-owned "last CTA" tickets of the decode kernels used by d2d_layer_fwd (zero at creation, reset by the kernel
-    // that used them): word 0 router, word 16 experts.  Like the side stream, they make concurrent d2d_layer_fwd calls on
-    // ONE layer object from several streams unsafe; use one layer object per stream for that.
+    // that used them): word 0 decode router, word 16 decode experts, word 32 tile counter of the up projection.  Like the
+    // side stream, they make concurrent d2d_layer_fwd calls on ONE layer object from several streams unsafe; use one
+    // layer object per stream for that.  A call that ended in D2D_ERR_TIMEOUT may leave them non-zero: recreate the layer.
     unsigned int *tickets;
 };
 

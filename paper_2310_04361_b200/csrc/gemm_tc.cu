@@ -387,6 +387,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     ok = mbar_wait(smem_u32(&sched_empty[sl]), (use & 1u) ^ 1u, ep.status);
                     if (!ok) break;
                     item = atomicAdd(ep.tile_counter, 1);
+                    // every CTA draws exactly one value past the end; whoever draws the largest of them is the last to
+                    // touch the counter and leaves it at zero for the next launch
+                    if (item == total_tiles + (int)gridDim.x - 1) *ep.tile_counter = 0;
                     sched_item[sl] = item < total_tiles ? item : -1;
                     mbar_arrive(smem_u32(&sched_full[sl]));       // release: the slot's content is visible to whoever sees the phase
                 }

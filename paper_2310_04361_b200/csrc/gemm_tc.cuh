@@ -32,8 +32,9 @@ struct d2d_gemm_args {
     // converts.  For problems with so few output tiles that most SMs would idle (decode batches).
     int k_splits;
     float *partial;
-    // Dynamic tile scheduling: a device counter that is ZERO when the kernel starts (the caller clears it); CTAs draw
-    // work items from it instead of walking a fixed round-robin list.  NULL = static schedule.
+    // Dynamic tile scheduling: a device counter that is ZERO when the kernel starts; CTAs draw work items from it
+    // instead of walking a fixed round-robin list, and the last draw of a launch resets it to zero (a launch that ends
+    // in D2D_ERR_TIMEOUT may leave it non-zero).  NULL = static schedule.
     int *tile_counter;
     // 1: A, B and the bias do NOT depend on the previous kernel of the stream, only the epilogue inputs (the selection
     // mask) do.  With programmatic dependent launch the main loops then start while that kernel still runs and only the
