@@ -243,8 +243,12 @@ D2D_API d2d_status d2d_layer_fwd(const d2d_layer *layer, const void *x, int32_t 
 /* Host-buffer convenience: the same layer call, but x and y are HOST pointers
  * ([T,d] of desc.dtype).  The call copies x to the device, runs the layer,
  * copies y back and synchronises `stream`; all device memory it needs comes
- * from `ws` (device, at least d2d_layer_fwd_host_workspace_bytes bytes).  For
- * full copy/compute overlap the host buffers should be page-locked. */
+ * from `ws` (device, at least d2d_layer_fwd_host_workspace_bytes bytes).
+ * Batches of 2048 tokens or more are cut into four chunks and pipelined over
+ * two copy streams the layer owns (copy in / layer / copy out overlap; tokens
+ * are independent, so the result is the same); this needs page-locked host
+ * buffers to be effective.  Returns the data-dependent status as well
+ * (D2D_ERR_NONFINITE, D2D_ERR_TIMEOUT), read back after the synchronisation. */
 D2D_API size_t d2d_layer_fwd_host_workspace_bytes(const d2d_layer *layer, int32_t max_tokens);
 D2D_API d2d_status d2d_layer_fwd_host(const d2d_layer *layer, const void *x_host, int32_t T, float tau, void *y_host,
                               void *ws, size_t ws_bytes, void *stream);

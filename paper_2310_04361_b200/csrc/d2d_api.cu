@@ -201,12 +201,18 @@ d2d_status d2d_layer_create(const d2d_layer_desc *desc, const d2d_weights *w, vo
                          cudaEventCreateWithFlags(&L->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
                          cudaEventCreateWithFlags(&L->ev_join, cudaEventDisableTiming) != cudaSuccess))
         rc = D2D_ERR_CUDA;
+    if (rc == D2D_OK) {
+        bool ok = cudaStreamCreateWithFlags(&L->copy_in, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&L->copy_out, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&L->ev_begin, cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&L->ev_end, cudaEventDisableTiming) == cudaSuccess;
+        for (int c = 0; c < d2d_layer::kHostChunks && ok; ++c)
+            ok = cudaEventCreateWithFlags(&L->ev_in[c], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&L->ev_done[c], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) rc = D2D_ERR_CUDA;
+    }
     if (rc != D2D_OK) {
-        if (L->ev_join) cudaEventDestroy(L->ev_join);
-        if (L->ev_fork) cudaEventDestroy(L->ev_fork);
-        if (L->side_stream) cudaStreamDestroy(L->side_stream);
-        cudaFree(L->slab);
-        delete L;
+        d2d_layer_destroy(L);
         return rc;
     }
     *out = L;
@@ -219,6 +225,14 @@ d2d_status d2d_layer_destroy(d2d_layer *layer)
     if (layer->ev_join) cudaEventDestroy(layer->ev_join);
     if (layer->ev_fork) cudaEventDestroy(layer->ev_fork);
     if (layer->side_stream) cudaStreamDestroy(layer->side_stream);
+    for (int c = 0; c < d2d_layer::kHostChunks; ++c) {
+        if (layer->ev_in[c]) cudaEventDestroy(layer->ev_in[c]);
+        if (layer->ev_done[c]) cudaEventDestroy(layer->ev_done[c]);
+    }
+    if (layer->ev_begin) cudaEventDestroy(layer->ev_begin);
+    if (layer->ev_end) cudaEventDestroy(layer->ev_end);
+    if (layer->copy_in) cudaStreamDestroy(layer->copy_in);
+    if (layer->copy_out) cudaStreamDestroy(layer->copy_out);
     cudaError_t e = cudaFree(layer->slab);
     delete layer;
     return e == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
@@ -373,6 +387,17 @@ d2d_status d2d_layer_fwd(const d2d_layer *layer, const void *x, int32_t T, float
     return d2d_launch_moe_ffn(layer, x, T, routing, y, base + w.ffn_off, w.total - w.ffn_off, st);
 }
 
+// Data-dependent conditions of a finished host call: the largest device status word (0 = ok).
+static d2d_status host_status(const int32_t *status_dev, int n)
+{
+    int32_t h[d2d_layer::kHostChunks] = {0, 0, 0, 0};
+    if (n > d2d_layer::kHostChunks) n = d2d_layer::kHostChunks;
+    if (cudaMemcpy(h, status_dev, sizeof(int32_t) * (size_t)n, cudaMemcpyDeviceToHost) != cudaSuccess) return D2D_ERR_CUDA;
+    int32_t worst = 0;
+    for (int i = 0; i < n; ++i) worst = h[i] > worst ? h[i] : worst;
+    return (d2d_status)worst;
+}
+
 // Carves routing buffers + x/y staging + the layer workspace out of one device buffer.
 struct host_call_layout {
     size_t x_off, y_off, mask_off, k_off, counts_off, offsets_off, perm_off, scalars_off, ws_off, total;
@@ -391,7 +416,7 @@ static host_call_layout host_layout(const d2d_layer *L, int T)
     h.counts_off = take(E * 4);
     h.offsets_off = take((E + 1) * 4);
     h.perm_off = take(Tn * E * 4);
-    h.scalars_off = take(2 * 4);
+    h.scalars_off = take((2 + d2d_layer::kHostChunks) * 4);     // n_sel, then one status word per chunk
     h.ws_off = off;
     off += layout_for(L, (int)Tn).total;
     h.total = off;
@@ -414,8 +439,8 @@ d2d_status d2d_layer_fwd_host(const d2d_layer *layer, const void *x_host, int32_
     if (ws_bytes < h.total) return D2D_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     char *base = (char *)ws;
-    const size_t row_bytes = (size_t)T * layer->desc.d * layer->elem;
-    D2D_CUDA_TRY(cudaMemcpyAsync(base + h.x_off, x_host, row_bytes, cudaMemcpyHostToDevice, st));
+    const size_t tok_bytes = (size_t)layer->desc.d * layer->elem;
+    const size_t row_bytes = (size_t)T * tok_bytes;
     d2d_routing r;
     memset(&r, 0, sizeof(r));
     r.mask = (uint32_t *)(base + h.mask_off);
@@ -426,12 +451,54 @@ d2d_status d2d_layer_fwd_host(const d2d_layer *layer, const void *x_host, int32_
     r.n_sel = (int32_t *)(base + h.scalars_off);
     r.status = r.n_sel + 1;
     r.perm_capacity = (int64_t)T * layer->desc.n_experts;
-    d2d_status rc = d2d_layer_fwd(layer, base + h.x_off, T, tau, base + h.y_off, nullptr, &r,
-                                  base + h.ws_off, h.total - h.ws_off, st);
+    // Tokens are independent, so a large batch is cut into chunks (multiples of 128 tokens) and pipelined: the copy of
+    // chunk c+1 to the device (copy-in stream), the layer on chunk c (`stream`) and the copy of chunk c-1 back to the
+    // host (copy-out stream) run at the same time; PCIe carries both directions at once.  The routing buffers and the
+    // layer workspace are reused chunk after chunk, which is safe because the layer calls are serial on `stream`.
+    const int n_chunks = T >= 2048 ? d2d_layer::kHostChunks : 1;
+    if (n_chunks == 1) {
+        D2D_CUDA_TRY(cudaMemcpyAsync(base + h.x_off, x_host, row_bytes, cudaMemcpyHostToDevice, st));
+        d2d_status rc = d2d_layer_fwd(layer, base + h.x_off, T, tau, base + h.y_off, nullptr, &r,
+                                      base + h.ws_off, h.total - h.ws_off, st);
+        if (rc != D2D_OK) return rc;
+        D2D_CUDA_TRY(cudaMemcpyAsync(y_host, base + h.y_off, row_bytes, cudaMemcpyDeviceToHost, st));
+        D2D_CUDA_TRY(cudaStreamSynchronize(st));
+        return host_status(r.status, 1);
+    }
+    const int chunk = d2d_cdiv(d2d_cdiv(T, n_chunks), 128) * 128;
+    // the copies may not start before work already queued on `stream` (which may still use ws) has finished
+    D2D_CUDA_TRY(cudaEventRecord(layer->ev_begin, st));
+    D2D_CUDA_TRY(cudaStreamWaitEvent(layer->copy_in, layer->ev_begin, 0));
+    D2D_CUDA_TRY(cudaStreamWaitEvent(layer->copy_out, layer->ev_begin, 0));
+    for (int c = 0, t0 = 0; t0 < T; ++c, t0 += chunk) {
+        const int tc = T - t0 < chunk ? T - t0 : chunk;
+        D2D_CUDA_TRY(cudaMemcpyAsync(base + h.x_off + (size_t)t0 * tok_bytes, (const char *)x_host + (size_t)t0 * tok_bytes,
+                                     (size_t)tc * tok_bytes, cudaMemcpyHostToDevice, layer->copy_in));
+        D2D_CUDA_TRY(cudaEventRecord(layer->ev_in[c], layer->copy_in));
+    }
+    d2d_status rc = D2D_OK;
+    int32_t *const status0 = r.status;
+    int n_used = 0;
+    for (int c = 0, t0 = 0; t0 < T; ++c, t0 += chunk, ++n_used) {
+        const int tc = T - t0 < chunk ? T - t0 : chunk;
+        r.status = status0 + c;                              // one status word per chunk (the layer call clears its own)
+        D2D_CUDA_TRY(cudaStreamWaitEvent(st, layer->ev_in[c], 0));
+        rc = d2d_layer_fwd(layer, base + h.x_off + (size_t)t0 * tok_bytes, tc, tau, base + h.y_off + (size_t)t0 * tok_bytes,
+                           nullptr, &r, base + h.ws_off, h.total - h.ws_off, st);
+        if (rc != D2D_OK) break;
+        D2D_CUDA_TRY(cudaEventRecord(layer->ev_done[c], st));
+        D2D_CUDA_TRY(cudaStreamWaitEvent(layer->copy_out, layer->ev_done[c], 0));
+        D2D_CUDA_TRY(cudaMemcpyAsync((char *)y_host + (size_t)t0 * tok_bytes, base + h.y_off + (size_t)t0 * tok_bytes,
+                                     (size_t)tc * tok_bytes, cudaMemcpyDeviceToHost, layer->copy_out));
+    }
+    // join both copy streams back into `stream` (also on the error path, so nothing is left running on them)
+    cudaEventRecord(layer->ev_end, layer->copy_out);
+    cudaStreamWaitEvent(st, layer->ev_end, 0);
+    cudaEventRecord(layer->ev_end, layer->copy_in);
+    cudaStreamWaitEvent(st, layer->ev_end, 0);
     if (rc != D2D_OK) return rc;
-    D2D_CUDA_TRY(cudaMemcpyAsync(y_host, base + h.y_off, row_bytes, cudaMemcpyDeviceToHost, st));
     D2D_CUDA_TRY(cudaStreamSynchronize(st));
-    return D2D_OK;
+    return host_status(status0, n_used);
 }
 
 }  // extern "C"

@@ -24,6 +24,11 @@ struct d2d_layer {
     // expert GEMMs, which do not read it
     cudaStream_t side_stream;
     cudaEvent_t ev_fork, ev_join;
+    // d2d_layer_fwd_host: copy-in and copy-out streams and per-chunk events, so that the host -> device copy of one
+    // chunk of tokens, the layer on the previous chunk and the device -> host copy of the one before overlap
+    static const int kHostChunks = 4;
+    cudaStream_t copy_in, copy_out;
+    cudaEvent_t ev_in[kHostChunks], ev_done[kHostChunks], ev_begin, ev_end;
     // layer-owned "last CTA" tickets of the decode kernels used by d2d_layer_fwd (zero at creation, reset by the kernel
     // that used them): word 0 decode router, word 16 decode experts, word 32 tile counter of the up projection.  Like the
     // side stream, they make concurrent d2d_layer_fwd calls on ONE layer object from several streams unsafe; use one
