@@ -346,6 +346,42 @@ def test_layer_fwd_host_buffers(api):
     assert torch.equal(yh, y_dev.cpu())
 
 
+def test_layer_fwd_host_chunked_pipeline_matches_device_call(api):
+    """2048 tokens or more: the host call runs in four pipelined chunks (ragged last chunk here); tokens are
+    independent, so the result equals one device call on the whole batch."""
+    T = 2048 + 300
+    cfg, w, x, layer = _setup(api, "bert", T)
+    xh = torch.from_numpy(x).to(torch.bfloat16).pin_memory()
+    yh = torch.empty_like(xh).pin_memory()
+    ws = layer.host_workspace(T)
+    for _ in range(2):                          # twice: buffers, events and tickets are reusable
+        yh.zero_()
+        layer.layer_fwd_host(xh, 0.3, yh, ws)
+        y_dev, _ = layer.layer_fwd(xh.cuda(), 0.3)
+        torch.cuda.synchronize()
+        assert torch.equal(yh, y_dev.cpu())
+
+
+def test_layer_fwd_host_reports_nonfinite_scores(api):
+    """An infinite token row makes its router scores non-finite: the host call returns the data-dependent status."""
+    T = 2048 + 64
+    cfg, w, x, layer = _setup(api, "bert", T)
+    xb = x.copy()
+    # a row aligned with the signs of one router row overflows that hidden unit to +inf (NaN or mixed infinities would
+    # be absorbed by the ReLU's max); the token sits in the last chunk
+    xb[T - 5, :] = 3e38 * np.sign(np.asarray(w["w_r1"], dtype=np.float32)[0])
+    xh = torch.from_numpy(xb).to(torch.bfloat16).pin_memory()
+    yh = torch.empty_like(xh).pin_memory()
+    ws = layer.host_workspace(T)
+    with pytest.raises(api.D2DError) as e:
+        layer.layer_fwd_host(xh, 0.3, yh, ws)
+    assert api.STATUS_NAMES[e.value.code] == "NONFINITE"
+    # the layer object stays usable
+    xh2 = torch.from_numpy(x).to(torch.bfloat16).pin_memory()
+    layer.layer_fwd_host(xh2, 0.3, yh, ws)
+    assert torch.isfinite(yh.float()).all()
+
+
 @pytest.mark.parametrize("name,T,tau", [("bert", 333, 0.3), ("llama", 150, 0.4)])
 def test_expert_up_then_down_matches_oracle(api, name, T, tau):
     """The two halves of the tensor-core expert step, called on their own: H is zero exactly where the token
