@@ -95,7 +95,7 @@ static d2d_status launch_dense_masked(const d2d_layer *L, const void *x, int T, 
     d2d_gemm_args up = {};
     up.tile_counter = up_counter;
     up.pdl_late_wait = up_counter != nullptr;
-    up.a = x; up.b = L->w1; up.b_gate = D.gated ? L->w_gate : nullptr; up.bias = L->b1; up.out = ws;
+    up.a = x; up.b = L->w1; up.b_gate = D.gated ? L->w_gate : nullptr; up.b_cat = L->w1g; up.b_cat_block = 128; up.bias = L->b1; up.out = ws;
     up.M = T; up.N = D.d_ff; up.K = D.d; up.epilogue = D2D_EPI_UP_MASKED; up.act = D.act;
     up.mask = r->mask; up.mask_words = (D.n_experts + 31) / 32; up.expert_size = D.expert_size; up.status = r->status;
     d2d_status rc = d2d_gemm_tc(up, st);
@@ -175,6 +175,12 @@ d2d_status d2d_layer_create(const d2d_layer_desc *desc, const d2d_weights *w, vo
     size_t total = 256;                                   // the ticket words (see d2d_layer::tickets)
     for (const piece &p : pieces)
         if (p.src) total += d2d_align_up(p.n * el, 256);
+    // gated bf16 layers: W1 and W_gate once more, interleaved in blocks of 128 rows for the tensor-core up projection
+    const int cat_block = 128;
+    const size_t cat_rows = (size_t)2 * cat_block * d2d_cdiv(D.d_ff, cat_block);
+    const bool want_cat = D.gated && D.dtype == D2D_BF16;
+    const size_t cat_off = total;
+    if (want_cat) total += d2d_align_up(cat_rows * D.d * el, 256);
     cudaStream_t st = (cudaStream_t)stream;
     if (cudaMalloc(&L->slab, total) != cudaSuccess) {
         delete L;
@@ -195,6 +201,20 @@ d2d_status d2d_layer_create(const d2d_layer_desc *desc, const d2d_weights *w, vo
             rc = D2D_ERR_CUDA;
         }
         if (rc != D2D_OK) break;
+    }
+    if (rc == D2D_OK && want_cat) {
+        char *cat = (char *)L->slab + cat_off;
+        const size_t row_b = (size_t)D.d * el;
+        if (cudaMemsetAsync(cat, 0, cat_rows * row_b, st) != cudaSuccess) rc = D2D_ERR_CUDA;
+        for (int r0 = 0, b = 0; r0 < D.d_ff && rc == D2D_OK; r0 += cat_block, ++b) {
+            const size_t rows = (size_t)(D.d_ff - r0 < cat_block ? D.d_ff - r0 : cat_block);
+            char *dst = cat + (size_t)b * 2 * cat_block * row_b;
+            if (cudaMemcpyAsync(dst, (const char *)w->w1 + (size_t)r0 * row_b, rows * row_b, cudaMemcpyDeviceToDevice, st) != cudaSuccess ||
+                cudaMemcpyAsync(dst + (size_t)cat_block * row_b, (const char *)w->w_gate + (size_t)r0 * row_b, rows * row_b,
+                                cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+                rc = D2D_ERR_CUDA;
+        }
+        L->w1g = cat;
     }
     if (rc == D2D_OK && cudaStreamSynchronize(st) != cudaSuccess) rc = D2D_ERR_CUDA;
     if (rc == D2D_OK && (cudaStreamCreateWithFlags(&L->side_stream, cudaStreamNonBlocking) != cudaSuccess ||
@@ -311,7 +331,7 @@ d2d_status d2d_expert_up_fwd(const d2d_layer *layer, const void *x, int32_t T, c
     if (layer->desc.dtype != D2D_BF16 || layer->desc.d_ff % 8 || !d2d_gemm_tc_available()) return D2D_ERR_UNSUPPORTED;
     const d2d_layer_desc &D = layer->desc;
     d2d_gemm_args up = {};
-    up.a = x; up.b = layer->w1; up.b_gate = D.gated ? layer->w_gate : nullptr; up.bias = layer->b1; up.out = H;
+    up.a = x; up.b = layer->w1; up.b_gate = D.gated ? layer->w_gate : nullptr; up.b_cat = layer->w1g; up.b_cat_block = 128; up.bias = layer->b1; up.out = H;
     up.M = T; up.N = D.d_ff; up.K = D.d; up.epilogue = D2D_EPI_UP_MASKED; up.act = D.act;
     up.mask = routing->mask; up.mask_words = (D.n_experts + 31) / 32; up.expert_size = D.expert_size;
     up.status = routing->status;

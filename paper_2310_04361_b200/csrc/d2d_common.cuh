@@ -18,6 +18,7 @@ struct d2d_layer {
     // w2t = W2 transposed to [d_ff, d] so that an expert's slice is s contiguous rows too
     void *w1, *b1, *w_gate, *w2t, *b2;
     void *w2;               // W2 as given ([d, d_ff]): the K-major B operand of the dense down projection
+    void *w1g;              // gated bf16 layers: W1 and W_gate interleaved in blocks of 128 rows (see d2d_gemm_args::b_cat)
     void *slab;             // one allocation backing all of the above
     size_t slab_bytes;
     // side stream + events: the per-expert metadata (counts, offsets, token lists) is built beside the

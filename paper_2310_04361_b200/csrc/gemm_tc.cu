@@ -152,7 +152,23 @@ struct EpiParams {
     uint32_t inv_expert_size;        // ceil(2^32 / expert_size): column / expert_size = umulhi(column, inv) for columns < 2^16
     int *tile_counter;               // device counter (zero at launch) for dynamic tile scheduling, NULL = static round-robin
     int late_wait;                   // 1: only the epilogue waits for the previous kernel of the stream (see below)
+    int gate_cat;                    // 1 (gated): tm_b covers up and gate rows interleaved in blocks of BN, one load brings both
+    int band_rows;                   // > 0: tiles are walked column-major inside bands of this many row tiles (L2 reuse)
 };
+
+// Tile index -> (row tile, column tile).  Plain order is row-major: CTAs that run together share a few rows of A and
+// sweep all of B, so B is streamed from HBM once per wave when A and B together exceed L2.  With bands, the tiles of
+// `band` consecutive row tiles are walked column by column: the band's rows of A stay in L2 while B is streamed once
+// per band.
+__device__ __forceinline__ void tile_coords(int tile, int rows, int cols, int band, int &r, int &c)
+{
+    if (band <= 0) { r = tile / cols; c = tile - r * cols; return; }
+    const int per_band = band * cols;
+    const int b = tile / per_band, idx = tile - b * per_band;
+    const int h = rows - b * band < band ? rows - b * band : band;      // height of this band (the last may be short)
+    c = idx / h;
+    r = b * band + (idx - c * h);
+}
 
 // Activations of the bf16 tensor-core path.  Results are rounded to bf16 (8 bits of mantissa,
 // 2^-9 relative), and the epilogue of the up projection is issue-bound (K = d is short compared
@@ -396,7 +412,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 if (item >= total_tiles) break;
                 const int tile = item / k_splits, sp = item - tile * k_splits;
                 const int kb0 = (int)((long long)sp * nkb / k_splits), kb1 = (int)((long long)(sp + 1) * nkb / k_splits);
-                const int m0 = (tile / n_tiles) * TM + (int)rank * BM, n0 = (tile % n_tiles) * BN + (int)rank * B_ROWS;
+                int tr, tc;
+                tile_coords(tile, (M + TM - 1) / TM, n_tiles, ep.band_rows, tr, tc);
+                const int m0 = tr * TM + (int)rank * BM, n0 = tc * BN + (int)rank * B_ROWS;
                 for (int kb = kb0; kb < kb1; ++kb, ++it) {
                     const uint32_t s = it % STAGES, round = it / STAGES;
                     ok = mbar_wait(smem_u32(&bar_empty[s]), (round & 1u) ^ 1u, ep.status);
@@ -413,8 +431,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                         const uint32_t full = smem_u32(&bar_full[s]);
                         mbar_expect_tx(full, (uint32_t)STAGE_BYTES);
                         tma_load_2d(dst, &tm_a, kb * BK, m0, full);
-                        tma_load_2d(dst + A_BYTES, &tm_b, kb * BK, n0, full);
-                        if (GATED) tma_load_2d(dst + A_BYTES + B_BYTES, &tm_b2, kb * BK, n0, full);
+                        if (GATED && ep.gate_cat) {
+                            // up rows [n0, n0+BN) and gate rows [n0, n0+BN) are adjacent in the interleaved copy: one
+                            // 2*BN-row box (the producer thread's time per k-block is what bounds the gated main loop)
+                            tma_load_2d(dst + A_BYTES, &tm_b, kb * BK, 2 * n0, full);
+                        } else {
+                            tma_load_2d(dst + A_BYTES, &tm_b, kb * BK, n0, full);
+                            if (GATED) tma_load_2d(dst + A_BYTES + B_BYTES, &tm_b2, kb * BK, n0, full);
+                        }
                     }
                 }
             }
@@ -508,7 +532,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             }
             if (item >= total_tiles) break;
             const int tile = item / k_splits;
-            const int m0 = (tile / n_tiles) * TM + (int)rank * BM, n0 = (tile % n_tiles) * BN;
+            int tr, tc;
+            tile_coords(tile, (M + TM - 1) / TM, n_tiles, ep.band_rows, tr, tc);
+            const int m0 = tr * TM + (int)rank * BM, n0 = tc * BN;
             const int row = m0 + quad * 32 + lane;
             // this row's selection words go to registers before the wait, so their latency is hidden
             uint32_t mw[MASK_REGS];
@@ -722,6 +748,21 @@ int sm_count()
 
 bool pdl_enabled();
 
+// Band height (in row tiles) for the tile walk, 0 = plain row-major.  Row-major order re-reads B once per wave of
+// CTAs, which is free while B stays in L2 (126 MB) beside the streaming A; only a large B (Llama-sized weights) needs
+// bands.  The band is sized so that its rows of A take about 32 MB (measured best on the Llama-shaped layer: 32 row
+// tiles of 1 MB, 1050 us against 1427 us for the up projection).
+int band_rows_for(int M, int N, int K, int tile_m, bool gated)
+{
+    (void)M;
+    const double b_bytes = 2.0 * N * K * (gated ? 2 : 1);
+    if (b_bytes < 48e6) return 0;
+    const char *e = getenv("D2D_GEMM_BAND");
+    if (e) return atoi(e);
+    int band = (int)(32e6 / (2.0 * tile_m * K) + 0.5);
+    return band < 16 ? 16 : band;                           // shorter bands stream B too often (16 .. 32 measured alike)
+}
+
 template <int BN, int EPI, int ACT, bool GATED, bool PAIR>
 d2d_status launch(const d2d_gemm_args &g, cudaStream_t st)
 {
@@ -730,11 +771,18 @@ d2d_status launch(const d2d_gemm_args &g, cudaStream_t st)
     constexpr int STAGES = (200 * 1024) / STAGE_BYTES > 8 ? 8 : (200 * 1024) / STAGE_BYTES;   // 200 KB of operand stages (+ 24 KB bias cache)
     constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + 1024 + (size_t)BIAS_CACHE_ELEMS * 4;
     CUtensorMap ta, tb, tb2;
-    if (!make_map(&ta, g.a, g.M, g.K, BM) || !make_map(&tb, g.b, g.N, g.K, B_ROWS)) return D2D_ERR_CUDA;
-    if (GATED) {
-        if (!make_map(&tb2, g.b_gate, g.N, g.K, B_ROWS)) return D2D_ERR_CUDA;
-    } else {
+    const bool gate_cat = GATED && !PAIR && g.b_cat != nullptr && g.b_cat_block == BN;
+    if (!make_map(&ta, g.a, g.M, g.K, BM)) return D2D_ERR_CUDA;
+    if (gate_cat) {
+        if (!make_map(&tb, g.b_cat, 2 * BN * d2d_cdiv(g.N, BN), g.K, 2 * BN)) return D2D_ERR_CUDA;
         tb2 = tb;
+    } else {
+        if (!make_map(&tb, g.b, g.N, g.K, B_ROWS)) return D2D_ERR_CUDA;
+        if (GATED) {
+            if (!make_map(&tb2, g.b_gate, g.N, g.K, B_ROWS)) return D2D_ERR_CUDA;
+        } else {
+            tb2 = tb;
+        }
     }
     auto kern = gemm_tc_kernel<BN, STAGES, EPI, ACT, GATED, PAIR>;
     static bool attr_set = false;
@@ -745,7 +793,8 @@ d2d_status launch(const d2d_gemm_args &g, cudaStream_t st)
     const int es = g.expert_size > 0 ? g.expert_size : 1;
     EpiParams ep{(const __nv_bfloat16 *)g.bias, g.out, g.mask, g.mask_words, es, g.status,
                  (uint32_t)((0x100000000ull + (unsigned long long)es - 1) / (unsigned long long)es),
-                 PAIR ? nullptr : g.tile_counter, (g.pdl_late_wait && pdl_enabled()) ? 1 : 0};
+                 PAIR ? nullptr : g.tile_counter, (g.pdl_late_wait && pdl_enabled()) ? 1 : 0, gate_cat ? 1 : 0,
+                 band_rows_for(g.M, g.N, g.K, PAIR ? 2 * BM : BM, GATED)};
     const int k_splits = g.k_splits > 1 ? g.k_splits : 1;
     const int tiles = d2d_cdiv(g.N, BN) * d2d_cdiv(g.M, PAIR ? 2 * BM : BM) * k_splits;
     const int workers = PAIR ? sm_count() / 2 : sm_count();

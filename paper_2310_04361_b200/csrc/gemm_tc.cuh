@@ -18,6 +18,10 @@ struct d2d_gemm_args {
     const void *a;           // [M, K] bf16 row-major (activations)
     const void *b;           // [N, K] bf16 row-major (weights, nn.Linear layout)
     const void *b_gate;      // [N, K] second weight matrix for the gated up projection, else NULL
+    // optional copy of b and b_gate interleaved in blocks of b_cat_block rows: [b rows of block 0 | gate rows of block 0 |
+    // b rows of block 1 | ...], the last block zero padded; lets the gated kernel fetch both tiles with one load
+    const void *b_cat;
+    int b_cat_block;
     const void *bias;        // [N] bf16 or NULL
     void *out;               // [M, N] bf16 or f32, row-major, leading dimension N
     int M, N, K;
