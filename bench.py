@@ -329,7 +329,7 @@ def run_ours(args):
             # decode regime: the expert kernel is bound by HBM traffic on the touched expert slices
             touched = n_used * (cfg.n_mat * cfg.s * cfg.d + cfg.s) * elem + 2 * T * cfg.d * elem + cfg.d * elem
             achieved = touched / (t_ffn * 1e-3) / 1e9
-            roofline = {"bound": "hbm", "kernel": "moe_ffn_fwd (small_ffn_kernel)" if T <= 8 else "moe_ffn_fwd", "achieved": achieved,
+            roofline = {"bound": "hbm", "kernel": "moe_ffn_fwd (small_ffn_kernel)" if T <= 4 else "moe_ffn_fwd", "achieved": achieved,
                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
                         "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, T, args.tau)),
                         "peak_source": f"{peaks['source']} HBM copy", "algorithmic_bytes_per_launch": touched,

@@ -226,7 +226,7 @@ D2D_API d2d_status d2d_expert_down_fwd(const d2d_layer *layer, const void *H, in
 /* The whole layer with no host synchronisation in between:
  * router_fwd -> select_dynk -> moe_ffn_fwd (Sec. 3.2-3.4).  R_out: optional
  * device [T,E] float32 output of the router scores; with NULL the scores may
- * never reach memory (for bf16 batches of 9 or more tokens the router kernel
+ * never reach memory (for bf16 batches of 5 or more tokens the router kernel
  * thresholds them on chip).  `routing` supplies the metadata buffers
  * (required; they are outputs).  Work is enqueued on `stream`; the per-expert
  * metadata may be built on a stream the layer owns, joined back into `stream`

@@ -51,21 +51,29 @@ ws_layout layout_for(const d2d_layer *L, int T)
 
 }  // namespace
 
-// Tokens from which the dense tensor-core path (masked hidden activations, two GEMMs) is used
-// instead of the token-major CUDA-core kernel.
-static const int kDenseMaskedMinTokens = 9;
+// Measured on the GPT-2-medium-shaped FFN (us per layer call, decode kernels / tensor-core path): T = 3: 31 / 39,
+// T = 4: 33 / 39, T = 5: 41 / 40, T = 8: 43 / 39.
+int d2d_decode_max_tokens()
+{
+    static const int v = [] {
+        const char *e = getenv("D2D_DECODE_MAX_TOKENS");
+        const int n = e ? atoi(e) : 4;
+        return n < 0 ? 0 : n > 8 ? 8 : n;
+    }();
+    return v;
+}
 
 static bool use_dense_masked(const d2d_layer *L, int T)
 {
-    return L->desc.dtype == D2D_BF16 && T >= kDenseMaskedMinTokens && L->desc.d_ff % 8 == 0 && d2d_gemm_tc_available();
+    return L->desc.dtype == D2D_BF16 && T > d2d_decode_max_tokens() && L->desc.d_ff % 8 == 0 && d2d_gemm_tc_available();
 }
 
 // Up to this many tokens the expert-per-CTA kernel (each kept expert's slice read once) is used.
-static const int kSmallFfnMaxTokens = 8;
 
 static bool use_small_ffn(const d2d_layer *L, int T)
 {
-    return T <= kSmallFfnMaxTokens && d2d_small_ffn_supports(L->desc);
+    const int lim = L->desc.dtype == D2D_BF16 ? d2d_decode_max_tokens() : 8;      // fp32 layers have no tensor-core path
+    return T <= lim && d2d_small_ffn_supports(L->desc);
 }
 
 size_t d2d_moe_ffn_ws_bytes(const d2d_layer *L, int T)
@@ -73,7 +81,7 @@ size_t d2d_moe_ffn_ws_bytes(const d2d_layer *L, int T)
     size_t need = 256;
     if (use_small_ffn(L, T)) need = d2d_small_ffn_ws_bytes(L, T);
     // hidden activations H [T, d_ff] bf16 of the dense-masked path
-    if (L->desc.dtype == D2D_BF16 && T >= kDenseMaskedMinTokens) {
+    if (L->desc.dtype == D2D_BF16 && T > d2d_decode_max_tokens()) {
         size_t h = d2d_align_up((size_t)T * L->desc.d_ff * 2, 256);
         if (d2d_gemm_tc_splits(T, L->desc.d, L->desc.d_ff) > 1) h += d2d_align_up((size_t)T * L->desc.d * 4, 256);   // split-K partial sums
         if (h > need) need = h;

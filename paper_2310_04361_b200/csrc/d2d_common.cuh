@@ -47,6 +47,10 @@ struct d2d_layer {
 extern unsigned long long d2d_launch_counter;
 #define D2D_LAUNCHED(n) __atomic_fetch_add(&d2d_launch_counter, (unsigned long long)(n), __ATOMIC_RELAXED)
 
+// Largest batch served by the decode kernels (cp.async CUDA-core kernels, two launches per layer call); larger bf16
+// batches take the tensor-core path.  4 by default, D2D_DECODE_MAX_TOKENS=n (0 .. 8) overrides it for tuning.
+int d2d_decode_max_tokens();
+
 static inline size_t d2d_align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 static inline int d2d_cdiv(int a, int b) { return (a + b - 1) / b; }
 

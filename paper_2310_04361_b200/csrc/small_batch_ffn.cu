@@ -168,7 +168,7 @@ small_router_kernel(const TT *__restrict__ x, int T, int d, const TT *__restrict
         }
     }
     if (sel.enabled) {
-        // the scores of all T <= 8 tokens were written by this CTA: select from them right here
+        // the scores of all (at most 8) tokens were written by this CTA: select from them right here
         __syncthreads();
         uint32_t *smask = reinterpret_cast<uint32_t *>(us + (size_t)T * d_h);
         d2d_small::select_cta(R, T, E, (E + 31) / 32, sel.tau, sel.mask, sel.k, sel.counts, sel.offsets, sel.perm, sel.tok_off,
@@ -402,7 +402,7 @@ size_t d2d_small_router_ws_bytes(const d2d_layer *L, int T) { return 256 + d2d_a
 bool d2d_small_router_supports(const d2d_layer_desc &D, int T)
 {
     const size_t elem = D.dtype == D2D_F32 ? 4 : 2;
-    return T >= 1 && T <= 8 && D.d % 8 == 0 && D.d_h % 8 == 0 &&
+    return T >= 1 && T <= (D.dtype == D2D_BF16 ? d2d_decode_max_tokens() : 8) && D.d % 8 == 0 && D.d_h % 8 == 0 &&
            (size_t)(8 + MAX_TBLK) * D.d * elem + (size_t)T * D.d_h * 4 + (size_t)T * ((D.n_experts + 31) / 32) * 4 <= kSmemLimit;
 }
 

@@ -250,10 +250,11 @@ def test_other_activations_and_odd_expert_size(api, act):
 
 # ------------------------------------------------------------------------------------ whole layer
 
-# token counts on both sides of every dispatch boundary: decode kernels (T <= 8), tensor-core path with the split-K
-# down projection (9 <= T <= 128), one and several row tiles, ragged last tile
+# token counts on both sides of every dispatch boundary: decode kernels (T <= 4), tensor-core path with the split-K
+# down projection (5 <= T <= 128), one and several row tiles, ragged last tile
 LAYER_CASES = [("tiny", None, 0.5), ("bert", 1000, 0.3), ("vit", 900, 0.3), ("gpt2_ffn", 8, 0.2), ("llama", 64, 0.4),
-               ("gpt2_ffn", 1, 0.2), ("gpt2_ffn", 9, 0.2), ("gpt2_ffn", 16, 0.5), ("gpt2_attn", 100, 0.2),
+               ("gpt2_ffn", 1, 0.2), ("gpt2_ffn", 4, 0.5), ("gpt2_ffn", 5, 0.2), ("gpt2_ffn", 9, 0.2), ("gpt2_ffn", 16, 0.5),
+               ("gpt2_attn", 3, 0.2), ("gpt2_attn", 100, 0.2),
                ("gpt2_attn", 128, 0.5), ("bert", 129, 0.3), ("llama", 300, 0.4)]
 
 
