@@ -565,33 +565,32 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             }
             const bool bias_fast = ep.bias == nullptr || bias_cached;
             const bool wide_store = (N & 15) == 0 && (reinterpret_cast<uintptr_t>(ep.out) & 31) == 0;   // 32-byte aligned rows
-            const bool gran8 = EPI == D2D_EPI_UP_MASKED && mrow != nullptr && (ep.expert_size & 7) == 0;
-            // Non-gated: the next unit's accumulators are prefetched into a second register set.  Gated tiles need
-            // two accumulators per column; a second set would spill, so each unit is loaded when it is needed and
-            // the other epilogue warps of the SM sub-partition cover the latency.
+            const bool mask_on = EPI == D2D_EPI_UP_MASKED && ep.mask != nullptr;                         // CTA-uniform
+            // The common case gets a loop of its own with nothing else in it (the epilogue is sensitive to its
+            // instruction-cache footprint): a full-width tile, the bias in shared memory, vector-aligned rows and
+            // expert sizes that are multiples of 8.  Everything else (ragged last column tile, odd sizes, a bias too
+            // long for the cache) goes through the compact generic loop below.
+            const bool fast_tile = bias_fast && (N & 7) == 0 && n0 + BN <= N && (!mask_on || (ep.expert_size & 7) == 0);
             uint32_t ra[16], rb[GATED ? 1 : 16], ga[GATED ? 16 : 1];
-            if (!GATED) tmem_ld16_issue(tbase, ra);
+            if (fast_tile) {
+                // Non-gated: the next unit's accumulators are prefetched into a second register set.  Gated tiles need
+                // two accumulators per column; a second set would spill, so each unit is loaded when it is needed and
+                // the other epilogue warps of the SM sub-partition cover the latency.
+                if (!GATED) tmem_ld16_issue(tbase, ra);
 #pragma unroll
-            for (int u = 0; u < N_UNITS; ++u) {             // at most 4 units
-                const int col0 = colw + u * 16;
-                uint32_t (&r)[16] = GATED ? ra : ((u & 1) ? reinterpret_cast<uint32_t (&)[16]>(rb) : ra);
-                uint32_t (&g)[16] = reinterpret_cast<uint32_t (&)[16]>(ga);
-                if (col0 >= N) {                            // warp-uniform (ragged last column tile)
-                    if (!GATED) tmem_ld_wait();
-                    break;
-                }
-                if (GATED) {
-                    tmem_ld16_issue(tbase + u * 16, ra);
-                    tmem_ld16_issue(tbase + u * 16 + BN, reinterpret_cast<uint32_t (&)[16]>(ga));
-                }
-
-                // selection bits of this row for the 16 columns
-                uint32_t keep = 0xffffu;
-                if (EPI == D2D_EPI_UP_MASKED && mrow) {
-                    keep = 0u;
-                    if (gran8) {
-                        // expert sizes that are multiples of 8: each 8-column half of the unit belongs to one
-                        // expert; e = col / s by a multiply-high with the precomputed reciprocal
+                for (int u = 0; u < N_UNITS; ++u) {             // at most 4 units
+                    const int col0 = colw + u * 16;
+                    uint32_t (&r)[16] = GATED ? ra : ((u & 1) ? reinterpret_cast<uint32_t (&)[16]>(rb) : ra);
+                    uint32_t (&g)[16] = reinterpret_cast<uint32_t (&)[16]>(ga);
+                    if (GATED) {
+                        tmem_ld16_issue(tbase + u * 16, ra);
+                        tmem_ld16_issue(tbase + u * 16 + BN, reinterpret_cast<uint32_t (&)[16]>(ga));
+                    }
+                    // selection bits of this row: each 8-column half of the unit belongs to one expert;
+                    // e = col / s by a multiply-high with the precomputed reciprocal
+                    uint32_t keep = 0xffffu;
+                    if (mask_on && mrow) {
+                        keep = 0u;
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
                             const uint32_t ee = __umulhi((uint32_t)(col0 + 8 * h), ep.inv_expert_size);
@@ -608,40 +607,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                             }
                             if ((wd >> (ee & 31)) & 1u) keep |= 0xffu << (8 * h);
                         }
-                    } else {
-                        const int s = ep.expert_size;
-                        int ee = e, l = lo;
-                        while (l < 16) {
-                            if ((ee >> 5) != widx) {
-                                widx = ee >> 5;
-                                if (ep.mask_words <= MASK_REGS) {
-                                    word = 0u;
-#pragma unroll
-                                    for (int i = 0; i < MASK_REGS; ++i) word = (i == widx) ? mw[i] : word;
-                                } else {
-                                    word = __ldg(mrow + widx);
-                                }
-                            }
-                            const int hi = l + s;
-                            if ((word >> (ee & 31)) & 1u) {
-                                const int a = l < 0 ? 0 : l, b2 = hi > 16 ? 16 : hi;
-                                keep |= ((1u << b2) - 1u) & ~((1u << a) - 1u);
-                            }
-                            l = hi;
-                            ++ee;
-                        }
-                        // advance to the expert that owns the first column of the next unit
-                        lo -= 16;
-                        while (lo + s <= 0) { lo += s; ++e; }
                     }
-                }
-                tmem_ld_wait();                                               // this unit's accumulators have landed
-                if (!GATED && u + 1 < N_UNITS)                                // the next unit's load overlaps the math below
-                    tmem_ld16_issue(tbase + (u + 1) * 16, (u & 1) ? ra : reinterpret_cast<uint32_t (&)[16]>(rb));
+                    tmem_ld_wait();                                               // this unit's accumulators have landed
+                    if (!GATED && u + 1 < N_UNITS)                                // the next unit's load overlaps the math below
+                        tmem_ld16_issue(tbase + (u + 1) * 16, (u & 1) ? ra : reinterpret_cast<uint32_t (&)[16]>(rb));
 
-                if (col0 + 16 <= N && bias_fast && (N & 7) == 0) {   // (N % 8 also keeps the 16-byte vector accesses aligned)
                     float v[16];
-                    epilogue_16<EPI, ACT, GATED>(r, g, v, bias_f, ep.bias != nullptr, col0, keep, gran8);
+                    epilogue_16<EPI, ACT, GATED>(r, g, v, bias_f, ep.bias != nullptr, col0, keep, mask_on && mrow != nullptr);
                     if (row < M) {
                         if (EPI == D2D_EPI_PARTIAL_F32) {
                             float *o = (float *)ep.out + (size_t)row * N + col0;
@@ -671,9 +643,40 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                             }
                         }
                     }
-                } else {
-                    // rare: ragged last column tile, odd leading dimension, or a bias too long for the cache
-                    epilogue_16_slow<EPI, ACT, GATED>(r, g, ep.bias, ep.out, row, M, col0, N, keep);
+                }
+            } else {
+                // generic loop: one unit at a time, every bound checked, any expert size
+                uint32_t (&g)[16] = reinterpret_cast<uint32_t (&)[16]>(ga);
+#pragma unroll 1
+                for (int u = 0; u < N_UNITS; ++u) {
+                    const int col0 = colw + u * 16;
+                    if (col0 >= N) break;                       // warp-uniform (ragged last column tile)
+                    tmem_ld16_issue(tbase + u * 16, ra);
+                    if (GATED) tmem_ld16_issue(tbase + u * 16 + BN, g);
+                    uint32_t keep = 0xffffu;
+                    if (mask_on && mrow) {
+                        keep = 0u;
+                        const int s = ep.expert_size;
+                        int ee = e, l = lo;
+                        while (l < 16) {
+                            if ((ee >> 5) != widx) {
+                                widx = ee >> 5;
+                                word = __ldg(mrow + widx);
+                            }
+                            const int hi = l + s;
+                            if ((word >> (ee & 31)) & 1u) {
+                                const int a = l < 0 ? 0 : l, b2 = hi > 16 ? 16 : hi;
+                                keep |= ((1u << b2) - 1u) & ~((1u << a) - 1u);
+                            }
+                            l = hi;
+                            ++ee;
+                        }
+                        // advance to the expert that owns the first column of the next unit
+                        lo -= 16;
+                        while (lo + s <= 0) { lo += s; ++e; }
+                    }
+                    tmem_ld_wait();
+                    epilogue_16_slow<EPI, ACT, GATED>(ra, g, ep.bias, ep.out, row, M, col0, N, keep);
                 }
             }
             // all of this warp's TMEM reads of the buffer are complete: hand it back to the MMA warp
