@@ -577,6 +577,27 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 // two accumulators per column; a second set would spill, so each unit is loaded when it is needed and
                 // the other epilogue warps of the SM sub-partition cover the latency.
                 if (!GATED) tmem_ld16_issue(tbase, ra);
+                // selection bits of this row, one per 8-column group of the warp's columns (each group belongs to one
+                // expert; e = col / s by a multiply-high with the precomputed reciprocal); done once per tile so that the
+                // unrolled units below stay small
+                uint32_t kbits = 0xffffffffu;
+                if (mask_on && mrow) {
+                    kbits = 0u;
+#pragma unroll
+                    for (int h = 0; h < COLS_PER_WARP / 8; ++h) {
+                        const uint32_t ee = __umulhi((uint32_t)(colw + 8 * h), ep.inv_expert_size);
+                        const int wi = (int)(ee >> 5);
+                        uint32_t wd;
+                        if (ep.mask_words <= MASK_REGS) {
+                            wd = mw[0];
+#pragma unroll
+                            for (int i = 1; i < MASK_REGS; ++i) wd = (i == wi) ? mw[i] : wd;
+                        } else {
+                            wd = __ldg(mrow + wi);
+                        }
+                        kbits |= ((wd >> (ee & 31)) & 1u) << h;
+                    }
+                }
 #pragma unroll
                 for (int u = 0; u < N_UNITS; ++u) {             // at most 4 units
                     const int col0 = colw + u * 16;
@@ -586,34 +607,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                         tmem_ld16_issue(tbase + u * 16, ra);
                         tmem_ld16_issue(tbase + u * 16 + BN, reinterpret_cast<uint32_t (&)[16]>(ga));
                     }
-                    // selection bits of this row: each 8-column half of the unit belongs to one expert;
-                    // e = col / s by a multiply-high with the precomputed reciprocal
-                    uint32_t keep = 0xffffu;
-                    if (mask_on && mrow) {
-                        keep = 0u;
-#pragma unroll
-                        for (int h = 0; h < 2; ++h) {
-                            const uint32_t ee = __umulhi((uint32_t)(col0 + 8 * h), ep.inv_expert_size);
-                            const int wi = (int)(ee >> 5);
-                            uint32_t wd;
-                            if (ep.mask_words <= 4) {
-                                wd = wi == 0 ? mw[0] : wi == 1 ? mw[1] : wi == 2 ? mw[2] : mw[3];
-                            } else if (ep.mask_words <= MASK_REGS) {
-                                wd = mw[0];
-#pragma unroll
-                                for (int i = 1; i < MASK_REGS; ++i) wd = (i == wi) ? mw[i] : wd;
-                            } else {
-                                wd = __ldg(mrow + wi);
-                            }
-                            if ((wd >> (ee & 31)) & 1u) keep |= 0xffu << (8 * h);
-                        }
-                    }
+                    const uint32_t keep = ((kbits >> (2 * u)) & 1u ? 0x00ffu : 0u) | ((kbits >> (2 * u + 1)) & 1u ? 0xff00u : 0u);
                     tmem_ld_wait();                                               // this unit's accumulators have landed
                     if (!GATED && u + 1 < N_UNITS)                                // the next unit's load overlaps the math below
                         tmem_ld16_issue(tbase + (u + 1) * 16, (u & 1) ? ra : reinterpret_cast<uint32_t (&)[16]>(rb));
 
                     float v[16];
-                    epilogue_16<EPI, ACT, GATED>(r, g, v, bias_f, ep.bias != nullptr, col0, keep, mask_on && mrow != nullptr);
+                    epilogue_16<EPI, ACT, GATED>(r, g, v, bias_f, ep.bias != nullptr, col0, keep, EPI == D2D_EPI_UP_MASKED);
                     if (row < M) {
                         if (EPI == D2D_EPI_PARTIAL_F32) {
                             float *o = (float *)ep.out + (size_t)row * N + col0;
