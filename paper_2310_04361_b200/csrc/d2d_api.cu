@@ -483,7 +483,11 @@ d2d_status d2d_layer_fwd_host(const d2d_layer *layer, const void *x_host, int32_
     // chunk c+1 to the device (copy-in stream), the layer on chunk c (`stream`) and the copy of chunk c-1 back to the
     // host (copy-out stream) run at the same time; PCIe carries both directions at once.  The routing buffers and the
     // layer workspace are reused chunk after chunk, which is safe because the layer calls are serial on `stream`.
-    const int n_chunks = T >= 2048 ? d2d_layer::kHostChunks : 1;
+    int n_chunks = T >= 2048 ? d2d_layer::kHostChunks : 1;
+    if (const char *e = getenv("D2D_HOST_CHUNKS")) {          // 1 .. 4, for tuning
+        const int n = atoi(e);
+        if (n >= 1 && n <= d2d_layer::kHostChunks && T >= 128 * n) n_chunks = n;
+    }
     if (n_chunks == 1) {
         D2D_CUDA_TRY(cudaMemcpyAsync(base + h.x_off, x_host, row_bytes, cudaMemcpyHostToDevice, st));
         d2d_status rc = d2d_layer_fwd(layer, base + h.x_off, T, tau, base + h.y_off, nullptr, &r,
