@@ -244,7 +244,8 @@ D2D_API d2d_status d2d_layer_fwd(const d2d_layer *layer, const void *x, int32_t 
  * ([T,d] of desc.dtype).  The call copies x to the device, runs the layer,
  * copies y back and synchronises `stream`; all device memory it needs comes
  * from `ws` (device, at least d2d_layer_fwd_host_workspace_bytes bytes).
- * Batches of 2048 tokens or more are cut into four chunks and pipelined over
+ * Batches of 8192 tokens or more are cut into up to four chunks (of at least
+ * 4096 tokens) and pipelined over
  * two copy streams the layer owns (copy in / layer / copy out overlap; tokens
  * are independent, so the result is the same); this needs page-locked host
  * buffers to be effective.  Returns the data-dependent status as well

@@ -483,7 +483,10 @@ d2d_status d2d_layer_fwd_host(const d2d_layer *layer, const void *x_host, int32_
     // chunk c+1 to the device (copy-in stream), the layer on chunk c (`stream`) and the copy of chunk c-1 back to the
     // host (copy-out stream) run at the same time; PCIe carries both directions at once.  The routing buffers and the
     // layer workspace are reused chunk after chunk, which is safe because the layer calls are serial on `stream`.
-    int n_chunks = T >= 2048 ? d2d_layer::kHostChunks : 1;
+    // a chunk should still fill the GPU (a 1024-token layer call costs almost as much as a 4096-token one), so
+    // chunks hold at least 4096 tokens
+    int n_chunks = T / 4096;
+    n_chunks = n_chunks < 1 ? 1 : n_chunks > d2d_layer::kHostChunks ? d2d_layer::kHostChunks : n_chunks;
     if (const char *e = getenv("D2D_HOST_CHUNKS")) {          // 1 .. 4, for tuning
         const int n = atoi(e);
         if (n >= 1 && n <= d2d_layer::kHostChunks && T >= 128 * n) n_chunks = n;

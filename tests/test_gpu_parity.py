@@ -348,9 +348,9 @@ def test_layer_fwd_host_buffers(api):
 
 
 def test_layer_fwd_host_chunked_pipeline_matches_device_call(api):
-    """2048 tokens or more: the host call runs in four pipelined chunks (ragged last chunk here); tokens are
+    """8192 tokens or more: the host call runs in pipelined chunks (two here, the second ragged); tokens are
     independent, so the result equals one device call on the whole batch."""
-    T = 2048 + 300
+    T = 8192 + 300
     cfg, w, x, layer = _setup(api, "bert", T)
     xh = torch.from_numpy(x).to(torch.bfloat16).pin_memory()
     yh = torch.empty_like(xh).pin_memory()
@@ -365,7 +365,7 @@ def test_layer_fwd_host_chunked_pipeline_matches_device_call(api):
 
 def test_layer_fwd_host_reports_nonfinite_scores(api):
     """An infinite token row makes its router scores non-finite: the host call returns the data-dependent status."""
-    T = 2048 + 64
+    T = 8192 + 64
     cfg, w, x, layer = _setup(api, "bert", T)
     xb = x.copy()
     # a row aligned with the signs of one router row overflows that hidden unit to +inf (NaN or mixed infinities would
