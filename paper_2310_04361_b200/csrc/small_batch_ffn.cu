@@ -106,19 +106,28 @@ small_router_kernel(const TT *__restrict__ x, int T, int d, const TT *__restrict
     const int j0 = blockIdx.x * 8;
     const int rows = d_h - j0 < 8 ? d_h - j0 : 8;
 
+    // copy groups: [W_r1 rows + first token block] first, W_r2 (needed only by the last CTA, prefetched by all) second,
+    // so that layer 1 starts as soon as its own operands have landed and does not wait for the 2*E*d_h bytes of W_r2
     cta_copy_async(w1s, w_r1 + (size_t)j0 * d, (size_t)rows * d * sizeof(TT));
+    {
+        const int ntok0 = T < TBLK ? T : TBLK;
+        cta_copy_async(xs, x, (size_t)ntok0 * d * sizeof(TT));
+    }
     cp_async_commit();
-    if (stage_w2) cta_copy_async(w2s, w_r2, (size_t)E * d_h * sizeof(TT));     // needed only by the last CTA; prefetched by all
+    if (stage_w2) cta_copy_async(w2s, w_r2, (size_t)E * d_h * sizeof(TT));
     cp_async_commit();
 
     for (int t0 = 0; t0 < T; t0 += TBLK) {
         const int ntok = T - t0 < TBLK ? T - t0 : TBLK;
-        __syncthreads();                                          // previous block's readers of xs are done
-        cta_copy_async(xs, x + (size_t)t0 * d, (size_t)ntok * d * sizeof(TT));
+        if (t0 > 0) {
+            __syncthreads();                                      // previous block's readers of xs are done
+            cta_copy_async(xs, x + (size_t)t0 * d, (size_t)ntok * d * sizeof(TT));
+            cp_async_commit();
+        }
         if (ntok < TBLK)                                          // unused token slots read zeros
             for (int i = threadIdx.x; i < (TBLK - ntok) * d; i += NT) xs[(size_t)ntok * d + i] = d2d_from_float<TT>(0.0f);
-        cp_async_commit();
-        cp_async_wait<0>();                                       // everything issued so far has landed
+        if (t0 == 0) cp_async_wait<1>();                          // the first group: W_r1 rows and the first token block
+        else cp_async_wait<0>();
         __syncthreads();
         if (warp < rows) {
             float acc[TBLK];
