@@ -100,7 +100,10 @@ small_router_kernel(const TT *__restrict__ x, int T, int d, const TT *__restrict
     TT *w1s = reinterpret_cast<TT *>(smem_raw);
     TT *xs = w1s + (size_t)8 * d;
     TT *w2s = xs + (size_t)TBLK * d;
-    float *us = reinterpret_cast<float *>(w2s + (stage_w2 ? (size_t)E * d_h : 0));
+    // W_r2 rows are staged with a pitch of d_h + 16 bytes: in layer 2 each thread walks its own row, and with the
+    // natural pitch (a multiple of 128 bytes) all lanes of a warp would hit the same shared-memory banks
+    const int w2_pitch = d_h + (int)(16 / sizeof(TT));
+    float *us = reinterpret_cast<float *>(w2s + (stage_w2 ? (size_t)E * w2_pitch : 0));
     __shared__ unsigned int my_ticket;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int j0 = blockIdx.x * 8;
@@ -114,7 +117,14 @@ small_router_kernel(const TT *__restrict__ x, int T, int d, const TT *__restrict
         cta_copy_async(xs, x, (size_t)ntok0 * d * sizeof(TT));
     }
     cp_async_commit();
-    if (stage_w2) cta_copy_async(w2s, w_r2, (size_t)E * d_h * sizeof(TT));
+    if (stage_w2) {
+        const int cpr = d_h * (int)sizeof(TT) / 16;               // 16-byte chunks per row
+        for (int c = threadIdx.x; c < E * cpr; c += NT) {
+            const int row = c / cpr, w = c - row * cpr;
+            cp_async16(reinterpret_cast<char *>(w2s + (size_t)row * w2_pitch) + w * 16,
+                       reinterpret_cast<const char *>(w_r2 + (size_t)row * d_h) + w * 16);
+        }
+    }
     cp_async_commit();
 
     for (int t0 = 0; t0 < T; t0 += TBLK) {
@@ -162,7 +172,7 @@ small_router_kernel(const TT *__restrict__ x, int T, int d, const TT *__restrict
             for (int q = 0; q < TBLK; ++q) acc[q] = 0.0f;
             for (int c = 0; c < d_h; c += 8) {
                 float wv[8];
-                if (stage_w2) lds8(w2s + (size_t)i * d_h + c, wv);
+                if (stage_w2) lds8(w2s + (size_t)i * w2_pitch + c, wv);
                 else d2d_load8(w_r2 + (size_t)i * d_h + c, wv);
 #pragma unroll
                 for (int q = 0; q < TBLK; ++q) {
@@ -376,7 +386,7 @@ d2d_status launch_router_tb(const d2d_layer *L, const void *x, int T, float *R, 
 {
     const d2d_layer_desc &D = L->desc;
     const size_t base = (size_t)(8 + TBLK) * D.d * sizeof(TT) + (size_t)T * D.d_h * 4 + (size_t)T * ((D.n_experts + 31) / 32) * 4;
-    const size_t w2_bytes = (size_t)D.n_experts * D.d_h * sizeof(TT);
+    const size_t w2_bytes = (size_t)D.n_experts * (D.d_h * sizeof(TT) + 16);      // padded pitch, see the kernel
     const int stage_w2 = base + w2_bytes <= kSmemLimit ? 1 : 0;
     const size_t smem = base + (stage_w2 ? w2_bytes : 0);
     auto kern = small_router_kernel<TT, TBLK>;
