@@ -10,7 +10,7 @@
 //
 // Every mbarrier wait is bounded: when the limit runs out the role records D2D_ERR_TIMEOUT in the
 // status word and leaves its loop, all roles meet at the final barrier, TMEM is freed and the
-// kernel returns (no trap, no endless spin).  No multicast loads are used.
+// kernel returns (no trap, no endless spin).  Every load is a plain per-CTA load.
 #include "gemm_tc.cuh"
 
 #include <stdlib.h>
@@ -117,7 +117,7 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // TMA load issued by either CTA of a pair; the transaction bytes are credited to the barrier at `bar`
-// (a shared::cluster address, normally the leader CTA's barrier).  No multicast.
+// (a shared::cluster address, normally the leader CTA's barrier).  Each CTA loads its own data.
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar)
 {
     asm volatile(
@@ -134,12 +134,13 @@ __device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t da, uin
         ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
         : "memory");
 }
-// arrives on the barrier at the same shared-memory offset in both CTAs of the pair once the MMAs issued so far retire
+// arrives on the barrier at the same shared-memory offset in BOTH CTAs of the pair once the MMAs issued so far retire:
+// two commits, one per CTA's copy of the barrier (addressed through the cluster window)
 __device__ __forceinline__ void umma_commit_pair(uint32_t bar)
 {
-    const uint16_t both = 3;
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                 ::"r"(bar), "h"(both) : "memory");
+    const uint32_t b0 = map_to_cta(bar, 0), b1 = map_to_cta(bar, 1);
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(b0) : "memory");
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(b1) : "memory");
 }
 
 struct EpiParams {
@@ -297,8 +298,8 @@ __host__ __device__ constexpr int pow2_at_least(int v) { return v <= 32 ? 32 : v
 // PAIR: two CTAs of a cluster (adjacent SMs) compute one 256 x BN tile with tcgen05.mma.cta_group::2: each CTA
 // loads its own 128 rows of A and only HALF of the B tile, the MMA reads both halves, and each CTA ends up with
 // its 128 accumulator rows in its own TMEM.  This cuts the L2 -> SM operand traffic per FLOP by 1.5x without
-// any multicast load.  The even CTA issues the MMAs; barriers that both CTAs need are signalled with
-// multicast commits (stage release, accumulator ready) or remote arrives (accumulator drained).
+// any load that is shared between CTAs.  The even CTA issues the MMAs; barriers that both CTAs need are signalled
+// with one commit per CTA (stage release, accumulator ready) or remote arrives (accumulator drained).
 template <int BN, int STAGES, int EPI, int ACT, bool GATED, bool PAIR>
 __global__ void __launch_bounds__(NTHREADS_V2, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,

@@ -6,7 +6,7 @@
 // so the hidden activations never touch HBM, R is written once (the caller may want it) and the
 // mask kernel's extra pass over R disappears.  One CTA per 128 tokens; 18 warps: TMA producer,
 // MMA issuer, 16 epilogue warps (four per TMEM lane quadrant, each a quarter of the columns).
-// All mbarrier waits are bounded (status D2D_ERR_TIMEOUT); no multicast.
+// All mbarrier waits are bounded (status D2D_ERR_TIMEOUT); every load is a plain per-CTA load.
 #include <cuda.h>
 
 #include "d2d_common.cuh"
