@@ -254,6 +254,36 @@ D2D_API size_t d2d_layer_fwd_host_workspace_bytes(const d2d_layer *layer, int32_
 D2D_API d2d_status d2d_layer_fwd_host(const d2d_layer *layer, const void *x_host, int32_t T, float tau, void *y_host,
                               void *ws, size_t ws_bytes, void *stream);
 
+/* Layer groups (Sec. 3.5: every projection matrix of the attention layer is
+ * replaced by its own MoE layer, so a converted block has four MoE layers in
+ * the attention and one in the FFN).  The Q, K and V projections read the same
+ * token rows: a group holds n_layers (1..4) layers of ONE shape (equal desc)
+ * and runs them on a shared input as one launch sequence.  Each layer keeps
+ * its own router, its own threshold rule (max over ITS experts, Eq. 4) and its
+ * own output; the result equals n_layers separate d2d_layer_fwd calls.
+ *   layers   : host array of layer handles; the group does not own them and
+ *              they must outlive it; a layer may appear once.
+ *   x        : device [T, d] of desc.dtype, shared by all layers.
+ *   y        : device [n_layers, T, d] (layer l's output at y + l*T*d elements;
+ *              T*d*sizeof(elem) must be a multiple of 16).
+ *   routing  : host array of n_layers d2d_routing (outputs, all required as
+ *              in d2d_layer_fwd); routing[l] describes layer l.
+ *   ws       : device workspace of at least d2d_group_workspace_bytes bytes.
+ * bf16, not gated, d_h = 128, E a multiple of 32 and at most 256, d_ff a
+ * multiple of 64: the group owns stacked copies of the weights and the routers
+ * run as one grid, the up projections as one GEMM and the down projections as
+ * one batched GEMM (T of 5 or more); for T <= 4 (fp32: T <= 8) of any shape
+ * the decode kernels serve all layers in two launches.  Other shapes run the
+ * layers one after the other.  Device status: timeouts of the merged GEMMs
+ * are reported in routing[0].status.  Like a layer, a group (and its layers)
+ * serves one call at a time. */
+typedef struct d2d_group d2d_group;
+D2D_API d2d_status d2d_group_create(d2d_layer *const *layers, int32_t n_layers, void *stream, d2d_group **out);
+D2D_API d2d_status d2d_group_destroy(d2d_group *group);
+D2D_API size_t d2d_group_workspace_bytes(const d2d_group *group, int32_t max_tokens);
+D2D_API d2d_status d2d_group_fwd(const d2d_group *group, const void *x, int32_t T, float tau, void *y,
+                                 d2d_routing *routing, void *ws, size_t ws_bytes, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

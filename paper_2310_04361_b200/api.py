@@ -29,7 +29,7 @@ ACTS = {"relu": 0, "gelu_erf": 1, "gelu_tanh": 2, "silu": 3}
 EXPORTS = ["d2d_status_str", "d2d_launch_count", "d2d_layer_create", "d2d_layer_destroy", "d2d_workspace_bytes",
            "d2d_select_workspace_bytes", "d2d_router_fwd", "d2d_select_dynk", "d2d_select_dynk_static", "d2d_select_topk",
            "d2d_routing_from_mask", "d2d_moe_ffn_fwd", "d2d_expert_up_fwd", "d2d_expert_down_fwd", "d2d_layer_fwd", "d2d_layer_fwd_host_workspace_bytes",
-           "d2d_layer_fwd_host"]
+           "d2d_layer_fwd_host", "d2d_group_create", "d2d_group_destroy", "d2d_group_workspace_bytes", "d2d_group_fwd"]
 
 
 class LayerDesc(ctypes.Structure):
@@ -70,6 +70,12 @@ _lib.d2d_layer_fwd.argtypes = [c_void_p, c_void_p, c_int32, c_float, c_void_p, c
 _lib.d2d_layer_fwd_host_workspace_bytes.restype = c_size_t
 _lib.d2d_layer_fwd_host_workspace_bytes.argtypes = [c_void_p, c_int32]
 _lib.d2d_layer_fwd_host.argtypes = [c_void_p, c_void_p, c_int32, c_float, c_void_p, c_void_p, c_size_t, c_void_p]
+_lib.d2d_group_create.argtypes = [POINTER(c_void_p), c_int32, c_void_p, POINTER(c_void_p)]
+_lib.d2d_group_destroy.argtypes = [c_void_p]
+_lib.d2d_group_workspace_bytes.restype = c_size_t
+_lib.d2d_group_workspace_bytes.argtypes = [c_void_p, c_int32]
+_lib.d2d_group_fwd.argtypes = [c_void_p, c_void_p, c_int32, c_float, c_void_p, POINTER(RoutingStruct), c_void_p, c_size_t,
+                               c_void_p]
 
 
 def launch_count() -> int:
@@ -250,6 +256,51 @@ class Layer:
                                        c_void_p(y_host.data_ptr()), _ptr(ws), ws.numel(), _stream(stream)),
                "d2d_layer_fwd_host")
         return y_host
+
+
+class LayerGroup:
+    """Layers of one shape that read the same tokens (the Q, K and V projections of an attention layer): d2d_group_*."""
+
+    def __init__(self, layers: list):
+        self.layers = list(layers)                      # the group does not own the layers: keep them alive
+        self.device = self.layers[0].device if self.layers else torch.device("cuda:0")
+        arr = (c_void_p * len(self.layers))(*[l.handle for l in self.layers])
+        handle = c_void_p()
+        with torch.cuda.device(self.device):
+            _check(_lib.d2d_group_create(arr, len(self.layers), _stream(), ctypes.byref(handle)), "d2d_group_create")
+        self.handle = handle
+        self._ws = None
+
+    def close(self):
+        if getattr(self, "handle", None):
+            _lib.d2d_group_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def workspace(self, T: int):
+        need = int(_lib.d2d_group_workspace_bytes(self.handle, T))
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty((need,), dtype=torch.uint8, device=self.device)
+        return self._ws
+
+    def group_fwd(self, x, tau: float, y=None, routings: list | None = None, stream=None):
+        """y: [n_layers, T, d]; routings: one Routing per layer (outputs)."""
+        T = x.shape[0]
+        n, L0 = len(self.layers), self.layers[0]
+        if y is None:
+            y = torch.empty((n, T, L0.d), dtype=L0.tdtype, device=self.device)
+        if routings is None:
+            routings = [l.new_routing(T) for l in self.layers]
+        arr = (RoutingStruct * n)(*[r.struct for r in routings])
+        ws = self.workspace(T)
+        _check(_lib.d2d_group_fwd(self.handle, _ptr(x), T, c_float(tau), _ptr(y), arr, _ptr(ws), ws.numel(),
+                                  _stream(stream)), "d2d_group_fwd")
+        return y, routings
 
 
 def select_dynk(R, tau: float, routing: Routing | None = None, dual: bool = False, stream=None,

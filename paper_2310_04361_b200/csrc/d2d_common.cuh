@@ -37,6 +37,25 @@ struct d2d_layer {
     unsigned int *tickets;
 };
 
+// Layers of one shape that read the same token rows (the Q, K and V projections of one attention layer) and run as
+// one launch sequence; see d2d_group_fwd.
+#define D2D_MAX_GROUP 4
+struct d2d_router_weights {
+    const void *w_r1, *b_r1, *w_r2, *b_r2;
+};
+struct d2d_group {
+    int n;
+    d2d_layer *layers[D2D_MAX_GROUP];        // not owned
+    d2d_layer_desc desc;                     // the common shape
+    int merged;                              // 1: the stacked copies below exist and the merged tensor-core path may be used
+    // stacked copies: routers [n*d_h, d], [n*d_h], [n*E, d_h], [n*E]; W1 [n*d_ff, d], b1 [n*d_ff]; W2 [n*d, d_ff], b2 [n*d]
+    void *w_r1, *b_r1, *w_r2, *b_r2, *w1, *b1, *w2, *b2;
+    void *slab;
+    int *up_counter;                         // tile counter of the merged up projection (inside the slab, self-resetting)
+    cudaStream_t side_stream;
+    cudaEvent_t ev_fork, ev_join;
+};
+
 #define D2D_CUDA_TRY(expr)                                   \
     do {                                                     \
         cudaError_t err__ = (expr);                          \
@@ -76,6 +95,10 @@ d2d_status d2d_small_select(const float *R, int T, int E, float tau, const d2d_r
 bool d2d_router_fused_supports(const d2d_layer_desc &D, int T);
 d2d_status d2d_router_fused(const d2d_layer *L, const void *x, int T, float tau, int do_mask, float *R, uint32_t *mask,
                             int32_t *k, int32_t *status, cudaStream_t st);
+d2d_status d2d_router_fused_group(const d2d_layer_desc &D, const d2d_router_weights &w, int n_layers, const void *x, int T,
+                                  float tau, const d2d_routing *routing, uint32_t *mask_cat, int cat_words, cudaStream_t st);
+d2d_status d2d_small_group_fwd(const d2d_layer *const *layers, int n, const void *x, int T, float tau, const d2d_routing *routing,
+                               float *const *R, float *const *u, float *const *y32, void *y, cudaStream_t st);
 bool d2d_small_router_supports(const d2d_layer_desc &D, int T);
 size_t d2d_small_router_ws_bytes(const d2d_layer *L, int T);
 // select_into != NULL: the kernel's last CTA also performs the dynamic-k selection (threshold tau) and writes the routing

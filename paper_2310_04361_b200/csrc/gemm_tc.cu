@@ -155,6 +155,7 @@ struct EpiParams {
     int late_wait;                   // 1: only the epilogue waits for the previous kernel of the stream (see below)
     int gate_cat;                    // 1 (gated): tm_b covers up and gate rows interleaved in blocks of BN, one load brings both
     int band_rows;                   // > 0: tiles are walked column-major inside bands of this many row tiles (L2 reuse)
+    int batch;                       // >= 1 problems of one shape: A columns, B rows, bias entries and out advance per problem
 };
 
 // Tile index -> (row tile, column tile).  Plain order is row-major: CTAs that run together share a few rows of A and
@@ -327,17 +328,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     constexpr int MASK_REGS = 8;                                     // selection words of a row kept in registers (E <= 256; wider masks are read through L1)
     // the whole bias vector is staged once, as float32, behind the operand stages when it fits
     float *bias_f = reinterpret_cast<float *>(smem + (size_t)STAGES * STAGE_BYTES);
-    const bool bias_cached = ep.bias != nullptr && N <= BIAS_CACHE_ELEMS && (N & 3) == 0;
+    const int NB = N * ep.batch;                                     // bias entries of all problems
+    const bool bias_cached = ep.bias != nullptr && NB <= BIAS_CACHE_ELEMS && (N & 3) == 0;
     if (bias_cached) {
         // 16-byte loads, all issued before the first use: the fill costs one memory latency, not N / threads of them
-        for (int i = threadIdx.x * 8; i < N; i += NTHREADS_V2 * 8) {
+        for (int i = threadIdx.x * 8; i < NB; i += NTHREADS_V2 * 8) {
             float b8[8];
-            if (i + 8 <= N) {
+            if (i + 8 <= NB) {
                 d2d_load8(ep.bias + i, b8);
 #pragma unroll
                 for (int q = 0; q < 8; ++q) bias_f[i + q] = b8[q];
             } else {
-                for (int q = 0; i + q < N; ++q) bias_f[i + q] = __bfloat162float(ep.bias[i + q]);
+                for (int q = 0; i + q < NB; ++q) bias_f[i + q] = __bfloat162float(ep.bias[i + q]);
             }
         }
     }
@@ -347,7 +349,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     const int n_tiles = (N + BN - 1) / BN;
     // work item = (output tile, K split); with k_splits > 1 every item accumulates a slice of K and the
     // epilogue adds its partial sums to a float32 buffer (small-M problems that would leave most SMs idle)
-    const int total_tiles = ((M + TM - 1) / TM) * n_tiles * k_splits;
+    const int tiles_pp = ((M + TM - 1) / TM) * n_tiles;            // output tiles per problem
+    const int total_tiles = tiles_pp * ep.batch * k_splits;
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;           // 0 = the CTA that issues the MMAs
     const int worker = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
     const int n_workers = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
@@ -411,11 +414,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     mbar_arrive(smem_u32(&sched_full[sl]));       // release: the slot's content is visible to whoever sees the phase
                 }
                 if (item >= total_tiles) break;
-                const int tile = item / k_splits, sp = item - tile * k_splits;
+                int tile = item / k_splits;
+                const int sp = item - tile * k_splits;
                 const int kb0 = (int)((long long)sp * nkb / k_splits), kb1 = (int)((long long)(sp + 1) * nkb / k_splits);
+                int prob = 0;
+                if (ep.batch > 1) { prob = tile / tiles_pp; tile -= prob * tiles_pp; }
                 int tr, tc;
                 tile_coords(tile, (M + TM - 1) / TM, n_tiles, ep.band_rows, tr, tc);
-                const int m0 = tr * TM + (int)rank * BM, n0 = tc * BN + (int)rank * B_ROWS;
+                const int m0 = tr * TM + (int)rank * BM, n0 = prob * N + tc * BN + (int)rank * B_ROWS;
+                const int ka = prob * K;                      // problem p reads columns [p*K, (p+1)*K) of A
                 for (int kb = kb0; kb < kb1; ++kb, ++it) {
                     const uint32_t s = it % STAGES, round = it / STAGES;
                     ok = mbar_wait(smem_u32(&bar_empty[s]), (round & 1u) ^ 1u, ep.status);
@@ -425,13 +432,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                         // both CTAs' bytes are credited to the leader's barrier (where the MMAs are issued)
                         const uint32_t full = map_to_cta(smem_u32(&bar_full[s]), 0);
                         if (rank == 0) mbar_expect_tx(smem_u32(&bar_full[s]), 2u * (uint32_t)STAGE_BYTES);
-                        tma_load_2d_pair(dst, &tm_a, kb * BK, m0, full);
+                        tma_load_2d_pair(dst, &tm_a, ka + kb * BK, m0, full);
                         tma_load_2d_pair(dst + A_BYTES, &tm_b, kb * BK, n0, full);
                         if (GATED) tma_load_2d_pair(dst + A_BYTES + B_BYTES, &tm_b2, kb * BK, n0, full);
                     } else {
                         const uint32_t full = smem_u32(&bar_full[s]);
                         mbar_expect_tx(full, (uint32_t)STAGE_BYTES);
-                        tma_load_2d(dst, &tm_a, kb * BK, m0, full);
+                        tma_load_2d(dst, &tm_a, ka + kb * BK, m0, full);
                         if (GATED && ep.gate_cat) {
                             // up rows [n0, n0+BN) and gate rows [n0, n0+BN) are adjacent in the interleaved copy: one
                             // 2*BN-row box (the producer thread's time per k-block is what bounds the gated main loop)
@@ -532,10 +539,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 if (item < 0) break;
             }
             if (item >= total_tiles) break;
-            const int tile = item / k_splits;
+            int tile = item / k_splits;
+            int prob = 0;
+            if (ep.batch > 1) { prob = tile / tiles_pp; tile -= prob * tiles_pp; }
             int tr, tc;
             tile_coords(tile, (M + TM - 1) / TM, n_tiles, ep.band_rows, tr, tc);
             const int m0 = tr * TM + (int)rank * BM, n0 = tc * BN;
+            // this problem's bias entries and output matrix
+            const float *bias_p = bias_f + prob * N;
+            const __nv_bfloat16 *bias_g = ep.bias ? ep.bias + prob * N : nullptr;
+            void *out_p = (char *)ep.out + (size_t)prob * M * N * ((EPI == D2D_EPI_ABS_F32 || EPI == D2D_EPI_PARTIAL_F32) ? 4 : 2);
             const int row = m0 + quad * 32 + lane;
             // this row's selection words go to registers before the wait, so their latency is hidden
             uint32_t mw[MASK_REGS];
@@ -565,7 +578,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 lo = e * ep.expert_size - colw;             // first column of expert e relative to the current unit (<= 0)
             }
             const bool bias_fast = ep.bias == nullptr || bias_cached;
-            const bool wide_store = (N & 15) == 0 && (reinterpret_cast<uintptr_t>(ep.out) & 31) == 0;   // 32-byte aligned rows
+            const bool wide_store = (N & 15) == 0 && (reinterpret_cast<uintptr_t>(out_p) & 31) == 0;   // 32-byte aligned rows
             const bool mask_on = EPI == D2D_EPI_UP_MASKED && ep.mask != nullptr;                         // CTA-uniform
             // The common case gets a loop of its own with nothing else in it (the epilogue is sensitive to its
             // instruction-cache footprint): a full-width tile, the bias in shared memory, vector-aligned rows and
@@ -614,20 +627,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                         tmem_ld16_issue(tbase + (u + 1) * 16, (u & 1) ? ra : reinterpret_cast<uint32_t (&)[16]>(rb));
 
                     float v[16];
-                    epilogue_16<EPI, ACT, GATED>(r, g, v, bias_f, ep.bias != nullptr, col0, keep, EPI == D2D_EPI_UP_MASKED);
+                    epilogue_16<EPI, ACT, GATED>(r, g, v, bias_p, ep.bias != nullptr, col0, keep, EPI == D2D_EPI_UP_MASKED);
                     if (row < M) {
                         if (EPI == D2D_EPI_PARTIAL_F32) {
-                            float *o = (float *)ep.out + (size_t)row * N + col0;
+                            float *o = (float *)out_p + (size_t)row * N + col0;
 #pragma unroll
                             for (int j = 0; j < 16; j += 4)
                                 asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(o + j), "f"(v[j]), "f"(v[j + 1]),
                                              "f"(v[j + 2]), "f"(v[j + 3]) : "memory");
                         } else if (EPI == D2D_EPI_ABS_F32) {
-                            float *o = (float *)ep.out + (size_t)row * N + col0;
+                            float *o = (float *)out_p + (size_t)row * N + col0;
 #pragma unroll
                             for (int j = 0; j < 16; j += 4) *reinterpret_cast<float4 *>(o + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
                         } else {
-                            __nv_bfloat16 *o = (__nv_bfloat16 *)ep.out + (size_t)row * N + col0;
+                            __nv_bfloat16 *o = (__nv_bfloat16 *)out_p + (size_t)row * N + col0;
                             uint32_t pk[8];
 #pragma unroll
                             for (int j = 0; j < 8; ++j) {
@@ -677,7 +690,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                         while (lo + s <= 0) { lo += s; ++e; }
                     }
                     tmem_ld_wait();
-                    epilogue_16_slow<EPI, ACT, GATED>(ra, g, ep.bias, ep.out, row, M, col0, N, keep);
+                    epilogue_16_slow<EPI, ACT, GATED>(ra, g, bias_g, out_p, row, M, col0, N, keep);
                 }
             }
             // all of this warp's TMEM reads of the buffer are complete: hand it back to the MMA warp
@@ -776,12 +789,14 @@ d2d_status launch(const d2d_gemm_args &g, cudaStream_t st)
     constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + 1024 + (size_t)BIAS_CACHE_ELEMS * 4;
     CUtensorMap ta, tb, tb2;
     const bool gate_cat = GATED && !PAIR && g.b_cat != nullptr && g.b_cat_block == BN;
-    if (!make_map(&ta, g.a, g.M, g.K, BM)) return D2D_ERR_CUDA;
+    const int batch = g.batch > 1 ? g.batch : 1;
+    if (batch > 1 && (GATED || PAIR || g.K % BK != 0)) return D2D_ERR_UNSUPPORTED;
+    if (!make_map(&ta, g.a, g.M, g.K * batch, BM)) return D2D_ERR_CUDA;
     if (gate_cat) {
         if (!make_map(&tb, g.b_cat, 2 * BN * d2d_cdiv(g.N, BN), g.K, 2 * BN)) return D2D_ERR_CUDA;
         tb2 = tb;
     } else {
-        if (!make_map(&tb, g.b, g.N, g.K, B_ROWS)) return D2D_ERR_CUDA;
+        if (!make_map(&tb, g.b, g.N * batch, g.K, B_ROWS)) return D2D_ERR_CUDA;
         if (GATED) {
             if (!make_map(&tb2, g.b_gate, g.N, g.K, B_ROWS)) return D2D_ERR_CUDA;
         } else {
@@ -798,9 +813,9 @@ d2d_status launch(const d2d_gemm_args &g, cudaStream_t st)
     EpiParams ep{(const __nv_bfloat16 *)g.bias, g.out, g.mask, g.mask_words, es, g.status,
                  (uint32_t)((0x100000000ull + (unsigned long long)es - 1) / (unsigned long long)es),
                  PAIR ? nullptr : g.tile_counter, (g.pdl_late_wait && pdl_enabled()) ? 1 : 0, gate_cat ? 1 : 0,
-                 band_rows_for(g.M, g.N, g.K, PAIR ? 2 * BM : BM, GATED)};
+                 band_rows_for(g.M, g.N, g.K, PAIR ? 2 * BM : BM, GATED), batch};
     const int k_splits = g.k_splits > 1 ? g.k_splits : 1;
-    const int tiles = d2d_cdiv(g.N, BN) * d2d_cdiv(g.M, PAIR ? 2 * BM : BM) * k_splits;
+    const int tiles = d2d_cdiv(g.N, BN) * d2d_cdiv(g.M, PAIR ? 2 * BM : BM) * k_splits * batch;
     const int workers = PAIR ? sm_count() / 2 : sm_count();
     const int grid = (tiles < workers ? tiles : workers) * (PAIR ? 2 : 1);
     cudaLaunchConfig_t cfg = {};
@@ -825,13 +840,13 @@ d2d_status launch(const d2d_gemm_args &g, cudaStream_t st)
 
 // Tile width that wastes the fewest SM-rounds: tiles / (rounds * workers), wider tiles preferred on ties
 // (fewer re-reads of A, fewer per-tile overheads).  A "worker" is an SM, or an SM pair for the 2-CTA variant.
-int pick_bn(int M, int N, int tile_m, int workers, const int *cands, int n_cands, double *eff_out)
+int pick_bn(int M, int N, int tile_m, int workers, const int *cands, int n_cands, double *eff_out, int batch = 1)
 {
     int best = cands[0];
     double best_eff = -1.0;
     for (int i = 0; i < n_cands; ++i) {
         const int bn = cands[i];
-        const long tiles = (long)d2d_cdiv(N, bn) * d2d_cdiv(M, tile_m);
+        const long tiles = (long)d2d_cdiv(N, bn) * d2d_cdiv(M, tile_m) * batch;
         const long rounds = (tiles + workers - 1) / workers;
         const double useful = (double)N / ((double)d2d_cdiv(N, bn) * bn);       // ragged last column tile
         const double eff = useful * (double)tiles / (double)(rounds * workers) * (bn >= 128 ? 1.0 : 0.85);
@@ -875,8 +890,8 @@ d2d_status launch_bn(const d2d_gemm_args &g, cudaStream_t st)
         const int cands1[4] = {256, 192, 128, 64};
         double eff2 = 0.0, eff1 = 0.0;
         const int bn2 = pick_bn(g.M, g.N, 2 * BM, sms / 2, cands2, 3, &eff2);
-        const int bn1 = pick_bn(g.M, g.N, BM, sms, cands1, 4, &eff1);
-        if (pair_mode_enabled() && g.M > BM && eff2 >= 0.8 * eff1) {
+        const int bn1 = pick_bn(g.M, g.N, BM, sms, cands1, 4, &eff1, g.batch > 1 ? g.batch : 1);
+        if (pair_mode_enabled() && g.M > BM && g.batch <= 1 && eff2 >= 0.8 * eff1) {
             switch (bn2) {
             case 256: return launch<256, EPI, ACT, false, true>(g, st);
             case 192: return launch<192, EPI, ACT, false, true>(g, st);
@@ -906,15 +921,15 @@ d2d_status launch_up(const d2d_gemm_args &g, cudaStream_t st)
 
 }  // namespace
 
-// y = bf16(partial + bias) after a split-K GEMM
+// y = bf16(partial + bias) after a split-K GEMM; `batch` problems back to back ([batch, M, N] sums, [batch, N] bias)
 __global__ void __launch_bounds__(256)
 splitk_finalize_kernel(const float *__restrict__ partial, const __nv_bfloat16 *__restrict__ bias, __nv_bfloat16 *__restrict__ out,
-                       int M, int N)
+                       int M, int N, int batch)
 {
-    const size_t total = (size_t)M * N;
+    const size_t per = (size_t)M * N, total = per * batch;
     for (size_t i = ((size_t)blockIdx.x * 256 + threadIdx.x) * 4; i < total; i += (size_t)gridDim.x * 1024) {
         const float4 v = __ldcg(reinterpret_cast<const float4 *>(partial + i));
-        const int c = (int)(i % N);
+        const int c = (int)(i / per) * N + (int)(i % N);
         const float o[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int q = 0; q < 4; ++q) out[i + q] = __float2bfloat16_rn(o[q] + (bias ? __bfloat162float(bias[c + q]) : 0.0f));
@@ -923,11 +938,11 @@ splitk_finalize_kernel(const float *__restrict__ partial, const __nv_bfloat16 *_
 
 bool d2d_gemm_tc_available() { return get_encode() != nullptr; }
 
-int d2d_gemm_tc_splits(int M, int N, int K)
+int d2d_gemm_tc_splits(int M, int N, int K, int batch)
 {
     // only single-row-tile problems whose column tiles would occupy less than half of the SMs
     if (M > BM || (N & 3)) return 1;
-    const int tiles = d2d_cdiv(N, 64);
+    const int tiles = d2d_cdiv(N, 64) * (batch > 1 ? batch : 1);
     const int nkb = d2d_cdiv(K, BK);
     int splits = sm_count() / (tiles > 0 ? tiles : 1);
     if (splits > nkb / 2) splits = nkb / 2;          // at least two k-blocks per slice
@@ -943,16 +958,17 @@ d2d_status d2d_gemm_tc(const d2d_gemm_args &g, cudaStream_t st)
     case D2D_EPI_ABS_F32: return launch_bn<D2D_EPI_ABS_F32, 0, false>(g, st);
     case D2D_EPI_BIAS_BF16:
         if (g.k_splits > 1 && g.partial) {
-            if (cudaMemsetAsync(g.partial, 0, (size_t)g.M * g.N * sizeof(float), st) != cudaSuccess) return D2D_ERR_CUDA;
+            const int batch = g.batch > 1 ? g.batch : 1;
+            if (cudaMemsetAsync(g.partial, 0, (size_t)batch * g.M * g.N * sizeof(float), st) != cudaSuccess) return D2D_ERR_CUDA;
             d2d_gemm_args p = g;
             p.epilogue = D2D_EPI_PARTIAL_F32;
             p.bias = nullptr;
             p.out = g.partial;
             const d2d_status rc = launch<64, D2D_EPI_PARTIAL_F32, 0, false, false>(p, st);
             if (rc != D2D_OK) return rc;
-            const int blocks = d2d_cdiv(g.M * g.N, 1024);
+            const int blocks = d2d_cdiv(batch * g.M * g.N, 1024);
             splitk_finalize_kernel<<<blocks < 148 ? blocks : 148, 256, 0, st>>>(g.partial, (const __nv_bfloat16 *)g.bias,
-                                                                                 (__nv_bfloat16 *)g.out, g.M, g.N);
+                                                                                 (__nv_bfloat16 *)g.out, g.M, g.N, batch);
             D2D_LAUNCHED(1);
             return cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
         }

@@ -44,10 +44,15 @@ struct d2d_gemm_args {
     // mask) do.  With programmatic dependent launch the main loops then start while that kernel still runs and only the
     // epilogue waits for it.  Never set this when A may be written by the preceding kernel.
     int pdl_late_wait;
+    // Batched problems with one shape (the down projections of several layers that ran as one merged up projection):
+    // with batch > 1, A is [M, batch*K] and problem p reads its columns [p*K, (p+1)*K); B is [batch*N, K] and bias is
+    // [batch*N], problem p owns rows / entries [p*N, (p+1)*N); out is [batch, M, N] (problem p at out + p*M*N).
+    // Requires K % 64 == 0.  0 and 1 both mean a single problem.
+    int batch;
 };
 
 // Number of K slices d2d_gemm_tc would use for a [M,N,K] down projection (1 = no split) and the float32 scratch it needs.
-int d2d_gemm_tc_splits(int M, int N, int K);
+int d2d_gemm_tc_splits(int M, int N, int K, int batch = 1);
 
 // Enqueues C = epilogue(A B^T).  Requires K % 8 == 0 and 16-byte aligned base pointers.
 d2d_status d2d_gemm_tc(const d2d_gemm_args &g, cudaStream_t st);

@@ -94,20 +94,42 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+struct RouterLayerIO {
+    float *R;              // [T, E] scores or NULL
+    uint32_t *mask;        // [T, ceil(E/32)]
+    int32_t *k;            // [T]
+    int32_t *status;
+};
+struct RouterGroupIO {
+    RouterLayerIO l[D2D_MAX_GROUP];
+    uint32_t *mask_cat;    // merged mask [T, cat_words] or NULL
+    int cat_words;
+};
+
 // Shared memory (dynamic, 1024-byte aligned):
 //   [ STAGES x (x tile 128x64 | W_r1 tile DH x 64) ]        first GEMM operand ring
 //   [ u: DH/64 k-blocks x (128 rows x 128 B) ]              A operand of the second GEMM (written by epilogue 1)
 //   W_r2 (DH/64 k-blocks x 256 rows x 128 B, the B operand of the second GEMM) reuses the first stages of the ring:
 //   it is loaded as soon as the last k-blocks that used those stages have been consumed, under epilogue 1.
 // TMEM: columns [0, DH) accumulator of u, columns [256, 256 + E_pad) accumulator of R (E <= 256).
+// Several routers that read the same tokens (the Q, K and V projections of one attention layer) run as ONE grid:
+// blockIdx.y picks the router.  Their weights are stacked (W_r1 [n*DH, d], b_r1 [n*DH], W_r2 [n*E, DH], b_r2 [n*E]);
+// every router writes its own outputs and, when mask_cat is given, its mask words once more into a merged mask
+// [T, cat_words] at word offset l * ceil(E/32) (the selection mask of the merged up projection).
 template <int DH>
 __global__ void __launch_bounds__(NTHREADS, 1)
 router_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_w1,
-                    const __grid_constant__ CUtensorMap tm_w2, const __nv_bfloat16 *__restrict__ b_r1,
-                    const __nv_bfloat16 *__restrict__ b_r2, int T, int d, int E, int EN /* E rounded up to 16 */,
-                    float tau, int do_mask, float *__restrict__ R, uint32_t *__restrict__ mask, int32_t *__restrict__ k,
-                    int32_t *__restrict__ status)
+                    const __grid_constant__ CUtensorMap tm_w2, const __nv_bfloat16 *__restrict__ b_r1_all,
+                    const __nv_bfloat16 *__restrict__ b_r2_all, int T, int d, int E, int EN /* E rounded up to 16 */,
+                    float tau, int do_mask, const __grid_constant__ RouterGroupIO io)
 {
+    const int layer = blockIdx.y;
+    const __nv_bfloat16 *b_r1 = b_r1_all ? b_r1_all + layer * DH : nullptr;
+    const __nv_bfloat16 *b_r2 = b_r2_all ? b_r2_all + layer * E : nullptr;
+    float *__restrict__ R = io.l[layer].R;
+    uint32_t *__restrict__ mask = io.l[layer].mask;
+    int32_t *__restrict__ k = io.l[layer].k;
+    int32_t *__restrict__ status = io.l[layer].status;
     constexpr int KB2 = DH / BK;                          // k-blocks of the second GEMM
     constexpr int A_BYTES = BM * BK * 2, B1_BYTES = DH * BK * 2;
     constexpr int STAGE_BYTES = A_BYTES + B1_BYTES;
@@ -170,7 +192,7 @@ router_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_const
                 const uint32_t dst = smem_u32(smem + (size_t)s * STAGE_BYTES);
                 mbar_expect_tx(full, (uint32_t)STAGE_BYTES);
                 tma_load_2d(dst, &tm_x, kb * BK, m0, full);
-                tma_load_2d(dst + A_BYTES, &tm_w1, kb * BK, 0, full);
+                tma_load_2d(dst + A_BYTES, &tm_w1, kb * BK, layer * DH, full);
             }
             // W_r2 goes into stages 0 .. W2_STAGES-1 once the MMAs of the last k-block that used each of them have retired
             for (int s = 0; s < W2_STAGES && ok; ++s) {
@@ -182,7 +204,7 @@ router_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_const
             if (ok) {
                 mbar_expect_tx(smem_u32(&bar_w2), (uint32_t)(KB2 * W2_KB_BYTES));
                 for (int kb = 0; kb < KB2; ++kb)
-                    tma_load_2d(smem_u32(w2_s + (size_t)kb * W2_KB_BYTES), &tm_w2, kb * BK, 0, smem_u32(&bar_w2));
+                    tma_load_2d(smem_u32(w2_s + (size_t)kb * W2_KB_BYTES), &tm_w2, kb * BK, layer * E, smem_u32(&bar_w2));
             }
         }
     } else if (warp == 1) {
@@ -344,7 +366,10 @@ router_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_const
                                 const int i = w * 32 + j;
                                 if (i < E && (anybad || v[q][j] >= thr)) word |= 1u << j;
                             }
-                            if (row < T) mask[(size_t)row * W + w] = word;
+                            if (row < T) {
+                                mask[(size_t)row * W + w] = word;
+                                if (io.mask_cat) io.mask_cat[(size_t)row * io.cat_words + layer * W + w] = word;
+                            }
                             kt += __popc(word);
                         }
                     }
@@ -401,16 +426,15 @@ bool make_map(CUtensorMap *map, const void *base, int rows, int cols, int box_ro
 }
 
 template <int DH>
-d2d_status launch(const d2d_layer *L, const void *x, int T, float tau, int do_mask, float *R, uint32_t *mask, int32_t *k,
-                  int32_t *status, cudaStream_t st)
+d2d_status launch(const d2d_layer_desc &D, const d2d_router_weights &w, int n_layers, const void *x, int T, float tau, int do_mask,
+                  const RouterGroupIO &io, cudaStream_t st)
 {
-    const d2d_layer_desc &D = L->desc;
     constexpr int STAGE_BYTES = BM * BK * 2 + DH * BK * 2;
     constexpr int KB2 = DH / BK;
     constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + (size_t)KB2 * BM * 128 + 1024;
     CUtensorMap tx, tw1, tw2;
-    if (!make_map(&tx, x, T, D.d, BM) || !make_map(&tw1, L->w_r1, D.d_h, D.d, DH) ||
-        !make_map(&tw2, L->w_r2, D.n_experts, D.d_h, 256))
+    if (!make_map(&tx, x, T, D.d, BM) || !make_map(&tw1, w.w_r1, D.d_h * n_layers, D.d, DH) ||
+        !make_map(&tw2, w.w_r2, D.n_experts * n_layers, D.d_h, 256))
         return D2D_ERR_CUDA;
     auto kern = router_fused_kernel<DH>;
     static bool attr_set = false;
@@ -419,8 +443,8 @@ d2d_status launch(const d2d_layer *L, const void *x, int T, float tau, int do_ma
         attr_set = true;
     }
     const int EN = (D.n_experts + 15) / 16 * 16;
-    kern<<<d2d_cdiv(T, BM), NTHREADS, SMEM, st>>>(tx, tw1, tw2, (const __nv_bfloat16 *)L->b_r1, (const __nv_bfloat16 *)L->b_r2,
-                                                 T, D.d, D.n_experts, EN, tau, do_mask, R, mask, k, status);
+    kern<<<dim3(d2d_cdiv(T, BM), n_layers), NTHREADS, SMEM, st>>>(tx, tw1, tw2, (const __nv_bfloat16 *)w.b_r1, (const __nv_bfloat16 *)w.b_r2,
+                                                                 T, D.d, D.n_experts, EN, tau, do_mask, io);
     D2D_LAUNCHED(1);
     return cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
 }
@@ -437,5 +461,20 @@ bool d2d_router_fused_supports(const d2d_layer_desc &D, int T)
 d2d_status d2d_router_fused(const d2d_layer *L, const void *x, int T, float tau, int do_mask, float *R, uint32_t *mask,
                             int32_t *k, int32_t *status, cudaStream_t st)
 {
-    return launch<128>(L, x, T, tau, do_mask, R, mask, k, status, st);
+    RouterGroupIO io = {};
+    io.l[0] = {R, mask, k, status};
+    const d2d_router_weights w = {L->w_r1, L->b_r1, L->w_r2, L->b_r2};
+    return launch<128>(L->desc, w, 1, x, T, tau, do_mask, io, st);
+}
+
+// n routers of one shape with stacked weights, one grid; routing[l] receives mask, k and status of router l.
+d2d_status d2d_router_fused_group(const d2d_layer_desc &D, const d2d_router_weights &w, int n_layers, const void *x, int T,
+                                  float tau, const d2d_routing *routing, uint32_t *mask_cat, int cat_words, cudaStream_t st)
+{
+    if (n_layers < 1 || n_layers > D2D_MAX_GROUP) return D2D_ERR_INVALID_ARG;
+    RouterGroupIO io = {};
+    for (int l = 0; l < n_layers; ++l) io.l[l] = {nullptr, routing[l].mask, routing[l].k, routing[l].status};
+    io.mask_cat = mask_cat;
+    io.cat_words = cat_words;
+    return launch<128>(D, w, n_layers, x, T, tau, 1, io, st);
 }

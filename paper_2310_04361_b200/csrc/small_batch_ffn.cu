@@ -85,15 +85,36 @@ struct SmallSel {
     long long capacity;
 };
 
+// Per-layer arguments; blockIdx.y picks the layer, so that several layers of one shape that read the same tokens
+// (the Q, K and V projections of an attention layer) run as one grid.
+struct SmallRouterLayer {
+    const void *w_r1, *b_r1, *w_r2, *b_r2;
+    float *u, *R;
+    unsigned int *ticket;
+    float *zero;
+    SmallSel sel;
+};
+struct SmallRouterArgs {
+    SmallRouterLayer l[D2D_MAX_GROUP];
+};
+
 // dynamic shared memory: [ W_r1 rows of this CTA: 8*d | token block: TBLK*d | W_r2: E*d_h (if staged) | u: T*d_h floats |
 //                          selection words: T*ceil(E/32) ]
 template <typename TT, int TBLK>
 __global__ void __launch_bounds__(NT)
-small_router_kernel(const TT *__restrict__ x, int T, int d, const TT *__restrict__ w_r1, const TT *__restrict__ b_r1,
-                    int d_h, const TT *__restrict__ w_r2, const TT *__restrict__ b_r2, int E, int stage_w2,
-                    float *__restrict__ u, float *R, unsigned int *__restrict__ ticket, SmallSel sel, float *__restrict__ zero,
-                    int zero_words)
+small_router_kernel(const TT *__restrict__ x, int T, int d, int d_h, int E, int stage_w2, int zero_words,
+                    const __grid_constant__ SmallRouterArgs args)
 {
+    const SmallRouterLayer &P = args.l[blockIdx.y];
+    const TT *__restrict__ w_r1 = static_cast<const TT *>(P.w_r1);
+    const TT *__restrict__ b_r1 = static_cast<const TT *>(P.b_r1);
+    const TT *__restrict__ w_r2 = static_cast<const TT *>(P.w_r2);
+    const TT *__restrict__ b_r2 = static_cast<const TT *>(P.b_r2);
+    float *__restrict__ u = P.u;
+    float *R = P.R;
+    unsigned int *__restrict__ ticket = P.ticket;
+    float *__restrict__ zero = P.zero;
+    const SmallSel &sel = P.sel;
     // clear the float32 accumulator of the expert kernel that follows on the stream (saves a memset node)
     for (int i = blockIdx.x * NT + threadIdx.x; i < zero_words; i += gridDim.x * NT) zero[i] = 0.0f;
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -204,13 +225,32 @@ __device__ __forceinline__ void red_add_v4(float *addr, float a, float b, float 
 
 // dynamic shared memory: [ W1 rows: rc*d | W_gate rows: rc*d (gated) | W2T rows: rc*d | token block: TBLK*d | h: TBLK*rc floats ]
 // rc = neurons handled per pass (the whole expert when its slices fit).
+struct SmallFfnLayer {
+    const void *w1, *b1, *w_gate, *w2t, *b2;
+    const int32_t *offsets, *perm;
+    float *y32;
+    unsigned int *ticket;
+    void *y;
+};
+struct SmallFfnArgs {
+    SmallFfnLayer l[D2D_MAX_GROUP];
+};
+
 template <typename TT, int ACT, bool GATED, int TBLK>
 __global__ void __launch_bounds__(NT)
-small_ffn_kernel(const TT *__restrict__ x, int T, int d, int s, int rc, const TT *__restrict__ w1,
-                 const TT *__restrict__ b1, const TT *__restrict__ w_gate, const TT *__restrict__ w2t,
-                 const TT *__restrict__ b2, const int32_t *__restrict__ offsets, const int32_t *__restrict__ perm,
-                 float *__restrict__ y32, unsigned int *__restrict__ ticket, TT *__restrict__ y)
+small_ffn_kernel(const TT *__restrict__ x, int T, int d, int s, int rc, const __grid_constant__ SmallFfnArgs args)
 {
+    const SmallFfnLayer &P = args.l[blockIdx.y];
+    const TT *__restrict__ w1 = static_cast<const TT *>(P.w1);
+    const TT *__restrict__ b1 = static_cast<const TT *>(P.b1);
+    const TT *__restrict__ w_gate = static_cast<const TT *>(P.w_gate);
+    const TT *__restrict__ w2t = static_cast<const TT *>(P.w2t);
+    const TT *__restrict__ b2 = static_cast<const TT *>(P.b2);
+    const int32_t *__restrict__ offsets = P.offsets;
+    const int32_t *__restrict__ perm = P.perm;
+    float *__restrict__ y32 = P.y32;
+    unsigned int *__restrict__ ticket = P.ticket;
+    TT *__restrict__ y = static_cast<TT *>(P.y);
     extern __shared__ __align__(16) unsigned char smem_raw[];
     TT *w1s = reinterpret_cast<TT *>(smem_raw);
     TT *wgs = w1s + (size_t)rc * d;
@@ -328,10 +368,8 @@ int rows_per_pass(const d2d_layer_desc &D, size_t elem, int tb = MAX_TBLK)
 int token_block(int T) { return T <= 1 ? 1 : T <= 2 ? 2 : T <= 4 ? 4 : 8; }
 
 template <typename TT, int ACT, bool GATED, int TBLK>
-d2d_status launch_ffn_tb(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y, float *y32,
-                         unsigned int *ticket, cudaStream_t st)
+d2d_status launch_ffn_tb(const d2d_layer_desc &D, int n_layers, const SmallFfnArgs &args, const void *x, int T, cudaStream_t st)
 {
-    const d2d_layer_desc &D = L->desc;
     const int rc = rows_per_pass(D, sizeof(TT), TBLK);
     if (rc <= 0) return D2D_ERR_UNSUPPORTED;
     const size_t smem = (size_t)(GATED ? 3 : 2) * rc * D.d * sizeof(TT) + (size_t)TBLK * D.d * sizeof(TT) + (size_t)TBLK * rc * 4;
@@ -341,50 +379,44 @@ d2d_status launch_ffn_tb(const d2d_layer *L, const void *x, int T, const d2d_rou
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess) return D2D_ERR_CUDA;
         attr_smem = kSmemLimit;
     }
-    kern<<<D.n_experts, NT, smem, st>>>((const TT *)x, T, D.d, D.expert_size, rc, (const TT *)L->w1, (const TT *)L->b1,
-                                        (const TT *)L->w_gate, (const TT *)L->w2t, (const TT *)L->b2, r->offsets, r->perm,
-                                        y32, ticket, (TT *)y);
+    kern<<<dim3(D.n_experts, n_layers), NT, smem, st>>>((const TT *)x, T, D.d, D.expert_size, rc, args);
     D2D_LAUNCHED(1);
     return cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
 }
 
 template <typename TT, int ACT, bool GATED>
-d2d_status launch_ffn(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y, float *y32,
-                      unsigned int *ticket, cudaStream_t st)
+d2d_status launch_ffn(const d2d_layer_desc &D, int n, const SmallFfnArgs &a, const void *x, int T, cudaStream_t st)
 {
     switch (token_block(T)) {
-    case 1: return launch_ffn_tb<TT, ACT, GATED, 1>(L, x, T, r, y, y32, ticket, st);
-    case 2: return launch_ffn_tb<TT, ACT, GATED, 2>(L, x, T, r, y, y32, ticket, st);
-    case 4: return launch_ffn_tb<TT, ACT, GATED, 4>(L, x, T, r, y, y32, ticket, st);
-    default: return launch_ffn_tb<TT, ACT, GATED, 8>(L, x, T, r, y, y32, ticket, st);
+    case 1: return launch_ffn_tb<TT, ACT, GATED, 1>(D, n, a, x, T, st);
+    case 2: return launch_ffn_tb<TT, ACT, GATED, 2>(D, n, a, x, T, st);
+    case 4: return launch_ffn_tb<TT, ACT, GATED, 4>(D, n, a, x, T, st);
+    default: return launch_ffn_tb<TT, ACT, GATED, 8>(D, n, a, x, T, st);
     }
 }
 
 template <typename TT, int ACT>
-d2d_status launch_ffn_gated(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y, float *y32,
-                            unsigned int *ticket, cudaStream_t st)
+d2d_status launch_ffn_gated(const d2d_layer_desc &D, int n, const SmallFfnArgs &a, const void *x, int T, cudaStream_t st)
 {
-    if (L->desc.gated) return launch_ffn<TT, ACT, true>(L, x, T, r, y, y32, ticket, st);
-    return launch_ffn<TT, ACT, false>(L, x, T, r, y, y32, ticket, st);
+    if (D.gated) return launch_ffn<TT, ACT, true>(D, n, a, x, T, st);
+    return launch_ffn<TT, ACT, false>(D, n, a, x, T, st);
 }
 
 template <typename TT>
-d2d_status launch_ffn_dtype(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y, float *y32,
-                            unsigned int *ticket, cudaStream_t st)
+d2d_status launch_ffn_dtype(const d2d_layer_desc &D, int n, const SmallFfnArgs &a, const void *x, int T, cudaStream_t st)
 {
-    switch (L->desc.act) {
-    case D2D_ACT_RELU: return launch_ffn_gated<TT, D2D_ACT_RELU>(L, x, T, r, y, y32, ticket, st);
-    case D2D_ACT_GELU_ERF: return launch_ffn_gated<TT, D2D_ACT_GELU_ERF>(L, x, T, r, y, y32, ticket, st);
-    case D2D_ACT_GELU_TANH: return launch_ffn_gated<TT, D2D_ACT_GELU_TANH>(L, x, T, r, y, y32, ticket, st);
-    default: return launch_ffn_gated<TT, D2D_ACT_SILU>(L, x, T, r, y, y32, ticket, st);
+    switch (D.act) {
+    case D2D_ACT_RELU: return launch_ffn_gated<TT, D2D_ACT_RELU>(D, n, a, x, T, st);
+    case D2D_ACT_GELU_ERF: return launch_ffn_gated<TT, D2D_ACT_GELU_ERF>(D, n, a, x, T, st);
+    case D2D_ACT_GELU_TANH: return launch_ffn_gated<TT, D2D_ACT_GELU_TANH>(D, n, a, x, T, st);
+    default: return launch_ffn_gated<TT, D2D_ACT_SILU>(D, n, a, x, T, st);
     }
 }
 
 template <typename TT, int TBLK>
-d2d_status launch_router_tb(const d2d_layer *L, const void *x, int T, float *R, float *u, unsigned int *ticket, cudaStream_t st,
-                            const SmallSel &sel, float *zero, int zero_words)
+d2d_status launch_router_tb(const d2d_layer_desc &D, int n_layers, const SmallRouterArgs &args, const void *x, int T,
+                            int zero_words, cudaStream_t st)
 {
-    const d2d_layer_desc &D = L->desc;
     const size_t base = (size_t)(8 + TBLK) * D.d * sizeof(TT) + (size_t)T * D.d_h * 4 + (size_t)T * ((D.n_experts + 31) / 32) * 4;
     const size_t w2_bytes = (size_t)D.n_experts * (D.d_h * sizeof(TT) + 16);      // padded pitch, see the kernel
     const int stage_w2 = base + w2_bytes <= kSmemLimit ? 1 : 0;
@@ -395,22 +427,35 @@ d2d_status launch_router_tb(const d2d_layer *L, const void *x, int T, float *R, 
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess) return D2D_ERR_CUDA;
         attr_set = true;
     }
-    kern<<<d2d_cdiv(D.d_h, 8), NT, smem, st>>>((const TT *)x, T, D.d, (const TT *)L->w_r1, (const TT *)L->b_r1, D.d_h,
-                                                (const TT *)L->w_r2, (const TT *)L->b_r2, D.n_experts, stage_w2, u, R, ticket, sel, zero, zero_words);
+    kern<<<dim3(d2d_cdiv(D.d_h, 8), n_layers), NT, smem, st>>>((const TT *)x, T, D.d, D.d_h, D.n_experts, stage_w2, zero_words, args);
     D2D_LAUNCHED(1);
     return cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
 }
 
 template <typename TT>
-d2d_status launch_router(const d2d_layer *L, const void *x, int T, float *R, float *u, unsigned int *ticket, cudaStream_t st,
-                         const SmallSel &sel, float *zero, int zero_words)
+d2d_status launch_router(const d2d_layer_desc &D, int n, const SmallRouterArgs &a, const void *x, int T, int zero_words,
+                         cudaStream_t st)
 {
     switch (token_block(T)) {
-    case 1: return launch_router_tb<TT, 1>(L, x, T, R, u, ticket, st, sel, zero, zero_words);
-    case 2: return launch_router_tb<TT, 2>(L, x, T, R, u, ticket, st, sel, zero, zero_words);
-    case 4: return launch_router_tb<TT, 4>(L, x, T, R, u, ticket, st, sel, zero, zero_words);
-    default: return launch_router_tb<TT, 8>(L, x, T, R, u, ticket, st, sel, zero, zero_words);
+    case 1: return launch_router_tb<TT, 1>(D, n, a, x, T, zero_words, st);
+    case 2: return launch_router_tb<TT, 2>(D, n, a, x, T, zero_words, st);
+    case 4: return launch_router_tb<TT, 4>(D, n, a, x, T, zero_words, st);
+    default: return launch_router_tb<TT, 8>(D, n, a, x, T, zero_words, st);
     }
+}
+
+SmallSel make_sel(const d2d_routing *into, float tau)
+{
+    SmallSel sel = {};
+    if (into) {
+        sel.enabled = 1;
+        sel.tau = tau;
+        sel.mask = into->mask; sel.k = into->k; sel.counts = into->counts;
+        sel.offsets = into->offsets; sel.perm = into->perm; sel.tok_off = into->tok_off;
+        sel.tok_exp = into->tok_exp; sel.n_sel = into->n_sel; sel.status = into->status;
+        sel.capacity = (long long)into->perm_capacity;
+    }
+    return sel;
 }
 
 }  // namespace
@@ -431,17 +476,33 @@ d2d_status d2d_small_router(const d2d_layer *L, const void *x, int T, float *R, 
     unsigned int *ticket = fused ? L->tickets : (unsigned int *)ws;
     float *u = (float *)((char *)ws + 256);
     if (!fused) D2D_CUDA_TRY(cudaMemsetAsync(ticket, 0, sizeof(unsigned int), st));
-    SmallSel sel = {};
-    if (select_into) {
-        sel.enabled = 1;
-        sel.tau = tau;
-        sel.mask = select_into->mask; sel.k = select_into->k; sel.counts = select_into->counts;
-        sel.offsets = select_into->offsets; sel.perm = select_into->perm; sel.tok_off = select_into->tok_off;
-        sel.tok_exp = select_into->tok_exp; sel.n_sel = select_into->n_sel; sel.status = select_into->status;
-        sel.capacity = (long long)select_into->perm_capacity;
+    SmallRouterArgs a = {};
+    a.l[0] = {L->w_r1, L->b_r1, L->w_r2, L->b_r2, u, R, ticket, zero, make_sel(select_into, tau)};
+    if (L->desc.dtype == D2D_F32) return launch_router<float>(L->desc, 1, a, x, T, zero_words, st);
+    return launch_router<__nv_bfloat16>(L->desc, 1, a, x, T, zero_words, st);
+}
+
+// Decode batches of a layer group (layers of one shape reading the same tokens): ONE router launch (+ selection +
+// metadata) and ONE expert launch for all layers.  Uses the layer-owned tickets; R[l], u[l] and y32[l] are scratch of the
+// group's workspace; y is [n, T, d].
+d2d_status d2d_small_group_fwd(const d2d_layer *const *layers, int n, const void *x, int T, float tau, const d2d_routing *routing,
+                               float *const *R, float *const *u, float *const *y32, void *y, cudaStream_t st)
+{
+    if (n < 1 || n > D2D_MAX_GROUP) return D2D_ERR_INVALID_ARG;
+    const d2d_layer_desc &D = layers[0]->desc;
+    const size_t el = layers[0]->elem;
+    SmallRouterArgs ra = {};
+    SmallFfnArgs fa = {};
+    for (int l = 0; l < n; ++l) {
+        const d2d_layer *L = layers[l];
+        ra.l[l] = {L->w_r1, L->b_r1, L->w_r2, L->b_r2, u[l], R[l], L->tickets, y32[l], make_sel(&routing[l], tau)};
+        fa.l[l] = {L->w1, L->b1, L->w_gate, L->w2t, L->b2, routing[l].offsets, routing[l].perm, y32[l], L->tickets + 16,
+                   (char *)y + (size_t)l * T * D.d * el};
     }
-    if (L->desc.dtype == D2D_F32) return launch_router<float>(L, x, T, R, u, ticket, st, sel, zero, zero_words);
-    return launch_router<__nv_bfloat16>(L, x, T, R, u, ticket, st, sel, zero, zero_words);
+    d2d_status rc = D.dtype == D2D_F32 ? launch_router<float>(D, n, ra, x, T, T * D.d, st)
+                                       : launch_router<__nv_bfloat16>(D, n, ra, x, T, T * D.d, st);
+    if (rc != D2D_OK) return rc;
+    return D.dtype == D2D_F32 ? launch_ffn_dtype<float>(D, n, fa, x, T, st) : launch_ffn_dtype<__nv_bfloat16>(D, n, fa, x, T, st);
 }
 
 // ws: [ticket (256 bytes) | y32: T*d floats]
@@ -459,6 +520,8 @@ d2d_status d2d_small_ffn(const d2d_layer *L, const void *x, int T, const d2d_rou
     float *y32 = (float *)((char *)ws + 256);
     // the ticket and the float32 accumulator must start at zero
     if (!fused) D2D_CUDA_TRY(cudaMemsetAsync(ws, 0, 256 + (size_t)T * L->desc.d * 4, st));
-    if (L->desc.dtype == D2D_F32) return launch_ffn_dtype<float>(L, x, T, r, y, y32, ticket, st);
-    return launch_ffn_dtype<__nv_bfloat16>(L, x, T, r, y, y32, ticket, st);
+    SmallFfnArgs a = {};
+    a.l[0] = {L->w1, L->b1, L->w_gate, L->w2t, L->b2, r->offsets, r->perm, y32, ticket, y};
+    if (L->desc.dtype == D2D_F32) return launch_ffn_dtype<float>(L->desc, 1, a, x, T, st);
+    return launch_ffn_dtype<__nv_bfloat16>(L->desc, 1, a, x, T, st);
 }

@@ -306,6 +306,85 @@ def test_layer_fwd_without_scores_output_matches_the_run_with_it(api, name, T, t
         assert _rel_err(y2.float().cpu().numpy(), y1) <= (0 if (T > 128) else 1e-2)
 
 
+# ------------------------------------------------------------------------------------ layer groups (shared input)
+
+GROUP_CASES = [("gpt2_attn", 3, 1, 0.2), ("gpt2_attn", 3, 4, 0.5), ("gpt2_attn", 3, 5, 0.2), ("gpt2_attn", 3, 64, 0.2),
+               ("gpt2_attn", 3, 129, 0.5), ("gpt2_attn", 3, 300, 0.2), ("bert", 4, 200, 0.3), ("vit", 2, 260, 0.3),
+               ("gpt2_attn", 1, 3, 0.2), ("gpt2_attn", 1, 200, 0.2),
+               ("tiny", 2, 6, 0.5), ("tiny", 3, 128, 0.5), ("llama", 2, 40, 0.4)]
+
+
+@pytest.mark.parametrize("name,n,T,tau", GROUP_CASES)
+def test_group_fwd_matches_oracle_and_separate_layer_calls(api, name, n, T, tau):
+    """n layers of one shape on a shared input (the Q, K, V projections of an attention layer, Sec. 3.5): every
+    layer's routing is exact for its own scores' rule, its y matches the oracle given its mask, and both equal what
+    a separate d2d_layer_fwd call on that layer produces."""
+    from dataclasses import replace
+    _cache.clear()
+    cfg = wl.with_tokens(wl.CONFIGS[name], T)
+    act = oracle.ACT_BY_NAME[cfg.act]
+    x = wl.make_tokens(cfg)
+    ws = [wl.make_weights(replace(cfg, seed=cfg.seed + 17 * l)) for l in range(n)]
+    layers = [api.Layer.from_config(cfg, w) for w in ws]
+    group = api.LayerGroup(layers)
+    xd = api.to_device(x, cfg.dtype)
+    routings = [L.new_routing(T, dual=True) for L in layers]
+    for rep in range(2):                                   # twice: tickets and tile counters must reset themselves
+        y, rs = group.group_fwd(xd, tau, routings=routings)
+        torch.cuda.synchronize()
+        eps = TOL_R[cfg.dtype]
+        for l in range(n):
+            r = rs[l]
+            assert r.status == 0
+            G = oracle.unpack_mask(r.mask_u32(), cfg.E)
+            _check_routing(r, G, dual=True)                # k, counts, offsets, perm, dual: exact for this mask
+            ref = oracle.layer(x, ws[l], act, tau)
+            m = ref["R"].max(1, keepdims=True)
+            diff = G != ref["G"]
+            near = np.abs(ref["R"] - np.float32(tau) * m) <= 4 * eps * m
+            assert (~diff | near).all() and diff.mean() < 0.01
+            w = ws[l]
+            y_ref = oracle.moe_ffn(x, w["w1"], w["b1"], w["w_gate"], w["w2"], w["b2"], act, G)
+            assert _rel_err(y[l].float().cpu().numpy(), y_ref) <= TOL_Y[cfg.dtype]
+            if rep == 0:
+                y1, r1 = layers[l].layer_fwd(xd, tau)
+                torch.cuda.synchronize()
+                assert np.array_equal(r1.mask_u32(), r.mask_u32())
+                assert _rel_err(y[l].float().cpu().numpy(), y1.float().cpu().numpy()) <= 1e-2
+    group.close()
+    for L in layers:
+        L.close()
+
+
+def test_group_rejects_mixed_shapes_and_repeated_layers(api):
+    cfg = wl.with_tokens(wl.CONFIGS["gpt2_attn"], 8)
+    a = api.Layer.from_config(cfg, wl.make_weights(cfg))
+    b = api.Layer.from_config(wl.CONFIGS["tiny"], wl.make_weights(wl.CONFIGS["tiny"]))
+    for bad in ([a, b], [a, a], []):
+        with pytest.raises(api.D2DError) as e:
+            api.LayerGroup(bad)
+        assert api.STATUS_NAMES[e.value.code] == "INVALID_ARG"
+    g = api.LayerGroup([a])
+    with pytest.raises(api.D2DError) as e:
+        g.group_fwd(api.to_device(wl.make_tokens(cfg), cfg.dtype), 1.5)
+    assert api.STATUS_NAMES[e.value.code] == "INVALID_ARG"
+    g.close(); a.close(); b.close()
+
+
+def test_group_fwd_zero_tokens(api):
+    cfg = wl.with_tokens(wl.CONFIGS["gpt2_attn"], 8)
+    layers = [api.Layer.from_config(cfg, wl.make_weights(cfg)) for _ in range(2)]
+    g = api.LayerGroup(layers)
+    x0 = torch.empty((0, cfg.d), dtype=torch.bfloat16, device="cuda")
+    y, rs = g.group_fwd(x0, 0.3)
+    torch.cuda.synchronize()
+    for r in rs:
+        assert r.status == 0 and r.n_sel == 0 and int(r.offsets.abs().sum().item()) == 0
+    g.close()
+    for L in layers:
+        L.close()
+
+
 # ------------------------------------------------------------------------------------ full-size sampled checks
 
 FULL_CASES = [("bert", 0.3, 96), ("vit", 0.3, 64), ("llama", 0.4, 24), ("paper", None, 48)]
