@@ -49,6 +49,9 @@ def parse_args():
     p.add_argument("--sweep", action="store_true", help="also time the workload's whole tau grid")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a captured CUDA graph")
+    p.add_argument("--group", type=int, default=0,
+                   help="also time N layers of the workload's shape on the shared input as one d2d_group_fwd call "
+                        "(the Q, K, V projections of an attention layer) against N separate d2d_layer_fwd calls")
     return p.parse_args()
 
 
@@ -379,6 +382,53 @@ def run_ours(args):
                 sweep.append({"tau": tau, "rho": routing.n_sel / (T * cfg.E), "ms": statistics.mean(ts),
                               "speedup_vs_dense": t_dense / statistics.mean(ts)})
 
+        group = None
+        if args.group > 1:
+            from dataclasses import replace
+            n = args.group
+            gws = [weights] + [wl.make_weights(replace(cfg, seed=cfg.seed + 17 * l)) for l in range(1, n)]
+            glayers = [layer] + [api.Layer.from_config(cfg, w, device=dev) for w in gws[1:]]
+            grp = api.LayerGroup(glayers)
+            gy = torch.empty((n, T, cfg.d), dtype=tdt, device=dev)
+            grs = [L.new_routing(T) for L in glayers]
+            grp.workspace(T)
+            for L in glayers:
+                L.workspace(T)
+
+            def group_step():
+                grp.group_fwd(x, args.tau, y=gy, routings=grs)
+
+            def separate_step():
+                for l, L in enumerate(glayers):
+                    L.layer_fwd(x, args.tau, y=gy[l], routing=grs[l])
+
+            gdense_w = [(torch.from_numpy(w["w1"]).to(dev, tdt), None if w["b1"] is None else torch.from_numpy(w["b1"]).to(dev, tdt),
+                         torch.from_numpy(w["w2"]).to(dev, tdt), None if w["b2"] is None else torch.from_numpy(w["b2"]).to(dev, tdt))
+                        for w in gws]
+
+            def dense_group():
+                return [F.linear(actf(F.linear(x, a, b)), c, e) for a, b, c, e in gdense_w]
+
+            group_step()
+            l0 = api.launch_count()
+            group_step()
+            g_launches = api.launch_count() - l0
+            separate_step()
+            l0 = api.launch_count()
+            separate_step()
+            s_launches = api.launch_count() - l0
+            t_group = statistics.mean(timed_loop(runner(group_step), args.steps, 3))
+            t_sep = statistics.mean(timed_loop(runner(separate_step), args.steps, 3))
+            t_gdense = None if cfg.gated else statistics.mean(timed_loop(runner(dense_group), args.steps, 3))
+            torch.cuda.synchronize()
+            assert all(r.status == 0 for r in grs)
+            group = {"n_layers": n, "group_fwd_ms": t_group, "separate_layer_fwd_ms": t_sep, "dense_ms": t_gdense,
+                     "launches_group": g_launches, "launches_separate": s_launches,
+                     "speedup_vs_separate": t_sep / t_group, "speedup_vs_dense": None if t_gdense is None else t_gdense / t_group,
+                     "rho": [r.n_sel / (T * cfg.E) for r in grs],
+                     "tokens_per_s": T / (t_group * 1e-3)}
+            grp.close()
+
         cpu = None
         if not args.no_cpu_baseline:
             cpu = time_cpu_oracle(cfg, weights, x_np, args.tau)
@@ -402,6 +452,8 @@ def run_ours(args):
         }
         if sweep is not None:
             line["tau_sweep"] = sweep
+        if group is not None:
+            line["group"] = group
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.barrier()
