@@ -330,19 +330,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     float *bias_f = reinterpret_cast<float *>(smem + (size_t)STAGES * STAGE_BYTES);
     const int NB = N * ep.batch;                                     // bias entries of all problems
     const bool bias_cached = ep.bias != nullptr && NB <= BIAS_CACHE_ELEMS && (N & 3) == 0;
-    if (bias_cached) {
-        // 16-byte loads, all issued before the first use: the fill costs one memory latency, not N / threads of them
-        for (int i = threadIdx.x * 8; i < NB; i += NTHREADS_V2 * 8) {
-            float b8[8];
-            if (i + 8 <= NB) {
-                d2d_load8(ep.bias + i, b8);
-#pragma unroll
-                for (int q = 0; q < 8; ++q) bias_f[i + q] = b8[q];
-            } else {
-                for (int q = 0; i + q < NB; ++q) bias_f[i + q] = __bfloat162float(ep.bias[i + q]);
-            }
-        }
-    }
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nkb = (K + BK - 1) / BK;
@@ -392,14 +379,44 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     // With late_wait only the epilogue depends on that kernel (the selection mask written by the router): the
     // operand loads and the MMAs of the first tiles then overlap it, and only the epilogue warps wait.
     const bool dyn = !PAIR && ep.tile_counter != nullptr;
-    if (!ep.late_wait || warp >= 2) asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (bias_cached && warp >= 2) {
+        // The epilogue warps stage the bias (a parameter: no need to wait for the previous kernel) while the producer
+        // and the MMA thread are already at work.  16-byte loads, all issued before the first use: the fill costs one
+        // memory latency, not N / threads of them.
+        for (int i = ((int)threadIdx.x - 64) * 8; i < NB; i += N_EPI_WARPS * 32 * 8) {
+            float b8[8];
+            if (i + 8 <= NB) {
+                d2d_load8(ep.bias + i, b8);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) bias_f[i + q] = b8[q];
+            } else {
+                for (int q = 0; i + q < NB; ++q) bias_f[i + q] = __bfloat162float(ep.bias[i + q]);
+            }
+        }
+        asm volatile("bar.sync 1, %0;" ::"r"(N_EPI_WARPS * 32) : "memory");
+    }
+    // early_b: the B operand (weights) does not depend on the previous kernel either, so the producer requests the B
+    // tiles of its first k-blocks BEFORE it waits for that kernel and only the A tiles after (static schedule only)
+    const bool early_b = !PAIR && !dyn && !ep.late_wait;
+    if (warp >= 2 || (!ep.late_wait && !(early_b && warp == 0))) asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            uint32_t it = 0;
+            uint32_t it = 0, pre = 0;
             bool ok = true;
+            // B tile(s) of k-block kb into the stage at dst (single-CTA form)
+            auto load_b = [&](uint32_t dst, uint32_t full, int kb, int n0) {
+                if (GATED && ep.gate_cat) {
+                    // up rows [n0, n0+BN) and gate rows [n0, n0+BN) are adjacent in the interleaved copy: one
+                    // 2*BN-row box (the producer thread's time per k-block is what bounds the gated main loop)
+                    tma_load_2d(dst + A_BYTES, &tm_b, kb * BK, 2 * n0, full);
+                } else {
+                    tma_load_2d(dst + A_BYTES, &tm_b, kb * BK, n0, full);
+                    if (GATED) tma_load_2d(dst + A_BYTES + B_BYTES, &tm_b2, kb * BK, n0, full);
+                }
+            };
             for (uint32_t local = 0; ok; ++local) {
                 int item = worker + (int)local * n_workers;
                 if (dyn) {
@@ -423,8 +440,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 tile_coords(tile, (M + TM - 1) / TM, n_tiles, ep.band_rows, tr, tc);
                 const int m0 = tr * TM + (int)rank * BM, n0 = prob * N + tc * BN + (int)rank * B_ROWS;
                 const int ka = prob * K;                      // problem p reads columns [p*K, (p+1)*K) of A
+                if (early_b && local == 0) {
+                    // arm the first stages and request their B tiles, then wait for the previous kernel (A may be its output)
+                    for (int kb = kb0; kb < kb1 && pre < (uint32_t)STAGES; ++kb, ++pre) {
+                        const uint32_t full = smem_u32(&bar_full[pre]);
+                        mbar_expect_tx(full, (uint32_t)STAGE_BYTES);
+                        load_b(smem_u32(smem + (size_t)pre * STAGE_BYTES), full, kb, n0);
+                    }
+                    asm volatile("griddepcontrol.wait;" ::: "memory");
+                }
                 for (int kb = kb0; kb < kb1; ++kb, ++it) {
                     const uint32_t s = it % STAGES, round = it / STAGES;
+                    if (it < pre) {                           // armed above, B already requested
+                        tma_load_2d(smem_u32(smem + (size_t)s * STAGE_BYTES), &tm_a, ka + kb * BK, m0, smem_u32(&bar_full[s]));
+                        continue;
+                    }
                     ok = mbar_wait(smem_u32(&bar_empty[s]), (round & 1u) ^ 1u, ep.status);
                     if (!ok) break;
                     const uint32_t dst = smem_u32(smem + (size_t)s * STAGE_BYTES);
@@ -439,14 +469,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                         const uint32_t full = smem_u32(&bar_full[s]);
                         mbar_expect_tx(full, (uint32_t)STAGE_BYTES);
                         tma_load_2d(dst, &tm_a, ka + kb * BK, m0, full);
-                        if (GATED && ep.gate_cat) {
-                            // up rows [n0, n0+BN) and gate rows [n0, n0+BN) are adjacent in the interleaved copy: one
-                            // 2*BN-row box (the producer thread's time per k-block is what bounds the gated main loop)
-                            tma_load_2d(dst + A_BYTES, &tm_b, kb * BK, 2 * n0, full);
-                        } else {
-                            tma_load_2d(dst + A_BYTES, &tm_b, kb * BK, n0, full);
-                            if (GATED) tma_load_2d(dst + A_BYTES + B_BYTES, &tm_b2, kb * BK, n0, full);
-                        }
+                        load_b(dst, full, kb, n0);
                     }
                 }
             }
@@ -940,9 +963,9 @@ bool d2d_gemm_tc_available() { return get_encode() != nullptr; }
 
 int d2d_gemm_tc_splits(int M, int N, int K, int batch)
 {
-    // only single-row-tile problems whose column tiles would occupy less than half of the SMs
-    if (M > BM || (N & 3)) return 1;
-    const int tiles = d2d_cdiv(N, 64) * (batch > 1 ? batch : 1);
+    // only problems whose 128 x 64 output tiles would occupy less than half of the SMs (a few hundred tokens at most)
+    if (N & 3) return 1;
+    const int tiles = d2d_cdiv(M, BM) * d2d_cdiv(N, 64) * (batch > 1 ? batch : 1);
     const int nkb = d2d_cdiv(K, BK);
     int splits = sm_count() / (tiles > 0 ? tiles : 1);
     if (splits > nkb / 2) splits = nkb / 2;          // at least two k-blocks per slice
