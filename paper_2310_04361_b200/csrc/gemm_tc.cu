@@ -207,6 +207,60 @@ template <int ACT> __device__ __forceinline__ float fast_act(float z)
     return z * fmaf(0.5f, t, 0.5f);
 }
 
+// ---- packed float32 pairs (sm_100 issues add / mul / fma on two float32 values per instruction; same IEEE results
+// as the scalar forms).  The epilogue is bound by instruction issue, so its per-element math runs on pairs.
+__device__ __forceinline__ uint64_t pack2(float a, float b)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float &a, float &b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t dup2(float a) { return pack2(a, a); }
+
+// fast_act on a pair; the same operations in the same order as the scalar form, so the results are identical
+template <int ACT> __device__ __forceinline__ uint64_t fast_act2(uint64_t z)
+{
+    float a, b;
+    if (ACT == D2D_ACT_RELU) {
+        unpack2(z, a, b);
+        return pack2(fmaxf(a, 0.0f), fmaxf(b, 0.0f));
+    }
+    uint64_t arg;
+    if (ACT == D2D_ACT_GELU_ERF) {
+        unpack2(mul2(z, z), a, b);
+        const uint64_t z2 = pack2(fminf(a, 64.0f), fminf(b, 64.0f));
+        const uint64_t q = fma2(fma2(dup2(-3.15807042e-4f), z2, dup2(3.67982560e-2f)), z2, dup2(7.97717834e-1f));
+        arg = mul2(z, q);
+    } else if (ACT == D2D_ACT_GELU_TANH) {
+        const uint64_t q = fma2(dup2(0.79788456080286536f * 0.044715f), mul2(z, z), dup2(0.79788456080286536f));
+        arg = mul2(z, q);
+    } else {
+        arg = mul2(dup2(0.5f), z);                          // SiLU
+    }
+    unpack2(arg, a, b);
+    const uint64_t t = pack2(fast_tanh(a), fast_tanh(b));
+    return mul2(z, fma2(dup2(0.5f), t, dup2(0.5f)));
+}
+
 __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
@@ -239,14 +293,15 @@ __device__ __forceinline__ void epilogue_16(const uint32_t (&r)[16], const uint3
         for (int j = 0; j < 16; ++j) bias[j] = 0.0f;
     }
     if (EPI == D2D_EPI_UP_MASKED && halves) {
-        // each 8-column half belongs to one expert: one predicate per half, one select per element
-        const bool k0 = (keep & 1u) != 0, k1 = (keep & 0x100u) != 0;
+        // the common case of the up projection: math on pairs; the selection is applied by the caller on the packed
+        // bf16 words (each 8-column half belongs to one expert)
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            const float z = __uint_as_float(r[j]) + bias[j];
+        for (int j = 0; j < 16; j += 2) {
             // first accumulator = up projection (+ bias), second = gate
-            const float h = GATED ? fast_act<ACT>(__uint_as_float(g[j])) * z : fast_act<ACT>(z);
-            v[j] = (j < 8 ? k0 : k1) ? h : 0.0f;
+            const uint64_t z = add2(pack2(__uint_as_float(r[j]), __uint_as_float(r[j + 1])), pack2(bias[j], bias[j + 1]));
+            const uint64_t h = GATED ? mul2(fast_act2<ACT>(pack2(__uint_as_float(g[j]), __uint_as_float(g[j + 1]))), z)
+                                     : fast_act2<ACT>(z);
+            unpack2(h, v[j], v[j + 1]);
         }
         return;
     }
@@ -669,6 +724,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                             for (int j = 0; j < 8; ++j) {
                                 __nv_bfloat162 t = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
                                 pk[j] = *reinterpret_cast<uint32_t *>(&t);
+                                // selection: an expert the token did not keep contributes zeros (also when its
+                                // pre-activations are not finite)
+                                if (EPI == D2D_EPI_UP_MASKED) pk[j] = (keep >> (2 * j)) & 1u ? pk[j] : 0u;
                             }
                             if (wide_store) {
                                 // one 32-byte store per row and unit: a whole sector per lane, half as many store instructions
