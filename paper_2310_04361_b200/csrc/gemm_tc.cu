@@ -51,6 +51,20 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t
     return false;
 }
 
+// One non-blocking test of the phase with the given parity.
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity)
+{
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return done != 0;
+}
+
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar)
 {
     asm volatile(
@@ -538,6 +552,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             const uint32_t idesc = instr_desc_bf16(TM, (GATED && !PAIR) ? 2 * BN : BN);
             uint32_t it = 0, local = 0;
             bool ok = true;
+            // The tensor core accepts only a few instructions ahead, so whatever this thread executes between the last
+            // MMA of one k-block and the first MMA of the next is a bubble in the MMA pipe.  The barrier of the NEXT
+            // k-block is therefore tested between the MMAs of the current one (`have` carries the answer across
+            // k-blocks and tiles), and nothing but the commit sits between two k-blocks whose data has landed.
+            bool have = false;
             for (;; ++local) {
                 int item = worker + (int)local * n_workers;
                 if (dyn) {
@@ -558,17 +577,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 const uint32_t acc = tmem_base + buf * BUF_COLS;
                 for (int kb = kb0; kb < kb1; ++kb, ++it) {
                     const uint32_t s = it % STAGES, round = it / STAGES;
-                    ok = mbar_wait(smem_u32(&bar_full[s]), round & 1u, ep.status);
-                    if (!ok) break;
-                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    if (!have) {
+                        ok = mbar_wait(smem_u32(&bar_full[s]), round & 1u, ep.status);
+                        if (!ok) break;
+                    }
                     const uint32_t a_addr = smem_u32(smem + (size_t)s * STAGE_BYTES);
                     const uint64_t da = smem_desc_sw128(a_addr);
                     const uint64_t db = smem_desc_sw128(a_addr + A_BYTES);
                     const uint64_t db2 = smem_desc_sw128(a_addr + A_BYTES + B_BYTES);
+                    const uint32_t s_next = (it + 1) % STAGES, round_next = (it + 1) / STAGES;
 #pragma unroll
                     for (int k = 0; k < BK / UMMA_K; ++k) {
                         const uint64_t koff = (uint64_t)((k * UMMA_K * 2) >> 4);    // 32 bytes per K step inside the swizzle row
                         const uint32_t accum = (kb > kb0 || k != 0) ? 1u : 0u;
+                        // before the last MMA of this k-block: has the next k-block (of this or the next tile) landed?
+                        if (k == BK / UMMA_K - 1) have = mbar_test(smem_u32(&bar_full[s_next]), round_next & 1u);
                         if (PAIR) {
                             umma_bf16_pair(acc, da + koff, db + koff, idesc, accum);
                             if (GATED) umma_bf16_pair(acc + BN, da + koff, db2 + koff, idesc, accum);
