@@ -492,17 +492,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     const uint32_t sl = local & 1u, use = local >> 1;
                     ok = mbar_wait(smem_u32(&sched_empty[sl]), (use & 1u) ^ 1u, ep.status);
                     if (!ok) break;
-                    item = atomicAdd(ep.tile_counter, 1);
-                    // every CTA draws exactly one value past the end; whoever draws the largest of them is the last to
-                    // touch the counter and leaves it at zero for the next launch
-                    if (item == total_tiles + (int)gridDim.x - 1) *ep.tile_counter = 0;
+                    // A CTA's first item is its own index (no round trip to the counter before the first loads); the
+                    // counter hands out the items from gridDim.x on.  Every CTA draws exactly one value past the end,
+                    // total_tiles draws in all: whoever gets the last one leaves the counter at zero for the next launch.
+                    if (local > 0) {
+                        const int c = atomicAdd(ep.tile_counter, 1);
+                        if (c == total_tiles - 1) *ep.tile_counter = 0;
+                        item = (int)gridDim.x + c;
+                    }
                     sched_item[sl] = item < total_tiles ? item : -1;
                     mbar_arrive(smem_u32(&sched_full[sl]));       // release: the slot's content is visible to whoever sees the phase
                 }
                 if (item >= total_tiles) break;
-                int tile = item / k_splits;
+                int tile = (!GATED && k_splits == 1) ? item : item / k_splits;
                 const int sp = item - tile * k_splits;
-                const int kb0 = (int)((long long)sp * nkb / k_splits), kb1 = (int)((long long)(sp + 1) * nkb / k_splits);
+                // no split is the common case: skip the divisions (measured: faster for the plain kernels, slower for the
+                // gated one, whose code layout is at its limit)
+                const bool one = !GATED && k_splits == 1;
+                const int kb0 = one ? 0 : (int)((long long)sp * nkb / k_splits), kb1 = one ? nkb : (int)((long long)(sp + 1) * nkb / k_splits);
                 int prob = 0;
                 if (ep.batch > 1) { prob = tile / tiles_pp; tile -= prob * tiles_pp; }
                 int tr, tc;
@@ -568,8 +575,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     if (item < 0) break;
                 }
                 if (item >= total_tiles) break;
-                const int sp = item % k_splits;
-                const int kb0 = (int)((long long)sp * nkb / k_splits), kb1 = (int)((long long)(sp + 1) * nkb / k_splits);
+                const int sp = (!GATED && k_splits == 1) ? 0 : item % k_splits;
+                // no split is the common case: skip the divisions (measured: faster for the plain kernels, slower for the
+                // gated one, whose code layout is at its limit)
+                const bool one = !GATED && k_splits == 1;
+                const int kb0 = one ? 0 : (int)((long long)sp * nkb / k_splits), kb1 = one ? nkb : (int)((long long)(sp + 1) * nkb / k_splits);
                 const uint32_t buf = local & 1u, use = local >> 1;
                 ok = mbar_wait(smem_u32(&bar_acc_empty[buf]), (use & 1u) ^ 1u, ep.status);   // epilogue drained this buffer
                 if (!ok) break;
@@ -640,7 +650,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 if (item < 0) break;
             }
             if (item >= total_tiles) break;
-            int tile = item / k_splits;
+            int tile = (!GATED && k_splits == 1) ? item : item / k_splits;
             int prob = 0;
             if (ep.batch > 1) { prob = tile / tiles_pp; tile -= prob * tiles_pp; }
             int tr, tc;
