@@ -53,6 +53,11 @@ def test_status_strings_and_host_side_validation(lib):
     assert lib.d2d_router_fwd(None, None, 4, None, None, 0, None) == 1
     assert lib.d2d_select_dynk(None, 4, 16, ctypes.c_float(0.5), None, None, 0, None) == 1
     assert lib.d2d_moe_ffn_fwd(None, None, 4, None, None, None, 0, None) == 1
+    assert lib.d2d_group_create(None, 3, None, None) == 1
+    assert lib.d2d_group_destroy(None) == 0
+    lib.d2d_group_workspace_bytes.restype = ctypes.c_size_t
+    assert lib.d2d_group_workspace_bytes(None, 16) == 0
+    assert lib.d2d_group_fwd(None, None, 4, ctypes.c_float(0.5), None, None, None, 0, None) == 1
 
 
 def test_product_does_not_reach_the_oracle():

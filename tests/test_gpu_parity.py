@@ -385,6 +385,42 @@ def test_group_fwd_zero_tokens(api):
         L.close()
 
 
+def test_group_full_size_on_sampled_tokens(api):
+    """The Q/K/V group at the size the benchmark times (T = 4096, merged tensor-core path): metadata in full,
+    the oracle recomputes sampled tokens of every layer from that layer's own mask."""
+    from dataclasses import replace
+    _cache.clear()
+    n, T, tau = 3, 4096, 0.2
+    cfg = wl.with_tokens(wl.CONFIGS["gpt2_attn"], T)
+    act = oracle.ACT_BY_NAME[cfg.act]
+    x = wl.make_tokens(cfg)
+    ws = [wl.make_weights(replace(cfg, seed=cfg.seed + 17 * l)) for l in range(n)]
+    layers = [api.Layer.from_config(cfg, w) for w in ws]
+    group = api.LayerGroup(layers)
+    y, rs = group.group_fwd(api.to_device(x, cfg.dtype), tau)
+    torch.cuda.synchronize()
+    rng = np.random.default_rng(3)
+    for l in range(n):
+        assert rs[l].status == 0
+        G = oracle.unpack_mask(rs[l].mask_u32(), cfg.E)
+        _check_routing(rs[l], G, dual=False)
+        k = G.sum(1)
+        assert k.min() >= 1
+        sample = np.unique(np.concatenate([rng.choice(T, 48, replace=False), [int(k.argmin()), int(k.argmax()), 0, T - 1]]))
+        w = ws[l]
+        # the mask itself: the rule applied to the oracle's scores, except where a score sits on the threshold
+        ref = oracle.layer(x[sample], w, act, tau)
+        m = ref["R"].max(1, keepdims=True)
+        diff = G[sample] != ref["G"]
+        assert (~diff | (np.abs(ref["R"] - np.float32(tau) * m) <= 4 * TOL_R[cfg.dtype] * m)).all()
+        y_ref = oracle.moe_ffn(x[sample], w["w1"], w["b1"], w["w_gate"], w["w2"], w["b2"], act, G[sample])
+        yg = y[l][torch.from_numpy(sample).cuda()].float().cpu().numpy()
+        assert _rel_err(yg, y_ref) <= TOL_Y[cfg.dtype]
+    group.close()
+    for L in layers:
+        L.close()
+
+
 # ------------------------------------------------------------------------------------ full-size sampled checks
 
 FULL_CASES = [("bert", 0.3, 96), ("vit", 0.3, 64), ("llama", 0.4, 24), ("paper", None, 48)]
