@@ -65,6 +65,36 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity)
     return done != 0;
 }
 
+// Bounded wait for whole warps: try_wait may suspend the warp in hardware until the phase completes or a time
+// limit passes, so thirty-two waiting lanes cost no issue slots.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, int32_t *status)
+{
+    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (done) return true;
+    }
+    if (status) atomicMax(status, (int32_t)D2D_ERR_TIMEOUT);
+    return false;
+}
+// true in exactly one lane of a converged warp
+__device__ __forceinline__ bool elect_one()
+{
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
+}
+
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar)
 {
     asm volatile(
@@ -552,7 +582,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0 && rank == 0) {
+        // The whole warp walks the loop, so that waits, indices and descriptors are warp-uniform (the tensor-core
+        // instructions take their operands from uniform registers); one elected lane issues the MMAs and commits.
+        if (rank == 0) {
             // Gated (single CTA): the up and gate tiles sit back to back in shared memory, so they are ONE K-major
             // B operand of 2*BN rows and one MMA fills both accumulators (columns [0,BN) up, [BN,2BN) gate).
             // Two N=BN instructions would each pay the full A-operand read and run at half the rate.
@@ -568,10 +600,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 int item = worker + (int)local * n_workers;
                 if (dyn) {
                     const uint32_t sl = local & 1u, su = local >> 1;
-                    ok = mbar_wait(smem_u32(&sched_full[sl]), su & 1u, ep.status);
+                    ok = mbar_wait_warp(smem_u32(&sched_full[sl]), su & 1u, ep.status);
                     if (!ok) break;
                     item = sched_item[sl];
-                    mbar_arrive(smem_u32(&sched_empty[sl]));
+                    __syncwarp();                              // every lane has read the slot before it is handed back
+                    if (elect_one()) mbar_arrive(smem_u32(&sched_empty[sl]));
                     if (item < 0) break;
                 }
                 if (item >= total_tiles) break;
@@ -581,14 +614,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 const bool one = !GATED && k_splits == 1;
                 const int kb0 = one ? 0 : (int)((long long)sp * nkb / k_splits), kb1 = one ? nkb : (int)((long long)(sp + 1) * nkb / k_splits);
                 const uint32_t buf = local & 1u, use = local >> 1;
-                ok = mbar_wait(smem_u32(&bar_acc_empty[buf]), (use & 1u) ^ 1u, ep.status);   // epilogue drained this buffer
+                ok = mbar_wait_warp(smem_u32(&bar_acc_empty[buf]), (use & 1u) ^ 1u, ep.status);   // epilogue drained this buffer
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t acc = tmem_base + buf * BUF_COLS;
                 for (int kb = kb0; kb < kb1; ++kb, ++it) {
                     const uint32_t s = it % STAGES, round = it / STAGES;
                     if (!have) {
-                        ok = mbar_wait(smem_u32(&bar_full[s]), round & 1u, ep.status);
+                        ok = mbar_wait_warp(smem_u32(&bar_full[s]), round & 1u, ep.status);
                         if (!ok) break;
                     }
                     const uint32_t a_addr = smem_u32(smem + (size_t)s * STAGE_BYTES);
@@ -596,27 +629,37 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     const uint64_t db = smem_desc_sw128(a_addr + A_BYTES);
                     const uint64_t db2 = smem_desc_sw128(a_addr + A_BYTES + B_BYTES);
                     const uint32_t s_next = (it + 1) % STAGES, round_next = (it + 1) / STAGES;
-#pragma unroll
-                    for (int k = 0; k < BK / UMMA_K; ++k) {
+                    auto issue = [&](int k) {
                         const uint64_t koff = (uint64_t)((k * UMMA_K * 2) >> 4);    // 32 bytes per K step inside the swizzle row
                         const uint32_t accum = (kb > kb0 || k != 0) ? 1u : 0u;
-                        // before the last MMA of this k-block: has the next k-block (of this or the next tile) landed?
-                        if (k == BK / UMMA_K - 1) have = mbar_test(smem_u32(&bar_full[s_next]), round_next & 1u);
                         if (PAIR) {
                             umma_bf16_pair(acc, da + koff, db + koff, idesc, accum);
                             if (GATED) umma_bf16_pair(acc + BN, da + koff, db2 + koff, idesc, accum);
                         } else {
                             umma_bf16(acc, da + koff, db + koff, idesc, accum);
                         }
+                    };
+                    if (elect_one()) {
+#pragma unroll
+                        for (int k = 0; k < BK / UMMA_K - 1; ++k) issue(k);
                     }
-                    // stage reusable (in both CTAs of a pair) once these MMAs have read it
-                    if (PAIR) umma_commit_pair(smem_u32(&bar_empty[s]));
-                    else umma_commit(smem_u32(&bar_empty[s]));
+                    // before the last MMA of this k-block: has the next k-block (of this or the next tile) landed?
+                    have = __all_sync(0xffffffffu, mbar_test(smem_u32(&bar_full[s_next]), round_next & 1u));
+                    if (elect_one()) {
+                        issue(BK / UMMA_K - 1);
+                        // stage reusable (in both CTAs of a pair) once these MMAs have read it
+                        if (PAIR) umma_commit_pair(smem_u32(&bar_empty[s]));
+                        else umma_commit(smem_u32(&bar_empty[s]));
+                    }
+                    __syncwarp();
                 }
                 if (!ok) break;
                 // accumulator of this tile complete (each CTA of a pair holds its own 128 rows)
-                if (PAIR) umma_commit_pair(smem_u32(&bar_acc_full[buf]));
-                else umma_commit(smem_u32(&bar_acc_full[buf]));
+                if (elect_one()) {
+                    if (PAIR) umma_commit_pair(smem_u32(&bar_acc_full[buf]));
+                    else umma_commit(smem_u32(&bar_acc_full[buf]));
+                }
+                __syncwarp();
             }
         }
     } else {
