@@ -69,6 +69,8 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity)
 // limit passes, so thirty-two waiting lanes cost no issue slots.
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, int32_t *status)
 {
+    // how long one try may suspend is up to the hardware, so the bound is in time: about a second by the global timer
+    unsigned long long t0 = 0;
     for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
         uint32_t done;
         asm volatile(
@@ -79,6 +81,12 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, in
             : "r"(bar), "r"(parity)
             : "memory");
         if (done) return true;
+        if ((it & 31u) == 31u) {                               // rarely reached: a try normally ends with the phase complete
+            unsigned long long now;
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > 1000000000ull) break;
+        }
     }
     if (status) atomicMax(status, (int32_t)D2D_ERR_TIMEOUT);
     return false;
