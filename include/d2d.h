@@ -98,7 +98,9 @@ typedef struct {
 /* Routing of one batch: the outputs of d2d_select_dynk and the input of
  * d2d_moe_ffn_fwd.  All pointers are device pointers owned by the caller.
  * mask, k, counts, offsets, perm, n_sel and status are required; the
- * token-major dual (tok_off, tok_exp) is optional (both NULL or both set). */
+ * token-major dual (tok_off, tok_exp) is optional (both NULL or both set).
+ * d2d_layer_fwd alone also accepts a routing whose per-expert lists are absent
+ * as a set (counts, offsets, perm, n_sel, tok_off, tok_exp all NULL); see there. */
 typedef struct {
     uint32_t *mask;      /* [T, ceil(E/32)]  expert i of token t = bit i%32 of word i/32       */
     int32_t *k;          /* [T]              experts kept by token t                           */
@@ -131,6 +133,39 @@ D2D_API d2d_status d2d_layer_create(const d2d_layer_desc *desc, const d2d_weight
 
 /* Frees the handle and its device copies.  NULL is a no-op. */
 D2D_API d2d_status d2d_layer_destroy(d2d_layer *layer);
+
+/* How the expert step of bf16 batches above the decode sizes computes the up
+ * projection H = G * A(x W1^T + b1) (Sec. 3.4).  Both forms give the same H;
+ * the choice changes speed only.
+ *   D2D_PATH_DENSE   one contraction over all d_ff neurons with the selection
+ *                    applied as a mask: time independent of the selection.
+ *   D2D_PATH_GATHER  tokens are bucketed by groups of `group` adjacent experts
+ *                    and each group runs a contraction over the tokens that keep
+ *                    one of its experts (the grouped form of Listing 1): time
+ *                    proportional to the number of kept (token, group) pairs.
+ *   D2D_PATH_AUTO    (default) decided per call on the device from the number of
+ *                    selected pairs of that batch: gathered when
+ *                    n_sel <= rho_max * T * E and T >= 512, dense otherwise.  Both
+ *                    kernels are enqueued and the one not needed returns at once,
+ *                    so there is no host synchronisation.
+ * group: experts per group, 0 = library default for the shape (a power of two
+ * that divides E, group * expert_size a multiple of 16 and at most 256, 128 for
+ * gated layers).  rho_max: crossover density of D2D_PATH_AUTO, negative =
+ * library default for the shape.  Returns D2D_ERR_UNSUPPORTED when the shape
+ * cannot take the gathered path (fp32 layers, expert sizes that are not a
+ * multiple of 8) and it, or a group, was asked for. */
+typedef enum { D2D_PATH_AUTO = 0, D2D_PATH_DENSE = 1, D2D_PATH_GATHER = 2 } d2d_expert_path;
+D2D_API d2d_status d2d_layer_set_expert_path(d2d_layer *layer, d2d_expert_path path, int32_t group, double rho_max);
+/* Current setting; any output pointer may be NULL.  *group is 0 when the shape
+ * cannot take the gathered path. */
+D2D_API d2d_status d2d_layer_get_expert_path(const d2d_layer *layer, int32_t *path, int32_t *group, double *rho_max);
+
+/* Clears the layer-owned device counters (the "last CTA" tickets, the tile and
+ * sub-chunk counters of the expert kernels).  They reset themselves when a
+ * call completes; a call that ended with D2D_ERR_TIMEOUT in the status word
+ * may have left them non-zero, and the next call would then skip work.  Enqueue
+ * this on the stream after such a call (it is a 1-2 KB memset). */
+D2D_API d2d_status d2d_layer_reset_counters(d2d_layer *layer, void *stream);
 
 /* Bytes of device workspace that any call on `layer` with up to max_tokens
  * tokens needs (256-byte aligned buffer).  Returns 0 for a NULL layer. */
@@ -215,11 +250,16 @@ D2D_API d2d_status d2d_moe_ffn_fwd(const d2d_layer *layer, const void *x, int32_
  * for every neuron n of the original FFN: the expert up projections of all
  * kept (token, expert) pairs as one dense contraction with the selection
  * applied as a mask.  x: device [T, d]; H: device [T, d_ff] bf16 (caller's).
+ * d2d_expert_up_gather_fwd: the same H through the gathered kernel
+ * (D2D_PATH_GATHER with the layer's group size), whatever path the layer is
+ * set to; D2D_ERR_UNSUPPORTED for shapes the gathered path cannot take.
  * d2d_expert_down_fwd (Sec. 3.2, 3.4): y = H W2^T + b2, which is
  * b2 + sum over kept experts of W2[:, blk] h_blk.  y: device [T, d] bf16;
  * status: device status word (receives D2D_ERR_TIMEOUT), may be NULL. */
 D2D_API d2d_status d2d_expert_up_fwd(const d2d_layer *layer, const void *x, int32_t T, const d2d_routing *routing,
                                      void *H, void *stream);
+D2D_API d2d_status d2d_expert_up_gather_fwd(const d2d_layer *layer, const void *x, int32_t T, const d2d_routing *routing,
+                                            void *H, void *stream);
 D2D_API d2d_status d2d_expert_down_fwd(const d2d_layer *layer, const void *H, int32_t T, void *y, int32_t *status,
                                        void *stream);
 
@@ -227,8 +267,12 @@ D2D_API d2d_status d2d_expert_down_fwd(const d2d_layer *layer, const void *H, in
  * router_fwd -> select_dynk -> moe_ffn_fwd (Sec. 3.2-3.4).  R_out: optional
  * device [T,E] float32 output of the router scores; with NULL the scores may
  * never reach memory (for bf16 batches of 5 or more tokens the router kernel
- * thresholds them on chip).  `routing` supplies the metadata buffers
- * (required; they are outputs).  Work is enqueued on `stream`; the per-expert
+ * thresholds them on chip).  `routing` supplies the metadata buffers (they
+ * are outputs): mask, k and status are required; the per-expert lists
+ * (counts, offsets, perm, n_sel and the dual) may be NULL as a set, in which
+ * case they are not built -- allowed where the expert kernels read only the
+ * mask (bf16 batches of 5 or more tokens with d_h = 128 and E <= 256),
+ * D2D_ERR_INVALID_ARG elsewhere.  Work is enqueued on `stream`; the per-expert
  * metadata may be built on a stream the layer owns, joined back into `stream`
  * before the call's last operation, so everything the call writes is ordered
  * before whatever the caller enqueues on `stream` next.  The layer object

@@ -26,7 +26,9 @@ STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "WORKSPACE", 4: 
                 6: "TIMEOUT", 7: "CAPACITY"}
 D2D_F32, D2D_BF16 = 0, 1
 ACTS = {"relu": 0, "gelu_erf": 1, "gelu_tanh": 2, "silu": 3}
+PATHS = {"auto": 0, "dense": 1, "gather": 2}
 EXPORTS = ["d2d_status_str", "d2d_launch_count", "d2d_layer_create", "d2d_layer_destroy", "d2d_workspace_bytes",
+           "d2d_layer_set_expert_path", "d2d_layer_get_expert_path", "d2d_layer_reset_counters", "d2d_expert_up_gather_fwd",
            "d2d_select_workspace_bytes", "d2d_router_fwd", "d2d_select_dynk", "d2d_select_dynk_static", "d2d_select_topk",
            "d2d_routing_from_mask", "d2d_moe_ffn_fwd", "d2d_expert_up_fwd", "d2d_expert_down_fwd", "d2d_layer_fwd", "d2d_layer_fwd_host_workspace_bytes",
            "d2d_layer_fwd_host", "d2d_group_create", "d2d_group_destroy", "d2d_group_workspace_bytes", "d2d_group_fwd"]
@@ -64,6 +66,10 @@ _lib.d2d_select_topk.argtypes = [c_void_p, c_int32, c_int32, c_int32, POINTER(Ro
 _lib.d2d_routing_from_mask.argtypes = [c_int32, c_int32, POINTER(RoutingStruct), c_void_p, c_size_t, c_void_p]
 _lib.d2d_moe_ffn_fwd.argtypes = [c_void_p, c_void_p, c_int32, POINTER(RoutingStruct), c_void_p, c_void_p, c_size_t, c_void_p]
 _lib.d2d_expert_up_fwd.argtypes = [c_void_p, c_void_p, c_int32, POINTER(RoutingStruct), c_void_p, c_void_p]
+_lib.d2d_expert_up_gather_fwd.argtypes = [c_void_p, c_void_p, c_int32, POINTER(RoutingStruct), c_void_p, c_void_p]
+_lib.d2d_layer_set_expert_path.argtypes = [c_void_p, c_int, c_int32, ctypes.c_double]
+_lib.d2d_layer_get_expert_path.argtypes = [c_void_p, POINTER(c_int32), POINTER(c_int32), POINTER(ctypes.c_double)]
+_lib.d2d_layer_reset_counters.argtypes = [c_void_p, c_void_p]
 _lib.d2d_expert_down_fwd.argtypes = [c_void_p, c_void_p, c_int32, c_void_p, c_void_p, c_void_p]
 _lib.d2d_layer_fwd.argtypes = [c_void_p, c_void_p, c_int32, c_float, c_void_p, c_void_p, POINTER(RoutingStruct),
                                c_void_p, c_size_t, c_void_p]
@@ -110,19 +116,27 @@ def torch_dtype(name: str):
 class Routing:
     """Caller-owned device buffers for the routing of one batch (d2d_routing)."""
 
-    def __init__(self, T: int, E: int, device, dual: bool = False, perm_capacity: int | None = None):
+    def __init__(self, T: int, E: int, device, dual: bool = False, perm_capacity: int | None = None, lists: bool = True):
+        """lists=False leaves out the per-expert lists (counts, offsets, perm, n_sel): d2d_layer_fwd then does not build them."""
         W = (E + 31) // 32
         cap = T * E if perm_capacity is None else int(perm_capacity)
         i32 = dict(dtype=torch.int32, device=device)
         self.T, self.E, self.W = T, E, W
         self.mask = torch.zeros((max(T, 1), W), **i32)     # raw uint32 words kept in an int32 tensor
         self.k = torch.zeros((max(T, 1),), **i32)
+        self.scalars = torch.zeros((2,), **i32)            # n_sel, status
+        self.lists = lists
+        if not lists:
+            self.counts = self.offsets = self.perm = self.tok_off = self.tok_exp = None
+            self.struct = RoutingStruct(mask=self.mask.data_ptr(), k=self.k.data_ptr(), counts=None, offsets=None, perm=None,
+                                        tok_off=None, tok_exp=None, n_sel=None, status=self.scalars.data_ptr() + 4,
+                                        perm_capacity=0)
+            return
         self.counts = torch.zeros((E,), **i32)
         self.offsets = torch.zeros((E + 1,), **i32)
         self.perm = torch.zeros((max(cap, 1),), **i32)
         self.tok_off = torch.zeros((T + 1,), **i32) if dual else None
         self.tok_exp = torch.zeros((max(cap, 1),), **i32) if dual else None
-        self.scalars = torch.zeros((2,), **i32)            # n_sel, status
         self.struct = RoutingStruct(
             mask=self.mask.data_ptr(), k=self.k.data_ptr(), counts=self.counts.data_ptr(),
             offsets=self.offsets.data_ptr(), perm=self.perm.data_ptr(),
@@ -132,6 +146,9 @@ class Routing:
 
     @property
     def n_sel(self) -> int:
+        """Selected (token, expert) pairs: the library's n_sel, or the sum of k when the lists were not built."""
+        if not self.lists:
+            return int(self.k[: self.T].sum().item())
         return int(self.scalars[0].item())
 
     @property
@@ -194,8 +211,23 @@ class Layer:
             self._ws = torch.empty((need,), dtype=torch.uint8, device=self.device)
         return self._ws
 
-    def new_routing(self, T: int, dual: bool = False, perm_capacity: int | None = None) -> Routing:
-        return Routing(T, self.E, self.device, dual, perm_capacity)
+    def new_routing(self, T: int, dual: bool = False, perm_capacity: int | None = None, lists: bool = True) -> Routing:
+        return Routing(T, self.E, self.device, dual, perm_capacity, lists)
+
+    # -- which up projection the tensor-core expert step uses --------------------------------
+    def set_expert_path(self, path: str = "auto", group: int = 0, rho_max: float = -1.0) -> None:
+        """path: "auto" | "dense" | "gather"; group: experts per group (0 = default); rho_max: crossover density of
+        "auto" (negative = default).  See d2d_layer_set_expert_path."""
+        _check(_lib.d2d_layer_set_expert_path(self.handle, PATHS[path], int(group), float(rho_max)), "d2d_layer_set_expert_path")
+
+    def get_expert_path(self):
+        path, group, rho = c_int32(), c_int32(), ctypes.c_double()
+        _check(_lib.d2d_layer_get_expert_path(self.handle, ctypes.byref(path), ctypes.byref(group), ctypes.byref(rho)),
+               "d2d_layer_get_expert_path")
+        return {v: k for k, v in PATHS.items()}[path.value], group.value, rho.value
+
+    def reset_counters(self, stream=None) -> None:
+        _check(_lib.d2d_layer_reset_counters(self.handle, _stream(stream)), "d2d_layer_reset_counters")
 
     # -- the calls of the C ABI -------------------------------------------------------------
     def router_fwd(self, x, R=None, stream=None):
@@ -223,6 +255,15 @@ class Layer:
             H = torch.empty((T, self.d_ff), dtype=torch.bfloat16, device=self.device)
         _check(_lib.d2d_expert_up_fwd(self.handle, _ptr(x), T, ctypes.byref(routing.struct), _ptr(H), _stream(stream)),
                "d2d_expert_up_fwd")
+        return H
+
+    def expert_up_gather_fwd(self, x, routing: Routing, H=None, stream=None):
+        """The same H through the gathered, grouped kernel (tokens bucketed by groups of adjacent experts)."""
+        T = x.shape[0]
+        if H is None:
+            H = torch.empty((T, self.d_ff), dtype=torch.bfloat16, device=self.device)
+        _check(_lib.d2d_expert_up_gather_fwd(self.handle, _ptr(x), T, ctypes.byref(routing.struct), _ptr(H), _stream(stream)),
+               "d2d_expert_up_gather_fwd")
         return H
 
     def expert_down_fwd(self, H, y=None, stream=None):

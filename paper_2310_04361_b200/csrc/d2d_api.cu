@@ -7,6 +7,7 @@
 #include "d2d_common.cuh"
 #include <stdlib.h>
 #include "gemm_tc.cuh"
+#include "moe_gather.cuh"
 
 bool d2d_token_path_supports(const d2d_layer_desc &D);
 d2d_status d2d_launch_moe_ffn_token(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y,
@@ -18,11 +19,16 @@ namespace {
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-bool routing_ok(const d2d_routing *r, bool need_mask_only)
+bool has_lists(const d2d_routing *r) { return r->counts && r->offsets && r->perm && r->n_sel; }
+
+// lists_optional: the per-expert lists (counts, offsets, perm, n_sel) may be absent as a set (d2d_layer_fwd then
+// does not build them); mask, k and status are always required
+bool routing_ok(const d2d_routing *r, bool lists_optional)
 {
-    if (!r || !r->mask) return false;
-    if (need_mask_only) return true;
-    if (!r->k || !r->counts || !r->offsets || !r->perm || !r->n_sel || !r->status) return false;
+    if (!r || !r->mask || !r->k || !r->status) return false;
+    const bool none = !r->counts && !r->offsets && !r->perm && !r->n_sel && !r->tok_off && !r->tok_exp;
+    if (lists_optional && none) return true;
+    if (!has_lists(r)) return false;
     if ((r->tok_off == nullptr) != (r->tok_exp == nullptr)) return false;
     return r->perm_capacity >= 0;
 }
@@ -89,25 +95,63 @@ size_t d2d_moe_ffn_ws_bytes(const d2d_layer *L, int T)
     return need;
 }
 
-// Large batches: every expert is used by some token of a 128-token tile, so the expert FFN runs
-// as two dense tensor-core GEMMs; the selection enters as a mask on the hidden activations
-// (h_n of an expert the token did not keep is zeroed in the epilogue), which is exactly
-// y = b2 + sum over kept experts.
+// Density above which the masked dense up projection is faster than the gathered one for this shape (the automatic
+// choice).  The gathered kernel's cost is proportional to the fraction of (token, group) pairs u = 1 - (1 - rho)^g
+// (independent selections; correlated ones only lower u) times a per-row cost relative to the dense kernel that
+// depends on how wide one MMA of the group is; the constants are fitted to measurements on B200.
+static double default_gather_rho_max(const d2d_layer_desc &D, int g)
+{
+    if (g <= 0) return -1.0;
+    const int n_mma = g * D.expert_size * (D.gated ? 2 : 1);
+    const double cost = n_mma >= 256 ? 1.05 : n_mma >= 128 ? 1.2 : n_mma >= 96 ? 1.5 : 2.2;
+    const double u_max = 0.92 / cost;
+    return u_max >= 1.0 ? 1.0 : 1.0 - pow(1.0 - u_max, 1.0 / g);
+}
+
+// Expert step of bf16 batches above the decode sizes, on the tensor cores.
+//   up projection    two kernels that compute the same H = G * A(x W1^T + b1):
+//     masked dense   one GEMM over all of d_ff, the selection applied as a mask in the epilogue; its time does not
+//                    depend on the selection (every expert is kept by some token of a 128-token tile)
+//     gathered       per group of adjacent experts, a contraction over the tokens that keep the group (moe_gather.cu);
+//                    its time is proportional to the number of (token, group) pairs
+//   down projection  y = H W2^T + b2 as a dense GEMM: exactly b2 + the sum over kept experts, since the h of an expert
+//                    the token did not keep is zero
+// Which up projection runs is decided per call from the number of selected pairs of THIS batch.  D2D_PATH_AUTO
+// launches both kernels with complementary rules on a device word (n_sel) that is valid once the preceding kernel of
+// the stream has completed; the one that is not needed returns at once, so no host synchronisation is involved.
 // up_counter (optional): a zeroed device counter; its presence also states that the kernel launched just before
-// on this stream is the router, which writes only the mask (and R, k), so that the up projection's main loops may
-// overlap it and draw their tiles dynamically.
-static d2d_status launch_dense_masked(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y,
-                                      void *ws, cudaStream_t st, int *up_counter)
+// on this stream is the router, which writes only the mask (and R, k), so that a forced masked dense up projection
+// may overlap it with its main loops and draw its tiles dynamically.
+static d2d_status launch_tc_experts(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y,
+                                    void *ws, cudaStream_t st, int *up_counter, const int32_t *n_sel)
 {
     const d2d_layer_desc &D = L->desc;
-    d2d_gemm_args up = {};
-    up.tile_counter = up_counter;
-    up.pdl_late_wait = up_counter != nullptr;
-    up.a = x; up.b = L->w1; up.b_gate = D.gated ? L->w_gate : nullptr; up.b_cat = L->w1g; up.b_cat_block = 128; up.bias = L->b1; up.out = ws;
-    up.M = T; up.N = D.d_ff; up.K = D.d; up.epilogue = D2D_EPI_UP_MASKED; up.act = D.act;
-    up.mask = r->mask; up.mask_words = (D.n_experts + 31) / 32; up.expert_size = D.expert_size; up.status = r->status;
-    d2d_status rc = d2d_gemm_tc(up, st);
-    if (rc != D2D_OK) return rc;
+    int path = L->expert_path;
+    if (L->gather_group <= 0) path = D2D_PATH_DENSE;
+    if (path == D2D_PATH_AUTO && (T < 512 || !n_sel)) path = D2D_PATH_DENSE;      // small batches: every weight row is read either way
+    const long long n_sel_max = (long long)(L->gather_rho_max * (double)T * (double)D.n_experts);
+    d2d_status rc;
+    if (path != D2D_PATH_GATHER) {
+        d2d_gemm_args up = {};
+        const bool forced = path == D2D_PATH_DENSE;
+        up.tile_counter = forced ? up_counter : nullptr;
+        up.pdl_late_wait = forced && up_counter != nullptr;
+        up.n_sel = forced ? nullptr : n_sel; up.n_sel_max = n_sel_max;
+        up.a = x; up.b = L->w1; up.b_gate = D.gated ? L->w_gate : nullptr; up.b_cat = L->w1g; up.b_cat_block = 128; up.bias = L->b1; up.out = ws;
+        up.M = T; up.N = D.d_ff; up.K = D.d; up.epilogue = D2D_EPI_UP_MASKED; up.act = D.act;
+        up.mask = r->mask; up.mask_words = (D.n_experts + 31) / 32; up.expert_size = D.expert_size; up.status = r->status;
+        rc = d2d_gemm_tc(up, st);
+        if (rc != D2D_OK) return rc;
+    }
+    if (path != D2D_PATH_DENSE) {
+        d2d_gather_args ga = {};
+        ga.x = x; ga.w1 = L->w1; ga.w_gate = D.gated ? L->w_gate : nullptr; ga.b1 = L->b1; ga.mask = r->mask; ga.H = ws;
+        ga.T = T; ga.d = D.d; ga.d_ff = D.d_ff; ga.n_experts = D.n_experts; ga.s = D.expert_size; ga.g = L->gather_group;
+        ga.act = D.act; ga.status = r->status; ga.ctr = L->gather_ctr;
+        ga.n_sel = path == D2D_PATH_AUTO ? n_sel : nullptr; ga.n_sel_max = n_sel_max;
+        rc = d2d_moe_gather_up(ga, st);
+        if (rc != D2D_OK) return rc;
+    }
     d2d_gemm_args dn = {};
     dn.a = ws; dn.b = L->w2; dn.bias = L->b2; dn.out = y;
     dn.M = T; dn.N = D.d; dn.K = D.d_ff; dn.epilogue = D2D_EPI_BIAS_BF16; dn.status = r->status;
@@ -118,11 +162,11 @@ static d2d_status launch_dense_masked(const d2d_layer *L, const void *x, int T, 
 }
 
 d2d_status d2d_launch_moe_ffn(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y,
-                              void *ws, size_t ws_bytes, cudaStream_t st, int *up_counter, int small_fused)
+                              void *ws, size_t ws_bytes, cudaStream_t st, int *up_counter, int small_fused, const int32_t *n_sel)
 {
     if (ws_bytes < d2d_moe_ffn_ws_bytes(L, T)) return D2D_ERR_WORKSPACE;
-    if (use_small_ffn(L, T)) return d2d_small_ffn(L, x, T, r, y, ws, st, small_fused);
-    if (use_dense_masked(L, T)) return launch_dense_masked(L, x, T, r, y, ws, st, up_counter);
+    if (use_small_ffn(L, T)) return has_lists(r) ? d2d_small_ffn(L, x, T, r, y, ws, st, small_fused) : D2D_ERR_INVALID_ARG;
+    if (use_dense_masked(L, T)) return launch_tc_experts(L, x, T, r, y, ws, st, up_counter, n_sel ? n_sel : r->n_sel);
     return d2d_launch_moe_ffn_token(L, x, T, r, y, st);
 }
 
@@ -181,6 +225,12 @@ d2d_status d2d_layer_create(const d2d_layer_desc *desc, const d2d_weights *w, vo
         {&L->b2, w->b2, (size_t)D.d, false}, {&L->w2, w->w2, n_w, false},
     };
     size_t total = 256;                                   // the ticket words (see d2d_layer::tickets)
+    L->gather_group = d2d_gather_group_for(D, 0);
+    L->gather_rho_max = default_gather_rho_max(D, L->gather_group);
+    L->expert_path = D2D_PATH_AUTO;
+    L->gather_ctr_words = D.n_experts + 64;               // enough for any group size: E / g counters + the exit ticket
+    const size_t ctr_off = total;
+    total += d2d_align_up((size_t)L->gather_ctr_words * sizeof(int), 256);
     for (const piece &p : pieces)
         if (p.src) total += d2d_align_up(p.n * el, 256);
     // gated bf16 layers: W1 and W_gate once more, interleaved in blocks of 128 rows for the tensor-core up projection
@@ -196,8 +246,9 @@ d2d_status d2d_layer_create(const d2d_layer_desc *desc, const d2d_weights *w, vo
     }
     L->slab_bytes = total;
     L->tickets = (unsigned int *)L->slab;
-    size_t off = 256;
-    d2d_status rc = cudaMemsetAsync(L->tickets, 0, 256, st) == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
+    L->gather_ctr = (int *)((char *)L->slab + ctr_off);
+    size_t off = ctr_off + d2d_align_up((size_t)L->gather_ctr_words * sizeof(int), 256);
+    d2d_status rc = cudaMemsetAsync(L->slab, 0, off, st) == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
     for (const piece &p : pieces) {
         if (!p.src || rc != D2D_OK) continue;
         void *dst = (char *)L->slab + off;
@@ -264,6 +315,33 @@ d2d_status d2d_layer_destroy(d2d_layer *layer)
     cudaError_t e = cudaFree(layer->slab);
     delete layer;
     return e == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
+}
+
+d2d_status d2d_layer_set_expert_path(d2d_layer *layer, d2d_expert_path path, int32_t group, double rho_max)
+{
+    if (!layer || path < D2D_PATH_AUTO || path > D2D_PATH_GATHER || group < 0) return D2D_ERR_INVALID_ARG;
+    const int g = d2d_gather_group_for(layer->desc, group);
+    if (g <= 0 && (path == D2D_PATH_GATHER || group > 0)) return D2D_ERR_UNSUPPORTED;
+    layer->gather_group = g;
+    layer->expert_path = path;
+    layer->gather_rho_max = rho_max >= 0.0 ? (rho_max > 1.0 ? 1.0 : rho_max) : default_gather_rho_max(layer->desc, g);
+    return D2D_OK;
+}
+
+d2d_status d2d_layer_get_expert_path(const d2d_layer *layer, int32_t *path, int32_t *group, double *rho_max)
+{
+    if (!layer) return D2D_ERR_INVALID_ARG;
+    if (path) *path = layer->expert_path;
+    if (group) *group = layer->gather_group;
+    if (rho_max) *rho_max = layer->gather_rho_max;
+    return D2D_OK;
+}
+
+d2d_status d2d_layer_reset_counters(d2d_layer *layer, void *stream)
+{
+    if (!layer) return D2D_ERR_INVALID_ARG;
+    const size_t bytes = 256 + d2d_align_up((size_t)layer->gather_ctr_words * sizeof(int), 256);
+    return cudaMemsetAsync(layer->slab, 0, bytes, (cudaStream_t)stream) == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
 }
 
 size_t d2d_workspace_bytes(const d2d_layer *layer, int32_t max_tokens)
@@ -346,6 +424,21 @@ d2d_status d2d_expert_up_fwd(const d2d_layer *layer, const void *x, int32_t T, c
     return d2d_gemm_tc(up, (cudaStream_t)stream);
 }
 
+d2d_status d2d_expert_up_gather_fwd(const d2d_layer *layer, const void *x, int32_t T, const d2d_routing *routing,
+                                    void *H, void *stream)
+{
+    if (!layer || T < 0) return D2D_ERR_INVALID_ARG;
+    if (T == 0) return D2D_OK;
+    if (!x || !H || !aligned16(x) || !aligned16(H) || !routing_ok(routing, false)) return D2D_ERR_INVALID_ARG;
+    if (layer->gather_group <= 0) return D2D_ERR_UNSUPPORTED;
+    const d2d_layer_desc &D = layer->desc;
+    d2d_gather_args ga = {};
+    ga.x = x; ga.w1 = layer->w1; ga.w_gate = D.gated ? layer->w_gate : nullptr; ga.b1 = layer->b1; ga.mask = routing->mask; ga.H = H;
+    ga.T = T; ga.d = D.d; ga.d_ff = D.d_ff; ga.n_experts = D.n_experts; ga.s = D.expert_size; ga.g = layer->gather_group;
+    ga.act = D.act; ga.status = routing->status; ga.ctr = layer->gather_ctr;
+    return d2d_moe_gather_up(ga, (cudaStream_t)stream);
+}
+
 d2d_status d2d_expert_down_fwd(const d2d_layer *layer, const void *H, int32_t T, void *y, int32_t *status, void *stream)
 {
     if (!layer || T < 0) return D2D_ERR_INVALID_ARG;
@@ -362,11 +455,12 @@ d2d_status d2d_expert_down_fwd(const d2d_layer *layer, const void *H, int32_t T,
 d2d_status d2d_layer_fwd(const d2d_layer *layer, const void *x, int32_t T, float tau, void *y,
                          float *R_out, d2d_routing *routing, void *ws, size_t ws_bytes, void *stream)
 {
-    if (!layer || T < 0 || !routing_ok(routing, false)) return D2D_ERR_INVALID_ARG;
+    if (!layer || T < 0 || !routing_ok(routing, true)) return D2D_ERR_INVALID_ARG;
     if (!(tau >= 0.0f && tau <= 1.0f)) return D2D_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     const int E = layer->desc.n_experts;
-    if (T == 0) return d2d_launch_select(nullptr, 0, E, tau, 0, routing, ws, st);
+    const bool lists = has_lists(routing);
+    if (T == 0) return lists ? d2d_launch_select(nullptr, 0, E, tau, 0, routing, ws, st) : D2D_OK;
     if (!x || !y || !aligned16(x) || !aligned16(y) || (R_out && !aligned16(R_out))) return D2D_ERR_INVALID_ARG;
     const ws_layout w = layout_for(layer, T);
     if (!ws || !aligned16(ws) || ws_bytes < w.total) return D2D_ERR_WORKSPACE;
@@ -381,23 +475,30 @@ d2d_status d2d_layer_fwd(const d2d_layer *layer, const void *x, int32_t T, float
         // memset node sits in front of the router (the up projection may begin while the router is still running)
         int *up_counter = dense ? (int *)(layer->tickets + 32) : nullptr;
         // the scores themselves are written only when the caller asked for them: mask and k come out of the same kernel
-        rc = d2d_router_fused(layer, x, T, tau, 1, R_out, routing->mask, routing->k, routing->status, st);
+        // the router also adds up k: the number of selected pairs, which decides between the two up projections
+        int32_t *ksum = (int32_t *)(layer->tickets + 40);
+        rc = d2d_router_fused(layer, x, T, tau, 1, R_out, routing->mask, routing->k, routing->status, st, dense ? ksum : nullptr);
         if (rc != D2D_OK) return rc;
         if (dense) {
-            // The dense-masked expert GEMMs read only the mask: build counts / offsets / token lists on the side
-            // stream while they run (the small metadata CTAs fit beside the persistent GEMM CTAs), join at the end.
-            if (cudaEventRecord(layer->ev_fork, st) != cudaSuccess ||
-                cudaStreamWaitEvent(layer->side_stream, layer->ev_fork, 0) != cudaSuccess)
-                return D2D_ERR_CUDA;
-            rc = d2d_launch_select(nullptr, T, E, tau, 0, routing, base + w.sel_off, layer->side_stream, 1);
-            if (rc != D2D_OK) return rc;
-            rc = d2d_launch_moe_ffn(layer, x, T, routing, y, base + w.ffn_off, w.total - w.ffn_off, st, up_counter);
-            if (cudaEventRecord(layer->ev_join, layer->side_stream) != cudaSuccess ||
-                cudaStreamWaitEvent(st, layer->ev_join, 0) != cudaSuccess)
+            // The tensor-core expert kernels read only the mask: the per-expert lists (when the caller wants them) are
+            // built on the side stream while they run (the small metadata CTAs fit beside the persistent CTAs), join at the end.
+            if (lists) {
+                if (cudaEventRecord(layer->ev_fork, st) != cudaSuccess ||
+                    cudaStreamWaitEvent(layer->side_stream, layer->ev_fork, 0) != cudaSuccess)
+                    return D2D_ERR_CUDA;
+                rc = d2d_launch_select(nullptr, T, E, tau, 0, routing, base + w.sel_off, layer->side_stream, 1);
+                if (rc != D2D_OK) return rc;
+            }
+            rc = d2d_launch_moe_ffn(layer, x, T, routing, y, base + w.ffn_off, w.total - w.ffn_off, st, up_counter, 0, ksum + 4);
+            if (lists && (cudaEventRecord(layer->ev_join, layer->side_stream) != cudaSuccess ||
+                          cudaStreamWaitEvent(st, layer->ev_join, 0) != cudaSuccess))
                 return D2D_ERR_CUDA;
             return rc;
         }
+        if (!lists) return D2D_ERR_INVALID_ARG;               // the expert kernels of this shape walk the per-expert lists
         rc = d2d_launch_select(nullptr, T, E, tau, 0, routing, base + w.sel_off, st, 1);
+    } else if (!lists) {
+        return D2D_ERR_INVALID_ARG;                           // every other path builds (and its expert kernels use) the lists
     } else if (d2d_small_router_supports(layer->desc, T)) {
         // decode batches: the router kernel's last CTA selects as well (one launch for router + selection)
         const bool small = use_small_ffn(layer, T);

@@ -31,10 +31,20 @@ struct d2d_layer {
     cudaStream_t copy_in, copy_out;
     cudaEvent_t ev_in[kHostChunks], ev_done[kHostChunks], ev_begin, ev_end;
     // layer-owned "last CTA" tickets of the decode kernels used by d2d_layer_fwd (zero at creation, reset by the kernel
-    // that used them): word 0 decode router, word 16 decode experts, word 32 tile counter of the up projection.  Like the
-    // side stream, they make concurrent d2d_layer_fwd calls on ONE layer object from several streams unsafe; use one
-    // layer object per stream for that.  A call that ended in D2D_ERR_TIMEOUT may leave them non-zero: recreate the layer.
+    // that used them): word 0 decode router, word 16 decode experts, word 32 tile counter of the up projection, words
+    // 40 / 41 sum of k and exit ticket of the fused router, word 44 the number of selected pairs the fused router
+    // publishes for the density-adaptive dispatch of the expert step.  Like the side stream, they make concurrent
+    // d2d_layer_fwd calls on ONE layer object from several streams unsafe; use one layer object per stream for that.
+    // A call that ended in D2D_ERR_TIMEOUT may leave them non-zero: d2d_layer_reset_counters clears them.
     unsigned int *tickets;
+    // gathered expert path (moe_gather.cu): per-group sub-chunk counters + exit ticket (self-resetting like the tickets),
+    // experts per group (0 = the shape cannot use the path), which path the expert step takes (d2d_expert_path) and
+    // the density up to which the automatic choice takes the gathered path
+    int *gather_ctr;
+    int gather_ctr_words;
+    int gather_group;
+    int expert_path;
+    double gather_rho_max;
 };
 
 // Layers of one shape that read the same token rows (the Q, K and V projections of one attention layer) and run as
@@ -83,9 +93,11 @@ size_t d2d_select_ws_bytes(int T, int E);
 d2d_status d2d_launch_select(const float *R, int T, int E, float tau, int topk, const d2d_routing *out,
                              void *ws, cudaStream_t st, int mask_ready = 0);
 
-// up_counter: see launch_dense_masked (NULL unless the fused router was launched just before on `st`)
+// up_counter: see launch_tc_experts (NULL unless the fused router was launched just before on `st`)
+// n_sel: device word that holds the number of selected pairs when the expert kernels start (NULL: r->n_sel)
 d2d_status d2d_launch_moe_ffn(const d2d_layer *L, const void *x, int T, const d2d_routing *r, void *y,
-                              void *ws, size_t ws_bytes, cudaStream_t st, int *up_counter = nullptr, int small_fused = 0);
+                              void *ws, size_t ws_bytes, cudaStream_t st, int *up_counter = nullptr, int small_fused = 0,
+                              const int32_t *n_sel = nullptr);
 size_t d2d_moe_ffn_ws_bytes(const d2d_layer *L, int T);
 
 // small-batch (T <= 64) kernels
@@ -93,8 +105,10 @@ bool d2d_small_select_supports(int T, int E);
 d2d_status d2d_small_select(const float *R, int T, int E, float tau, const d2d_routing *out, cudaStream_t st,
                             int mask_ready = 0);
 bool d2d_router_fused_supports(const d2d_layer_desc &D, int T);
+// ksum (optional, 8 device ints, words 0 and 1 zero at launch and left at zero): the kernel adds up k over all tokens
+// and its last CTA publishes the total, the number of selected (token, expert) pairs, in ksum[4]
 d2d_status d2d_router_fused(const d2d_layer *L, const void *x, int T, float tau, int do_mask, float *R, uint32_t *mask,
-                            int32_t *k, int32_t *status, cudaStream_t st);
+                            int32_t *k, int32_t *status, cudaStream_t st, int32_t *ksum = nullptr);
 d2d_status d2d_router_fused_group(const d2d_layer_desc &D, const d2d_router_weights &w, int n_layers, const void *x, int T,
                                   float tau, const d2d_routing *routing, uint32_t *mask_cat, int cat_words, cudaStream_t st);
 d2d_status d2d_small_group_fwd(const d2d_layer *const *layers, int n, const void *x, int T, float tau, const d2d_routing *routing,

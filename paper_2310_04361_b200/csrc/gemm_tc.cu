@@ -12,190 +12,17 @@
 // status word and leaves its loop, all roles meet at the final barrier, TMEM is freed and the
 // kernel returns (no trap, no endless spin).  Every load is a plain per-CTA load.
 #include "gemm_tc.cuh"
+#include "tc_common.cuh"
 
 #include <stdlib.h>
 
 namespace {
 
+using namespace d2d_tc;
+
 constexpr int BM = 128;          // rows of A per CTA = TMEM lanes
 constexpr int BK = 64;           // 64 bf16 = one 128-byte swizzle row
 constexpr int UMMA_K = 16;
-constexpr uint32_t WAIT_LIMIT = 1u << 22;
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-// Bounded wait for the phase with the given parity; false (and status set) when the limit runs out.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t *status)
-{
-    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
-        uint32_t done;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done)
-            : "r"(bar), "r"(parity)
-            : "memory");
-        if (done) return true;
-        if (it > 64) __nanosleep(32);
-    }
-    if (status) atomicMax(status, (int32_t)D2D_ERR_TIMEOUT);
-    return false;
-}
-
-// One non-blocking test of the phase with the given parity.
-__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity)
-{
-    uint32_t done;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(done)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return done != 0;
-}
-
-// Bounded wait for whole warps: try_wait may suspend the warp in hardware until the phase completes or a time
-// limit passes, so thirty-two waiting lanes cost no issue slots.  Nothing in the loop depends on the lane (same
-// barrier, same parity, the timer is read by one warp instruction), so the lanes stay in step and take the same
-// decision; a vote at the end would make that explicit but measured 1.8 % slower on the ViT-shaped layer.
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, int32_t *status)
-{
-    // how long one try may suspend is up to the hardware, so the bound is in time: about a second by the global timer
-    unsigned long long t0 = 0;
-    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
-        uint32_t done;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done)
-            : "r"(bar), "r"(parity)
-            : "memory");
-        if (done) return true;
-        if ((it & 31u) == 31u) {                               // rarely reached: a try normally ends with the phase complete
-            unsigned long long now;
-            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > 1000000000ull) break;
-        }
-    }
-    if (status) atomicMax(status, (int32_t)D2D_ERR_TIMEOUT);
-    return false;
-}
-// true in exactly one lane of a converged warp
-__device__ __forceinline__ bool elect_one()
-{
-    uint32_t pred;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "elect.sync _|p, 0xffffffff;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(pred));
-    return pred != 0;
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
-        : "memory");
-}
-
-// K-major operand tile whose rows are 128 bytes, 128-byte swizzle: 8-row groups are 1024 bytes apart.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
-{
-    uint64_t d = 0;
-    d |= (uint64_t)((addr >> 4) & 0x3fffu);
-    d |= (uint64_t)1 << 16;                 // leading byte offset (not used by swizzled K-major layouts)
-    d |= (uint64_t)(1024 >> 4) << 32;       // stride byte offset between 8-row groups
-    d |= (uint64_t)1 << 46;                 // descriptor version of this architecture
-    d |= (uint64_t)2 << 61;                 // 128-byte swizzle
-    return d;
-}
-
-__device__ __forceinline__ uint32_t instr_desc_bf16(int m, int n)
-{
-    return (1u << 4)                        // fp32 accumulator
-           | (1u << 7) | (1u << 10)         // A and B are bf16
-           | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);   // both operands K-major
-}
-
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// ---- helpers of the 2-CTA (cta_group::2) variant: a CTA pair shares one 256-row tile ----
-__device__ __forceinline__ uint32_t cluster_ctarank()
-{
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ void cluster_sync_all()
-{
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_addr, uint32_t rank)
-{
-    uint32_t r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_addr), "r"(rank));
-    return r;
-}
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
-{
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-// TMA load issued by either CTA of a pair; the transaction bytes are credited to the barrier at `bar`
-// (a shared::cluster address, normally the leader CTA's barrier).  Each CTA loads its own data.
-__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
-        : "memory");
-}
-__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-// arrives on the barrier at the same shared-memory offset in BOTH CTAs of the pair once the MMAs issued so far retire:
-// two commits, one per CTA's copy of the barrier (addressed through the cluster window)
-__device__ __forceinline__ void umma_commit_pair(uint32_t bar)
-{
-    const uint32_t b0 = map_to_cta(bar, 0), b1 = map_to_cta(bar, 1);
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(b0) : "memory");
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(b1) : "memory");
-}
 
 struct EpiParams {
     const __nv_bfloat16 *bias;
@@ -210,6 +37,8 @@ struct EpiParams {
     int gate_cat;                    // 1 (gated): tm_b covers up and gate rows interleaved in blocks of BN, one load brings both
     int band_rows;                   // > 0: tiles are walked column-major inside bands of this many row tiles (L2 reuse)
     int batch;                       // >= 1 problems of one shape: A columns, B rows, bias entries and out advance per problem
+    const int32_t *n_sel;            // density-adaptive dispatch: do nothing when *n_sel <= n_sel_max (NULL: always run)
+    long long n_sel_max;
 };
 
 // Tile index -> (row tile, column tile).  Plain order is row-major: CTAs that run together share a few rows of A and
@@ -226,109 +55,6 @@ __device__ __forceinline__ void tile_coords(int tile, int rows, int cols, int ba
     r = b * band + (idx - c * h);
 }
 
-// Activations of the bf16 tensor-core path.  Results are rounded to bf16 (8 bits of mantissa,
-// 2^-9 relative), and the epilogue of the up projection is issue-bound (K = d is short compared
-// with the 128 x BN outputs of a tile), so every activation is built on ONE special-function
-// instruction, the hardware tanh (relative error about 2^-11):
-//   SiLU       z * sigmoid(z)            = z * (0.5 + 0.5 tanh(z / 2))
-//   GELU tanh  0.5 z (1 + tanh(c (z + 0.044715 z^3)))
-//   GELU erf   0.5 z (1 + erf(z / sqrt 2)),  erf(z / sqrt 2) ~= tanh(z (a + b z^2 + c z^4)), a quintic
-//              argument fitted to erf with maximum error 3.7e-5 (GELU: 5.4e-5 absolute before the tanh
-//              instruction's own error) -- well below what a bf16 result can represent.
-__device__ __forceinline__ float fast_tanh(float x)
-{
-    float y;
-    asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
-template <int ACT> __device__ __forceinline__ float fast_act(float z)
-{
-    if (ACT == D2D_ACT_RELU) return fmaxf(z, 0.0f);
-    if (ACT == D2D_ACT_GELU_ERF) {
-        // the quintic was fitted on |z| <= 8 and turns over beyond |z| ~ 11: clamp z^2 inside it (tanh is 1 there anyway)
-        const float z2 = fminf(z * z, 64.0f);
-        const float q = fmaf(fmaf(-3.15807042e-4f, z2, 3.67982560e-2f), z2, 7.97717834e-1f);
-        const float t = fast_tanh(z * q);
-        return z * fmaf(0.5f, t, 0.5f);
-    }
-    if (ACT == D2D_ACT_GELU_TANH) {
-        const float q = fmaf(0.79788456080286536f * 0.044715f, z * z, 0.79788456080286536f);
-        const float t = fast_tanh(z * q);
-        return z * fmaf(0.5f, t, 0.5f);
-    }
-    const float t = fast_tanh(0.5f * z);                   // SiLU
-    return z * fmaf(0.5f, t, 0.5f);
-}
-
-// ---- packed float32 pairs (sm_100 issues add / mul / fma on two float32 values per instruction; same IEEE results
-// as the scalar forms).  The epilogue is bound by instruction issue, so its per-element math runs on pairs.
-__device__ __forceinline__ uint64_t pack2(float a, float b)
-{
-    uint64_t r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
-    return r;
-}
-__device__ __forceinline__ void unpack2(uint64_t v, float &a, float &b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
-__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c)
-{
-    uint64_t d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
-__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b)
-{
-    uint64_t d;
-    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
-__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
-{
-    uint64_t d;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
-__device__ __forceinline__ uint64_t dup2(float a) { return pack2(a, a); }
-
-// fast_act on a pair; the same operations in the same order as the scalar form, so the results are identical
-template <int ACT> __device__ __forceinline__ uint64_t fast_act2(uint64_t z)
-{
-    float a, b;
-    if (ACT == D2D_ACT_RELU) {
-        unpack2(z, a, b);
-        return pack2(fmaxf(a, 0.0f), fmaxf(b, 0.0f));
-    }
-    uint64_t arg;
-    if (ACT == D2D_ACT_GELU_ERF) {
-        unpack2(mul2(z, z), a, b);
-        const uint64_t z2 = pack2(fminf(a, 64.0f), fminf(b, 64.0f));
-        const uint64_t q = fma2(fma2(dup2(-3.15807042e-4f), z2, dup2(3.67982560e-2f)), z2, dup2(7.97717834e-1f));
-        arg = mul2(z, q);
-    } else if (ACT == D2D_ACT_GELU_TANH) {
-        const uint64_t q = fma2(dup2(0.79788456080286536f * 0.044715f), mul2(z, z), dup2(0.79788456080286536f));
-        arg = mul2(z, q);
-    } else {
-        arg = mul2(dup2(0.5f), z);                          // SiLU
-    }
-    unpack2(arg, a, b);
-    const uint64_t t = pack2(fast_tanh(a), fast_tanh(b));
-    return mul2(z, fma2(dup2(0.5f), t, dup2(0.5f)));
-}
-
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr));
-}
 
 // 16 accumulator columns -> 16 output values: bias (float32, staged in shared memory), activation, selection mask.
 template <int EPI, int ACT, bool GATED>
@@ -405,18 +131,13 @@ __host__ __device__ constexpr int pow2_at_least(int v) { return v <= 32 ? 32 : v
 // Persistent kernel: CTA c computes tiles c, c + gridDim.x, ... (128 x BN each, column tiles
 // fastest).  Two accumulator buffers in TMEM let the epilogue of one tile overlap the MMAs of the
 // next.  GATED: two B tiles (up, gate) share the A tile; the epilogue forms A(gate) * (up + bias).
-// PAIR: two CTAs of a cluster (adjacent SMs) compute one 256 x BN tile with tcgen05.mma.cta_group::2: each CTA
-// loads its own 128 rows of A and only HALF of the B tile, the MMA reads both halves, and each CTA ends up with
-// its 128 accumulator rows in its own TMEM.  This cuts the L2 -> SM operand traffic per FLOP by 1.5x without
-// any load that is shared between CTAs.  The even CTA issues the MMAs; barriers that both CTAs need are signalled
-// with one commit per CTA (stage release, accumulator ready) or remote arrives (accumulator drained).
-template <int BN, int STAGES, int EPI, int ACT, bool GATED, bool PAIR>
+template <int BN, int STAGES, int EPI, int ACT, bool GATED>
 __global__ void __launch_bounds__(NTHREADS_V2, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
                const __grid_constant__ CUtensorMap tm_b2, EpiParams ep, int M, int N, int K, int k_splits)
 {
-    constexpr int TM = PAIR ? 2 * BM : BM;                // rows of the tile a CTA (pair) computes
-    constexpr int B_ROWS = PAIR ? BN / 2 : BN;            // rows of B this CTA stages
+    constexpr int TM = BM;                                // rows of the tile a CTA computes
+    constexpr int B_ROWS = BN;                            // rows of B this CTA stages
     constexpr int A_BYTES = BM * BK * 2;
     constexpr int B_BYTES = B_ROWS * BK * 2;
     constexpr int STAGE_BYTES = A_BYTES + (GATED ? 2 : 1) * B_BYTES;
@@ -447,9 +168,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     // epilogue adds its partial sums to a float32 buffer (small-M problems that would leave most SMs idle)
     const int tiles_pp = ((M + TM - 1) / TM) * n_tiles;            // output tiles per problem
     const int total_tiles = tiles_pp * ep.batch * k_splits;
-    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;           // 0 = the CTA that issues the MMAs
-    const int worker = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
-    const int n_workers = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+    const int worker = (int)blockIdx.x;
+    const int n_workers = (int)gridDim.x;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -458,28 +178,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&bar_acc_full[b]), 1);
-            mbar_init(smem_u32(&bar_acc_empty[b]), PAIR ? 2 * N_EPI_WARPS : N_EPI_WARPS);
+            mbar_init(smem_u32(&bar_acc_empty[b]), N_EPI_WARPS);
             mbar_init(smem_u32(&sched_full[b]), 1);
             mbar_init(smem_u32(&sched_empty[b]), 2);          // read by the MMA thread and by the epilogue's leader
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
-        if (PAIR) {
-            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_holder)),
-                         "r"((uint32_t)TMEM_COLS)
-                         : "memory");
-            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-        } else {
-            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_holder)),
-                         "r"((uint32_t)TMEM_COLS)
-                         : "memory");
-            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-        }
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_holder)),
+                     "r"((uint32_t)TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    if (PAIR) cluster_sync_all();          // the peer's barriers are initialised before anything signals them
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = tmem_base_holder;
     // Programmatic dependent launch: everything above (barriers, TMEM, the bias vector: parameters, not activations)
@@ -487,7 +199,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     // and its writes are visible.  The next kernel of the stream may be scheduled onto SMs as this grid frees them.
     // With late_wait only the epilogue depends on that kernel (the selection mask written by the router): the
     // operand loads and the MMAs of the first tiles then overlap it, and only the epilogue warps wait.
-    const bool dyn = !PAIR && ep.tile_counter != nullptr;
+    const bool dyn = ep.tile_counter != nullptr;
     if (bias_cached && warp >= 2) {
         // The epilogue warps stage the bias (a parameter: no need to wait for the previous kernel) while the producer
         // and the MMA thread are already at work.  16-byte loads, all issued before the first use: the fill costs one
@@ -506,11 +218,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
     }
     // early_b: the B operand (weights) does not depend on the previous kernel either, so the producer requests the B
     // tiles of its first k-blocks BEFORE it waits for that kernel and only the A tiles after (static schedule only)
-    const bool early_b = !PAIR && !dyn && !ep.late_wait;
+    const bool early_b = !dyn && !ep.late_wait && ep.n_sel == nullptr;
     if (warp >= 2 || (!ep.late_wait && !(early_b && warp == 0))) asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // density-adaptive dispatch: below the crossover the gathered kernel, launched next to this one, does the work
+    // (every thread has passed the dependency wait here: the host never combines n_sel with late_wait)
+    const bool run = ep.n_sel == nullptr || (long long)__ldcg(ep.n_sel) > ep.n_sel_max;
 
-    if (warp == 0) {
+    if (!run) {
+        // nothing to do
+    } else if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
         if (lane == 0) {
             uint32_t it = 0, pre = 0;
@@ -554,7 +271,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 if (ep.batch > 1) { prob = tile / tiles_pp; tile -= prob * tiles_pp; }
                 int tr, tc;
                 tile_coords(tile, (M + TM - 1) / TM, n_tiles, ep.band_rows, tr, tc);
-                const int m0 = tr * TM + (int)rank * BM, n0 = prob * N + tc * BN + (int)rank * B_ROWS;
+                const int m0 = tr * TM, n0 = prob * N + tc * BN;
                 const int ka = prob * K;                      // problem p reads columns [p*K, (p+1)*K) of A
                 if (early_b && local == 0) {
                     // arm the first stages and request their B tiles, then wait for the previous kernel (A may be its output)
@@ -574,19 +291,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     ok = mbar_wait(smem_u32(&bar_empty[s]), (round & 1u) ^ 1u, ep.status);
                     if (!ok) break;
                     const uint32_t dst = smem_u32(smem + (size_t)s * STAGE_BYTES);
-                    if (PAIR) {
-                        // both CTAs' bytes are credited to the leader's barrier (where the MMAs are issued)
-                        const uint32_t full = map_to_cta(smem_u32(&bar_full[s]), 0);
-                        if (rank == 0) mbar_expect_tx(smem_u32(&bar_full[s]), 2u * (uint32_t)STAGE_BYTES);
-                        tma_load_2d_pair(dst, &tm_a, ka + kb * BK, m0, full);
-                        tma_load_2d_pair(dst + A_BYTES, &tm_b, kb * BK, n0, full);
-                        if (GATED) tma_load_2d_pair(dst + A_BYTES + B_BYTES, &tm_b2, kb * BK, n0, full);
-                    } else {
-                        const uint32_t full = smem_u32(&bar_full[s]);
-                        mbar_expect_tx(full, (uint32_t)STAGE_BYTES);
-                        tma_load_2d(dst, &tm_a, ka + kb * BK, m0, full);
-                        load_b(dst, full, kb, n0);
-                    }
+                    const uint32_t full = smem_u32(&bar_full[s]);
+                    mbar_expect_tx(full, (uint32_t)STAGE_BYTES);
+                    tma_load_2d(dst, &tm_a, ka + kb * BK, m0, full);
+                    load_b(dst, full, kb, n0);
                 }
             }
         }
@@ -594,11 +302,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
         // ------------------------------------------------------------------ MMA issuer
         // The whole warp walks the loop, so that waits, indices and descriptors are warp-uniform (the tensor-core
         // instructions take their operands from uniform registers); one elected lane issues the MMAs and commits.
-        if (rank == 0) {
-            // Gated (single CTA): the up and gate tiles sit back to back in shared memory, so they are ONE K-major
+        {
+            // Gated: the up and gate tiles sit back to back in shared memory, so they are ONE K-major
             // B operand of 2*BN rows and one MMA fills both accumulators (columns [0,BN) up, [BN,2BN) gate).
             // Two N=BN instructions would each pay the full A-operand read and run at half the rate.
-            const uint32_t idesc = instr_desc_bf16(TM, (GATED && !PAIR) ? 2 * BN : BN);
+            const uint32_t idesc = instr_desc_bf16(TM, GATED ? 2 * BN : BN);
             uint32_t it = 0, local = 0;
             bool ok = true;
             // The tensor core accepts only a few instructions ahead, so whatever this thread executes between the last
@@ -642,12 +350,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     auto issue = [&](int k) {
                         const uint64_t koff = (uint64_t)((k * UMMA_K * 2) >> 4);    // 32 bytes per K step inside the swizzle row
                         const uint32_t accum = (kb > kb0 || k != 0) ? 1u : 0u;
-                        if (PAIR) {
-                            umma_bf16_pair(acc, da + koff, db + koff, idesc, accum);
-                            if (GATED) umma_bf16_pair(acc + BN, da + koff, db2 + koff, idesc, accum);
-                        } else {
-                            umma_bf16(acc, da + koff, db + koff, idesc, accum);
-                        }
+                        umma_bf16(acc, da + koff, db + koff, idesc, accum);
                     };
                     if (elect_one()) {
 #pragma unroll
@@ -657,18 +360,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                     have = __all_sync(0xffffffffu, mbar_test(smem_u32(&bar_full[s_next]), round_next & 1u));
                     if (elect_one()) {
                         issue(BK / UMMA_K - 1);
-                        // stage reusable (in both CTAs of a pair) once these MMAs have read it
-                        if (PAIR) umma_commit_pair(smem_u32(&bar_empty[s]));
-                        else umma_commit(smem_u32(&bar_empty[s]));
+                        umma_commit(smem_u32(&bar_empty[s]));        // stage reusable once these MMAs have read it
                     }
                     __syncwarp();
                 }
                 if (!ok) break;
-                // accumulator of this tile complete (each CTA of a pair holds its own 128 rows)
-                if (elect_one()) {
-                    if (PAIR) umma_commit_pair(smem_u32(&bar_acc_full[buf]));
-                    else umma_commit(smem_u32(&bar_acc_full[buf]));
-                }
+                if (elect_one()) umma_commit(smem_u32(&bar_acc_full[buf]));   // accumulator of this tile complete
                 __syncwarp();
             }
         }
@@ -708,7 +405,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             if (ep.batch > 1) { prob = tile / tiles_pp; tile -= prob * tiles_pp; }
             int tr, tc;
             tile_coords(tile, (M + TM - 1) / TM, n_tiles, ep.band_rows, tr, tc);
-            const int m0 = tr * TM + (int)rank * BM, n0 = tc * BN;
+            const int m0 = tr * TM, n0 = tc * BN;
             // this problem's bias entries and output matrix
             const float *bias_p = bias_f + prob * N;
             const __nv_bfloat16 *bias_g = ep.bias ? ep.bias + prob * N : nullptr;
@@ -863,74 +560,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
             // all of this warp's TMEM reads of the buffer are complete: hand it back to the MMA warp
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
-            if (lane == 0) {
-                if (PAIR) mbar_arrive_cluster(map_to_cta(smem_u32(&bar_acc_empty[buf]), 0));   // the leader waits for both CTAs
-                else mbar_arrive(smem_u32(&bar_acc_empty[buf]));
-            }
+            if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[buf]));
 
         }
     }
 
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    if (PAIR) cluster_sync_all();          // neither CTA releases shared memory or TMEM while the other may still use it
-    if (warp == 1) {
-        if (PAIR)
-            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
-        else
-            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
-    }
+    if (warp == 1)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
 }
 
 // ------------------------------------------------------------------------------------------ host side
-
-typedef CUresult (*encode_tiled_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                    const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-encode_tiled_fn get_encode()
-{
-    static encode_tiled_fn fn = [] {
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-            q != cudaDriverEntryPointSuccess)
-            p = nullptr;
-        return (encode_tiled_fn)p;
-    }();
-    return fn;
-}
-
-// [rows, cols] bf16 row-major matrix, box = box_rows x 64 columns, 128-byte swizzle, zero fill outside.
-bool make_map(CUtensorMap *map, const void *base, int rows, int cols, int box_rows)
-{
-    encode_tiled_fn enc = get_encode();
-    if (!enc) return false;
-    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-    cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
-    cuuint32_t estr[2] = {1, 1};
-    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-int g_sm_count = 0;
-
-int sm_count()
-{
-    if (g_sm_count == 0) {
-        int dev = 0, n = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess &&
-            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
-            g_sm_count = n;
-        else
-            return 148;
-    }
-    return g_sm_count;
-}
-
-bool pdl_enabled();
 
 // Band height (in row tiles) for the tile walk, 0 = plain row-major.  Row-major order re-reads B once per wave of
 // CTAs, which is free while B stays in L2 (126 MB) beside the streaming A; only a large B (Llama-sized weights) needs
@@ -947,67 +588,71 @@ int band_rows_for(int M, int N, int K, int tile_m, bool gated)
     return band < 16 ? 16 : band;                           // shorter bands stream B too often (16 .. 32 measured alike)
 }
 
-template <int BN, int EPI, int ACT, bool GATED, bool PAIR>
+// cudaFuncAttributeMaxDynamicSharedMemorySize is a per-device attribute: set it once per (kernel, device).
+template <typename K> bool ensure_smem_attr(K kern, size_t smem, bool (&done)[64])
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+    if (!__atomic_load_n(&done[dev], __ATOMIC_ACQUIRE)) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return false;
+        __atomic_store_n(&done[dev], true, __ATOMIC_RELEASE);
+    }
+    return true;
+}
+
+template <int BN, int EPI, int ACT, bool GATED>
 d2d_status launch(const d2d_gemm_args &g, cudaStream_t st)
 {
-    constexpr int B_ROWS = PAIR ? BN / 2 : BN;
-    constexpr int STAGE_BYTES = BM * BK * 2 + (GATED ? 2 : 1) * B_ROWS * BK * 2;
+    constexpr int STAGE_BYTES = BM * BK * 2 + (GATED ? 2 : 1) * BN * BK * 2;
     constexpr int STAGES = (200 * 1024) / STAGE_BYTES > 8 ? 8 : (200 * 1024) / STAGE_BYTES;   // 200 KB of operand stages (+ 24 KB bias cache)
     constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + 1024 + (size_t)BIAS_CACHE_ELEMS * 4;
     CUtensorMap ta, tb, tb2;
-    const bool gate_cat = GATED && !PAIR && g.b_cat != nullptr && g.b_cat_block == BN;
+    const bool gate_cat = GATED && g.b_cat != nullptr && g.b_cat_block == BN;
     const int batch = g.batch > 1 ? g.batch : 1;
-    if (batch > 1 && (GATED || PAIR || g.K % BK != 0)) return D2D_ERR_UNSUPPORTED;
-    if (!make_map(&ta, g.a, g.M, g.K * batch, BM)) return D2D_ERR_CUDA;
+    if (batch > 1 && (GATED || g.K % BK != 0)) return D2D_ERR_UNSUPPORTED;
+    if (!d2d_tc_make_map(&ta, g.a, g.M, g.K * batch, BM)) return D2D_ERR_CUDA;
     if (gate_cat) {
-        if (!make_map(&tb, g.b_cat, 2 * BN * d2d_cdiv(g.N, BN), g.K, 2 * BN)) return D2D_ERR_CUDA;
+        if (!d2d_tc_make_map(&tb, g.b_cat, 2 * BN * d2d_cdiv(g.N, BN), g.K, 2 * BN)) return D2D_ERR_CUDA;
         tb2 = tb;
     } else {
-        if (!make_map(&tb, g.b, g.N * batch, g.K, B_ROWS)) return D2D_ERR_CUDA;
+        if (!d2d_tc_make_map(&tb, g.b, g.N * batch, g.K, BN)) return D2D_ERR_CUDA;
         if (GATED) {
-            if (!make_map(&tb2, g.b_gate, g.N, g.K, B_ROWS)) return D2D_ERR_CUDA;
+            if (!d2d_tc_make_map(&tb2, g.b_gate, g.N, g.K, BN)) return D2D_ERR_CUDA;
         } else {
             tb2 = tb;
         }
     }
-    auto kern = gemm_tc_kernel<BN, STAGES, EPI, ACT, GATED, PAIR>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM) != cudaSuccess) return D2D_ERR_CUDA;
-        attr_set = true;
-    }
+    auto kern = gemm_tc_kernel<BN, STAGES, EPI, ACT, GATED>;
+    static bool attr_set[64] = {};
+    if (!ensure_smem_attr(kern, SMEM, attr_set)) return D2D_ERR_CUDA;
     const int es = g.expert_size > 0 ? g.expert_size : 1;
     EpiParams ep{(const __nv_bfloat16 *)g.bias, g.out, g.mask, g.mask_words, es, g.status,
                  (uint32_t)((0x100000000ull + (unsigned long long)es - 1) / (unsigned long long)es),
-                 PAIR ? nullptr : g.tile_counter, (g.pdl_late_wait && pdl_enabled()) ? 1 : 0, gate_cat ? 1 : 0,
-                 band_rows_for(g.M, g.N, g.K, PAIR ? 2 * BM : BM, GATED), batch};
+                 g.tile_counter, (g.pdl_late_wait && !g.n_sel && d2d_tc_pdl_enabled()) ? 1 : 0, gate_cat ? 1 : 0,
+                 band_rows_for(g.M, g.N, g.K, BM, GATED), batch, g.n_sel, g.n_sel_max};
     const int k_splits = g.k_splits > 1 ? g.k_splits : 1;
-    const int tiles = d2d_cdiv(g.N, BN) * d2d_cdiv(g.M, PAIR ? 2 * BM : BM) * k_splits * batch;
-    const int workers = PAIR ? sm_count() / 2 : sm_count();
-    const int grid = (tiles < workers ? tiles : workers) * (PAIR ? 2 : 1);
+    const int tiles = d2d_cdiv(g.N, BN) * d2d_cdiv(g.M, BM) * k_splits * batch;
+    const int workers = d2d_tc_sm_count();
+    const int grid = tiles < workers ? tiles : workers;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid, 1, 1);
     cfg.blockDim = dim3(NTHREADS_V2, 1, 1);
     cfg.dynamicSmemBytes = SMEM;
     cfg.stream = st;
-    cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = PAIR ? 2 : 1;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
+    cudaLaunchAttribute attr[1];
     // the kernel's prologue may overlap the tail of the previous kernel in the stream (see griddepcontrol.wait in the kernel)
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = pdl_enabled() ? 2 : 1;
+    cfg.numAttrs = d2d_tc_pdl_enabled() ? 1 : 0;
     const cudaError_t err = cudaLaunchKernelEx(&cfg, kern, ta, tb, tb2, ep, g.M, g.N, g.K, k_splits);
     D2D_LAUNCHED(1);
     return err == cudaSuccess && cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
 }
 
 // Tile width that wastes the fewest SM-rounds: tiles / (rounds * workers), wider tiles preferred on ties
-// (fewer re-reads of A, fewer per-tile overheads).  A "worker" is an SM, or an SM pair for the 2-CTA variant.
-int pick_bn(int M, int N, int tile_m, int workers, const int *cands, int n_cands, double *eff_out, int batch = 1)
+// (fewer re-reads of A, fewer per-tile overheads).
+int pick_bn(int M, int N, int tile_m, int workers, const int *cands, int n_cands, int batch = 1)
 {
     int best = cands[0];
     double best_eff = -1.0;
@@ -1019,58 +664,19 @@ int pick_bn(int M, int N, int tile_m, int workers, const int *cands, int n_cands
         const double eff = useful * (double)tiles / (double)(rounds * workers) * (bn >= 128 ? 1.0 : 0.85);
         if (eff > best_eff + 1e-9) { best_eff = eff; best = bn; }
     }
-    if (eff_out) *eff_out = best_eff;
     return best;
-}
-
-bool pdl_enabled()
-{
-    static const bool on = [] {
-        const char *e = getenv("D2D_GEMM_PDL");            // D2D_GEMM_PDL=0 launches every GEMM fully serialised
-        return !(e && e[0] == '0');
-    }();
-    return on;
-}
-
-bool pair_mode_enabled()
-{
-    static const bool on = [] {
-        // off by default: measured on B200 the pair variant is not faster (the main loops are bound by the
-        // MMA issue interval, ~145 cycles per instruction, not by operand traffic); D2D_GEMM_PAIR=1 enables it
-        const char *e = getenv("D2D_GEMM_PAIR");
-        return e && e[0] == '1';
-    }();
-    return on;
 }
 
 template <int EPI, int ACT, bool GATED>
 d2d_status launch_bn(const d2d_gemm_args &g, cudaStream_t st)
 {
-    const int sms = sm_count();
-    if (GATED) {
-        if (pair_mode_enabled() && g.M > BM) return launch<128, EPI, ACT, true, true>(g, st);
-        return launch<128, EPI, ACT, true, false>(g, st);
-    } else {
-        // 2-CTA pairs (256-row tiles, half of B per CTA) when the problem has at least two row tiles and the
-        // pairs can be kept about as busy as single CTAs would be
-        const int cands2[3] = {256, 192, 128};
-        const int cands1[4] = {256, 192, 128, 64};
-        double eff2 = 0.0, eff1 = 0.0;
-        const int bn2 = pick_bn(g.M, g.N, 2 * BM, sms / 2, cands2, 3, &eff2);
-        const int bn1 = pick_bn(g.M, g.N, BM, sms, cands1, 4, &eff1, g.batch > 1 ? g.batch : 1);
-        if (pair_mode_enabled() && g.M > BM && g.batch <= 1 && eff2 >= 0.8 * eff1) {
-            switch (bn2) {
-            case 256: return launch<256, EPI, ACT, false, true>(g, st);
-            case 192: return launch<192, EPI, ACT, false, true>(g, st);
-            default: return launch<128, EPI, ACT, false, true>(g, st);
-            }
-        }
-        switch (bn1) {
-        case 256: return launch<256, EPI, ACT, false, false>(g, st);
-        case 192: return launch<192, EPI, ACT, false, false>(g, st);
-        case 128: return launch<128, EPI, ACT, false, false>(g, st);
-        default: return launch<64, EPI, ACT, false, false>(g, st);
-        }
+    if (GATED) return launch<128, EPI, ACT, true>(g, st);
+    const int cands[4] = {256, 192, 128, 64};
+    switch (pick_bn(g.M, g.N, BM, d2d_tc_sm_count(), cands, 4, g.batch > 1 ? g.batch : 1)) {
+    case 256: return launch<256, EPI, ACT, false>(g, st);
+    case 192: return launch<192, EPI, ACT, false>(g, st);
+    case 128: return launch<128, EPI, ACT, false>(g, st);
+    default: return launch<64, EPI, ACT, false>(g, st);
     }
 }
 
@@ -1103,6 +709,64 @@ splitk_finalize_kernel(const float *__restrict__ partial, const __nv_bfloat16 *_
     }
 }
 
+namespace {
+
+typedef CUresult (*encode_tiled_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                    const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+encode_tiled_fn get_encode()
+{
+    static encode_tiled_fn fn = [] {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            p = nullptr;
+        return (encode_tiled_fn)p;
+    }();
+    return fn;
+}
+
+}  // namespace
+
+bool d2d_tc_make_map(CUtensorMap *map, const void *base, int rows, int cols, int box_rows)
+{
+    encode_tiled_fn enc = get_encode();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    cuuint32_t box[2] = {64u, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int d2d_tc_sm_count()
+{
+    static int cached = 0;
+    if (cached == 0) {
+        int dev = 0, n = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && n > 0)
+            cached = n;
+        else
+            return 148;
+    }
+    return cached;
+}
+
+// D2D_GEMM_PDL=0 launches every GEMM fully serialised (no programmatic dependent launch)
+bool d2d_tc_pdl_enabled()
+{
+    static const bool on = [] {
+        const char *e = getenv("D2D_GEMM_PDL");
+        return !(e && e[0] == '0');
+    }();
+    return on;
+}
+
 bool d2d_gemm_tc_available() { return get_encode() != nullptr; }
 
 int d2d_gemm_tc_splits(int M, int N, int K, int batch)
@@ -1111,7 +775,7 @@ int d2d_gemm_tc_splits(int M, int N, int K, int batch)
     if (N & 3) return 1;
     const int tiles = d2d_cdiv(M, BM) * d2d_cdiv(N, 64) * (batch > 1 ? batch : 1);
     const int nkb = d2d_cdiv(K, BK);
-    int splits = sm_count() / (tiles > 0 ? tiles : 1);
+    int splits = d2d_tc_sm_count() / (tiles > 0 ? tiles : 1);
     if (splits > nkb / 2) splits = nkb / 2;          // at least two k-blocks per slice
     return splits >= 2 ? splits : 1;
 }
@@ -1131,7 +795,7 @@ d2d_status d2d_gemm_tc(const d2d_gemm_args &g, cudaStream_t st)
             p.epilogue = D2D_EPI_PARTIAL_F32;
             p.bias = nullptr;
             p.out = g.partial;
-            const d2d_status rc = launch<64, D2D_EPI_PARTIAL_F32, 0, false, false>(p, st);
+            const d2d_status rc = launch<64, D2D_EPI_PARTIAL_F32, 0, false>(p, st);
             if (rc != D2D_OK) return rc;
             const int blocks = d2d_cdiv(batch * g.M * g.N, 1024);
             splitk_finalize_kernel<<<blocks < 148 ? blocks : 148, 256, 0, st>>>(g.partial, (const __nv_bfloat16 *)g.bias,

@@ -49,6 +49,12 @@ struct d2d_gemm_args {
     // [batch*N], problem p owns rows / entries [p*N, (p+1)*N); out is [batch, M, N] (problem p at out + p*M*N).
     // Requires K % 64 == 0.  0 and 1 both mean a single problem.
     int batch;
+    // Density-adaptive dispatch (D2D_EPI_UP_MASKED): when n_sel is given the kernel reads the number of selected
+    // (token, expert) pairs from it once the previous kernel of the stream has completed and returns without doing
+    // anything if it is at most n_sel_max (the gathered kernel, launched with the complementary rule, does the
+    // work).  Cannot be combined with pdl_late_wait.
+    const int32_t *n_sel;
+    long long n_sel_max;
 };
 
 // Number of K slices d2d_gemm_tc would use for a [M,N,K] down projection (1 = no split) and the float32 scratch it needs.

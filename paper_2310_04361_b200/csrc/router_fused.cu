@@ -11,87 +11,28 @@
 
 #include "d2d_common.cuh"
 #include "gemm_tc.cuh"
+#include "tc_common.cuh"
 
 namespace {
 
+using d2d_tc::smem_u32; using d2d_tc::mbar_init; using d2d_tc::mbar_expect_tx; using d2d_tc::mbar_arrive;
+using d2d_tc::tma_load_2d; using d2d_tc::smem_desc_sw128; using d2d_tc::instr_desc_bf16; using d2d_tc::umma_bf16;
+using d2d_tc::umma_commit; using d2d_tc::tmem_ld16_issue; using d2d_tc::tmem_ld_wait;
+
 constexpr int BM = 128, BK = 64, UMMA_K = 16;
 constexpr int STAGES = 5;          // 5 x 32 KB of operands in flight: the first GEMM's main loop is bound by load latency
-constexpr uint32_t WAIT_LIMIT = 1u << 22;
 constexpr int NTHREADS = 64 + 512;       // TMA warp, MMA warp, 16 epilogue warps
 
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
+// every barrier wait of this kernel: 4096 back-to-back polls, then one poll every 128 ns
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int32_t *status)
 {
-    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
-        uint32_t done;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done)
-            : "r"(bar), "r"(parity)
-            : "memory");
-        if (done) return true;
-        if (it > 4096) __nanosleep(128);
-    }
-    if (status) atomicMax(status, (int32_t)D2D_ERR_TIMEOUT);
-    return false;
+    return d2d_tc::mbar_wait<4096, 128>(bar, parity, status);
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar)
-        : "memory");
-}
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr)
-{
-    uint64_t d = 0;
-    d |= (uint64_t)((addr >> 4) & 0x3fffu);
-    d |= (uint64_t)1 << 16;
-    d |= (uint64_t)(1024 >> 4) << 32;
-    d |= (uint64_t)1 << 46;
-    d |= (uint64_t)2 << 61;
-    return d;
-}
-__device__ __forceinline__ uint32_t instr_desc_bf16(int m, int n)
-{
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
-}
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
+// 16 accumulator columns of this thread's TMEM lane, complete on return
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16])
 {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr));
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+    tmem_ld16_issue(taddr, r);
+    tmem_ld_wait();
 }
 
 struct RouterLayerIO {
@@ -104,6 +45,8 @@ struct RouterGroupIO {
     RouterLayerIO l[D2D_MAX_GROUP];
     uint32_t *mask_cat;    // merged mask [T, cat_words] or NULL
     int cat_words;
+    int32_t *ksum;         // single layer only, or NULL: [0] running sum of k, [1] CTA exit ticket (both zero at launch and
+                           // left at zero), [4] receives the total = number of selected (token, expert) pairs
 };
 
 // Shared memory (dynamic, 1024-byte aligned):
@@ -376,15 +319,35 @@ router_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_const
                 }
                 pk_s[part * BM + r_local] = kt;
                 asm volatile("bar.sync 1, 512;" ::: "memory");
+                int k_row = 0;
                 if (part == 0 && row < T) {
-                    k[row] = pk_s[r_local] + pk_s[BM + r_local] + pk_s[2 * BM + r_local] + pk_s[3 * BM + r_local];
+                    k_row = pk_s[r_local] + pk_s[BM + r_local] + pk_s[2 * BM + r_local] + pk_s[3 * BM + r_local];
+                    k[row] = k_row;
                     if (anybad) atomicMax(status, (int32_t)D2D_ERR_NONFINITE);
+                }
+                if (io.ksum) {
+                    // number of selected pairs of the whole batch, for the density-adaptive dispatch of the expert step
+                    if (part == 0) {
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) k_row += __shfl_xor_sync(0xffffffffu, k_row, o);
+                        if (lane == 0) atomicAdd(io.ksum, k_row);
+                    }
+                    asm volatile("bar.sync 1, 512;" ::: "memory");
+                    if (warp == 2 && lane == 0) {
+                        __threadfence();
+                        if (atomicAdd(io.ksum + 1, 1) == (int)(gridDim.x * gridDim.y) - 1) {
+                            __threadfence();
+                            io.ksum[4] = atomicExch(io.ksum, 0);         // the CTA that finishes last publishes and resets
+                            io.ksum[1] = 0;
+                        }
+                    }
                 }
             }
         } else if (do_mask) {
             // keep the named barrier balanced when a bounded wait ran out
             asm volatile("bar.sync 1, 512;" ::: "memory");
             asm volatile("bar.sync 1, 512;" ::: "memory");
+            if (io.ksum) asm volatile("bar.sync 1, 512;" ::: "memory");
         }
     }
 
@@ -395,36 +358,6 @@ router_fused_kernel(const __grid_constant__ CUtensorMap tm_x, const __grid_const
     }
 }
 
-typedef CUresult (*encode_tiled_fn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                    const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-encode_tiled_fn get_encode()
-{
-    static encode_tiled_fn fn = [] {
-        void *p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-            q != cudaDriverEntryPointSuccess)
-            p = nullptr;
-        return (encode_tiled_fn)p;
-    }();
-    return fn;
-}
-
-bool make_map(CUtensorMap *map, const void *base, int rows, int cols, int box_rows)
-{
-    encode_tiled_fn enc = get_encode();
-    if (!enc) return false;
-    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-    cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
-    cuuint32_t estr[2] = {1, 1};
-    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 template <int DH>
 d2d_status launch(const d2d_layer_desc &D, const d2d_router_weights &w, int n_layers, const void *x, int T, float tau, int do_mask,
                   const RouterGroupIO &io, cudaStream_t st)
@@ -433,14 +366,16 @@ d2d_status launch(const d2d_layer_desc &D, const d2d_router_weights &w, int n_la
     constexpr int KB2 = DH / BK;
     constexpr size_t SMEM = (size_t)STAGES * STAGE_BYTES + (size_t)KB2 * BM * 128 + 1024;
     CUtensorMap tx, tw1, tw2;
-    if (!make_map(&tx, x, T, D.d, BM) || !make_map(&tw1, w.w_r1, D.d_h * n_layers, D.d, DH) ||
-        !make_map(&tw2, w.w_r2, D.n_experts * n_layers, D.d_h, 256))
+    if (!d2d_tc_make_map(&tx, x, T, D.d, BM) || !d2d_tc_make_map(&tw1, w.w_r1, D.d_h * n_layers, D.d, DH) ||
+        !d2d_tc_make_map(&tw2, w.w_r2, D.n_experts * n_layers, D.d_h, 256))
         return D2D_ERR_CUDA;
     auto kern = router_fused_kernel<DH>;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[64] = {};                         // the attribute is per device
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return D2D_ERR_CUDA;
+    if (!__atomic_load_n(&attr_set[dev], __ATOMIC_ACQUIRE)) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM) != cudaSuccess) return D2D_ERR_CUDA;
-        attr_set = true;
+        __atomic_store_n(&attr_set[dev], true, __ATOMIC_RELEASE);
     }
     const int EN = (D.n_experts + 15) / 16 * 16;
     kern<<<dim3(d2d_cdiv(T, BM), n_layers), NTHREADS, SMEM, st>>>(tx, tw1, tw2, (const __nv_bfloat16 *)w.b_r1, (const __nv_bfloat16 *)w.b_r2,
@@ -454,15 +389,16 @@ d2d_status launch(const d2d_layer_desc &D, const d2d_router_weights &w, int n_la
 bool d2d_router_fused_supports(const d2d_layer_desc &D, int T)
 {
     // d_h = 128 (the paper's router width) and E <= 256: operand ring, u and W_r2 then fit in shared memory together
-    return D.dtype == D2D_BF16 && T > d2d_decode_max_tokens() && D.d_h == 128 && D.n_experts <= 256 && D.d % 8 == 0 && get_encode() != nullptr;
+    return D.dtype == D2D_BF16 && T > d2d_decode_max_tokens() && D.d_h == 128 && D.n_experts <= 256 && D.d % 8 == 0 && d2d_gemm_tc_available();
 }
 
 // R may be NULL when only the mask is wanted; mask / k / status are used when do_mask != 0.
 d2d_status d2d_router_fused(const d2d_layer *L, const void *x, int T, float tau, int do_mask, float *R, uint32_t *mask,
-                            int32_t *k, int32_t *status, cudaStream_t st)
+                            int32_t *k, int32_t *status, cudaStream_t st, int32_t *ksum)
 {
     RouterGroupIO io = {};
     io.l[0] = {R, mask, k, status};
+    io.ksum = do_mask ? ksum : nullptr;
     const d2d_router_weights w = {L->w_r1, L->b_r1, L->w_r2, L->b_r2};
     return launch<128>(L->desc, w, 1, x, T, tau, do_mask, io, st);
 }

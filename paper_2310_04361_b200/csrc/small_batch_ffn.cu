@@ -231,6 +231,7 @@ struct SmallFfnLayer {
     float *y32;
     unsigned int *ticket;
     void *y;
+    long long capacity;      // entries the caller's perm buffer holds: a list truncated by D2D_ERR_CAPACITY is never read past it
 };
 struct SmallFfnArgs {
     SmallFfnLayer l[D2D_MAX_GROUP];
@@ -261,7 +262,10 @@ small_ffn_kernel(const TT *__restrict__ x, int T, int d, int s, int rc, const __
     __shared__ int stok[TBLK];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int e = blockIdx.x;
-    const int beg = offsets[e], end = offsets[e + 1];
+    // perm may have been truncated at `capacity` entries (the selection then reported D2D_ERR_CAPACITY): stay inside it
+    const long long cap = P.capacity;
+    const int end = (long long)offsets[e + 1] < cap ? offsets[e + 1] : (int)cap;
+    const int beg = offsets[e] < end ? offsets[e] : end;
 
     if (beg < end) {
         for (int r0 = 0; r0 < s; r0 += rc) {
@@ -275,7 +279,10 @@ small_ffn_kernel(const TT *__restrict__ x, int T, int d, int s, int rc, const __
             for (int p0 = beg; p0 < end; p0 += TBLK) {
                 const int ntok = end - p0 < TBLK ? end - p0 : TBLK;
                 __syncthreads();                                  // previous token block fully consumed
-                if (threadIdx.x < TBLK) stok[threadIdx.x] = perm[p0 + (threadIdx.x < ntok ? threadIdx.x : 0)];
+                if (threadIdx.x < TBLK) {
+                    const int tok = perm[p0 + (threadIdx.x < ntok ? threadIdx.x : 0)];
+                    stok[threadIdx.x] = tok < 0 ? 0 : tok >= T ? T - 1 : tok;      // a corrupt list cannot address outside x and y
+                }
                 __syncthreads();
                 for (int i = 0; i < ntok; ++i) cta_copy_async(xs + (size_t)i * d, x + (size_t)stok[i] * d, (size_t)d * sizeof(TT));
                 if (ntok < TBLK)
@@ -497,7 +504,7 @@ d2d_status d2d_small_group_fwd(const d2d_layer *const *layers, int n, const void
         const d2d_layer *L = layers[l];
         ra.l[l] = {L->w_r1, L->b_r1, L->w_r2, L->b_r2, u[l], R[l], L->tickets, y32[l], make_sel(&routing[l], tau)};
         fa.l[l] = {L->w1, L->b1, L->w_gate, L->w2t, L->b2, routing[l].offsets, routing[l].perm, y32[l], L->tickets + 16,
-                   (char *)y + (size_t)l * T * D.d * el};
+                   (char *)y + (size_t)l * T * D.d * el, (long long)routing[l].perm_capacity};
     }
     d2d_status rc = D.dtype == D2D_F32 ? launch_router<float>(D, n, ra, x, T, T * D.d, st)
                                        : launch_router<__nv_bfloat16>(D, n, ra, x, T, T * D.d, st);
@@ -521,7 +528,7 @@ d2d_status d2d_small_ffn(const d2d_layer *L, const void *x, int T, const d2d_rou
     // the ticket and the float32 accumulator must start at zero
     if (!fused) D2D_CUDA_TRY(cudaMemsetAsync(ws, 0, 256 + (size_t)T * L->desc.d * 4, st));
     SmallFfnArgs a = {};
-    a.l[0] = {L->w1, L->b1, L->w_gate, L->w2t, L->b2, r->offsets, r->perm, y32, ticket, y};
+    a.l[0] = {L->w1, L->b1, L->w_gate, L->w2t, L->b2, r->offsets, r->perm, y32, ticket, y, (long long)r->perm_capacity};
     if (L->desc.dtype == D2D_F32) return launch_ffn_dtype<float>(L->desc, 1, a, x, T, st);
     return launch_ffn_dtype<__nv_bfloat16>(L->desc, 1, a, x, T, st);
 }

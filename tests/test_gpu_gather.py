@@ -1,0 +1,179 @@
+"""GPU parity of the gathered, grouped expert path (tokens bucketed by groups of adjacent experts, Sec. 3.4 /
+Listing 1) and of the density-adaptive dispatch between it and the masked dense up projection.
+
+Every case runs the same inputs through each side of the dispatch (forced through d2d_layer_set_expert_path)
+and through the automatic choice, and compares y with the CPU oracle on the same mask.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2310_04361_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+TOL_Y = 2e-2          # bf16 in/out, float32 accumulation: max|y - y_ref| / max|y_ref|
+
+
+@pytest.fixture(scope="module")
+def api():
+    from paper_2310_04361_b200 import api as _api
+    assert torch.cuda.is_available()
+    return _api
+
+
+def _rel_err(got, ref):
+    ref = np.asarray(ref, dtype=np.float64)
+    got = np.asarray(got, dtype=np.float64)
+    return float(np.abs(got - ref).max() / max(np.abs(ref).max(), 1e-30))
+
+
+def _per_token_err(got, ref):
+    """max_t ( max_j |got - ref| / max_j |ref| ): every token normalised by its own magnitude."""
+    ref = np.asarray(ref, dtype=np.float64)
+    got = np.asarray(got, dtype=np.float64)
+    return float((np.abs(got - ref).max(1) / np.maximum(np.abs(ref).max(1), 1e-30)).max())
+
+
+def _routing(api, G, E):
+    return api.routing_from_mask(torch.from_numpy(oracle.pack_mask(G).view(np.int32)).cuda(), E)
+
+
+def _structured_mask(cfg, T, p, seed):
+    """Bernoulli(p) with the degenerate columns and rows the bucketing has to survive: an expert nobody keeps, an
+    expert everybody keeps, a token that keeps nothing, a token that keeps everything."""
+    rng = np.random.default_rng(seed)
+    G = (rng.random((T, cfg.E)) < p).astype(np.uint8)
+    G[:, 1 % cfg.E] = 0
+    G[:, (cfg.E - 2) % cfg.E] = 1
+    G[T // 3] = 0
+    G[T // 2] = 1
+    return G
+
+
+# (workload, tokens, experts per group or 0 = default, densities)
+GATHER_CASES = [
+    ("bert", 700, 0, (0.0, 0.03, 0.3, 1.0)),        # s = 24, default g = 4 (96 columns), ragged 256-token sub-chunk
+    ("bert", 1024, 2, (0.2,)),                      # 48-column groups
+    ("bert", 1300, 8, (0.1,)),                      # 192-column groups
+    ("vit", 900, 0, (0.05, 0.5)),                   # s = 16, g = 8
+    ("vit", 515, 4, (0.3,)),                        # 64-column groups
+    ("paper", 2100, 0, (0.0, 0.3, 1.0)),            # s = 128, one expert per group (the paper's benchmark shape)
+    ("llama", 600, 0, (0.1, 0.6)),                  # gated, s = 32, g = 4: one MMA fills the up and gate accumulators
+    ("llama", 257, 2, (0.4,)),
+    ("gpt2_ffn", 513, 0, (0.15,)),                  # d = 1024
+]
+
+
+@pytest.mark.parametrize("name,T,g,ps", GATHER_CASES)
+def test_gathered_up_projection_equals_masked_dense_and_oracle(api, name, T, g, ps):
+    cfg = wl.with_tokens(wl.CONFIGS[name], T)
+    w, x = wl.make_weights(cfg), wl.make_tokens(cfg)
+    layer = api.Layer.from_config(cfg, w)
+    layer.set_expert_path("auto", group=g)
+    xd = api.to_device(x, cfg.dtype)
+    act = oracle.ACT_BY_NAME[cfg.act]
+    for i, p in enumerate(ps):
+        G = _structured_mask(cfg, T, p, seed=17 * i + T) if 0.0 < p < 1.0 else np.full((T, cfg.E), int(p), np.uint8)
+        r = _routing(api, G, cfg.E)
+        H_dense = layer.expert_up_fwd(xd, r)
+        H = torch.full((T, cfg.d_ff), float("nan"), dtype=torch.bfloat16, device="cuda")     # every element must be written
+        for rep in range(2):                                   # twice: the sub-chunk counters reset themselves
+            layer.expert_up_gather_fwd(xd, r, H=H)
+            torch.cuda.synchronize()
+            assert r.status == 0
+            Hn = H.float().cpu().numpy().reshape(T, cfg.E, cfg.s)
+            assert np.isfinite(Hn).all()
+            assert not Hn[G == 0].any()                        # zero exactly where the token did not keep the expert
+            # the same products accumulated in the same order on the same unit
+            assert torch.equal(H, H_dense), (name, p, float((H.float() - H_dense.float()).abs().max()))
+            H.fill_(float("nan"))
+        layer.expert_up_gather_fwd(xd, r, H=H)
+        y = layer.expert_down_fwd(H).float().cpu().numpy()
+        y_ref = oracle.moe_ffn(x, w["w1"], w["b1"], w["w_gate"], w["w2"], w["b2"], act, G)
+        assert _rel_err(y, y_ref) <= TOL_Y, (name, p, _rel_err(y, y_ref))
+    layer.close()
+
+
+PATH_CASES = [("bert", 1000, 0.5), ("bert", 640, 0.9), ("vit", 1500, 0.6), ("paper", 1500, 0.3), ("llama", 520, 0.6)]
+
+
+@pytest.mark.parametrize("name,T,tau", PATH_CASES)
+def test_layer_fwd_is_the_same_on_both_sides_of_the_dispatch(api, name, T, tau):
+    """d2d_layer_fwd and d2d_moe_ffn_fwd with the up projection forced dense, forced gathered, and chosen on the
+    device with the crossover moved to either extreme: identical masks, y equal to the oracle's on that mask."""
+    cfg = wl.with_tokens(wl.CONFIGS[name], T)
+    w, x = wl.make_weights(cfg), wl.make_tokens(cfg)
+    layer = api.Layer.from_config(cfg, w)
+    xd = api.to_device(x, cfg.dtype)
+    act = oracle.ACT_BY_NAME[cfg.act]
+    ref_mask, y_ref = None, None
+    settings = [("dense", -1.0), ("gather", -1.0), ("auto", 0.0), ("auto", 1.0), ("auto", -1.0)]
+    for path, rho_max in settings:
+        layer.set_expert_path(path, rho_max=rho_max)
+        for lists in (True, False):
+            if not lists and name == "llama":
+                continue                                       # this router shape builds the lists on the way
+            r = layer.new_routing(T, lists=lists)
+            y = torch.full((T, cfg.d), float("nan"), dtype=torch.bfloat16, device="cuda")
+            for rep in range(2):
+                layer.layer_fwd(xd, tau, y=y, routing=r)
+                torch.cuda.synchronize()
+                assert r.status == 0
+            m = r.mask_u32().copy()
+            if ref_mask is None:
+                ref_mask = m
+                G = oracle.unpack_mask(m, cfg.E)
+                y_ref = oracle.moe_ffn(x, w["w1"], w["b1"], w["w_gate"], w["w2"], w["b2"], act, G)
+            assert np.array_equal(m, ref_mask)
+            assert r.n_sel == int(oracle.unpack_mask(m, cfg.E).sum())
+            yg = y.float().cpu().numpy()
+            assert np.isfinite(yg).all()
+            assert _rel_err(yg, y_ref) <= TOL_Y, (path, rho_max, lists, _rel_err(yg, y_ref))
+            assert _per_token_err(yg, y_ref) <= 4 * TOL_Y, (path, rho_max, lists, _per_token_err(yg, y_ref))
+        # the stand-alone expert step on the same mask
+        r2 = _routing(api, oracle.unpack_mask(ref_mask, cfg.E), cfg.E)
+        y2 = layer.moe_ffn_fwd(xd, r2).float().cpu().numpy()
+        assert _rel_err(y2, y_ref) <= TOL_Y
+    layer.close()
+
+
+def test_expert_path_settings_and_errors(api):
+    cfg = wl.with_tokens(wl.CONFIGS["bert"], 64)
+    layer = api.Layer.from_config(cfg, wl.make_weights(cfg))
+    assert layer.get_expert_path()[:2] == ("auto", 4)
+    layer.set_expert_path("gather", group=8, rho_max=0.25)
+    assert layer.get_expert_path() == ("gather", 8, 0.25)
+    for bad_group in (3, 16, 5):                               # not a divisor of 32 and E, or wider than one MMA
+        with pytest.raises(api.D2DError) as e:
+            layer.set_expert_path("auto", group=bad_group)
+        assert api.STATUS_NAMES[e.value.code] == "UNSUPPORTED"
+    layer.reset_counters()
+    torch.cuda.synchronize()
+    layer.close()
+    tiny = wl.CONFIGS["tiny"]                                  # fp32 layers have no tensor-core expert path
+    lt = api.Layer.from_config(tiny, wl.make_weights(tiny))
+    assert lt.get_expert_path()[1] == 0
+    with pytest.raises(api.D2DError) as e:
+        lt.set_expert_path("gather")
+    assert api.STATUS_NAMES[e.value.code] == "UNSUPPORTED"
+    lt.close()
+
+
+def test_decode_batch_with_truncated_lists_stays_inside_its_buffers(api):
+    """A perm buffer smaller than the number of selected pairs: the selection reports D2D_ERR_CAPACITY and the decode
+    expert kernel, which walks the lists, must not read past the buffer; guard words behind it stay untouched."""
+    cfg = wl.with_tokens(wl.CONFIGS["gpt2_ffn"], 4)
+    w, x = wl.make_weights(cfg), wl.make_tokens(cfg)
+    layer = api.Layer.from_config(cfg, w)
+    cap = 16
+    r = layer.new_routing(4, perm_capacity=cap)
+    guard = torch.full((4096,), -7, dtype=torch.int32, device="cuda")      # allocated right after: poison would be used as tokens
+    y = torch.zeros((4, cfg.d), dtype=torch.bfloat16, device="cuda")
+    layer.layer_fwd(api.to_device(x, cfg.dtype), 0.2, y=y, routing=r)
+    torch.cuda.synchronize()
+    assert r.status == 7 and r.n_sel > cap
+    assert bool((guard == -7).all())
+    assert torch.isfinite(y.float()).all()
+    layer.close()
