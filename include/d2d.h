@@ -145,9 +145,13 @@ D2D_API d2d_status d2d_layer_destroy(d2d_layer *layer);
  *                    proportional to the number of kept (token, group) pairs.
  *   D2D_PATH_AUTO    (default) decided per call on the device from the number of
  *                    selected pairs of that batch: gathered when
- *                    n_sel <= rho_max * T * E and T >= 512, dense otherwise.  Both
- *                    kernels are enqueued and the one not needed returns at once,
- *                    so there is no host synchronisation.
+ *                    n_sel <= rho_max * T * E, dense otherwise.  Both pairs of
+ *                    kernels are enqueued and the pair not needed returns at once,
+ *                    so there is no host synchronisation.  Batches whose up
+ *                    projection is below about 1e11 FLOP (100 us of tensor-core
+ *                    time) always take the dense form: the gathered kernel's
+ *                    fixed costs leave it nothing to win there, and the dense
+ *                    kernel then keeps its overlap with the router.
  * group: experts per group, 0 = library default for the shape (a power of two
  * that divides E, group * expert_size a multiple of 16 and at most 256, 128 for
  * gated layers).  rho_max: crossover density of D2D_PATH_AUTO, negative =
@@ -250,9 +254,15 @@ D2D_API d2d_status d2d_moe_ffn_fwd(const d2d_layer *layer, const void *x, int32_
  * for every neuron n of the original FFN: the expert up projections of all
  * kept (token, expert) pairs as one dense contraction with the selection
  * applied as a mask.  x: device [T, d]; H: device [T, d_ff] bf16 (caller's).
- * d2d_expert_up_gather_fwd: the same H through the gathered kernel
- * (D2D_PATH_GATHER with the layer's group size), whatever path the layer is
- * set to; D2D_ERR_UNSUPPORTED for shapes the gathered path cannot take.
+ * d2d_expert_up_gather_fwd: the gathered kernel (D2D_PATH_GATHER with the
+ * layer's group size), whatever path the layer is set to.  It writes ONLY the
+ * cells H[t, group columns] of kept (token, group) pairs -- with the same
+ * values d2d_expert_up_fwd writes there -- and leaves every other cell of H
+ * untouched; D2D_ERR_UNSUPPORTED for shapes the gathered path cannot take.
+ * d2d_expert_down_masked_fwd: y = (G * H) W2^T + b2 with the selection applied
+ * while H is read (cells of unkept (token, expert) pairs are never read), the
+ * down projection that follows the gathered kernel; valid for any H whose kept
+ * cells hold the hidden activations.  Needs routing->mask and ->status only.
  * d2d_expert_down_fwd (Sec. 3.2, 3.4): y = H W2^T + b2, which is
  * b2 + sum over kept experts of W2[:, blk] h_blk.  y: device [T, d] bf16;
  * status: device status word (receives D2D_ERR_TIMEOUT), may be NULL. */
@@ -260,6 +270,8 @@ D2D_API d2d_status d2d_expert_up_fwd(const d2d_layer *layer, const void *x, int3
                                      void *H, void *stream);
 D2D_API d2d_status d2d_expert_up_gather_fwd(const d2d_layer *layer, const void *x, int32_t T, const d2d_routing *routing,
                                             void *H, void *stream);
+D2D_API d2d_status d2d_expert_down_masked_fwd(const d2d_layer *layer, const void *H, int32_t T, const d2d_routing *routing,
+                                              void *y, void *stream);
 D2D_API d2d_status d2d_expert_down_fwd(const d2d_layer *layer, const void *H, int32_t T, void *y, int32_t *status,
                                        void *stream);
 

@@ -28,7 +28,7 @@ D2D_F32, D2D_BF16 = 0, 1
 ACTS = {"relu": 0, "gelu_erf": 1, "gelu_tanh": 2, "silu": 3}
 PATHS = {"auto": 0, "dense": 1, "gather": 2}
 EXPORTS = ["d2d_status_str", "d2d_launch_count", "d2d_layer_create", "d2d_layer_destroy", "d2d_workspace_bytes",
-           "d2d_layer_set_expert_path", "d2d_layer_get_expert_path", "d2d_layer_reset_counters", "d2d_expert_up_gather_fwd",
+           "d2d_layer_set_expert_path", "d2d_layer_get_expert_path", "d2d_layer_reset_counters", "d2d_expert_up_gather_fwd", "d2d_expert_down_masked_fwd",
            "d2d_select_workspace_bytes", "d2d_router_fwd", "d2d_select_dynk", "d2d_select_dynk_static", "d2d_select_topk",
            "d2d_routing_from_mask", "d2d_moe_ffn_fwd", "d2d_expert_up_fwd", "d2d_expert_down_fwd", "d2d_layer_fwd", "d2d_layer_fwd_host_workspace_bytes",
            "d2d_layer_fwd_host", "d2d_group_create", "d2d_group_destroy", "d2d_group_workspace_bytes", "d2d_group_fwd"]
@@ -67,6 +67,7 @@ _lib.d2d_routing_from_mask.argtypes = [c_int32, c_int32, POINTER(RoutingStruct),
 _lib.d2d_moe_ffn_fwd.argtypes = [c_void_p, c_void_p, c_int32, POINTER(RoutingStruct), c_void_p, c_void_p, c_size_t, c_void_p]
 _lib.d2d_expert_up_fwd.argtypes = [c_void_p, c_void_p, c_int32, POINTER(RoutingStruct), c_void_p, c_void_p]
 _lib.d2d_expert_up_gather_fwd.argtypes = [c_void_p, c_void_p, c_int32, POINTER(RoutingStruct), c_void_p, c_void_p]
+_lib.d2d_expert_down_masked_fwd.argtypes = [c_void_p, c_void_p, c_int32, POINTER(RoutingStruct), c_void_p, c_void_p]
 _lib.d2d_layer_set_expert_path.argtypes = [c_void_p, c_int, c_int32, ctypes.c_double]
 _lib.d2d_layer_get_expert_path.argtypes = [c_void_p, POINTER(c_int32), POINTER(c_int32), POINTER(ctypes.c_double)]
 _lib.d2d_layer_reset_counters.argtypes = [c_void_p, c_void_p]
@@ -257,8 +258,18 @@ class Layer:
                "d2d_expert_up_fwd")
         return H
 
+    def expert_down_masked_fwd(self, H, routing: Routing, y=None, stream=None):
+        """y = (G * H) W2^T + b2, reading only the kept cells of H (the down projection after the gathered kernel)."""
+        T = H.shape[0]
+        if y is None:
+            y = torch.empty((T, self.d), dtype=torch.bfloat16, device=self.device)
+        _check(_lib.d2d_expert_down_masked_fwd(self.handle, _ptr(H), T, ctypes.byref(routing.struct), _ptr(y), _stream(stream)),
+               "d2d_expert_down_masked_fwd")
+        return y
+
     def expert_up_gather_fwd(self, x, routing: Routing, H=None, stream=None):
-        """The same H through the gathered, grouped kernel (tokens bucketed by groups of adjacent experts)."""
+        """The gathered, grouped kernel (tokens bucketed by groups of adjacent experts): writes only the kept
+        (token, group) cells of H, the same values expert_up_fwd writes there."""
         T = x.shape[0]
         if H is None:
             H = torch.empty((T, self.d_ff), dtype=torch.bfloat16, device=self.device)

@@ -1,5 +1,6 @@
 // Host side of the C ABI declared in include/d2d.h: argument validation, weight packing,
 // workspace carving and kernel dispatch.  No computation happens on the host.
+#include <limits.h>
 #include <math.h>
 #include <new>
 #include <string.h>
@@ -95,17 +96,18 @@ size_t d2d_moe_ffn_ws_bytes(const d2d_layer *L, int T)
     return need;
 }
 
-// Density above which the masked dense up projection is faster than the gathered one for this shape (the automatic
-// choice).  The gathered kernel's cost is proportional to the fraction of (token, group) pairs u = 1 - (1 - rho)^g
-// (independent selections; correlated ones only lower u) times a per-row cost relative to the dense kernel that
-// depends on how wide one MMA of the group is; the constants are fitted to measurements on B200.
+// Density up to which the gathered up projection (followed by the down projection that applies the selection while it
+// stages H) beats the masked dense pair for this shape: the default crossover of the automatic choice.  Measured on
+// B200: the gathered kernel is bound by the rate at which token rows can be copied into the A stages (about the same
+// time per 128 x 64 tile of gathered rows whatever the MMA width), so its cost relative to the dense kernel is about
+// (256 / MMA columns) per gathered row, plus a fixed part (scanning the mask, one ragged tile per group visit); it wins
+// while the fraction of (token, group) pairs u = 1 - (1 - rho)^g stays below the value tabulated here.
 static double default_gather_rho_max(const d2d_layer_desc &D, int g)
 {
     if (g <= 0) return -1.0;
     const int n_mma = g * D.expert_size * (D.gated ? 2 : 1);
-    const double cost = n_mma >= 256 ? 1.05 : n_mma >= 128 ? 1.2 : n_mma >= 96 ? 1.5 : 2.2;
-    const double u_max = 0.92 / cost;
-    return u_max >= 1.0 ? 1.0 : 1.0 - pow(1.0 - u_max, 1.0 / g);
+    const double u_max = n_mma >= 256 ? 0.60 : n_mma >= 192 ? 0.30 : n_mma >= 128 ? 0.25 : 0.15;
+    return 1.0 - pow(1.0 - u_max, 1.0 / g);
 }
 
 // Expert step of bf16 batches above the decode sizes, on the tensor cores.
@@ -115,7 +117,8 @@ static double default_gather_rho_max(const d2d_layer_desc &D, int g)
 //     gathered       per group of adjacent experts, a contraction over the tokens that keep the group (moe_gather.cu);
 //                    its time is proportional to the number of (token, group) pairs
 //   down projection  y = H W2^T + b2 as a dense GEMM: exactly b2 + the sum over kept experts, since the h of an expert
-//                    the token did not keep is zero
+//                    the token did not keep is zero (written as zero by the masked dense kernel, or zero-filled from
+//                    the mask while H is staged when the gathered kernel, which writes only kept cells, may have run)
 // Which up projection runs is decided per call from the number of selected pairs of THIS batch.  D2D_PATH_AUTO
 // launches both kernels with complementary rules on a device word (n_sel) that is valid once the preceding kernel of
 // the stream has completed; the one that is not needed returns at once, so no host synchronisation is involved.
@@ -128,7 +131,11 @@ static d2d_status launch_tc_experts(const d2d_layer *L, const void *x, int T, co
     const d2d_layer_desc &D = L->desc;
     int path = L->expert_path;
     if (L->gather_group <= 0) path = D2D_PATH_DENSE;
-    if (path == D2D_PATH_AUTO && (T < 512 || !n_sel)) path = D2D_PATH_DENSE;      // small batches: every weight row is read either way
+    // The automatic choice costs two launches that return at once and the overlap of the router with the masked dense
+    // kernel's main loops: only for problems whose up projection takes long enough (about 100 us of tensor-core time)
+    // that this is noise.  Below that the fixed costs of the gathered kernel leave it nothing to win anyway.
+    const double up_flop = 2.0 * (double)T * D.d * D.d_ff * (D.gated ? 2.0 : 1.0);
+    if (path == D2D_PATH_AUTO && (up_flop < 1e11 || !n_sel)) path = D2D_PATH_DENSE;
     const long long n_sel_max = (long long)(L->gather_rho_max * (double)T * (double)D.n_experts);
     d2d_status rc;
     if (path != D2D_PATH_GATHER) {
@@ -148,12 +155,20 @@ static d2d_status launch_tc_experts(const d2d_layer *L, const void *x, int T, co
         ga.x = x; ga.w1 = L->w1; ga.w_gate = D.gated ? L->w_gate : nullptr; ga.b1 = L->b1; ga.mask = r->mask; ga.H = ws;
         ga.T = T; ga.d = D.d; ga.d_ff = D.d_ff; ga.n_experts = D.n_experts; ga.s = D.expert_size; ga.g = L->gather_group;
         ga.act = D.act; ga.status = r->status; ga.ctr = L->gather_ctr;
-        ga.n_sel = path == D2D_PATH_AUTO ? n_sel : nullptr; ga.n_sel_max = n_sel_max;
+        ga.n_sel = n_sel; ga.n_sel_max = path == D2D_PATH_AUTO ? n_sel_max : LLONG_MAX;
         rc = d2d_moe_gather_up(ga, st);
         if (rc != D2D_OK) return rc;
     }
+    // The gathered kernel writes only the kept cells of H, so whenever it may have run the down projection is the one
+    // that applies the selection while it stages H (it is valid after the masked dense up projection as well).
+    // With the automatic choice both down projections are enqueued as well, each with the rule of its up projection.
+    if (path != D2D_PATH_DENSE) {
+        rc = d2d_moe_down_masked(D, ws, r->mask, L->w2, L->b2, y, T, r->status, st, path == D2D_PATH_AUTO ? n_sel : nullptr, n_sel_max);
+        if (rc != D2D_OK || path == D2D_PATH_GATHER) return rc;
+    }
     d2d_gemm_args dn = {};
     dn.a = ws; dn.b = L->w2; dn.bias = L->b2; dn.out = y;
+    dn.n_sel = path == D2D_PATH_AUTO ? n_sel : nullptr; dn.n_sel_max = n_sel_max;
     dn.M = T; dn.N = D.d; dn.K = D.d_ff; dn.epilogue = D2D_EPI_BIAS_BF16; dn.status = r->status;
     // decode-sized batches: split K over the SMs, partial sums in the float32 scratch behind H
     dn.k_splits = d2d_gemm_tc_splits(T, D.d, D.d_ff);
@@ -436,7 +451,18 @@ d2d_status d2d_expert_up_gather_fwd(const d2d_layer *layer, const void *x, int32
     ga.x = x; ga.w1 = layer->w1; ga.w_gate = D.gated ? layer->w_gate : nullptr; ga.b1 = layer->b1; ga.mask = routing->mask; ga.H = H;
     ga.T = T; ga.d = D.d; ga.d_ff = D.d_ff; ga.n_experts = D.n_experts; ga.s = D.expert_size; ga.g = layer->gather_group;
     ga.act = D.act; ga.status = routing->status; ga.ctr = layer->gather_ctr;
+    ga.n_sel = routing->n_sel; ga.n_sel_max = LLONG_MAX;
     return d2d_moe_gather_up(ga, (cudaStream_t)stream);
+}
+
+d2d_status d2d_expert_down_masked_fwd(const d2d_layer *layer, const void *H, int32_t T, const d2d_routing *routing, void *y,
+                                      void *stream)
+{
+    if (!layer || T < 0) return D2D_ERR_INVALID_ARG;
+    if (T == 0) return D2D_OK;
+    if (!H || !y || !aligned16(H) || !aligned16(y) || !routing_ok(routing, true)) return D2D_ERR_INVALID_ARG;
+    if (!d2d_moe_down_masked_supports(layer->desc)) return D2D_ERR_UNSUPPORTED;
+    return d2d_moe_down_masked(layer->desc, H, routing->mask, layer->w2, layer->b2, y, T, routing->status, (cudaStream_t)stream);
 }
 
 d2d_status d2d_expert_down_fwd(const d2d_layer *layer, const void *H, int32_t T, void *y, int32_t *status, void *stream)

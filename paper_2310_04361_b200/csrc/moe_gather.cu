@@ -5,21 +5,27 @@
 // enough to run the tensor pipe at its full rate) and the tokens that keep at least one expert of the group.  Those
 // token rows are gathered into the swizzled A stages, multiplied with the group's contiguous W1 (and W_gate) rows,
 // and the epilogue applies bias, activation and the per-(token, expert) selection bits and scatters the gs hidden
-// activations of each row to H[token, group columns].  Rows of H that no expert of the group keeps are written as
-// zeros by the scheduler warp, so H is complete and the dense down projection can follow.  Executed work is
-// proportional to the number of (token, group) pairs, not to T * d_ff.
+// activations of each row to H[token, group columns].  Cells of H whose (token, group) pair is not kept are NOT
+// written: the down projection that follows (moe_down_masked_kernel below) never reads them, it zero-fills those
+// pieces of its A operand from the selection mask instead.  Executed work is proportional to the number of
+// (token, group) pairs, not to T * d_ff.
 //
 // One persistent CTA per SM, 14 warps:
 //   warp 0      scheduler: draws 256-token sub-chunks of a group from per-group device counters (work stealing at
 //               256-token granularity, so the CTAs finish together whatever the distribution of tokens over experts),
-//               compacts the tokens that keep the group with ballots into a row FIFO in shared memory, writes the zero
-//               rows, and emits 128-row tiles (rows left over are carried into the next sub-chunk of the same group;
-//               only the last tile of a group visit is ragged)
+//               compacts the tokens that keep the group with ballots into a row FIFO in shared memory and emits 128-row
+//               tiles (rows left over are carried into the next sub-chunk of the same group; only the last tile of a
+//               group visit is ragged)
 //   warp 1      allocates TMEM, issues tcgen05.mma (M = 128, N = gs or 2 gs for gated layers), two accumulators
 //   warps 2-5   gather: thread (row, 16-byte chunk) copies x rows with cp.async into the 128-byte-swizzled K-major
-//               layout the MMA descriptors expect; a group of copies is made visible to the tensor-core (async) proxy
-//               with fence.proxy.async before the stage's barrier is signalled.  Warp 2 also requests the W1 tiles
-//               (plain per-CTA TMA loads).
+//               layout the MMA descriptors expect and lets the copies themselves arrive on the stage's barrier
+//               (cp.async.mbarrier.arrive), so the threads never wait for data; the MMA warp executes the
+//               generic-to-async proxy fence after it has seen the barrier complete.  Warp 2 also requests the W1
+//               tiles (plain per-CTA TMA loads).  Measured alternatives, all slower or equal on B200: a fence in every
+//               gather thread after cp.async.wait_group (the threads then wait for data); one warp per stage that
+//               copies, waits, fences and signals; eight gather warps; one fence for several k-blocks; four-row TMA
+//               gathers (cp.async.bulk.tensor tile::gather4: no fence, but about 80 cycles per 512-byte gather).
+//               The stage period stays at about half a microsecond per 128 x 64 tile of gathered rows.
 //   warps 6-13  epilogue: tcgen05.ld, bias, activation, selection bits, 32-byte stores to the token's row of H
 // Every wait is bounded (status D2D_ERR_TIMEOUT), all roles meet at the final barrier, TMEM is freed.
 #include "moe_gather.cuh"
@@ -31,11 +37,17 @@ using namespace d2d_tc;
 
 constexpr int BM = 128, BK = 64, UMMA_K = 16;
 constexpr int A_BYTES = BM * BK * 2;
-constexpr int SUB = 256;                 // tokens per scheduler draw
+constexpr int MAX_SUB = 1024;            // most tokens per scheduler draw (a multiple of 256 chosen per launch, see launch())
 constexpr int TR = 4;                    // tile descriptors in flight
-constexpr int FIFO_CAP = 2048;           // row entries; in use at any time: TR * 128 emitted + 127 pending + SUB new
+constexpr int FIFO_CAP = 2048;           // row entries; in use at any time: TR * 128 emitted + 127 pending + MAX_SUB new
 constexpr int MAX_STAGES = 8;
-constexpr int WARP_SCHED = 0, WARP_MMA = 1, WARP_GATHER0 = 2, N_GATHER_WARPS = 4, WARP_EPI0 = 6, N_EPI_WARPS = 8;
+#ifndef D2D_GATHER_WARPS
+#define D2D_GATHER_WARPS 4
+#endif
+constexpr int WARP_SCHED = 0, WARP_MMA = 1, WARP_GATHER0 = 2, N_GATHER_WARPS = D2D_GATHER_WARPS, WARP_EPI0 = WARP_GATHER0 + N_GATHER_WARPS,
+              N_EPI_WARPS = 8;
+constexpr int ROWS_PER_PASS = N_GATHER_WARPS * 4;      // rows one pass of the gather threads covers (8 threads per row)
+constexpr int PASSES = BM / ROWS_PER_PASS;              // rows per gather thread and k-block
 constexpr int NTHREADS = 32 * (WARP_EPI0 + N_EPI_WARPS);
 
 struct GatherParams {
@@ -50,7 +62,9 @@ struct GatherParams {
     int T, d, d_ff, W;
     int g, s, gs, n_groups;          // experts per group, expert size, g * s, E / g
     uint32_t inv_s;                  // ceil(2^32 / s)
-    int stages, stage_bytes, lag;
+    int stages, stage_bytes;
+    int window;                      // groups the CTAs work in at the same time (their weight rows stay in L2)
+    int sub;                         // tokens per scheduler draw
 };
 
 struct TileDesc {
@@ -61,21 +75,43 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, uint32
 {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void cp_async_wait_lag(int lag)
+// one arrival on the barrier (counted in its initial count) once all earlier cp.async of this thread have completed
+__device__ __forceinline__ void cp_async_arrive(uint32_t bar)
 {
-    switch (lag) {
-    case 0: asm volatile("cp.async.wait_group 0;" ::: "memory"); break;
-    case 1: asm volatile("cp.async.wait_group 1;" ::: "memory"); break;
-    case 2: asm volatile("cp.async.wait_group 2;" ::: "memory"); break;
-    case 3: asm volatile("cp.async.wait_group 3;" ::: "memory"); break;
-    case 4: asm volatile("cp.async.wait_group 4;" ::: "memory"); break;
-    default: asm volatile("cp.async.wait_group 5;" ::: "memory"); break;
-    }
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
 }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __host__ __device__ constexpr int pow2_cols(int v) { return v <= 32 ? 32 : v <= 64 ? 64 : v <= 128 ? 128 : 256; }
+
+// The MMA warp's work for one tile: nkb k-blocks from the stage ring into the accumulator at `acc`.  The A tiles were
+// written by cp.async (generic proxy) and their arrival is observed through the stage's barrier; the proxy fence that
+// makes them visible to the tensor core's (async-proxy) reads is executed here, between that observation and the MMAs.
+__device__ __forceinline__ bool mma_tile(uint8_t *smem, uint64_t *bar_full, uint64_t *bar_empty, uint64_t *acc_full, uint32_t acc,
+                                         uint32_t idesc, int nkb, int stages, int stage_bytes, uint32_t &it, int32_t *status)
+{
+    for (int kb = 0; kb < nkb; ++kb, ++it) {
+        const uint32_t s = it % (uint32_t)stages, round = it / (uint32_t)stages;
+        if (!mbar_wait_warp(smem_u32(&bar_full[s]), round & 1u, status)) return false;
+        fence_async_smem();
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t a_addr = smem_u32(smem + (size_t)s * stage_bytes);
+        const uint64_t da = smem_desc_sw128(a_addr), db = smem_desc_sw128(a_addr + A_BYTES);
+        if (elect_one()) {
+#pragma unroll
+            for (int k = 0; k < BK / UMMA_K; ++k) {
+                const uint64_t koff = (uint64_t)((k * UMMA_K * 2) >> 4);
+                umma_bf16(acc, da + koff, db + koff, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+            }
+            umma_commit(smem_u32(&bar_empty[s]));
+        }
+        __syncwarp();
+    }
+    if (elect_one()) umma_commit(smem_u32(acc_full));
+    __syncwarp();
+    return true;
+}
 
 template <int ACT, bool GATED>
 __global__ void __launch_bounds__(NTHREADS, 1)
@@ -83,11 +119,11 @@ moe_gather_up_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_con
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    uint32_t *fifo = reinterpret_cast<uint32_t *>(smem + (size_t)p.stages * p.stage_bytes);     // [FIFO_CAP] token | bits << 24
-    int *zlist = reinterpret_cast<int *>(fifo + FIFO_CAP);                                       // [SUB] tokens whose row of the group is zero
+    uint32_t *fifo = reinterpret_cast<uint32_t *>(smem + (size_t)p.stages * p.stage_bytes);     // [FIFO_CAP] token indices
     __shared__ uint64_t bar_full[MAX_STAGES], bar_empty[MAX_STAGES], bar_acc_full[2], bar_acc_empty[2], tile_full[TR], tile_empty[TR];
     __shared__ TileDesc tdesc[TR];
     __shared__ uint32_t tmem_base_holder;
+    __shared__ uint32_t live[64];                             // scheduler: groups that still have sub-chunks (one bit each, E <= 2048)
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nkb = (p.d + BK - 1) / BK;
@@ -97,7 +133,8 @@ moe_gather_up_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_con
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; ++s) {
-            mbar_init(smem_u32(&bar_full[s]), 1 + N_GATHER_WARPS);     // the W1 request (with its byte count) + one arrival per gather warp
+            // the W1 request (with its byte count) + one arrival per gather thread, triggered when its copies have landed
+            mbar_init(smem_u32(&bar_full[s]), 1 + N_GATHER_WARPS * 32);
             mbar_init(smem_u32(&bar_empty[s]), 1);
         }
         for (int b = 0; b < 2; ++b) {
@@ -123,15 +160,25 @@ moe_gather_up_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_con
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // density-adaptive dispatch: above the crossover the masked dense kernel, launched next to this one, does the work
-    const bool run = p.n_sel == nullptr || (long long)__ldcg(p.n_sel) <= p.n_sel_max;
+    const bool run = p.n_sel == nullptr || (long long)__ldcg(p.n_sel) <= p.n_sel_max;      // n_sel_max = LLONG_MAX: always
 
     if (run && warp == WARP_SCHED) {
         // ------------------------------------------------------------------ scheduler
-        const int Ng = p.n_groups, n_sub = (p.T + SUB - 1) / SUB;
+        const int Ng = p.n_groups, SUB = p.sub, n_sub = (p.T + SUB - 1) / SUB;        // SUB is a multiple of 256
+        // Groups the CTAs work in at the same time.  The host's value keeps that many groups' weight rows in L2.  When
+        // few tokens keep a group, a visit of a CTA to a group should still yield several full tiles (its last tile is
+        // ragged and costs as much as a full one), so the CTAs spread over more groups: with gridDim.x / Wn CTAs per
+        // group a visit collects about u * T * Wn / gridDim.x rows, u = 1 - (1 - rho)^g the expected kept fraction.
+        int Wn = p.window;
+        if (p.n_sel) {
+            const float rho = fminf((float)__ldcg(p.n_sel) / ((float)p.T * (float)(Ng * p.g)), 1.0f);
+            const float u = fmaxf(1.0f - __expf((float)p.g * log1pf(-fminf(rho, 0.999f))), 1e-6f);
+            const float need = 8.0f * (float)BM * (float)gridDim.x / (u * (float)p.T);
+            const int w = need >= (float)Ng ? Ng : (int)need;
+            Wn = w > Wn ? w : Wn;
+        }
         const uint32_t lower = (1u << lane) - 1u;
-        const uint32_t gm = (1u << p.g) - 1u;                 // g <= 8
-        const int ppr = p.gs >> 3;                            // 16-byte pieces per zero row
-        int G = (int)(((long long)blockIdx.x * Ng) / (long long)gridDim.x);
+        const uint32_t gm = p.g >= 32 ? 0xffffffffu : (1u << p.g) - 1u;
         uint32_t head = 0, emitted = 0, tile_seq = 0;
         bool ok = true;
         auto emit = [&](uint32_t start, int n_rows, int group) -> bool {
@@ -147,52 +194,72 @@ moe_gather_up_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_con
             ++tile_seq;
             return true;
         };
-        for (int visited = 0; visited < Ng && ok;) {
+        // Visiting order: the groups are dealt to Wn "lanes" (group G belongs to lane G % Wn).  A CTA first works through
+        // its own lane, then through the others, so that at any time the CTAs are busy in about Wn groups whose weight
+        // rows stay in L2 while the token rows stream by.  Before it picks its next group a CTA takes a snapshot of all
+        // counters (one round trip for the whole warp) and skips the groups that are used up: a counter only grows, so
+        // "used up" is final and the walk over the order below never has to go back.
+        int j = 0, G = (int)blockIdx.x % Wn;                  // position in the order: lane (blockIdx.x + j) % Wn, group G
+        while (ok) {
+            for (int base = 0; base < Ng; base += 32) {
+                const int gi = base + lane;
+                const bool alive = gi < Ng && *(volatile const int *)(p.ctr + gi) < n_sub;
+                const uint32_t b = __ballot_sync(0xffffffffu, alive);
+                if (lane == 0) live[base >> 5] = b;
+            }
+            __syncwarp();
+            while (j < Wn && !((live[G >> 5] >> (G & 31)) & 1u)) {
+                G += Wn;
+                if (G >= Ng) {
+                    ++j;
+                    G = ((int)blockIdx.x + j) % Wn;
+                }
+            }
+            __syncwarp();                                     // everyone has read the snapshot before it is rewritten
+            if (j >= Wn) break;               // every group is used up
+            const int e0 = G * p.g, w = e0 >> 5, sh = e0 & 31;
+            // Draws of this group, software-pipelined: the counter is bumped one draw ahead, and a draw is walked in
+            // pieces of 256 tokens (eight mask words per lane) whose loads are requested one piece ahead of the
+            // compaction, so the warp waits for one memory latency per draw, not per piece.
+            auto load_piece = [&](int t0, uint32_t (&bits)[8]) {
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const int t = t0 + q * 32 + lane;
+                    bits[q] = t < p.T ? ((__ldg(p.mask + (size_t)t * p.W + w) >> sh) & gm) : 0u;
+                }
+            };
             int c = 0;
             if (lane == 0) c = atomicAdd(p.ctr + G, 1);
             c = __shfl_sync(0xffffffffu, c, 0);
-            if (c >= n_sub) {
-                // this group has no sub-chunk left: flush the rows carried so far as a ragged tile and move on
-                if (head != emitted) {
-                    ok = emit(emitted % FIFO_CAP, (int)(head - emitted), G);
-                    emitted = head;
+            while (c < n_sub && ok) {
+                int c_next = 0;
+                if (lane == 0) c_next = atomicAdd(p.ctr + G, 1);       // its round trip overlaps this draw
+                const int t_end = min((c + 1) * SUB, p.T);
+                uint32_t bits[8], bits_next[8];
+                load_piece(c * SUB, bits);
+                for (int t0 = c * SUB; t0 < t_end && ok; t0 += 256) {
+                    if (t0 + 256 < t_end) load_piece(t0 + 256, bits_next);
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        const bool keep = bits[q] != 0u;
+                        const uint32_t bk = __ballot_sync(0xffffffffu, keep);
+                        if (keep) fifo[(head + __popc(bk & lower)) % FIFO_CAP] = (uint32_t)(t0 + q * 32 + lane);
+                        head += __popc(bk);
+                    }
+                    while (head - emitted >= (uint32_t)BM && ok) {
+                        ok = emit(emitted % FIFO_CAP, BM, G);
+                        emitted += BM;
+                    }
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) bits[q] = bits_next[q];
                 }
-                G = G + 1 == Ng ? 0 : G + 1;
-                ++visited;
-                continue;
+                c = __shfl_sync(0xffffffffu, c_next, 0);
             }
-            const int t0 = c * SUB;
-            const int e0 = G * p.g, w = e0 >> 5, sh = e0 & 31;
-            uint32_t bits[SUB / 32];
-#pragma unroll
-            for (int j = 0; j < SUB / 32; ++j) {
-                const int t = t0 + j * 32 + lane;
-                bits[j] = t < p.T ? ((__ldg(p.mask + (size_t)t * p.W + w) >> sh) & gm) : 0u;
+            // no sub-chunk of this group is left: the rows carried so far go out as a ragged tile
+            if (ok && head != emitted) {
+                ok = emit(emitted % FIFO_CAP, (int)(head - emitted), G);
+                emitted = head;
             }
-            int nz = 0;
-#pragma unroll
-            for (int j = 0; j < SUB / 32; ++j) {
-                const int t = t0 + j * 32 + lane;
-                const bool keep = bits[j] != 0u, zero = !keep && t < p.T;
-                const uint32_t bk = __ballot_sync(0xffffffffu, keep), bz = __ballot_sync(0xffffffffu, zero);
-                if (keep) fifo[(head + __popc(bk & lower)) % FIFO_CAP] = (uint32_t)t | (bits[j] << 24);
-                if (zero) zlist[nz + __popc(bz & lower)] = t;
-                head += __popc(bk);
-                nz += __popc(bz);
-            }
-            __syncwarp();
-            while (head - emitted >= (uint32_t)BM && ok) {
-                ok = emit(emitted % FIFO_CAP, BM, G);
-                emitted += BM;
-            }
-            // rows of H that no expert of this group keeps are zero (the dense down projection reads all of H)
-            const int pieces = nz * ppr;
-            for (int i = lane; i < pieces; i += 32) {
-                const int r = i / ppr, q = i - r * ppr;
-                __nv_bfloat16 *o = p.H + (size_t)zlist[r] * p.d_ff + (size_t)G * p.gs + q * 8;
-                *reinterpret_cast<uint4 *>(o) = make_uint4(0u, 0u, 0u, 0u);
-            }
-            __syncwarp();                                     // zlist is rewritten by the next draw
         }
         emit(0u, -1, 0);                                      // end of the tile stream
         // the CTA whose scheduler finishes last leaves the counters at zero for the next launch
@@ -221,85 +288,51 @@ moe_gather_up_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_con
             ok = mbar_wait_warp(smem_u32(&bar_acc_empty[buf]), (use & 1u) ^ 1u, p.status);
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t acc = tmem_base + buf * buf_cols;
-            for (int kb = 0; kb < nkb; ++kb, ++it) {
-                const uint32_t s = it % (uint32_t)p.stages, round = it / (uint32_t)p.stages;
-                ok = mbar_wait_warp(smem_u32(&bar_full[s]), round & 1u, p.status);
-                if (!ok) break;
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t a_addr = smem_u32(smem + (size_t)s * p.stage_bytes);
-                const uint64_t da = smem_desc_sw128(a_addr), db = smem_desc_sw128(a_addr + A_BYTES);
-                if (elect_one()) {
-#pragma unroll
-                    for (int k = 0; k < BK / UMMA_K; ++k) {
-                        const uint64_t koff = (uint64_t)((k * UMMA_K * 2) >> 4);
-                        umma_bf16(acc, da + koff, db + koff, idesc, (kb > 0 || k > 0) ? 1u : 0u);
-                    }
-                    umma_commit(smem_u32(&bar_empty[s]));
-                }
-                __syncwarp();
-            }
-            if (!ok) break;
-            if (elect_one()) umma_commit(smem_u32(&bar_acc_full[buf]));
-            __syncwarp();
+            ok = mma_tile(smem, bar_full, bar_empty, &bar_acc_full[buf], tmem_base + buf * buf_cols, idesc, nkb, p.stages, p.stage_bytes, it,
+                          p.status);
         }
     } else if (run && warp >= WARP_GATHER0 && warp < WARP_EPI0) {
         // ------------------------------------------------------------------ gather warps: x rows -> swizzled A stages
         const int gw = warp - WARP_GATHER0, tid_g = gw * 32 + lane;
-        const int chunk = tid_g & 7, rbase = tid_g >> 3;      // this thread copies chunk `chunk` of rows rbase + 16 j
+        const int chunk = tid_g & 7, rbase = tid_g >> 3;      // this thread copies chunk `chunk` of rows rbase + ROWS_PER_PASS * j
         const uint32_t swz = (uint32_t)(((chunk ^ (rbase & 7)) << 4) + (rbase & 7) * 128 + (rbase >> 3) * 1024);
-        uint32_t it = 0, signaled = 0;
+        uint32_t it = 0;
         bool ok = true;
-        auto drain = [&]() {
-            cp_async_wait_lag(0);
-            fence_async_smem();
-            __syncwarp();
-            for (; signaled < it; ++signaled)
-                if (lane == 0) mbar_arrive(smem_u32(&bar_full[signaled % (uint32_t)p.stages]));
-        };
         for (uint32_t ti = 0; ok; ++ti) {
-            const uint32_t sl = ti % TR, par = (ti / TR) & 1u;
-            if (!mbar_test(smem_u32(&tile_full[sl]), par)) drain();       // nothing to overlap with: release what is in flight
-            ok = mbar_wait_warp(smem_u32(&tile_full[sl]), par, p.status);
+            const uint32_t sl = ti % TR;
+            ok = mbar_wait_warp(smem_u32(&tile_full[sl]), (ti / TR) & 1u, p.status);
             if (!ok) break;
             const int start = tdesc[sl].start, n_rows = tdesc[sl].n_rows, G = tdesc[sl].group;
             if (n_rows < 0) break;
-            const __nv_bfloat16 *src[8];
+            const __nv_bfloat16 *src[PASSES];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                int r = rbase + 16 * j;
-                r = r < n_rows ? r : n_rows - 1;              // rows past the end of a ragged tile repeat its last row (never stored)
-                const uint32_t e = fifo[(uint32_t)(start + r) % FIFO_CAP];
-                src[j] = p.x + (size_t)(e & 0xffffffu) * p.d + chunk * 8;
+            for (int j = 0; j < PASSES; ++j) {
+                int r = rbase + ROWS_PER_PASS * j;
+                // rows past the end of a ragged tile are zero-filled (no memory traffic) and never stored
+                src[j] = r < n_rows ? p.x + (size_t)fifo[(uint32_t)(start + r) % FIFO_CAP] * p.d + chunk * 8 : nullptr;
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&tile_empty[sl]));
-            for (int kb = 0; kb < nkb; ++kb) {
+            for (int kb = 0; kb < nkb; ++kb, ++it) {
                 const uint32_t s = it % (uint32_t)p.stages, round = it / (uint32_t)p.stages;
                 ok = mbar_wait_warp(smem_u32(&bar_empty[s]), (round & 1u) ^ 1u, p.status);
                 if (!ok) break;
-                const uint32_t stage = smem_u32(smem + (size_t)s * p.stage_bytes);
+                const uint32_t stage = smem_u32(smem + (size_t)s * p.stage_bytes), full = smem_u32(&bar_full[s]);
                 if (gw == 0 && elect_one()) {
-                    const uint32_t full = smem_u32(&bar_full[s]);
                     mbar_expect_tx(full, (uint32_t)(p.stage_bytes - A_BYTES));
                     tma_load_2d(stage + A_BYTES, &tm_w1, kb * BK, G * p.gs, full);
                     if (GATED) tma_load_2d(stage + A_BYTES + p.gs * 128, &tm_wg, kb * BK, G * p.gs, full);
                 }
-                const uint32_t nbytes = kb * BK + chunk * 8 < p.d ? 16u : 0u;      // zero fill past K
+                const bool in_k = kb * BK + chunk * 8 < p.d;                       // zero fill past K
 #pragma unroll
-                for (int j = 0; j < 8; ++j) cp_async16(stage + swz + (uint32_t)j * 2048u, nbytes ? src[j] + kb * BK : p.x, nbytes);
-                cp_async_commit();
-                ++it;
-                if (it - signaled > (uint32_t)p.lag) {
-                    cp_async_wait_lag(p.lag);
-                    fence_async_smem();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&bar_full[signaled % (uint32_t)p.stages]));
-                    ++signaled;
+                for (int j = 0; j < PASSES; ++j) {
+                    const bool live_row = in_k && src[j] != nullptr;
+                    cp_async16(stage + swz + (uint32_t)(j * ROWS_PER_PASS * 128), live_row ? src[j] + kb * BK : p.x, live_row ? 16u : 0u);
                 }
+                cp_async_arrive(full);                        // arrives when this thread's copies above have landed
             }
         }
-        drain();
+        cp_async_wait_all();                                  // nothing of this thread is in flight when the CTA exits
     } else if (run && warp >= WARP_EPI0) {
         // ------------------------------------------------------------------ epilogue
         const int ew = warp - WARP_EPI0, quad = warp & 3, half = ew >> 2;
@@ -316,11 +349,13 @@ moe_gather_up_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_con
             if (n_rows < 0) break;
             const int r = quad * 32 + lane;
             const bool valid = r < n_rows;
-            const uint32_t e = valid ? fifo[(uint32_t)(start + r) % FIFO_CAP] : 0u;
+            const uint32_t tok = valid ? fifo[(uint32_t)(start + r) % FIFO_CAP] : 0u;
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&tile_empty[sl]));
-            const uint32_t bits = e >> 24;
-            __nv_bfloat16 *orow = p.H + (size_t)(e & 0xffffffu) * p.d_ff + (size_t)G * p.gs;
+            // which experts of the group this token keeps (the load is covered by the wait for the accumulator)
+            const int e0 = G * p.g;
+            const uint32_t bits = valid ? __ldg(p.mask + (size_t)tok * p.W + (e0 >> 5)) >> (e0 & 31) : 0u;
+            __nv_bfloat16 *orow = p.H + (size_t)tok * p.d_ff + (size_t)G * p.gs;
             const __nv_bfloat16 *brow = p.b1 ? p.b1 + (size_t)G * p.gs : nullptr;
             const uint32_t buf = ti & 1u, use = ti >> 1;
             ok = mbar_wait_warp(smem_u32(&bar_acc_full[buf]), use & 1u, p.status);
@@ -393,6 +428,207 @@ moe_gather_up_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_con
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
 }
 
+// ---------------------------------------------------------------------------------------------------------------
+// Down projection after the gathered up projection: y = Hm W2^T + b2, where Hm[t, n] = G[t, n / s] ? H[t, n] : 0.
+// The selection is applied while the A operand is staged: a 16-byte piece of a row of H (8 neurons of one expert)
+// is copied only if the token keeps that expert and is zero-filled otherwise (cp.async with a source size of 0), so
+// cells of H that the gathered kernel never wrote are never read, and the pieces that are skipped cost no L2 traffic.
+// The contraction itself is dense (every token of a 128-token tile keeps some expert of every 64-neuron k-block).
+// Same roles as above without the scheduler: tiles are (128 tokens) x (bn columns of y), walked round-robin.
+struct DownParams {
+    const __nv_bfloat16 *H;          // [T, d_ff]
+    const uint32_t *mask;            // [T, W]
+    const __nv_bfloat16 *b2;         // [d] or NULL
+    __nv_bfloat16 *y;                // [T, d]
+    int32_t *status;
+    const int32_t *n_sel;            // density-adaptive dispatch: do nothing when *n_sel > n_sel_max (NULL: always run)
+    long long n_sel_max;
+    int T, d, d_ff, W, s;
+    uint32_t inv_s;
+    int bn, stages, stage_bytes, band;
+};
+
+__global__ void __launch_bounds__(NTHREADS, 1)
+moe_down_masked_kernel(const __grid_constant__ CUtensorMap tm_w2, const DownParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    __shared__ uint64_t bar_full[MAX_STAGES], bar_empty[MAX_STAGES], bar_acc_full[2], bar_acc_empty[2];
+    __shared__ uint32_t tmem_base_holder;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nkb = (p.d_ff + BK - 1) / BK;
+    const int row_tiles = (p.T + BM - 1) / BM, col_tiles = (p.d + p.bn - 1) / p.bn, total = row_tiles * col_tiles;
+    const uint32_t buf_cols = (uint32_t)pow2_cols(p.bn);
+    const uint32_t tmem_cols = 2u * buf_cols;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) {
+            mbar_init(smem_u32(&bar_full[s]), 1 + N_GATHER_WARPS * 32);
+            mbar_init(smem_u32(&bar_empty[s]), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&bar_acc_full[b]), 1);
+            mbar_init(smem_u32(&bar_acc_empty[b]), N_EPI_WARPS);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == WARP_MMA) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_holder)), "r"(tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = tmem_base_holder;
+    asm volatile("griddepcontrol.wait;" ::: "memory");       // H is the previous kernel's output
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const bool run = p.n_sel == nullptr || (long long)__ldcg(p.n_sel) <= p.n_sel_max;
+
+    // tile index -> (row tile, column tile): row-major, or column by column inside bands of `band` row tiles when W2 is
+    // too large to stay in L2 beside the streaming H (the band's rows of H are then re-used from L2 for every column)
+    auto coords = [&](int tile, int &r, int &c) {
+        if (p.band <= 0) { r = tile / col_tiles; c = tile - r * col_tiles; return; }
+        const int per_band = p.band * col_tiles;
+        const int b = tile / per_band, idx = tile - b * per_band;
+        const int h = row_tiles - b * p.band < p.band ? row_tiles - b * p.band : p.band;
+        c = idx / h;
+        r = b * p.band + (idx - c * h);
+    };
+
+    if (!run) {
+        // the masked dense up projection ran: the plain dense down projection, launched next to this kernel, follows it
+    } else if (warp == WARP_MMA) {
+        const uint32_t idesc = instr_desc_bf16(BM, p.bn);
+        uint32_t it = 0, local = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x, ++local) {
+            const uint32_t buf = local & 1u, use = local >> 1;
+            ok = mbar_wait_warp(smem_u32(&bar_acc_empty[buf]), (use & 1u) ^ 1u, p.status);
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            ok = mma_tile(smem, bar_full, bar_empty, &bar_acc_full[buf], tmem_base + buf * buf_cols, idesc, nkb, p.stages, p.stage_bytes, it,
+                          p.status);
+        }
+    } else if (warp >= WARP_GATHER0 && warp < WARP_EPI0) {
+        const int gw = warp - WARP_GATHER0, tid_g = gw * 32 + lane;
+        const int chunk = tid_g & 7, rbase = tid_g >> 3;
+        const uint32_t swz = (uint32_t)(((chunk ^ (rbase & 7)) << 4) + (rbase & 7) * 128 + (rbase >> 3) * 1024);
+        uint32_t it = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
+            int tr, tc;
+            coords(tile, tr, tc);
+            const int m0 = tr * BM, n0 = tc * p.bn;
+            uint32_t mw[PASSES];                              // the mask word that holds the current expert, one per row of this thread
+            int cur_w = -1;
+            for (int kb = 0; kb < nkb; ++kb, ++it) {
+                const uint32_t s = it % (uint32_t)p.stages, round = it / (uint32_t)p.stages;
+                const int col = kb * BK + chunk * 8;
+                const bool in_k = col < p.d_ff;
+                const uint32_t e = __umulhi((uint32_t)col, p.inv_s);     // the expert that owns these 8 neurons
+                if (in_k && (int)(e >> 5) != cur_w) {
+                    cur_w = (int)(e >> 5);
+#pragma unroll
+                    for (int j = 0; j < PASSES; ++j) {
+                        const int t = m0 + rbase + ROWS_PER_PASS * j;
+                        mw[j] = t < p.T ? __ldg(p.mask + (size_t)t * p.W + cur_w) : 0u;
+                    }
+                }
+                ok = mbar_wait_warp(smem_u32(&bar_empty[s]), (round & 1u) ^ 1u, p.status);
+                if (!ok) break;
+                const uint32_t stage = smem_u32(smem + (size_t)s * p.stage_bytes), full = smem_u32(&bar_full[s]);
+                if (gw == 0 && elect_one()) {
+                    mbar_expect_tx(full, (uint32_t)(p.stage_bytes - A_BYTES));
+                    tma_load_2d(stage + A_BYTES, &tm_w2, kb * BK, n0, full);
+                }
+                const __nv_bfloat16 *src = p.H + (size_t)(m0 + rbase) * p.d_ff + col;
+#pragma unroll
+                for (int j = 0; j < PASSES; ++j) {
+                    const bool keep = in_k && ((mw[j] >> (e & 31u)) & 1u);
+                    cp_async16(stage + swz + (uint32_t)(j * ROWS_PER_PASS * 128), keep ? src + (size_t)(ROWS_PER_PASS * j) * p.d_ff : p.H,
+                               keep ? 16u : 0u);
+                }
+                cp_async_arrive(full);
+            }
+        }
+        cp_async_wait_all();
+    } else if (warp >= WARP_EPI0) {
+        const int ew = warp - WARP_EPI0, quad = warp & 3, half = ew >> 2;
+        const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+        const bool wide = (p.d & 15) == 0 && (reinterpret_cast<uintptr_t>(p.y) & 31) == 0;
+        uint32_t local = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x, ++local) {
+            int tr, tc;
+            coords(tile, tr, tc);
+            const int row = tr * BM + quad * 32 + lane, n0 = tc * p.bn;
+            const uint32_t buf = local & 1u, use = local >> 1;
+            ok = mbar_wait_warp(smem_u32(&bar_acc_full[buf]), use & 1u, p.status);
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t tbase = tmem_base + buf * buf_cols + lane_base;
+            const int n_units = p.bn >> 4;
+            for (int u = half; u < n_units; u += 2) {
+                const int col0 = n0 + u * 16;
+                if (col0 >= p.d) break;                         // ragged last column tile (d is a multiple of 16)
+                uint32_t ra[16];
+                tmem_ld16_issue(tbase + (uint32_t)(u * 16), ra);
+                float bias[16];
+                if (p.b2) {
+                    float b8[8];
+                    d2d_load8(p.b2 + col0, b8);
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) bias[q] = b8[q];
+                    d2d_load8(p.b2 + col0 + 8, b8);
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) bias[8 + q] = b8[q];
+                } else {
+#pragma unroll
+                    for (int q = 0; q < 16; ++q) bias[q] = 0.0f;
+                }
+                tmem_ld_wait();
+                uint32_t pk[8];
+#pragma unroll
+                for (int j = 0; j < 16; j += 2) {
+                    const __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(ra[j]) + bias[j], __uint_as_float(ra[j + 1]) + bias[j + 1]);
+                    pk[j >> 1] = *reinterpret_cast<const uint32_t *>(&t2);
+                }
+                if (row < p.T) {
+                    __nv_bfloat16 *o = p.y + (size_t)row * p.d + col0;
+                    if (wide) {
+                        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(o), "r"(pk[0]), "r"(pk[1]), "r"(pk[2]),
+                                     "r"(pk[3]), "r"(pk[4]), "r"(pk[5]), "r"(pk[6]), "r"(pk[7]) : "memory");
+                    } else {
+                        *reinterpret_cast<uint4 *>(o) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        *reinterpret_cast<uint4 *>(o + 8) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                    }
+                }
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bar_acc_empty[buf]));
+        }
+    }
+
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == WARP_MMA)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+}
+
+bool ensure_attr(const void *kern, bool (&done)[64])
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+    if (!__atomic_load_n(&done[dev], __ATOMIC_ACQUIRE)) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 208 * 1024) != cudaSuccess) return false;
+        __atomic_store_n(&done[dev], true, __ATOMIC_RELEASE);
+    }
+    return true;
+}
+
 template <int ACT, bool GATED>
 d2d_status launch(const d2d_gather_args &a, cudaStream_t st)
 {
@@ -407,8 +643,15 @@ d2d_status launch(const d2d_gather_args &a, cudaStream_t st)
     p.stage_bytes = A_BYTES + b_rows * 128;
     int stages = (192 * 1024) / p.stage_bytes;
     p.stages = stages > MAX_STAGES ? MAX_STAGES : stages;
-    p.lag = p.stages - 2 > 4 ? 4 : p.stages - 2;
-    const size_t smem = (size_t)p.stages * p.stage_bytes + FIFO_CAP * 4 + SUB * 4 + 1024;      // at most 192 + 8 + 1 + 1 KB
+    // about 48 MB of weight rows in flight: the rest of L2 holds the token rows and the outputs
+    const long long group_bytes = (long long)b_rows * a.d * 2;
+    long long window = (48ll << 20) / (group_bytes > 0 ? group_bytes : 1);
+    p.window = (int)(window < 4 ? 4 : window > p.n_groups ? p.n_groups : window);
+    if (p.window > p.n_groups) p.window = p.n_groups;
+    // tokens per draw: about eight draws per CTA (the CTAs then finish together), 256 .. 1024
+    const long long want = (long long)a.T * p.n_groups / (8ll * d2d_tc_sm_count());
+    p.sub = want >= 1024 ? 1024 : want >= 512 ? 512 : 256;
+    const size_t smem = (size_t)p.stages * p.stage_bytes + FIFO_CAP * 4 + 1024;      // at most 192 + 8 + 1 KB
     if (smem > 208 * 1024) return D2D_ERR_UNSUPPORTED;
     CUtensorMap tw1, twg;
     if (!d2d_tc_make_map(&tw1, a.w1, a.d_ff, a.d, gs)) return D2D_ERR_CUDA;
@@ -419,12 +662,7 @@ d2d_status launch(const d2d_gather_args &a, cudaStream_t st)
     }
     auto kern = moe_gather_up_kernel<ACT, GATED>;
     static bool attr_set[64] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return D2D_ERR_CUDA;
-    if (!__atomic_load_n(&attr_set[dev], __ATOMIC_ACQUIRE)) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 208 * 1024) != cudaSuccess) return D2D_ERR_CUDA;
-        __atomic_store_n(&attr_set[dev], true, __ATOMIC_RELEASE);
-    }
+    if (!ensure_attr((const void *)kern, attr_set)) return D2D_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(d2d_tc_sm_count(), 1, 1);
     cfg.blockDim = dim3(NTHREADS, 1, 1);
@@ -456,22 +694,80 @@ d2d_status launch_act(const d2d_gather_args &a, cudaStream_t st)
 
 int d2d_gather_group_for(const d2d_layer_desc &D, int want)
 {
-    if (D.dtype != D2D_BF16 || D.d % 8 || D.d_ff % 8 || D.expert_size % 8 || !d2d_gemm_tc_available()) return 0;
+    if (!d2d_moe_down_masked_supports(D)) return 0;           // the gathered kernel's H needs the down projection that reads only kept cells
     const int max_cols = D.gated ? 128 : 256;                 // one MMA holds gs (gated: 2 gs) accumulator columns
     auto fits = [&](int g) {
         const int gs = g * D.expert_size;
-        return g >= 1 && g <= 8 && D.n_experts % g == 0 && 32 % g == 0 && gs % 16 == 0 && gs >= 16 && gs <= max_cols;
+        return g >= 1 && g <= 32 && D.n_experts % g == 0 && 32 % g == 0 && gs % 16 == 0 && gs >= 16 && gs <= max_cols;
     };
     if (want > 0) return fits(want) ? want : 0;
-    // default: the widest group of at most 128 columns (a full-rate MMA without wasting rows on a larger union)
-    for (int g = 8; g >= 1; g >>= 1)
-        if (fits(g) && g * D.expert_size <= 128) return g;
-    return fits(1) ? 1 : 0;
+    // default: the widest group one MMA can hold.  The kernel is bound by the rate at which token rows can be gathered
+    // (about the same time per 128 x 64 tile of x whatever the width of the MMA that consumes it), so the more columns
+    // a gathered row serves the better, although a wider group is kept by more tokens.
+    for (int g = 32; g >= 1; g >>= 1)
+        if (fits(g)) return g;
+    return 0;
 }
 
 d2d_status d2d_moe_gather_up(const d2d_gather_args &a, cudaStream_t st)
 {
     if (a.T <= 0) return D2D_OK;
-    if (a.T >= (1 << 24) || a.g < 1 || a.g > 8) return D2D_ERR_UNSUPPORTED;
+    if (a.g < 1 || a.g > 32 || a.n_experts > 2048) return D2D_ERR_UNSUPPORTED;
     return a.w_gate ? launch_act<true>(a, st) : launch_act<false>(a, st);
+}
+
+bool d2d_moe_down_masked_supports(const d2d_layer_desc &D)
+{
+    return D.dtype == D2D_BF16 && D.d % 16 == 0 && D.d_ff % 8 == 0 && D.expert_size % 8 == 0 && D.d_ff < 65536 && d2d_gemm_tc_available();
+}
+
+d2d_status d2d_moe_down_masked(const d2d_layer_desc &D, const void *H, const uint32_t *mask, const void *w2, const void *b2, void *y, int T,
+                               int32_t *status, cudaStream_t st, const int32_t *n_sel, long long n_sel_max)
+{
+    if (T <= 0) return D2D_OK;
+    if (!d2d_moe_down_masked_supports(D)) return D2D_ERR_UNSUPPORTED;
+    const int sms = d2d_tc_sm_count();
+    // column tile that wastes the fewest SM rounds (wider preferred on ties: fewer passes over H)
+    int bn = 256;
+    double best = -1.0;
+    for (int cand : {256, 192, 128}) {
+        const long tiles = (long)d2d_cdiv(D.d, cand) * d2d_cdiv(T, BM);
+        const long rounds = (tiles + sms - 1) / sms;
+        const double eff = (double)D.d / ((double)d2d_cdiv(D.d, cand) * cand) * (double)tiles / (double)(rounds * sms);
+        if (eff > best + 1e-9) { best = eff; bn = cand; }
+    }
+    DownParams p = {};
+    p.H = (const __nv_bfloat16 *)H; p.mask = mask; p.b2 = (const __nv_bfloat16 *)b2; p.y = (__nv_bfloat16 *)y; p.status = status;
+    p.T = T; p.d = D.d; p.d_ff = D.d_ff; p.W = (D.n_experts + 31) / 32; p.s = D.expert_size;
+    p.inv_s = (uint32_t)((0x100000000ull + (unsigned long long)D.expert_size - 1) / (unsigned long long)D.expert_size);
+    p.bn = bn;
+    p.n_sel = n_sel; p.n_sel_max = n_sel_max;
+    p.stage_bytes = A_BYTES + bn * 128;
+    const int stages = (192 * 1024) / p.stage_bytes;
+    p.stages = stages > MAX_STAGES ? MAX_STAGES : stages;
+    // W2 of Llama-sized layers does not stay in L2 beside H: walk the tiles in bands of about 32 MB of H rows
+    p.band = 0;
+    if (2.0 * D.d * D.d_ff >= 48e6) {
+        const int band = (int)(32e6 / (2.0 * BM * D.d_ff) + 0.5);
+        p.band = band < 16 ? 16 : band;
+    }
+    const size_t smem = (size_t)p.stages * p.stage_bytes + 1024;
+    CUtensorMap tw2;
+    if (!d2d_tc_make_map(&tw2, w2, D.d, D.d_ff, bn)) return D2D_ERR_CUDA;
+    static bool attr_set[64] = {};
+    if (!ensure_attr((const void *)moe_down_masked_kernel, attr_set)) return D2D_ERR_CUDA;
+    const int tiles = d2d_cdiv(D.d, bn) * d2d_cdiv(T, BM);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(tiles < sms ? tiles : sms, 1, 1);
+    cfg.blockDim = dim3(NTHREADS, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = d2d_tc_pdl_enabled() ? 1 : 0;
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, moe_down_masked_kernel, tw2, p);
+    D2D_LAUNCHED(1);
+    return err == cudaSuccess && cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
 }

@@ -10,7 +10,8 @@ struct d2d_gather_args {
     const void *w_gate;      // [d_ff, d] bf16 or NULL
     const void *b1;          // [d_ff] bf16 or NULL
     const uint32_t *mask;    // [T, ceil(E/32)] selection mask
-    void *H;                 // [T, d_ff] bf16, every element is written (kept experts: activations, others: zeros)
+    void *H;                 // [T, d_ff] bf16; only the cells of kept (token, group) pairs are written (inside such a cell,
+                             // the neurons of experts the token did not keep are zero); feed it to d2d_moe_down_masked
     int T, d, d_ff, n_experts;
     int s;                   // expert size
     int g;                   // experts per group (from d2d_gather_group_for)
@@ -19,7 +20,8 @@ struct d2d_gather_args {
     int *ctr;                // n_experts / g + 1 device ints, zero before the first launch; the kernel leaves them at zero
     // Density-adaptive dispatch without a host synchronisation: when n_sel is given, the kernel reads the number of
     // selected pairs of this batch from it and returns at once if it exceeds n_sel_max (the caller launches the
-    // masked dense up projection with the complementary rule).  NULL = always run.
+    // masked dense up projection with the complementary rule; LLONG_MAX = always run).  The kernel also sizes its
+    // work distribution from that density.  NULL = always run, distribution sized for dense selections.
     const int32_t *n_sel;
     long long n_sel_max;
 };
@@ -29,3 +31,11 @@ struct d2d_gather_args {
 int d2d_gather_group_for(const d2d_layer_desc &D, int want);
 
 d2d_status d2d_moe_gather_up(const d2d_gather_args &a, cudaStream_t st);
+
+// Down projection that applies the selection while it stages H: y = (G * H) W2^T + b2, reading only the cells of H
+// whose (token, expert) pair is kept.  Follows d2d_moe_gather_up (which writes only those cells) and is equally valid
+// after the masked dense up projection.  w2: [d, d_ff] bf16 as given; requires d % 16 == 0 and s % 8 == 0.
+bool d2d_moe_down_masked_supports(const d2d_layer_desc &D);
+// n_sel / n_sel_max: as in d2d_gather_args (the kernel returns at once when *n_sel > n_sel_max; NULL = always run).
+d2d_status d2d_moe_down_masked(const d2d_layer_desc &D, const void *H, const uint32_t *mask, const void *w2, const void *b2, void *y, int T,
+                               int32_t *status, cudaStream_t st, const int32_t *n_sel = nullptr, long long n_sel_max = 0);

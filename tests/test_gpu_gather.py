@@ -77,22 +77,31 @@ def test_gathered_up_projection_equals_masked_dense_and_oracle(api, name, T, g, 
     for i, p in enumerate(ps):
         G = _structured_mask(cfg, T, p, seed=17 * i + T) if 0.0 < p < 1.0 else np.full((T, cfg.E), int(p), np.uint8)
         r = _routing(api, G, cfg.E)
-        H_dense = layer.expert_up_fwd(xd, r)
-        H = torch.full((T, cfg.d_ff), float("nan"), dtype=torch.bfloat16, device="cuda")     # every element must be written
+        H_dense = layer.expert_up_fwd(xd, r).view(torch.int16).cpu().numpy().reshape(T, cfg.E, cfg.s)
+        gg = layer.get_expert_path()[1]
+        kept_group = np.repeat(G.reshape(T, cfg.E // gg, gg).max(-1), gg, axis=1).astype(bool)     # [T, E]: some expert of the group kept
+        POISON = 0x7fc1                                        # a NaN pattern: cells the kernel must not touch, and must never read
+        H = torch.full((T, cfg.d_ff), POISON, dtype=torch.int16, device="cuda").view(torch.bfloat16)
+        y_ref = oracle.moe_ffn(x, w["w1"], w["b1"], w["w_gate"], w["w2"], w["b2"], act, G)
         for rep in range(2):                                   # twice: the sub-chunk counters reset themselves
             layer.expert_up_gather_fwd(xd, r, H=H)
             torch.cuda.synchronize()
             assert r.status == 0
-            Hn = H.float().cpu().numpy().reshape(T, cfg.E, cfg.s)
-            assert np.isfinite(Hn).all()
-            assert not Hn[G == 0].any()                        # zero exactly where the token did not keep the expert
-            # the same products accumulated in the same order on the same unit
-            assert torch.equal(H, H_dense), (name, p, float((H.float() - H_dense.float()).abs().max()))
-            H.fill_(float("nan"))
-        layer.expert_up_gather_fwd(xd, r, H=H)
-        y = layer.expert_down_fwd(H).float().cpu().numpy()
-        y_ref = oracle.moe_ffn(x, w["w1"], w["b1"], w["w_gate"], w["w2"], w["b2"], act, G)
-        assert _rel_err(y, y_ref) <= TOL_Y, (name, p, _rel_err(y, y_ref))
+            Hn = H.view(torch.int16).cpu().numpy().reshape(T, cfg.E, cfg.s)
+            # cells of kept (token, group) pairs: bit for bit what the masked dense kernel writes (the same products
+            # accumulated in the same order on the same unit), zero at experts of the group the token did not keep
+            assert np.array_equal(Hn[kept_group], H_dense[kept_group]), (name, p)
+            assert not Hn[kept_group & (G == 0)].any()
+            # every other cell is left alone ...
+            assert (Hn[~kept_group] == np.int16(POISON)).all()
+            # ... and the down projection that follows never reads it
+            y = layer.expert_down_masked_fwd(H, r).float().cpu().numpy()
+            assert np.isfinite(y).all()
+            assert _rel_err(y, y_ref) <= TOL_Y, (name, p, _rel_err(y, y_ref))
+            H.view(torch.int16).fill_(POISON)
+        # the same down projection after the masked dense kernel
+        y = layer.expert_down_masked_fwd(layer.expert_up_fwd(xd, r), r).float().cpu().numpy()
+        assert _rel_err(y, y_ref) <= TOL_Y
     layer.close()
 
 
@@ -139,12 +148,50 @@ def test_layer_fwd_is_the_same_on_both_sides_of_the_dispatch(api, name, T, tau):
     layer.close()
 
 
+@pytest.mark.parametrize("name,tau", [("vit", 0.6), ("llama", 0.6)])
+def test_device_side_choice_at_full_size(api, name, tau):
+    """Batches large enough for the automatic choice: the crossover is moved to either extreme so that the decision
+    taken on the device goes each way (both kernel pairs are enqueued, one returns at once); y is checked against
+    the oracle on sampled tokens, at least one from every 128-token row tile."""
+    cfg = wl.CONFIGS[name]
+    w, x = wl.make_weights(cfg), wl.make_tokens(cfg)
+    layer = api.Layer.from_config(cfg, w)
+    xd = api.to_device(x, cfg.dtype)
+    act = oracle.ACT_BY_NAME[cfg.act]
+    T = cfg.T
+    rng = np.random.default_rng(11)
+    tiles = np.arange(0, T, 128)
+    sample = np.unique(np.concatenate([tiles + rng.integers(0, 128, tiles.shape), [0, T - 1]]))
+    sample = sample[sample < T]
+    if name == "llama":
+        sample = sample[:: 2]                                  # the oracle needs about 0.1 s per Llama-sized token
+    ref = None
+    for rho_max in (0.0, 1.0):
+        layer.set_expert_path("auto", rho_max=rho_max)
+        r = layer.new_routing(T)
+        y = torch.full((T, cfg.d), float("nan"), dtype=torch.bfloat16, device="cuda")
+        for rep in range(2):
+            layer.layer_fwd(xd, tau, y=y, routing=r)
+            torch.cuda.synchronize()
+            assert r.status == 0
+        G = oracle.unpack_mask(r.mask_u32(), cfg.E)
+        assert r.n_sel == int(G.sum())
+        if ref is None:
+            ref = (G, oracle.moe_ffn(x[sample], w["w1"], w["b1"], w["w_gate"], w["w2"], w["b2"], act, G[sample]))
+        assert np.array_equal(G, ref[0])
+        yg = y.float().cpu().numpy()
+        assert np.isfinite(yg).all()
+        assert _rel_err(yg[sample], ref[1]) <= TOL_Y, (rho_max, _rel_err(yg[sample], ref[1]))
+        assert _per_token_err(yg[sample], ref[1]) <= 4 * TOL_Y
+    layer.close()
+
+
 def test_expert_path_settings_and_errors(api):
     cfg = wl.with_tokens(wl.CONFIGS["bert"], 64)
     layer = api.Layer.from_config(cfg, wl.make_weights(cfg))
-    assert layer.get_expert_path()[:2] == ("auto", 4)
-    layer.set_expert_path("gather", group=8, rho_max=0.25)
-    assert layer.get_expert_path() == ("gather", 8, 0.25)
+    assert layer.get_expert_path()[:2] == ("auto", 8)
+    layer.set_expert_path("gather", group=4, rho_max=0.25)
+    assert layer.get_expert_path() == ("gather", 4, 0.25)
     for bad_group in (3, 16, 5):                               # not a divisor of 32 and E, or wider than one MMA
         with pytest.raises(api.D2DError) as e:
             layer.set_expert_path("auto", group=bad_group)
