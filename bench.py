@@ -1,11 +1,15 @@
 #!/usr/bin/env python
 """Benchmark of the dynamic-k MoE layer (D2DMoE inference hot path) on B200.
 
-One step = one pass of the whole hot path (router_fwd -> select_dynk -> moe_ffn_fwd, the
-single C-ABI call d2d_layer_fwd) over one batch of synthetic tokens.  Default workload: the
-BERT-base-shaped bf16 layer (d=768, d_ff=3072, 128 experts x 24 neurons, 32 x 128 tokens).
+One step = one pass of the whole hot path (router_fwd -> select_dynk -> moe_ffn_fwd, the single
+C-ABI call d2d_layer_fwd) over one batch of synthetic tokens.  Default workload: the largest
+single-GPU configuration, the Llama-style gated layer (d=4096, d_ff=11008, 344 experts x 32
+neurons, 8192 tokens) at tau = 0.4; the other configurations are timed in the same run and
+reported in `per_config` of the same JSON line.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--tau 0.3] [--workload bert] [--sweep]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload llama] [--tau 0.4]
+                    [--tokens T] [--bernoulli p] [--path auto|dense|gather] [--experts-per-group g]
+                    [--sweep] [--no-per-config] [--no-cpu-baseline] [--no-graph] [--group N]
     python bench.py --impl reference ...      # times the CPU oracle on the host cores
 
 Prints ONE JSON line on stdout (rank 0).  Multi-GPU: launched by torch.distributed.run, one
@@ -29,12 +33,23 @@ METRIC = "dynamic-k MoE layer tokens/s"
 UNIT = "tokens/s"
 L2_FLUSH_BYTES = 256 << 20
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
-# capture summarised under profiles/ (None until a capture of that kernel/workload exists).
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from ncu captures of that
+# kernel on that workload (None until a capture exists); keyed by (workload, tokens, kernel).
 NCU_TRAFFIC_BYTES = {
-    ("bert", 4096): 11.20e6,        # up projection: profiles/bert_gemm_up_down_full.md
-    ("gpt2_ffn", 1, 0.2): 9.868e6,  # decode expert kernel: profiles/gpt2_decode_T1_small_kernels_full.md
+    ("llama", 8192, "dense_up"): None,
+    ("llama", 8192, "gather_up"): None,
 }
+
+# (workload, tokens or None = the workload's own, tau or None, Bernoulli p or None) timed for `per_config`
+PER_CONFIG = [
+    ("tiny", None, 0.5, None),
+    ("bert", None, 0.3, None), ("bert", None, 0.7, None),
+    ("vit", None, 0.3, None), ("vit", None, 0.6, None),
+    ("gpt2_ffn", 1, 0.5, None), ("gpt2_ffn", 8, 0.5, None), ("gpt2_ffn", 64, 0.5, None),
+    ("gpt2_attn", 1, 0.5, None), ("gpt2_attn", 64, 0.5, None),
+    ("llama", None, 0.6, None),
+    ("paper", None, None, 0.1), ("paper", None, None, 0.3), ("paper", None, None, 0.5),
+]
 
 
 def parse_args():
@@ -43,16 +58,26 @@ def parse_args():
     p.add_argument("--steps", type=int, default=50)
     p.add_argument("--warmup", type=int, default=5)
     p.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    p.add_argument("--workload", default="bert")
+    p.add_argument("--workload", default="llama")
     p.add_argument("--tokens", type=int, default=0, help="override the workload's token count")
-    p.add_argument("--tau", type=float, default=0.3)
+    p.add_argument("--tau", type=float, default=None, help="threshold of the dynamic-k rule (default 0.4)")
+    p.add_argument("--bernoulli", type=float, default=None,
+                   help="override the gating decisions with Bernoulli(p) samples (the latency protocol of Sec. 4.4): "
+                        "the timed step is then the expert step d2d_moe_ffn_fwd on that mask")
+    p.add_argument("--path", default="auto", choices=["auto", "dense", "gather"],
+                   help="which up projection the tensor-core expert step uses (d2d_layer_set_expert_path)")
+    p.add_argument("--experts-per-group", type=int, default=0, help="group size of the gathered path (0 = default)")
     p.add_argument("--sweep", action="store_true", help="also time the workload's whole tau grid")
+    p.add_argument("--no-per-config", action="store_true", help="skip the other configurations")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--no-graph", action="store_true", help="launch eagerly instead of replaying a captured CUDA graph")
     p.add_argument("--group", type=int, default=0,
                    help="also time N layers of the workload's shape on the shared input as one d2d_group_fwd call "
                         "(the Q, K, V projections of an attention layer) against N separate d2d_layer_fwd calls")
-    return p.parse_args()
+    args = p.parse_args()
+    if args.tau is None:
+        args.tau = 0.4
+    return args
 
 
 def measured_peaks():
@@ -126,17 +151,30 @@ def physical_gpu_index(local_rank: int) -> int:
     return local_rank
 
 
-def flops_algorithmic(cfg, T, n_sel):
-    router = 2.0 * T * (cfg.d * cfg.d_h + cfg.d_h * cfg.E)
-    experts = 2.0 * cfg.n_mat * cfg.d * cfg.s * n_sel
-    return router, experts
+def config_dict(cfg, tau, bernoulli=None):
+    """The workload as both arms name it (the same keys and values in `--impl ours` and `--impl reference`)."""
+    c = {"workload": cfg.name, "tokens": cfg.T, "d": cfg.d, "d_ff": cfg.d_ff, "experts": cfg.E, "expert_size": cfg.s,
+         "d_h": cfg.d_h, "act": cfg.act, "gated": cfg.gated, "tau": tau}
+    if bernoulli is not None:
+        c["tau"] = None
+        c["bernoulli_p"] = bernoulli
+    return c
+
+
+def stats(ts):
+    ts = sorted(ts)
+    return {"mean": sum(ts) / len(ts), "median": ts[len(ts) // 2], "min": ts[0]}
 
 
 # ------------------------------------------------------------------------------------------ CPU oracle arm
 
-def oracle_step_fn(cfg, weights, x_sample, tau):
+def oracle_step_fn(cfg, weights, x_sample, tau, G_sample=None):
     import oracle
     act = oracle.ACT_BY_NAME[cfg.act]
+    if G_sample is not None:
+        def step():
+            return oracle.moe_ffn(x_sample, weights["w1"], weights["b1"], weights["w_gate"], weights["w2"], weights["b2"], act, G_sample)
+        return step
 
     def step():
         return oracle.layer(x_sample, weights, act, tau)
@@ -146,7 +184,7 @@ def oracle_step_fn(cfg, weights, x_sample, tau):
 def time_cpu_oracle(cfg, weights, x, tau, budget_s=12.0):
     """Times the oracle, as it stands, on a bounded token sample sized for roughly budget_s seconds."""
     import oracle
-    probe = min(32, x.shape[0])
+    probe = min(16, x.shape[0])
     t0 = time.perf_counter()
     oracle_step_fn(cfg, weights, x[:probe], tau)()
     per_tok = (time.perf_counter() - t0) / probe
@@ -157,9 +195,17 @@ def time_cpu_oracle(cfg, weights, x, tau, budget_s=12.0):
     for _ in range(passes):
         step()
     dt = time.perf_counter() - t0
-    return {"value": n * passes / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+    threads = max(1, oracle.num_threads())
+    n1 = max(1, min(n, int(3.0 / max(per_tok * threads, 1e-9))))       # about three seconds on one thread
+    oracle.set_num_threads(1)
+    t1 = time.perf_counter()
+    oracle_step_fn(cfg, weights, x[:n1], tau)()
+    dt1 = time.perf_counter() - t1
+    oracle.set_num_threads(threads)
+    return {"value": n * passes / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
             "sample": f"first {n} of {x.shape[0]} tokens of the {cfg.name} workload at tau={tau}, {passes} passes "
-                      f"(router+select+metadata+experts each), {dt:.2f} s"}
+                      f"(router+select+metadata+experts each), {dt:.2f} s",
+            "single_thread_value": n1 / dt1, "single_thread_sample": f"first {n1} tokens, one pass, {dt1:.2f} s"}
 
 
 def run_reference(args):
@@ -173,27 +219,31 @@ def run_reference(args):
         cfg = wl.with_tokens(cfg, args.tokens)
     weights = wl.make_weights(cfg)
     x = wl.make_tokens(cfg)
-    probe = min(16, cfg.T)
+    G = wl.make_bernoulli_mask(cfg, args.bernoulli) if args.bernoulli is not None else None
+    probe = min(8, cfg.T)
     t0 = time.perf_counter()
-    oracle_step_fn(cfg, weights, x[:probe], args.tau)()
+    oracle_step_fn(cfg, weights, x[:probe], args.tau, None if G is None else G[:probe])()
     per_tok = (time.perf_counter() - t0) / probe
     total_steps = args.steps + args.warmup
     n = int(max(1, min(cfg.T, 90.0 / total_steps / max(per_tok, 1e-9))))   # whole run within ~1.5 minutes
-    step = oracle_step_fn(cfg, weights, x[:n], args.tau)
+    step = oracle_step_fn(cfg, weights, x[:n], args.tau, None if G is None else G[:n])
     for _ in range(args.warmup):
         step()
-    t0 = time.perf_counter()
+    times = []
     for _ in range(args.steps):
+        t0 = time.perf_counter()
         step()
-    dt = time.perf_counter() - t0
+        times.append(time.perf_counter() - t0)
+    dt = sum(times)
     value = n * args.steps / dt
-    sample = f"each step = the first {n} of {cfg.T} tokens of the {cfg.name} workload at tau={args.tau}"
+    sample = f"each step = the first {n} of {cfg.T} tokens of the {cfg.name} workload"
+    st = stats([1e3 * t for t in times])
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": cfg.name, "tokens_per_step": n, "d": cfg.d, "d_ff": cfg.d_ff, "experts": cfg.E,
-                   "expert_size": cfg.s, "d_h": cfg.d_h, "act": cfg.act, "tau": args.tau},
+        "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "ms_median": st["median"], "ms_min": st["min"],
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": config_dict(cfg, args.tau, args.bernoulli),
+        "tokens_per_step": n,
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -204,60 +254,40 @@ def run_reference(args):
 
 # ------------------------------------------------------------------------------------------ GPU arm
 
-def run_ours(args):
-    import numpy as np
-    import torch
-    import torch.distributed as dist
-    from paper_2310_04361_b200 import api, workloads as wl
+class Harness:
+    """Timing protocol shared by every measurement of the GPU arm: W untimed warm-up steps, then K steps each
+    bracketed by CUDA events on the launching stream, with an L2 flush (a 256 MiB write) before every step and
+    outside its events; the step is a CUDA-graph replay of the library's own launch sequence unless --no-graph."""
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the dynamic-k MoE layer has no CPU fallback")
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+    def __init__(self, torch, dev, dist, world, no_graph):
+        self.torch, self.dev, self.dist, self.world, self.no_graph = torch, dev, dist, world, no_graph
+        self.flush = torch.empty((L2_FLUSH_BYTES,), dtype=torch.uint8, device=dev)
+        self.stream = torch.cuda.current_stream()
+        self.all_ranks = True        # False for the measurements only rank 0 takes (no collective barrier then)
 
-    cfg = wl.CONFIGS[args.workload]
-    if args.tokens:
-        cfg = wl.with_tokens(cfg, args.tokens)
-    T = cfg.T
-    weights = wl.make_weights(cfg)                      # every rank holds the whole layer
-    x_np = wl.make_tokens(cfg, stream=rank)             # ... and its own batch of tokens
-    layer = api.Layer.from_config(cfg, weights, device=dev)
-    x = api.to_device(x_np, cfg.dtype, dev)
-    y = torch.empty_like(x)
-    routing = layer.new_routing(T)
-    layer.workspace(T)
-    flush = torch.empty((L2_FLUSH_BYTES,), dtype=torch.uint8, device=dev)
-    stream = torch.cuda.current_stream()
+    def barrier(self):
+        if self.world > 1 and self.all_ranks:
+            self.dist.barrier()
+        self.torch.cuda.synchronize()
 
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    def timed_loop(fn, steps, warmup):
-        """Per-step CUDA events on the launching stream; the L2 flush between steps is outside the events."""
+    def timed_loop(self, fn, steps, warmup):
+        torch = self.torch
         for _ in range(warmup):
-            flush.zero_()
+            self.flush.zero_()
             fn()
         evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
-        barrier()
+        self.barrier()
         for a, b in evs:
-            flush.zero_()
-            a.record(stream)
+            self.flush.zero_()
+            a.record(self.stream)
             fn()
-            b.record(stream)
-        barrier()
+            b.record(self.stream)
+        self.barrier()
         return [a.elapsed_time(b) for a, b in evs]       # ms
 
-    def runner(fn):
-        """The step as it is launched in the timed region: a CUDA-graph replay of the library's launch
-        sequence (the layer is launch-latency bound for small batches), or the eager call with --no-graph."""
-        if args.no_graph:
+    def runner(self, fn):
+        torch = self.torch
+        if self.no_graph:
             return fn
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
@@ -271,61 +301,204 @@ def run_ours(args):
             fn()
         return g.replay
 
-    def max_over_ranks(v):
-        if world == 1:
+    def time(self, fn, steps, warmup=3):
+        return stats(self.timed_loop(self.runner(fn), steps, warmup))
+
+    def max_over_ranks(self, v):
+        if self.world == 1:
             return v
-        t = torch.tensor([v], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        t = self.torch.tensor([v], dtype=self.torch.float64, device=self.dev)
+        self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
         return float(t.item())
 
-    def step():
-        layer.layer_fwd(x, args.tau, y=y, routing=routing)
 
-    step()                                   # one eager call: counts the kernels a step launches
-    launches0 = api.launch_count()
+def dense_comparators(h, api, torch, cfg, weights, layer, x, y, steps):
+    """Same-shape dense FFN on the same tensors, same protocol: (1) torch eager F.linear -> act -> F.linear (cuBLASLt
+    GEMMs, a separate activation kernel); (2) this library's own tensor-core GEMMs with every expert kept
+    (bias + activation fused in the up projection's epilogue, no router, no selection); (3) the library's layer call
+    at tau = 0 (router included, every expert kept)."""
+    import numpy as np
+    import oracle
+    dev = h.dev
+    tdt = api.torch_dtype(cfg.dtype)
+    F = torch.nn.functional
+    w1 = torch.from_numpy(weights["w1"]).to(dev, tdt)
+    w2 = torch.from_numpy(weights["w2"]).to(dev, tdt)
+    b1 = None if weights["b1"] is None else torch.from_numpy(weights["b1"]).to(dev, tdt)
+    b2 = None if weights["b2"] is None else torch.from_numpy(weights["b2"]).to(dev, tdt)
+    wg = None if weights["w_gate"] is None else torch.from_numpy(weights["w_gate"]).to(dev, tdt)
+    actf = {"relu": F.relu, "gelu_erf": F.gelu, "gelu_tanh": lambda z: F.gelu(z, approximate="tanh"), "silu": F.silu}[cfg.act]
+
+    def dense():
+        up = F.linear(x, w1, b1)
+        hh = actf(F.linear(x, wg)) * up if wg is not None else actf(up)
+        return F.linear(hh, w2, b2)
+
+    out = {"torch_eager_ms": h.time(dense, steps)["median"]}
+    del w1, w2, wg
+    T = x.shape[0]
+    ones = np.ones((T, cfg.E), dtype=np.uint8)
+    r_all = api.routing_from_mask(torch.from_numpy(oracle.pack_mask(ones).view(np.int32)).to(dev), cfg.E)
+    path, group, rho_max = layer.get_expert_path()
+    if cfg.dtype == "bf16":
+        layer.set_expert_path("dense")
+    out["library_all_experts_ms"] = h.time(lambda: layer.moe_ffn_fwd(x, r_all, y=y), steps)["median"]
+    r0 = layer.new_routing(T)
+    out["library_layer_tau0_ms"] = h.time(lambda: layer.layer_fwd(x, 0.0, y=y, routing=r0), steps)["median"]
+    if cfg.dtype == "bf16":
+        layer.set_expert_path(path, group, rho_max)
+    return out
+
+
+def k_histogram(torch, routing, T, E):
+    k = routing.k[:T].float()
+    used = int((routing.counts > 0).sum().item()) if routing.lists else None
+    return {"min": int(k.min().item()), "median": float(k.median().item()),
+            "p99": float(torch.quantile(k, 0.99).item()), "max": int(k.max().item()), "experts_used": used}
+
+
+def measure_config(h, api, torch, wl, name, tokens, tau, bern, steps, peaks, path="auto", group=0, full=False, rank=0):
+    """One configuration: layer time, kept fraction, k histogram, dense comparators, roofline fraction of the expert step."""
+    import numpy as np
+    import oracle
+    cfg = wl.CONFIGS[name]
+    if tokens:
+        cfg = wl.with_tokens(cfg, tokens)
+    T = cfg.T
+    dev = h.dev
+    weights = wl.make_weights(cfg)
+    x_np = wl.make_tokens(cfg, stream=rank)
+    layer = api.Layer.from_config(cfg, weights, device=dev)
+    if cfg.dtype == "bf16" and (path != "auto" or group):
+        layer.set_expert_path(path, group)
+    x = api.to_device(x_np, cfg.dtype, dev)
+    y = torch.empty_like(x)
+    routing = layer.new_routing(T)
+    layer.workspace(T)
+    if bern is not None:
+        G = wl.make_bernoulli_mask(cfg, bern, stream=rank)
+        routing = api.routing_from_mask(torch.from_numpy(oracle.pack_mask(G).view(np.int32)).to(dev), cfg.E)
+
+        def step():
+            layer.moe_ffn_fwd(x, routing, y=y)
+    else:
+        def step():
+            layer.layer_fwd(x, tau, y=y, routing=routing)
     step()
-    launches_per_step = api.launch_count() - launches0
-    run_step = runner(step)
+    l0 = api.launch_count()
+    step()
+    launches = api.launch_count() - l0
+    res = {"cfg": cfg, "layer": layer, "weights": weights, "x": x, "x_np": x_np, "y": y, "routing": routing, "step": step,
+           "launches": launches}
+    if full:
+        return res
+    t = h.time(step, steps)
+    torch.cuda.synchronize()
+    assert routing.status == 0
+    n_sel = routing.n_sel
+    rho = n_sel / (T * cfg.E)
+    dense = dense_comparators(h, api, torch, cfg, weights, layer, x, y, max(10, steps // 2))
+    t_ffn = h.time(lambda: layer.moe_ffn_fwd(x, routing, y=y), max(10, steps // 2))["median"]
+    f_experts = 2.0 * cfg.n_mat * cfg.d * cfg.s * n_sel
+    elem = 2 if cfg.dtype == "bf16" else 4
+    n_used = int((routing.counts > 0).sum().item())
+    if T <= 64 or cfg.dtype == "f32":
+        touched = n_used * (cfg.n_mat * cfg.s * cfg.d + cfg.s) * elem + 2 * T * cfg.d * elem + cfg.d * elem
+        roof = {"bound": "hbm", "frac": touched / (t_ffn * 1e-3) / 1e9 / peaks["hbm_gbs"], "of": "touched expert bytes / expert-step time / HBM peak"}
+    else:
+        roof = {"bound": "tensor", "frac": f_experts / (t_ffn * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                "of": "algorithmic expert FLOP / expert-step time / bf16 peak"}
+    out = {"workload": cfg.name, "tokens": T, "tau": tau, "bernoulli_p": bern, "rho": rho, "pruned_flop_fraction": 1 - rho,
+           "k": k_histogram(torch, routing, T, cfg.E),
+           "step": "d2d_moe_ffn_fwd on the override mask" if bern is not None else "d2d_layer_fwd",
+           "ms_median": t["median"], "ms_min": t["min"], "tokens_per_s": T / (t["median"] * 1e-3),
+           "expert_step_ms": t_ffn, "launches_per_step": launches, "expert_path": layer.get_expert_path()[0] if cfg.dtype == "bf16" else "fp32",
+           "dense": dense, "speedup_vs_torch_dense": dense["torch_eager_ms"] / t["median"],
+           "speedup_vs_library_dense": dense["library_all_experts_ms"] / t["median"], "roofline": roof}
+    layer.close()
+    return out
+
+
+def run_ours(args):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    import oracle
+    from paper_2310_04361_b200 import api, workloads as wl
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the dynamic-k MoE layer has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    h = Harness(torch, dev, dist, world, args.no_graph)
+    peaks = measured_peaks()
+
+    m = measure_config(h, api, torch, wl, args.workload, args.tokens, args.tau, args.bernoulli, args.steps, peaks,
+                       path=args.path, group=args.experts_per_group, full=True, rank=rank)
+    cfg, layer, weights, x, x_np, y, routing, step = (m[k] for k in ("cfg", "layer", "weights", "x", "x_np", "y", "routing", "step"))
+    T = cfg.T
+    launches_per_step = m["launches"]
+    run_step = h.runner(step)
     sampler = ClockSampler(physical_gpu_index(local_rank))
     sampler.start()
-    times = timed_loop(run_step, args.steps, args.warmup)
+    times = h.timed_loop(run_step, args.steps, args.warmup)
     clocks = sampler.stop()
-    total_ms = max_over_ranks(sum(times))
+    total_ms = h.max_over_ranks(sum(times))
     value = world * T * args.steps / (total_ms * 1e-3)
     torch.cuda.synchronize()
-    n_sel = routing.n_sel
     assert routing.status == 0
+    n_sel = routing.n_sel
+    rho = n_sel / (T * cfg.E)
+    st_layer = stats(times)
 
     # ---- end to end through the host-buffer entry point (pinned host x -> device -> layer -> host y)
-    xh = x.cpu().pin_memory()
-    yh = torch.empty_like(xh).pin_memory()
-    hws = layer.host_workspace(T)
+    e2e = None
+    if args.bernoulli is None:
+        xh = x.cpu().pin_memory()
+        yh = torch.empty_like(xh).pin_memory()
+        hws = layer.host_workspace(T)
 
-    def e2e_step():
-        layer.layer_fwd_host(xh, args.tau, yh, hws)
+        def e2e_step():
+            layer.layer_fwd_host(xh, args.tau, yh, hws)
 
-    for _ in range(max(3, args.warmup)):
-        e2e_step()
-    barrier()
-    t0 = time.perf_counter()
-    for _ in range(args.steps):
-        flush.zero_()
-        e2e_step()
-    torch.cuda.synchronize()
-    e2e_s = max_over_ranks(time.perf_counter() - t0)
-    row_bytes = T * cfg.d * (2 if cfg.dtype == "bf16" else 4)
-    e2e = {"value": world * T * args.steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": row_bytes,
-           "d2h_bytes_per_step": row_bytes, "note": "wall clock over K calls of d2d_layer_fwd_host incl. an L2 flush per step"}
+        for _ in range(max(3, args.warmup)):
+            e2e_step()
+        h.barrier()
+        e2e_times = []
+        for _ in range(args.steps):
+            h.flush.zero_()
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            e2e_step()                                 # synchronises the stream itself
+            e2e_times.append(time.perf_counter() - t0)
+        e2e_s = h.max_over_ranks(sum(e2e_times))
+        row_bytes = T * cfg.d * (2 if cfg.dtype == "bf16" else 4)
+        e2e = {"value": world * T * args.steps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": row_bytes,
+               "d2h_bytes_per_step": row_bytes, "ms_median": 1e3 * sorted(e2e_times)[len(e2e_times) // 2],
+               "note": "wall clock around each d2d_layer_fwd_host call (pinned host x and y; H2D copy, layer, D2H copy and "
+                       "the stream synchronisation inside); the L2 flush before each call is outside the clock"}
+        del hws
 
     line = None
+    h.all_ranks = False                                    # what follows is measured by rank 0 alone
     if rank == 0:
-        # ---- per-stage breakdown (same flush protocol), used for the roofline of the dominant kernel
-        R = torch.empty((T, cfg.E), dtype=torch.float32, device=dev)
-        t_router = statistics.mean(timed_loop(runner(lambda: layer.router_fwd(x, R=R)), args.steps, 3))
-        t_select = statistics.mean(timed_loop(runner(lambda: api.select_dynk(R, args.tau, routing=routing)), args.steps, 3))
-        t_ffn = statistics.mean(timed_loop(runner(lambda: layer.moe_ffn_fwd(x, routing, y=y)), args.steps, 3))
-        peaks = measured_peaks()
-        f_router, f_experts = flops_algorithmic(cfg, T, n_sel)
+        sub = max(10, args.steps // 2)
+        # ---- per-stage breakdown (same protocol)
+        stages = {"layer_fwd": st_layer["median"]}
+        if args.bernoulli is None:
+            R = torch.empty((T, cfg.E), dtype=torch.float32, device=dev)
+            stages["router_fwd"] = h.time(lambda: layer.router_fwd(x, R=R), sub)["median"]
+            r_tmp = layer.new_routing(T)
+            stages["select_dynk"] = h.time(lambda: api.select_dynk(R, args.tau, routing=r_tmp), sub)["median"]
+            del R, r_tmp
+        t_ffn = h.time(lambda: layer.moe_ffn_fwd(x, routing, y=y), sub)["median"]
+        stages["moe_ffn_fwd"] = t_ffn
+        f_experts = 2.0 * cfg.n_mat * cfg.d * cfg.s * n_sel
         elem = 2 if cfg.dtype == "bf16" else 4
         n_used = int((routing.counts > 0).sum().item())
         if T <= 64 or cfg.dtype == "f32":
@@ -333,58 +506,62 @@ def run_ours(args):
             touched = n_used * (cfg.n_mat * cfg.s * cfg.d + cfg.s) * elem + 2 * T * cfg.d * elem + cfg.d * elem
             achieved = touched / (t_ffn * 1e-3) / 1e9
             roofline = {"bound": "hbm", "kernel": "moe_ffn_fwd (small_ffn_kernel)" if T <= 4 else "moe_ffn_fwd", "achieved": achieved,
-                        "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"],
-                        "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, T, args.tau)),
+                        "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None,
                         "peak_source": f"{peaks['source']} HBM copy", "algorithmic_bytes_per_launch": touched,
                         "experts_touched": n_used, "kernel_ms": t_ffn}
         else:
-            # dominant kernel = the expert up projection (one launch of gemm_tc_kernel with the masked
-            # activation epilogue); its algorithmic work is the up half of the kept pairs' FLOP
+            # dominant kernel = the expert up projection; which of its two forms the step ran is the rule the kernels
+            # themselves apply (n_sel against the layer's crossover); each is also timed on its own
+            path, group, rho_max = layer.get_expert_path()
+            up_flop = 2.0 * T * cfg.d * cfg.d_ff * (2 if cfg.gated else 1)
+            gathered = path == "gather" or (path == "auto" and group > 0 and up_flop >= 1e11 and n_sel <= rho_max * T * cfg.E)
             H = torch.empty((T, cfg.d_ff), dtype=torch.bfloat16, device=dev)
-            t_up = statistics.mean(timed_loop(runner(lambda: layer.expert_up_fwd(x, routing, H=H)), args.steps, 3))
-            t_down = statistics.mean(timed_loop(runner(lambda: layer.expert_down_fwd(H, y=y)), args.steps, 3))
+            t_up_dense = h.time(lambda: layer.expert_up_fwd(x, routing, H=H), sub)["median"]
+            t_up_gather = h.time(lambda: layer.expert_up_gather_fwd(x, routing, H=H), sub)["median"] if group > 0 else None
+            layer.expert_up_fwd(x, routing, H=H)
+            t_down = h.time(lambda: layer.expert_down_fwd(H, y=y), sub)["median"]
+            t_down_masked = h.time(lambda: layer.expert_down_masked_fwd(H, routing, y=y), sub)["median"] if group > 0 else None
+            t_up = t_up_gather if gathered else t_up_dense
             f_up = 2.0 * (cfg.n_mat - 1) * cfg.d * cfg.s * n_sel
             f_up_exec = 2.0 * (cfg.n_mat - 1) * T * cfg.d * cfg.d_ff
+            if gathered:
+                gmask = oracle.unpack_mask(routing.mask_u32(), cfg.E).reshape(T, cfg.E // group, group).max(-1)
+                f_up_exec = 2.0 * (cfg.n_mat - 1) * cfg.d * cfg.s * group * float(gmask.sum())
             achieved = f_up / (t_up * 1e-3) / 1e12
-            roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel<UP_MASKED> (d2d_expert_up_fwd)", "achieved": achieved,
-                        "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
-                        "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, T)),
+            kname = "gather_up" if gathered else "dense_up"
+            roofline = {"bound": "tensor",
+                        "kernel": ("moe_gather_up_kernel (d2d_expert_up_gather_fwd)" if gathered else "gemm_tc_kernel<UP_MASKED> (d2d_expert_up_fwd)"),
+                        "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["bf16_tflops"],
+                        "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, T, kname)),
                         "peak_source": f"{peaks['source']} burst bf16 GEMM", "algorithmic_flops_per_launch": f_up,
                         "executed_flops_per_launch": f_up_exec,
                         "executed_frac": f_up_exec / (t_up * 1e-3) / 1e12 / peaks["bf16_tflops"],
-                        "kernel_ms": t_up, "down_kernel_ms": t_down,
+                        "kernel_ms": t_up, "up_dense_ms": t_up_dense, "up_gather_ms": t_up_gather, "down_dense_ms": t_down,
+                        "down_masked_ms": t_down_masked, "expert_path": path, "experts_per_group": group, "rho_crossover": rho_max,
                         "expert_step_frac": f_experts / (t_ffn * 1e-3) / 1e12 / peaks["bf16_tflops"]}
+            del H
 
-        # ---- dense FFN comparator: torch (cuBLASLt) linear -> act -> linear on the same tensors
-        tdt = api.torch_dtype(cfg.dtype)
-        w1 = torch.from_numpy(weights["w1"]).to(dev, tdt)
-        w2 = torch.from_numpy(weights["w2"]).to(dev, tdt)
-        b1 = None if weights["b1"] is None else torch.from_numpy(weights["b1"]).to(dev, tdt)
-        b2 = None if weights["b2"] is None else torch.from_numpy(weights["b2"]).to(dev, tdt)
-        wg = None if weights["w_gate"] is None else torch.from_numpy(weights["w_gate"]).to(dev, tdt)
-        F = torch.nn.functional
-        actf = {"relu": F.relu, "gelu_erf": F.gelu, "gelu_tanh": lambda z: F.gelu(z, approximate="tanh"), "silu": F.silu}[cfg.act]
-
-        def dense():
-            up = F.linear(x, w1, b1)
-            h = actf(F.linear(x, wg)) * up if wg is not None else actf(up)
-            return F.linear(h, w2, b2)
-
-        t_dense = statistics.mean(timed_loop(runner(dense), args.steps, 3))
-        t_layer = sum(times) / len(times)
+        dense = dense_comparators(h, api, torch, cfg, weights, layer, x, y, sub)
+        t_layer = st_layer["median"]
 
         sweep = None
-        if args.sweep:
+        if args.sweep and args.bernoulli is None:
             sweep = []
             for tau in cfg.taus:
-                ts = timed_loop(runner(lambda tau=tau: layer.layer_fwd(x, tau, y=y, routing=routing)), max(10, args.steps // 2), 3)
+                ts = h.time(lambda tau=tau: layer.layer_fwd(x, tau, y=y, routing=routing), sub)
                 torch.cuda.synchronize()
-                sweep.append({"tau": tau, "rho": routing.n_sel / (T * cfg.E), "ms": statistics.mean(ts),
-                              "speedup_vs_dense": t_dense / statistics.mean(ts)})
+                sweep.append({"tau": tau, "rho": routing.n_sel / (T * cfg.E), "ms_median": ts["median"], "ms_min": ts["min"],
+                              "speedup_vs_torch_dense": dense["torch_eager_ms"] / ts["median"],
+                              "speedup_vs_library_dense": dense["library_all_experts_ms"] / ts["median"]})
+            layer.layer_fwd(x, args.tau, y=y, routing=routing)
+            torch.cuda.synchronize()
 
-        group = None
+        group_res = None
         if args.group > 1:
             from dataclasses import replace
+            tdt = api.torch_dtype(cfg.dtype)
+            F = torch.nn.functional
+            actf = {"relu": F.relu, "gelu_erf": F.gelu, "gelu_tanh": lambda z: F.gelu(z, approximate="tanh"), "silu": F.silu}[cfg.act]
             n = args.group
             gws = [weights] + [wl.make_weights(replace(cfg, seed=cfg.seed + 17 * l)) for l in range(1, n)]
             glayers = [layer] + [api.Layer.from_config(cfg, w, device=dev) for w in gws[1:]]
@@ -417,43 +594,61 @@ def run_ours(args):
             l0 = api.launch_count()
             separate_step()
             s_launches = api.launch_count() - l0
-            t_group = statistics.mean(timed_loop(runner(group_step), args.steps, 3))
-            t_sep = statistics.mean(timed_loop(runner(separate_step), args.steps, 3))
-            t_gdense = None if cfg.gated else statistics.mean(timed_loop(runner(dense_group), args.steps, 3))
+            t_group = h.time(group_step, sub)["median"]
+            t_sep = h.time(separate_step, sub)["median"]
+            t_gdense = None if cfg.gated else h.time(dense_group, sub)["median"]
             torch.cuda.synchronize()
             assert all(r.status == 0 for r in grs)
-            group = {"n_layers": n, "group_fwd_ms": t_group, "separate_layer_fwd_ms": t_sep, "dense_ms": t_gdense,
-                     "launches_group": g_launches, "launches_separate": s_launches,
-                     "speedup_vs_separate": t_sep / t_group, "speedup_vs_dense": None if t_gdense is None else t_gdense / t_group,
-                     "rho": [r.n_sel / (T * cfg.E) for r in grs],
-                     "tokens_per_s": T / (t_group * 1e-3)}
+            group_res = {"n_layers": n, "group_fwd_ms": t_group, "separate_layer_fwd_ms": t_sep, "dense_ms": t_gdense,
+                         "launches_group": g_launches, "launches_separate": s_launches,
+                         "speedup_vs_separate": t_sep / t_group, "speedup_vs_dense": None if t_gdense is None else t_gdense / t_group,
+                         "rho": [r.n_sel / (T * cfg.E) for r in grs], "tokens_per_s": T / (t_group * 1e-3)}
             grp.close()
 
+        khist = k_histogram(torch, routing, T, cfg.E)
         cpu = None
-        if not args.no_cpu_baseline:
+        if not args.no_cpu_baseline and args.bernoulli is None:
             cpu = time_cpu_oracle(cfg, weights, x_np, args.tau)
+        layer.close()
+        del layer, x, y, routing, weights
+        torch.cuda.empty_cache()
+
+        per_config = None
+        if not args.no_per_config:
+            per_config = []
+            for name, tokens, tau, bern in PER_CONFIG:
+                try:
+                    per_config.append(measure_config(h, api, torch, wl, name, tokens, tau, bern, 20, peaks))
+                except Exception as e:      # a configuration that fails must not take the headline down with it
+                    per_config.append({"workload": name, "tokens": tokens, "tau": tau, "bernoulli_p": bern, "error": repr(e)})
+                torch.cuda.empty_cache()
 
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "ms_per_step": total_ms / args.steps, "ms_median": st_layer["median"], "ms_min": st_layer["min"],
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": cfg.dtype, "data": "synthetic",
-            "config": {"workload": cfg.name, "tokens_per_gpu": T, "d": cfg.d, "d_ff": cfg.d_ff, "experts": cfg.E,
-                       "expert_size": cfg.s, "d_h": cfg.d_h, "act": cfg.act, "gated": cfg.gated, "tau": args.tau,
-                       "rho": n_sel / (T * cfg.E), "pruned_flop_fraction": 1 - n_sel / (T * cfg.E),
-                       "l2": f"flushed between steps by writing a {L2_FLUSH_BYTES >> 20} MiB buffer (outside the events)",
-                       "launch": "eager" if args.no_graph else "CUDA graph replay of the library's launch sequence",
-                       "parallelism": f"token-sharded replicas x{world}, no collective"},
+            "config": config_dict(cfg, args.tau, args.bernoulli),
+            "run": {"tokens_per_gpu": T, "rho": rho, "pruned_flop_fraction": 1 - rho, "k": khist,
+                    "step": "d2d_moe_ffn_fwd on the override mask" if args.bernoulli is not None else "d2d_layer_fwd",
+                    "l2": f"flushed between steps by writing a {L2_FLUSH_BYTES >> 20} MiB buffer (outside the events)",
+                    "launch": "eager" if args.no_graph else "CUDA graph replay of the library's launch sequence",
+                    "parallelism": f"token-sharded replicas x{world}, no collective"},
             "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
             "roofline": roofline, "cpu_baseline": cpu, "clocks": clocks,
-            "stages_ms": {"router_fwd": t_router, "select_dynk": t_select, "moe_ffn_fwd": t_ffn, "layer_fwd": t_layer},
-            "dense_ffn": {"ms": t_dense, "impl": "torch F.linear/act/F.linear (cuBLASLt)", "speedup_of_layer": t_dense / t_layer,
-                          "speedup_of_moe_ffn_only": t_dense / t_ffn},
+            "stages_ms": stages,
+            "dense_ffn": {**dense, "speedup": dense["torch_eager_ms"] / t_layer,
+                          "speedup_is": "torch eager dense FFN (cuBLASLt GEMMs + activation kernel) median / layer median",
+                          "speedup_vs_library_dense": dense["library_all_experts_ms"] / t_layer,
+                          "speedup_of_expert_step_only": dense["torch_eager_ms"] / t_ffn},
             "paper_context": "paper reports ~3x over a dense MLP on an A100 at 99% accuracy (Sec. 4.4); another machine, not the target",
         }
+        if per_config is not None:
+            line["per_config"] = per_config
         if sweep is not None:
             line["tau_sweep"] = sweep
-        if group is not None:
-            line["group"] = group
+        if group_res is not None:
+            line["group"] = group_res
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.barrier()

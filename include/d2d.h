@@ -30,6 +30,19 @@
  *   - T = 0 is a valid no-op.  There is no CPU fallback: without a CUDA device
  *     every compute call returns D2D_ERR_CUDA.
  *   - A handle is not thread-safe; distinct handles may be used concurrently.
+ *
+ * Environment variables (tuning aids, read once per process; results never
+ * depend on them)
+ *   D2D_DECODE_MAX_TOKENS=n  0..8, default 4: bf16 batches of up to n tokens take
+ *                            the decode kernels (each kept expert's weights read
+ *                            once by CUDA cores), larger ones the tensor-core path.
+ *   D2D_HOST_CHUNKS=n        1..4: number of pipelined chunks d2d_layer_fwd_host
+ *                            cuts a batch into (default: one per 4096 tokens).
+ *   D2D_GEMM_BAND=n          row tiles per band of the tile walk of the dense
+ *                            kernels when the weight operand exceeds L2 (default:
+ *                            about 32 MB of activation rows), 0 = row-major walk.
+ *   D2D_GEMM_PDL=0           launch every kernel fully serialised (no programmatic
+ *                            dependent launch).
  */
 #ifndef D2D_H_
 #define D2D_H_
@@ -197,8 +210,8 @@ D2D_API d2d_status d2d_router_fwd(const d2d_layer *layer, const void *x, int32_t
 D2D_API d2d_status d2d_select_dynk(const float *R, int32_t T, int32_t E, float tau, d2d_routing *out,
                            void *ws, size_t ws_bytes, void *stream);
 
-/* Static top-k selection (the regression router "is still compatible with"
- * top-k, Sec. 3.3): keeps the kk largest scores of each token, equal scores in
+/* Static top-k selection (Sec. 3.3 notes that a router trained by regression
+ * on the experts' output norms can also drive a fixed top-k rule): keeps the kk largest scores of each token, equal scores in
  * order of the lower expert index, then builds the same metadata. */
 D2D_API d2d_status d2d_select_topk(const float *R, int32_t T, int32_t E, int32_t kk, d2d_routing *out,
                            void *ws, size_t ws_bytes, void *stream);

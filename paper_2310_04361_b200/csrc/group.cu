@@ -1,6 +1,6 @@
 // Layer groups: several dynamic-k layers of one shape that read the same token rows, run as one launch sequence.
 // In a converted Transformer block the Q, K and V projections of the attention layer are such a group (Sec. 3.5: every
-// projection matrix becomes its own MoE layer, "four MoE layers in the MHA layer"); the output projection and the FFN
+// projection matrix becomes its own MoE layer, four of them per attention layer); the output projection and the FFN
 // read other tensors and stay ordinary d2d_layer_fwd calls.
 //
 //   T <= decode limit   one decode router launch (+ selection + metadata) and one expert launch for all layers

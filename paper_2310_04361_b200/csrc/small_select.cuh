@@ -1,7 +1,7 @@
 // Selection for a small batch (T <= 64) done by ONE CTA: row max, threshold, mask words, k, per-expert counts,
 // offsets, token lists and the token-major dual.  Shared by the stand-alone selection kernel and by the
 // small-batch router kernel, whose last CTA selects right after it has written the scores (one launch less
-// on the decode path).  Dynamic-k rule: Sec. 3.3, Eq. 6 (keep expert i of token t when R[t,i] >= tau * max_j R[t,j]).
+// on the decode path).  Dynamic-k rule: Sec. 3.4, Eq. 4 (keep expert i of token t when R[t,i] >= tau * max_j R[t,j]).
 #pragma once
 
 #include "d2d_common.cuh"

@@ -51,6 +51,36 @@ def _rel_err(got, ref):
     return float(np.abs(got - ref).max() / max(np.abs(ref).max(), 1e-30))
 
 
+def _per_token_err(got, ref):
+    """max over tokens of max_j |got - ref| / max_j |ref|: every token normalised by its own magnitude (with lognormal
+    token scales the global maximum is set by the few largest tokens)."""
+    ref = np.asarray(ref, dtype=np.float64)
+    got = np.asarray(got, dtype=np.float64)
+    return float((np.abs(got - ref).max(1) / np.maximum(np.abs(ref).max(1), 1e-30)).max())
+
+
+# per-token bound: a token's own maximum can be a few times smaller than the largest entry the tolerance refers to
+PER_TOKEN_FACTOR = 4
+
+
+def _poison(t):
+    """NaN-fill a tensor that a checked call must overwrite completely."""
+    if t.dtype in (torch.float32, torch.bfloat16):
+        t.fill_(float("nan"))
+    else:
+        t.view(torch.uint8).fill_(0xFF)
+    return t
+
+
+def _tile_sample(T, rng, extra=()):
+    """At least one token from EVERY 128-token row tile (a defect confined to one tile cannot hide), plus the first
+    and last row of the first and last tiles, plus `extra`."""
+    starts = np.arange(0, T, 128)
+    pick = starts + rng.integers(0, 128, starts.shape)
+    s = np.concatenate([pick, [0, min(127, T - 1), (T - 1) // 128 * 128, T - 1], np.asarray(extra, dtype=np.int64)])
+    return np.unique(s[s < T])
+
+
 def _check_routing(r, G, dual=True):
     meta = oracle.metadata(G)
     T, E = G.shape
@@ -255,7 +285,8 @@ def test_other_activations_and_odd_expert_size(api, act):
 LAYER_CASES = [("tiny", None, 0.5), ("bert", 1000, 0.3), ("vit", 900, 0.3), ("gpt2_ffn", 8, 0.2), ("llama", 64, 0.4),
                ("gpt2_ffn", 1, 0.2), ("gpt2_ffn", 4, 0.5), ("gpt2_ffn", 5, 0.2), ("gpt2_ffn", 9, 0.2), ("gpt2_ffn", 16, 0.5),
                ("gpt2_attn", 3, 0.2), ("gpt2_attn", 100, 0.2),
-               ("gpt2_attn", 128, 0.5), ("bert", 129, 0.3), ("llama", 300, 0.4)]
+               ("gpt2_attn", 128, 0.5), ("bert", 129, 0.3), ("llama", 300, 0.4),
+               ("gpt2_ffn", 64, 0.5), ("gpt2_attn", 1, 0.2), ("gpt2_attn", 8, 0.5)]
 
 
 @pytest.mark.parametrize("name,T,tau", LAYER_CASES)
@@ -263,8 +294,10 @@ def test_layer_fwd_end_to_end(api, name, T, tau):
     cfg, w, x, layer = _setup(api, name, T)
     ref = oracle.layer(x, w, oracle.ACT_BY_NAME[cfg.act], tau)
     Tn = x.shape[0]
-    R_out = torch.empty((Tn, cfg.E), dtype=torch.float32, device="cuda")
-    y, r = layer.layer_fwd(api.to_device(x, cfg.dtype), tau, R_out=R_out)
+    R_out = _poison(torch.empty((Tn, cfg.E), dtype=torch.float32, device="cuda"))
+    y = _poison(torch.empty((Tn, cfg.d), dtype=api.torch_dtype(cfg.dtype), device="cuda"))
+    _poison(layer.workspace(Tn))                           # nothing the call reads may be left over from an earlier call
+    y, r = layer.layer_fwd(api.to_device(x, cfg.dtype), tau, y=y, R_out=R_out)
     torch.cuda.synchronize()
     assert r.status == 0
     R = R_out.cpu().numpy()
@@ -280,9 +313,17 @@ def test_layer_fwd_end_to_end(api, name, T, tau):
     near = np.abs(ref["R"] - np.float32(tau) * m) <= 4 * eps * m
     assert (~diff | near).all()
     same = ~diff.any(1)
-    assert diff.mean() < 0.01 and same.mean() > 0.3
+    # measured: at most 0.2 % of the (token, expert) decisions differ and at least 70 % of the tokens have the
+    # all-oracle mask in every case of this list (bf16 scores carry 1e-3 of noise, E up to 344 decisions per token)
+    print(f"layer_fwd {name} T={Tn} tau={tau}: pairs that differ {diff.mean():.2e}, tokens with the oracle's mask {same.mean():.3f}")
+    assert diff.mean() < 0.005 and same.mean() >= 0.5
     yg = y.float().cpu().numpy()
+    assert np.isfinite(yg).all()
     assert _rel_err(yg[same], ref["y"][same]) <= TOL_Y[cfg.dtype]
+    # every token, against the oracle's expert step on the mask the library itself selected
+    y_self = oracle.moe_ffn(x, w["w1"], w["b1"], w["w_gate"], w["w2"], w["b2"], oracle.ACT_BY_NAME[cfg.act], G_gpu)
+    assert _rel_err(yg, y_self) <= TOL_Y[cfg.dtype]
+    assert _per_token_err(yg, y_self) <= PER_TOKEN_FACTOR * TOL_Y[cfg.dtype]
 
 
 @pytest.mark.parametrize("name,T,tau", [("bert", 700, 0.3), ("gpt2_ffn", 5, 0.2), ("gpt2_ffn", 40, 0.2)])
@@ -423,32 +464,44 @@ def test_group_full_size_on_sampled_tokens(api):
 
 # ------------------------------------------------------------------------------------ full-size sampled checks
 
-FULL_CASES = [("bert", 0.3, 96), ("vit", 0.3, 64), ("llama", 0.4, 24), ("paper", None, 48)]
+FULL_CASES = [("bert", 0.3, 1), ("vit", 0.3, 1), ("llama", 0.4, 1), ("paper", None, 2)]
 
 
-@pytest.mark.parametrize("name,tau,n_sample", FULL_CASES)
-def test_full_size_layer_on_sampled_tokens(api, name, tau, n_sample):
-    """Full workload size in the launch configuration the benchmark times; the oracle recomputes sampled tokens."""
+@pytest.mark.parametrize("name,tau,stride", FULL_CASES)
+def test_full_size_layer_on_sampled_tokens(api, name, tau, stride):
+    """Full workload size in the launch configuration the benchmark times; the oracle recomputes one token of every
+    128-token row tile (every `stride`-th tile where the oracle would take minutes), the edge rows of the first and
+    last tiles, and the tokens with the fewest and the most experts."""
     cfg, w, x, layer = _setup(api, name, None)
     act = oracle.ACT_BY_NAME[cfg.act]
     xd = api.to_device(x, cfg.dtype)
     T = x.shape[0]
+    y = _poison(torch.empty((T, cfg.d), dtype=torch.bfloat16, device="cuda"))
+    _poison(layer.workspace(T))
     if tau is None:       # the paper's protocol: Bernoulli override of the gating decisions (Sec. 4.4)
         G_full = wl.make_bernoulli_mask(cfg, 0.3)
         r = api.routing_from_mask(torch.from_numpy(oracle.pack_mask(G_full).view(np.int32)).cuda(), cfg.E)
-        y = layer.moe_ffn_fwd(xd, r)
+        y = layer.moe_ffn_fwd(xd, r, y=y)
     else:
-        y, r = layer.layer_fwd(xd, tau)
+        y, r = layer.layer_fwd(xd, tau, y=y)
     torch.cuda.synchronize()
     assert r.status == 0
     G = oracle.unpack_mask(r.mask_u32(), cfg.E)
     _check_routing(r, G, dual=False)                       # metadata consistent with the mask, in full
     k = G.sum(1)
     rng = np.random.default_rng(1)
-    sample = np.unique(np.concatenate([rng.choice(T, n_sample, replace=False), [int(k.argmin()), int(k.argmax()), 0, T - 1]]))
+    sample = _tile_sample(T, rng, extra=[int(k.argmin()), int(k.argmax())])
+    if stride > 1:
+        keep = (sample // 128) % stride == 0
+        keep[[0, -1]] = True
+        sample = sample[keep | np.isin(sample, [int(k.argmin()), int(k.argmax())])]
     y_ref = oracle.moe_ffn(x[sample], w["w1"], w["b1"], w["w_gate"], w["w2"], w["b2"], act, G[sample])
     yg = y[torch.from_numpy(sample).cuda()].float().cpu().numpy()
-    assert _rel_err(yg, y_ref) <= TOL_Y[cfg.dtype]
+    assert torch.isfinite(y.float()).all().item()
+    err, err_tok = _rel_err(yg, y_ref), _per_token_err(yg, y_ref)
+    print(f"full size {name}: {sample.size} sampled tokens, rel err {err:.2e}, per-token {err_tok:.2e}")
+    assert err <= TOL_Y[cfg.dtype]
+    assert err_tok <= PER_TOKEN_FACTOR * TOL_Y[cfg.dtype]
 
 
 def test_layer_fwd_host_buffers(api):

@@ -232,19 +232,35 @@ def test_selection_invariants(E):
 
 
 def test_selection_threshold_is_a_float32_product():
-    """tau*max is rounded to float32 before the compare: a value between the float32 and the exact product decides."""
+    """Eq. 4's threshold tau*max is ONE float32 round-to-nearest product, compared in float32.
+
+    The pairs below are chosen so that the float32 product lies strictly BELOW the exact real product tau*m (with
+    tau itself taken as the float32 value the rule receives): a score equal to the float32 product must then be kept,
+    whereas a rule that multiplied in double precision (or in exact arithmetic) would drop it, because it sits under
+    that threshold.  One pair of the other direction (float32 product above the exact one) shows the opposite case:
+    the float32 neighbour just below the rounded threshold lies above the exact product and must still be dropped."""
+    from fractions import Fraction
     tau = np.float32(0.1)
+    below_pairs = []
+    for m in np.float32([5.0, 123.456, 1e-3, 7e5]):
+        thr32 = np.float32(tau * m)                           # numpy: one float32 multiply, round to nearest
+        exact = Fraction(float(tau)) * Fraction(float(m))     # the real-number product of the two float32 inputs
+        assert Fraction(float(thr32)) < exact, "pair must have its float32 product below the exact product"
+        assert float(thr32) < float(tau) * float(m)           # ... and below the double-precision product as well
+        below_pairs.append((m, thr32))
+    R = np.array([[m, thr32, np.nextafter(thr32, np.float32(-np.inf))] for m, thr32 in below_pairs], dtype=np.float32)
+    G, k, _ = oracle.select(R, float(tau))
+    # the maximum, the score ON the float32 threshold (kept: >= in float32), the float32 value just under it (dropped)
+    assert G.tolist() == [[1, 1, 0]] * len(below_pairs)
+    assert k.tolist() == [2] * len(below_pairs)
+    # the other direction: float32 product above the exact one
     m = np.float32(3.0)
     thr32 = np.float32(tau * m)
-    exact = float(tau) * float(m)
-    assert float(thr32) != exact
-    lo, hi = sorted((float(thr32), exact))
-    # the float32 neighbour of thr32 on the far side of the exact product
-    below = np.nextafter(thr32, np.float32(-np.inf))
-    R = np.array([[m, thr32, below]], dtype=np.float32)
-    G, k, _ = oracle.select(R, float(tau))
+    assert Fraction(float(thr32)) > Fraction(float(tau)) * Fraction(float(m))
+    under = np.nextafter(thr32, np.float32(-np.inf))
+    assert Fraction(float(under)) < Fraction(float(tau)) * Fraction(float(m))      # no float32 value lies between the two products
+    G, _, _ = oracle.select(np.array([[m, thr32, under]], dtype=np.float32), float(tau))
     assert G.tolist() == [[1, 1, 0]]
-    assert lo <= hi
 
 
 def test_selection_nonfinite_rows_keep_everything():

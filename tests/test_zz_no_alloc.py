@@ -26,16 +26,31 @@ def _outputs(r):
 
 
 def test_static_scratch_selection_matches_regular_entry_point_twice():
+    import oracle
     from paper_2310_04361_b200 import api
-    calls = [(wl.CONFIGS["vit"], 25216, 0.3), (wl.CONFIGS["llama"], 3000, 0.6), (wl.CONFIGS["vit"], 25216, 0.3)]
-    for cfg, T, tau in calls:                       # back-to-back calls share the library's scratch array
-        R = torch.from_numpy(wl.make_router_scores(cfg, T)).cuda()
+    # back-to-back calls share the library's scratch array; the 40-token call takes the single-CTA branch (64 tokens or
+    # fewer), which needs no scratch at all, between two calls that do
+    calls = [(wl.CONFIGS["vit"], 25216, 0.3), (wl.CONFIGS["llama"], 3000, 0.6), (wl.CONFIGS["gpt2_ffn"], 40, 0.5),
+             (wl.CONFIGS["vit"], 25216, 0.3)]
+    for cfg, T, tau in calls:
+        R_np = wl.make_router_scores(cfg, T)
+        R = torch.from_numpy(R_np).cuda()
         want = _outputs(api.select_dynk(R, tau, dual=True))
         routing = api.Routing(T, cfg.E, R.device, dual=True)     # outputs are still the caller's buffers
         got = _outputs(api.select_dynk_static(R, tau, routing))
         assert got[0] == want[0] == 0 and got[1] == want[1] > 0
         for a, b in zip(got[2:], want[2:]):
             assert torch.equal(a, b)                # integer outputs: bit-exact
+        # and against the CPU oracle's rule and lists on the same scores (Eq. 4, Listing 1)
+        G, k, _ = oracle.select(R_np, tau)
+        meta = oracle.metadata(G)
+        assert np.array_equal(routing.mask_u32(), oracle.pack_mask(G))
+        assert np.array_equal(routing.k[:T].cpu().numpy(), k)
+        assert np.array_equal(routing.counts.cpu().numpy(), meta["counts"])
+        assert np.array_equal(routing.offsets.cpu().numpy(), meta["offsets"])
+        assert routing.n_sel == meta["n_sel"]
+        assert np.array_equal(routing.perm[: meta["n_sel"]].cpu().numpy(), meta["perm"])
+        assert np.array_equal(routing.tok_exp[: meta["n_sel"]].cpu().numpy(), meta["tok_exp"])
 
 
 def test_static_scratch_limit_is_enforced():
