@@ -288,6 +288,16 @@ D2D_API d2d_status d2d_expert_down_masked_fwd(const d2d_layer *layer, const void
 D2D_API d2d_status d2d_expert_down_fwd(const d2d_layer *layer, const void *H, int32_t T, void *y, int32_t *status,
                                        void *stream);
 
+/* Test aid for the library's failure handling (no counterpart in the paper).
+ * kind = 1: the NEXT d2d_expert_up_fwd call launches its kernel with one
+ * operand load left out in one CTA, so that the bounded waits inside that CTA
+ * run out (about a second): the kernel records D2D_ERR_TIMEOUT in the status
+ * word, every warp role reaches the final barrier, tensor memory is freed and
+ * the kernel returns normally -- nothing traps and no wait is unbounded.  H is
+ * incomplete after such a call.  kind = 0 clears a pending request.  Follow a
+ * timed-out call with d2d_layer_reset_counters before the layer is used again. */
+D2D_API d2d_status d2d_test_inject_fault(int32_t kind);
+
 /* The whole layer with no host synchronisation in between:
  * router_fwd -> select_dynk -> moe_ffn_fwd (Sec. 3.2-3.4).  R_out: optional
  * device [T,E] float32 output of the router scores; with NULL the scores may

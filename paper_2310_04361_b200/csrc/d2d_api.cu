@@ -15,6 +15,7 @@ d2d_status d2d_launch_moe_ffn_token(const d2d_layer *L, const void *x, int T, co
                                     cudaStream_t st);
 
 unsigned long long d2d_launch_counter = 0;
+static int g_test_fault = 0;       // d2d_test_inject_fault: consumed by the next d2d_expert_up_fwd
 
 namespace {
 
@@ -436,7 +437,15 @@ d2d_status d2d_expert_up_fwd(const d2d_layer *layer, const void *x, int32_t T, c
     up.M = T; up.N = D.d_ff; up.K = D.d; up.epilogue = D2D_EPI_UP_MASKED; up.act = D.act;
     up.mask = routing->mask; up.mask_words = (D.n_experts + 31) / 32; up.expert_size = D.expert_size;
     up.status = routing->status;
+    up.test_skip_load = __atomic_exchange_n(&g_test_fault, 0, __ATOMIC_RELAXED) == 1;
     return d2d_gemm_tc(up, (cudaStream_t)stream);
+}
+
+d2d_status d2d_test_inject_fault(int32_t kind)
+{
+    if (kind != 0 && kind != 1) return D2D_ERR_INVALID_ARG;
+    __atomic_store_n(&g_test_fault, kind, __ATOMIC_RELAXED);
+    return D2D_OK;
 }
 
 d2d_status d2d_expert_up_gather_fwd(const d2d_layer *layer, const void *x, int32_t T, const d2d_routing *routing,

@@ -39,6 +39,7 @@ struct EpiParams {
     int batch;                       // >= 1 problems of one shape: A columns, B rows, bias entries and out advance per problem
     const int32_t *n_sel;            // density-adaptive dispatch: do nothing when *n_sel <= n_sel_max (NULL: always run)
     long long n_sel_max;
+    int test_skip_load;              // test aid: CTA 0 never requests the A tile of its first k-block (see d2d_gemm_args)
 };
 
 // Tile index -> (row tile, column tile).  Plain order is row-major: CTAs that run together share a few rows of A and
@@ -285,6 +286,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__
                 for (int kb = kb0; kb < kb1; ++kb, ++it) {
                     const uint32_t s = it % STAGES, round = it / STAGES;
                     if (it < pre) {                           // armed above, B already requested
+                        // host-made fault for the failure-handling test: this stage's byte count is never reached, so the
+                        // MMA warp's wait, then the epilogue's and this thread's own, run out and the CTA leaves in order
+                        if (ep.test_skip_load && it == 0 && blockIdx.x == 0) continue;
                         tma_load_2d(smem_u32(smem + (size_t)s * STAGE_BYTES), &tm_a, ka + kb * BK, m0, smem_u32(&bar_full[s]));
                         continue;
                     }
@@ -629,7 +633,8 @@ d2d_status launch(const d2d_gemm_args &g, cudaStream_t st)
     EpiParams ep{(const __nv_bfloat16 *)g.bias, g.out, g.mask, g.mask_words, es, g.status,
                  (uint32_t)((0x100000000ull + (unsigned long long)es - 1) / (unsigned long long)es),
                  g.tile_counter, (g.pdl_late_wait && !g.n_sel && d2d_tc_pdl_enabled()) ? 1 : 0, gate_cat ? 1 : 0,
-                 band_rows_for(g.M, g.N, g.K, BM, GATED), batch, g.n_sel, g.n_sel_max};
+                 band_rows_for(g.M, g.N, g.K, BM, GATED), batch, g.n_sel, g.n_sel_max,
+                 (g.test_skip_load && !g.tile_counter && !g.pdl_late_wait && !g.n_sel) ? 1 : 0};
     const int k_splits = g.k_splits > 1 ? g.k_splits : 1;
     const int tiles = d2d_cdiv(g.N, BN) * d2d_cdiv(g.M, BM) * k_splits * batch;
     const int workers = d2d_tc_sm_count();

@@ -55,6 +55,11 @@ struct d2d_gemm_args {
     // work).  Cannot be combined with pdl_late_wait.
     const int32_t *n_sel;
     long long n_sel_max;
+    // Test aid for the failure-handling test (host-made fault, nothing traps or spins without bound): CTA 0 leaves out
+    // the load of the A tile of its first k-block, so the barrier of that stage never completes; the bounded waits of
+    // the MMA warp, the epilogue and the producer run out, D2D_ERR_TIMEOUT is recorded, every role reaches the final
+    // barrier, TMEM is freed and the kernel returns.  Only honoured by the statically scheduled launch.
+    int test_skip_load;
 };
 
 // Number of K slices d2d_gemm_tc would use for a [M,N,K] down projection (1 = no split) and the float32 scratch it needs.

@@ -569,6 +569,34 @@ def test_expert_up_then_down_matches_oracle(api, name, T, tau):
     assert _rel_err(y, y_ref) <= TOL_Y[cfg.dtype]
 
 
+# ------------------------------------------------------------------------------------ failure handling
+
+def test_bounded_waits_run_out_and_the_library_recovers(api):
+    """A host-made fault (one operand load of one CTA left out) makes the bounded waits inside the tensor-core kernel
+    run out: the call returns, the status word holds D2D_ERR_TIMEOUT, the context stays usable, and after
+    d2d_layer_reset_counters the same layer object computes correct results again."""
+    cfg, w, x, layer = _setup(api, "bert", 640)
+    xd = api.to_device(x, cfg.dtype)
+    G = wl.make_bernoulli_mask(cfg, 0.4, T=640)
+    r = api.routing_from_mask(torch.from_numpy(oracle.pack_mask(G).view(np.int32)).cuda(), cfg.E)
+    y_ref = oracle.moe_ffn(x, w["w1"], w["b1"], w["w_gate"], w["w2"], w["b2"], oracle.ACT_BY_NAME[cfg.act], G)
+    assert api._lib.d2d_test_inject_fault(1) == 0
+    H = layer.expert_up_fwd(xd, r)
+    torch.cuda.synchronize()                               # about a second: the waits give up, the kernel returns
+    assert r.status == 6                                   # D2D_ERR_TIMEOUT
+    layer.reset_counters()
+    r.scalars.zero_()
+    H = layer.expert_up_fwd(xd, r)                         # the request was consumed: this launch is a normal one
+    y = layer.expert_down_fwd(H).float().cpu().numpy()
+    torch.cuda.synchronize()
+    assert r.status == 0
+    assert _rel_err(y, y_ref) <= TOL_Y[cfg.dtype]
+    r2 = layer.new_routing(640)
+    y2, _ = layer.layer_fwd(xd, 0.3, routing=r2)
+    torch.cuda.synchronize()
+    assert r2.status == 0 and torch.isfinite(y2.float()).all().item()
+
+
 # ------------------------------------------------------------------------------------ argument errors
 
 def test_argument_errors(api):
