@@ -171,7 +171,7 @@ D2D_API d2d_status d2d_layer_destroy(d2d_layer *layer);
  * library default for the shape.  Returns D2D_ERR_UNSUPPORTED when the shape
  * cannot take the gathered path (fp32 layers, expert sizes that are not a
  * multiple of 8) and it, or a group, was asked for. */
-typedef enum { D2D_PATH_AUTO = 0, D2D_PATH_DENSE = 1, D2D_PATH_GATHER = 2 } d2d_expert_path;
+typedef enum { D2D_PATH_AUTO = 0, D2D_PATH_DENSE = 1, D2D_PATH_GATHER = 2, D2D_PATH_FUSED = 3 } d2d_expert_path;
 D2D_API d2d_status d2d_layer_set_expert_path(d2d_layer *layer, d2d_expert_path path, int32_t group, double rho_max);
 /* Current setting; any output pointer may be NULL.  *group is 0 when the shape
  * cannot take the gathered path. */

@@ -26,7 +26,7 @@ STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "WORKSPACE", 4: 
                 6: "TIMEOUT", 7: "CAPACITY"}
 D2D_F32, D2D_BF16 = 0, 1
 ACTS = {"relu": 0, "gelu_erf": 1, "gelu_tanh": 2, "silu": 3}
-PATHS = {"auto": 0, "dense": 1, "gather": 2}
+PATHS = {"auto": 0, "dense": 1, "gather": 2, "fused": 3}
 EXPORTS = ["d2d_status_str", "d2d_launch_count", "d2d_layer_create", "d2d_layer_destroy", "d2d_workspace_bytes",
            "d2d_layer_set_expert_path", "d2d_layer_get_expert_path", "d2d_layer_reset_counters", "d2d_expert_up_gather_fwd", "d2d_expert_down_masked_fwd", "d2d_test_inject_fault",
            "d2d_select_workspace_bytes", "d2d_router_fwd", "d2d_select_dynk", "d2d_select_dynk_static", "d2d_select_topk",

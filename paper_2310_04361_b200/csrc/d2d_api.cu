@@ -139,6 +139,24 @@ static d2d_status launch_tc_experts(const d2d_layer *L, const void *x, int T, co
     if (path == D2D_PATH_AUTO && (up_flop < 1e11 || !n_sel)) path = D2D_PATH_DENSE;
     const long long n_sel_max = (long long)(L->gather_rho_max * (double)T * (double)D.n_experts);
     d2d_status rc;
+    // Fused gathered step (plain layers): up projection, activation, down projection and the merge in one kernel whose
+    // time is proportional to the kept (token, group) pairs; the float32 accumulator takes the place of H.
+    long long n_sel_fused = -1;
+    if (L->fused_group > 0 && (path == D2D_PATH_FUSED || (path == D2D_PATH_AUTO && L->fused_rho_max > 0.0))) {
+        d2d_gather_args fa = {};
+        fa.x = x; fa.w1 = L->w1; fa.b1 = L->b1; fa.mask = r->mask;
+        fa.T = T; fa.d = D.d; fa.d_ff = D.d_ff; fa.n_experts = D.n_experts; fa.s = D.expert_size; fa.g = L->fused_group;
+        fa.act = D.act; fa.status = r->status; fa.ctr = L->gather_ctr;
+        if (path == D2D_PATH_AUTO) {
+            n_sel_fused = (long long)(L->fused_rho_max * (double)T * (double)D.n_experts);
+            if (n_sel_fused > n_sel_max) n_sel_fused = n_sel_max;
+            fa.n_sel = n_sel; fa.n_sel_min = -1; fa.n_sel_max = n_sel_fused;
+        }
+        rc = d2d_moe_gather_ffn(fa, (float *)ws, y, L->w2, L->b2, st);
+        if (rc != D2D_OK || path == D2D_PATH_FUSED) return rc;
+    } else if (path == D2D_PATH_FUSED) {
+        return D2D_ERR_UNSUPPORTED;
+    }
     if (path != D2D_PATH_GATHER) {
         d2d_gemm_args up = {};
         const bool forced = path == D2D_PATH_DENSE;
@@ -156,7 +174,7 @@ static d2d_status launch_tc_experts(const d2d_layer *L, const void *x, int T, co
         ga.x = x; ga.w1 = L->w1; ga.w_gate = D.gated ? L->w_gate : nullptr; ga.b1 = L->b1; ga.mask = r->mask; ga.H = ws;
         ga.T = T; ga.d = D.d; ga.d_ff = D.d_ff; ga.n_experts = D.n_experts; ga.s = D.expert_size; ga.g = L->gather_group;
         ga.act = D.act; ga.status = r->status; ga.ctr = L->gather_ctr;
-        ga.n_sel = n_sel; ga.n_sel_max = path == D2D_PATH_AUTO ? n_sel_max : LLONG_MAX;
+        ga.n_sel = n_sel; ga.n_sel_min = n_sel_fused; ga.n_sel_max = path == D2D_PATH_AUTO ? n_sel_max : LLONG_MAX;
         rc = d2d_moe_gather_up(ga, st);
         if (rc != D2D_OK) return rc;
     }
@@ -164,7 +182,7 @@ static d2d_status launch_tc_experts(const d2d_layer *L, const void *x, int T, co
     // that applies the selection while it stages H (it is valid after the masked dense up projection as well).
     // With the automatic choice both down projections are enqueued as well, each with the rule of its up projection.
     if (path != D2D_PATH_DENSE) {
-        rc = d2d_moe_down_masked(D, ws, r->mask, L->w2, L->b2, y, T, r->status, st, path == D2D_PATH_AUTO ? n_sel : nullptr, n_sel_max);
+        rc = d2d_moe_down_masked(D, ws, r->mask, L->w2, L->b2, y, T, r->status, st, path == D2D_PATH_AUTO ? n_sel : nullptr, n_sel_fused, n_sel_max);
         if (rc != D2D_OK || path == D2D_PATH_GATHER) return rc;
     }
     d2d_gemm_args dn = {};
@@ -244,6 +262,8 @@ d2d_status d2d_layer_create(const d2d_layer_desc *desc, const d2d_weights *w, vo
     L->gather_group = d2d_gather_group_for(D, 0);
     L->gather_rho_max = default_gather_rho_max(D, L->gather_group);
     L->expert_path = D2D_PATH_AUTO;
+    L->fused_group = d2d_gather_ffn_group_for(D);
+    L->fused_rho_max = 0.0;
     L->gather_ctr_words = D.n_experts + 64;               // enough for any group size: E / g counters + the exit ticket
     const size_t ctr_off = total;
     total += d2d_align_up((size_t)L->gather_ctr_words * sizeof(int), 256);
@@ -335,7 +355,21 @@ d2d_status d2d_layer_destroy(d2d_layer *layer)
 
 d2d_status d2d_layer_set_expert_path(d2d_layer *layer, d2d_expert_path path, int32_t group, double rho_max)
 {
-    if (!layer || path < D2D_PATH_AUTO || path > D2D_PATH_GATHER || group < 0) return D2D_ERR_INVALID_ARG;
+    if (!layer || path < D2D_PATH_AUTO || path > D2D_PATH_FUSED || group < 0) return D2D_ERR_INVALID_ARG;
+    if (path == D2D_PATH_FUSED) {
+        // the group size applies to the fused kernel, whose groups hold at most 128 neurons
+        const d2d_layer_desc &D = layer->desc;
+        int g = d2d_gather_ffn_group_for(D);
+        if (g <= 0) return D2D_ERR_UNSUPPORTED;
+        if (group > 0) {
+            const int gs = group * D.expert_size;
+            if ((group & (group - 1)) || group > 32 || D.n_experts % group || gs % 16 || gs > 128) return D2D_ERR_UNSUPPORTED;
+            g = group;
+        }
+        layer->fused_group = g;
+        layer->expert_path = path;
+        return D2D_OK;
+    }
     const int g = d2d_gather_group_for(layer->desc, group);
     if (g <= 0 && (path == D2D_PATH_GATHER || group > 0)) return D2D_ERR_UNSUPPORTED;
     layer->gather_group = g;
@@ -348,7 +382,7 @@ d2d_status d2d_layer_get_expert_path(const d2d_layer *layer, int32_t *path, int3
 {
     if (!layer) return D2D_ERR_INVALID_ARG;
     if (path) *path = layer->expert_path;
-    if (group) *group = layer->gather_group;
+    if (group) *group = layer->expert_path == D2D_PATH_FUSED ? layer->fused_group : layer->gather_group;
     if (rho_max) *rho_max = layer->gather_rho_max;
     return D2D_OK;
 }
@@ -460,7 +494,7 @@ d2d_status d2d_expert_up_gather_fwd(const d2d_layer *layer, const void *x, int32
     ga.x = x; ga.w1 = layer->w1; ga.w_gate = D.gated ? layer->w_gate : nullptr; ga.b1 = layer->b1; ga.mask = routing->mask; ga.H = H;
     ga.T = T; ga.d = D.d; ga.d_ff = D.d_ff; ga.n_experts = D.n_experts; ga.s = D.expert_size; ga.g = layer->gather_group;
     ga.act = D.act; ga.status = routing->status; ga.ctr = layer->gather_ctr;
-    ga.n_sel = routing->n_sel; ga.n_sel_max = LLONG_MAX;
+    ga.n_sel = routing->n_sel; ga.n_sel_min = -1; ga.n_sel_max = LLONG_MAX;
     return d2d_moe_gather_up(ga, (cudaStream_t)stream);
 }
 

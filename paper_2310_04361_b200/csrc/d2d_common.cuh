@@ -45,6 +45,8 @@ struct d2d_layer {
     int gather_group;
     int expert_path;
     double gather_rho_max;
+    int fused_group;              // experts per group of the fused gathered kernel (0: shape not supported)
+    double fused_rho_max;         // automatic choice: the fused kernel runs while n_sel <= fused_rho_max * T * E (0: never)
 };
 
 // Layers of one shape that read the same token rows (the Q, K and V projections of one attention layer) and run as

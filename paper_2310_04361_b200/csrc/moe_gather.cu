@@ -58,7 +58,7 @@ struct GatherParams {
     int32_t *status;
     int *ctr;                        // [n_groups] sub-chunk counters + [1] exit ticket, zero at launch, reset by the last CTA
     const int32_t *n_sel;            // selected (token, expert) pairs of this batch, or NULL
-    long long n_sel_max;             // the kernel does nothing when *n_sel > n_sel_max (the masked dense path runs instead)
+    long long n_sel_min, n_sel_max;  // the kernel works only when n_sel_min < *n_sel <= n_sel_max (another path runs otherwise)
     int T, d, d_ff, W;
     int g, s, gs, n_groups;          // experts per group, expert size, g * s, E / g
     uint32_t inv_s;                  // ceil(2^32 / s)
@@ -113,6 +113,121 @@ __device__ __forceinline__ bool mma_tile(uint8_t *smem, uint64_t *bar_full, uint
     return true;
 }
 
+// The scheduler warp's whole job (see the file header): draws sub-chunks of groups from the device counters, compacts
+// the tokens that keep the group into the FIFO, emits tiles through the descriptor ring, ends the stream with a
+// sentinel, and lets the CTA that finishes last reset the counters.
+__device__ __forceinline__ void run_scheduler(const GatherParams &p, uint32_t *fifo, uint64_t *tile_full, uint64_t *tile_empty,
+                                              TileDesc *tdesc, uint32_t *live, int lane)
+{
+    const int Ng = p.n_groups, SUB = p.sub, n_sub = (p.T + SUB - 1) / SUB;        // SUB is a multiple of 256
+    // Groups the CTAs work in at the same time.  The host's value keeps that many groups' weight rows in L2.  When
+    // few tokens keep a group, a visit of a CTA to a group should still yield several full tiles (its last tile is
+    // ragged and costs as much as a full one), so the CTAs spread over more groups: with gridDim.x / Wn CTAs per
+    // group a visit collects about u * T * Wn / gridDim.x rows, u = 1 - (1 - rho)^g the expected kept fraction.
+    int Wn = p.window;
+    if (p.n_sel) {
+        const float rho = fminf((float)__ldcg(p.n_sel) / ((float)p.T * (float)(Ng * p.g)), 1.0f);
+        const float u = fmaxf(1.0f - __expf((float)p.g * log1pf(-fminf(rho, 0.999f))), 1e-6f);
+        const float need = 8.0f * (float)BM * (float)gridDim.x / (u * (float)p.T);
+        const int w = need >= (float)Ng ? Ng : (int)need;
+        Wn = w > Wn ? w : Wn;
+    }
+    const uint32_t lower = (1u << lane) - 1u;
+    const uint32_t gm = p.g >= 32 ? 0xffffffffu : (1u << p.g) - 1u;
+    uint32_t head = 0, emitted = 0, tile_seq = 0;
+    bool ok = true;
+    auto emit = [&](uint32_t start, int n_rows, int group) -> bool {
+        const uint32_t sl = tile_seq % TR, use = tile_seq / TR;
+        if (!mbar_wait_warp(smem_u32(&tile_empty[sl]), (use & 1u) ^ 1u, p.status)) return false;
+        __syncwarp();                                     // the FIFO entries written by all lanes are ordered before the arrival
+        if (lane == 0) {
+            tdesc[sl].start = (int)start;
+            tdesc[sl].n_rows = n_rows;
+            tdesc[sl].group = group;
+            mbar_arrive(smem_u32(&tile_full[sl]));
+        }
+        ++tile_seq;
+        return true;
+    };
+    // Visiting order: the groups are dealt to Wn "lanes" (group G belongs to lane G % Wn).  A CTA first works through
+    // its own lane, then through the others, so that at any time the CTAs are busy in about Wn groups whose weight
+    // rows stay in L2 while the token rows stream by.  Before it picks its next group a CTA takes a snapshot of all
+    // counters (one round trip for the whole warp) and skips the groups that are used up: a counter only grows, so
+    // "used up" is final and the walk over the order below never has to go back.
+    int j = 0, G = (int)blockIdx.x % Wn;                  // position in the order: lane (blockIdx.x + j) % Wn, group G
+    while (ok) {
+        for (int base = 0; base < Ng; base += 32) {
+            const int gi = base + lane;
+            const bool alive = gi < Ng && *(volatile const int *)(p.ctr + gi) < n_sub;
+            const uint32_t b = __ballot_sync(0xffffffffu, alive);
+            if (lane == 0) live[base >> 5] = b;
+        }
+        __syncwarp();
+        while (j < Wn && !((live[G >> 5] >> (G & 31)) & 1u)) {
+            G += Wn;
+            if (G >= Ng) {
+                ++j;
+                G = ((int)blockIdx.x + j) % Wn;
+            }
+        }
+        __syncwarp();                                     // everyone has read the snapshot before it is rewritten
+        if (j >= Wn) break;               // every group is used up
+        const int e0 = G * p.g, w = e0 >> 5, sh = e0 & 31;
+        // Draws of this group, software-pipelined: the counter is bumped one draw ahead, and a draw is walked in
+        // pieces of 256 tokens (eight mask words per lane) whose loads are requested one piece ahead of the
+        // compaction, so the warp waits for one memory latency per draw, not per piece.
+        auto load_piece = [&](int t0, uint32_t (&bits)[8]) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const int t = t0 + q * 32 + lane;
+                bits[q] = t < p.T ? ((__ldg(p.mask + (size_t)t * p.W + w) >> sh) & gm) : 0u;
+            }
+        };
+        int c = 0;
+        if (lane == 0) c = atomicAdd(p.ctr + G, 1);
+        c = __shfl_sync(0xffffffffu, c, 0);
+        while (c < n_sub && ok) {
+            int c_next = 0;
+            if (lane == 0) c_next = atomicAdd(p.ctr + G, 1);       // its round trip overlaps this draw
+            const int t_end = min((c + 1) * SUB, p.T);
+            uint32_t bits[8], bits_next[8];
+            load_piece(c * SUB, bits);
+            for (int t0 = c * SUB; t0 < t_end && ok; t0 += 256) {
+                if (t0 + 256 < t_end) load_piece(t0 + 256, bits_next);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const bool keep = bits[q] != 0u;
+                    const uint32_t bk = __ballot_sync(0xffffffffu, keep);
+                    if (keep) fifo[(head + __popc(bk & lower)) % FIFO_CAP] = (uint32_t)(t0 + q * 32 + lane);
+                    head += __popc(bk);
+                }
+                while (head - emitted >= (uint32_t)BM && ok) {
+                    ok = emit(emitted % FIFO_CAP, BM, G);
+                    emitted += BM;
+                }
+#pragma unroll
+                for (int q = 0; q < 8; ++q) bits[q] = bits_next[q];
+            }
+            c = __shfl_sync(0xffffffffu, c_next, 0);
+        }
+        // no sub-chunk of this group is left: the rows carried so far go out as a ragged tile
+        if (ok && head != emitted) {
+            ok = emit(emitted % FIFO_CAP, (int)(head - emitted), G);
+            emitted = head;
+        }
+    }
+    emit(0u, -1, 0);                                      // end of the tile stream
+    // the CTA whose scheduler finishes last leaves the counters at zero for the next launch
+    if (lane == 0) {
+        __threadfence();
+        const int done = atomicAdd(p.ctr + Ng, 1);
+        if (done == (int)gridDim.x - 1) {
+            for (int i = 0; i <= Ng; ++i) p.ctr[i] = 0;
+            __threadfence();
+        }
+    }
+}
+
 template <int ACT, bool GATED>
 __global__ void __launch_bounds__(NTHREADS, 1)
 moe_gather_up_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__ CUtensorMap tm_wg, const GatherParams p)
@@ -160,117 +275,11 @@ moe_gather_up_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_con
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // density-adaptive dispatch: above the crossover the masked dense kernel, launched next to this one, does the work
-    const bool run = p.n_sel == nullptr || (long long)__ldcg(p.n_sel) <= p.n_sel_max;      // n_sel_max = LLONG_MAX: always
+    const long long n_sel_now = p.n_sel ? (long long)__ldcg(p.n_sel) : 0;
+    const bool run = p.n_sel == nullptr || (n_sel_now > p.n_sel_min && n_sel_now <= p.n_sel_max);      // (-1, LLONG_MAX]: always
 
     if (run && warp == WARP_SCHED) {
-        // ------------------------------------------------------------------ scheduler
-        const int Ng = p.n_groups, SUB = p.sub, n_sub = (p.T + SUB - 1) / SUB;        // SUB is a multiple of 256
-        // Groups the CTAs work in at the same time.  The host's value keeps that many groups' weight rows in L2.  When
-        // few tokens keep a group, a visit of a CTA to a group should still yield several full tiles (its last tile is
-        // ragged and costs as much as a full one), so the CTAs spread over more groups: with gridDim.x / Wn CTAs per
-        // group a visit collects about u * T * Wn / gridDim.x rows, u = 1 - (1 - rho)^g the expected kept fraction.
-        int Wn = p.window;
-        if (p.n_sel) {
-            const float rho = fminf((float)__ldcg(p.n_sel) / ((float)p.T * (float)(Ng * p.g)), 1.0f);
-            const float u = fmaxf(1.0f - __expf((float)p.g * log1pf(-fminf(rho, 0.999f))), 1e-6f);
-            const float need = 8.0f * (float)BM * (float)gridDim.x / (u * (float)p.T);
-            const int w = need >= (float)Ng ? Ng : (int)need;
-            Wn = w > Wn ? w : Wn;
-        }
-        const uint32_t lower = (1u << lane) - 1u;
-        const uint32_t gm = p.g >= 32 ? 0xffffffffu : (1u << p.g) - 1u;
-        uint32_t head = 0, emitted = 0, tile_seq = 0;
-        bool ok = true;
-        auto emit = [&](uint32_t start, int n_rows, int group) -> bool {
-            const uint32_t sl = tile_seq % TR, use = tile_seq / TR;
-            if (!mbar_wait_warp(smem_u32(&tile_empty[sl]), (use & 1u) ^ 1u, p.status)) return false;
-            __syncwarp();                                     // the FIFO entries written by all lanes are ordered before the arrival
-            if (lane == 0) {
-                tdesc[sl].start = (int)start;
-                tdesc[sl].n_rows = n_rows;
-                tdesc[sl].group = group;
-                mbar_arrive(smem_u32(&tile_full[sl]));
-            }
-            ++tile_seq;
-            return true;
-        };
-        // Visiting order: the groups are dealt to Wn "lanes" (group G belongs to lane G % Wn).  A CTA first works through
-        // its own lane, then through the others, so that at any time the CTAs are busy in about Wn groups whose weight
-        // rows stay in L2 while the token rows stream by.  Before it picks its next group a CTA takes a snapshot of all
-        // counters (one round trip for the whole warp) and skips the groups that are used up: a counter only grows, so
-        // "used up" is final and the walk over the order below never has to go back.
-        int j = 0, G = (int)blockIdx.x % Wn;                  // position in the order: lane (blockIdx.x + j) % Wn, group G
-        while (ok) {
-            for (int base = 0; base < Ng; base += 32) {
-                const int gi = base + lane;
-                const bool alive = gi < Ng && *(volatile const int *)(p.ctr + gi) < n_sub;
-                const uint32_t b = __ballot_sync(0xffffffffu, alive);
-                if (lane == 0) live[base >> 5] = b;
-            }
-            __syncwarp();
-            while (j < Wn && !((live[G >> 5] >> (G & 31)) & 1u)) {
-                G += Wn;
-                if (G >= Ng) {
-                    ++j;
-                    G = ((int)blockIdx.x + j) % Wn;
-                }
-            }
-            __syncwarp();                                     // everyone has read the snapshot before it is rewritten
-            if (j >= Wn) break;               // every group is used up
-            const int e0 = G * p.g, w = e0 >> 5, sh = e0 & 31;
-            // Draws of this group, software-pipelined: the counter is bumped one draw ahead, and a draw is walked in
-            // pieces of 256 tokens (eight mask words per lane) whose loads are requested one piece ahead of the
-            // compaction, so the warp waits for one memory latency per draw, not per piece.
-            auto load_piece = [&](int t0, uint32_t (&bits)[8]) {
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    const int t = t0 + q * 32 + lane;
-                    bits[q] = t < p.T ? ((__ldg(p.mask + (size_t)t * p.W + w) >> sh) & gm) : 0u;
-                }
-            };
-            int c = 0;
-            if (lane == 0) c = atomicAdd(p.ctr + G, 1);
-            c = __shfl_sync(0xffffffffu, c, 0);
-            while (c < n_sub && ok) {
-                int c_next = 0;
-                if (lane == 0) c_next = atomicAdd(p.ctr + G, 1);       // its round trip overlaps this draw
-                const int t_end = min((c + 1) * SUB, p.T);
-                uint32_t bits[8], bits_next[8];
-                load_piece(c * SUB, bits);
-                for (int t0 = c * SUB; t0 < t_end && ok; t0 += 256) {
-                    if (t0 + 256 < t_end) load_piece(t0 + 256, bits_next);
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        const bool keep = bits[q] != 0u;
-                        const uint32_t bk = __ballot_sync(0xffffffffu, keep);
-                        if (keep) fifo[(head + __popc(bk & lower)) % FIFO_CAP] = (uint32_t)(t0 + q * 32 + lane);
-                        head += __popc(bk);
-                    }
-                    while (head - emitted >= (uint32_t)BM && ok) {
-                        ok = emit(emitted % FIFO_CAP, BM, G);
-                        emitted += BM;
-                    }
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) bits[q] = bits_next[q];
-                }
-                c = __shfl_sync(0xffffffffu, c_next, 0);
-            }
-            // no sub-chunk of this group is left: the rows carried so far go out as a ragged tile
-            if (ok && head != emitted) {
-                ok = emit(emitted % FIFO_CAP, (int)(head - emitted), G);
-                emitted = head;
-            }
-        }
-        emit(0u, -1, 0);                                      // end of the tile stream
-        // the CTA whose scheduler finishes last leaves the counters at zero for the next launch
-        if (lane == 0) {
-            __threadfence();
-            const int done = atomicAdd(p.ctr + Ng, 1);
-            if (done == (int)gridDim.x - 1) {
-                for (int i = 0; i <= Ng; ++i) p.ctr[i] = 0;
-                __threadfence();
-            }
-        }
+        run_scheduler(p, fifo, tile_full, tile_empty, tdesc, live, lane);
     } else if (run && warp == WARP_MMA) {
         // ------------------------------------------------------------------ MMA issuer (whole warp walks, one lane issues)
         const uint32_t idesc = instr_desc_bf16(BM, n_mma);
@@ -441,8 +450,8 @@ struct DownParams {
     const __nv_bfloat16 *b2;         // [d] or NULL
     __nv_bfloat16 *y;                // [T, d]
     int32_t *status;
-    const int32_t *n_sel;            // density-adaptive dispatch: do nothing when *n_sel > n_sel_max (NULL: always run)
-    long long n_sel_max;
+    const int32_t *n_sel;            // density-adaptive dispatch: work only when n_sel_min < *n_sel <= n_sel_max (NULL: always)
+    long long n_sel_min, n_sel_max;
     int T, d, d_ff, W, s;
     uint32_t inv_s;
     int bn, stages, stage_bytes, band;
@@ -484,7 +493,8 @@ moe_down_masked_kernel(const __grid_constant__ CUtensorMap tm_w2, const DownPara
     const uint32_t tmem_base = tmem_base_holder;
     asm volatile("griddepcontrol.wait;" ::: "memory");       // H is the previous kernel's output
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    const bool run = p.n_sel == nullptr || (long long)__ldcg(p.n_sel) <= p.n_sel_max;
+    const long long n_sel_now = p.n_sel ? (long long)__ldcg(p.n_sel) : 0;
+    const bool run = p.n_sel == nullptr || (n_sel_now > p.n_sel_min && n_sel_now <= p.n_sel_max);
 
     // tile index -> (row tile, column tile): row-major, or column by column inside bands of `band` row tiles when W2 is
     // too large to stay in L2 beside the streaming H (the band's rows of H are then re-used from L2 for every column)
@@ -618,6 +628,389 @@ moe_down_masked_kernel(const __grid_constant__ CUtensorMap tm_w2, const DownPara
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
 }
 
+// ---------------------------------------------------------------------------------------------------------------
+// Fused gathered expert step (plain FFN): for every (group, 128-row tile of the tokens that keep it)
+//   up projection -> bias, activation, selection bits -> H tile in shared memory -> down projection with the group's
+//   columns of W2 -> the [rows, d] partial outputs are ADDED to a float32 accumulator at the rows of their tokens.
+// This is the expert-major form of Listing 1 with its atomic merge (App. C): the hidden activations never leave the
+// SM, nothing of the down projection is computed for pairs that were not kept, and the whole expert step costs time
+// in proportion to the number of (token, group) pairs.  What bounds it on B200 is the merge: 4 d bytes of vector
+// reductions per pair at about 5.5 TB/s for the whole chip, so it wins while few tokens keep a group.
+// The caller pre-fills y32 with b2 and converts it to the output type afterwards (kernels below).
+//
+// 16 warps: scheduler, up-MMA issuer, down-MMA issuer, W2 producer (TMA), four gather warps, four warps for the first
+// epilogue (up accumulator -> H tile) and four for the second (down accumulator -> staged, row-contiguous
+// red.global.add.v4.f32).  TMEM: two 128-column up accumulators and two 128-column down accumulators, so gs <= 128.
+constexpr int F_SCHED = 0, F_MMA_UP = 1, F_MMA_DN = 2, F_W2 = 3, F_GATHER0 = 4, F_EPI1_0 = 8, F_EPI2_0 = 12;
+constexpr int F_NTHREADS = 512;
+constexpr int F_CHUNK = 128;                 // columns of y per down accumulator
+constexpr int F_STG_ROW = 272;               // staged accumulator row: 64 floats + 16 bytes of padding
+
+struct FfnParams {
+    GatherParams g;                  // scheduler and gather part (g.H unused)
+    float *y32;                      // [T, d]
+    int n_chunks, kb2;               // ceil(d / 128), ceil(gs / 64)
+};
+
+template <int ACT>
+__global__ void __launch_bounds__(F_NTHREADS, 1)
+moe_gather_ffn_kernel(const __grid_constant__ CUtensorMap tm_w1, const __grid_constant__ CUtensorMap tm_w2, const FfnParams fp)
+{
+    const GatherParams &p = fp.g;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t *hs = smem + (size_t)p.stages * p.stage_bytes;                    // H tile: kb2 x (128 rows x 128 B), swizzled
+    uint8_t *w2s = hs + (size_t)fp.kb2 * A_BYTES;                             // two slots of kb2 W2 tiles (128 rows x 128 B)
+    uint8_t *stg = w2s + (size_t)2 * fp.kb2 * A_BYTES;                        // 128 staged accumulator rows
+    uint32_t *fifo = reinterpret_cast<uint32_t *>(stg + 128 * F_STG_ROW);     // [FIFO_CAP] token indices
+    __shared__ uint64_t bar_full[MAX_STAGES], bar_empty[MAX_STAGES], tile_full[TR], tile_empty[TR];
+    __shared__ uint64_t up_full[2], up_empty[2], h_full, h_empty, w2_full[2], w2_empty[2], dn_full[2], dn_empty[2];
+    __shared__ TileDesc tdesc[TR];
+    __shared__ uint32_t tmem_base_holder;
+    __shared__ uint32_t live[64];
+    __shared__ int tok_s[BM];                                                 // tokens of the tile the second epilogue works on
+    __shared__ volatile int e2_rows, e2_ok;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nkb = (p.d + BK - 1) / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) {
+            mbar_init(smem_u32(&bar_full[s]), 1 + N_GATHER_WARPS * 32);
+            mbar_init(smem_u32(&bar_empty[s]), 1);
+        }
+        for (int t = 0; t < TR; ++t) {
+            mbar_init(smem_u32(&tile_full[t]), 1);
+            mbar_init(smem_u32(&tile_empty[t]), N_GATHER_WARPS + 3 + 4 + 1);  // gather, two MMA warps, W2 producer, epilogue 1, leader of epilogue 2
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&up_full[b]), 1);
+            mbar_init(smem_u32(&up_empty[b]), 4);
+            mbar_init(smem_u32(&w2_full[b]), 1);
+            mbar_init(smem_u32(&w2_empty[b]), 1);
+            mbar_init(smem_u32(&dn_full[b]), 1);
+            mbar_init(smem_u32(&dn_empty[b]), 4);
+        }
+        mbar_init(smem_u32(&h_full), 4);
+        mbar_init(smem_u32(&h_empty), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == F_MMA_UP) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_holder)), "r"(512u)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = tmem_base_holder;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const long long n_sel_now = p.n_sel ? (long long)__ldcg(p.n_sel) : 0;
+    const bool run = p.n_sel == nullptr || (n_sel_now > p.n_sel_min && n_sel_now <= p.n_sel_max);
+
+    if (!run) {
+        // another path does the work
+    } else if (warp == F_SCHED) {
+        run_scheduler(p, fifo, tile_full, tile_empty, tdesc, live, lane);
+    } else if (warp == F_MMA_UP) {
+        const uint32_t idesc = instr_desc_bf16(BM, p.gs);
+        uint32_t it = 0;
+        bool ok = true;
+        for (uint32_t ti = 0; ok; ++ti) {
+            const uint32_t sl = ti % TR;
+            ok = mbar_wait_warp(smem_u32(&tile_full[sl]), (ti / TR) & 1u, p.status);
+            if (!ok) break;
+            const int n_rows = tdesc[sl].n_rows;
+            __syncwarp();
+            if (n_rows < 0) break;
+            if (elect_one()) mbar_arrive(smem_u32(&tile_empty[sl]));
+            const uint32_t ub = ti & 1u, use = ti >> 1;
+            ok = mbar_wait_warp(smem_u32(&up_empty[ub]), (use & 1u) ^ 1u, p.status);
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            ok = mma_tile(smem, bar_full, bar_empty, &up_full[ub], tmem_base + ub * 128u, idesc, nkb, p.stages, p.stage_bytes, it, p.status);
+        }
+    } else if (warp == F_MMA_DN) {
+        // down projection of each tile: A = the H tile, B = the group's columns of W2, 128 output columns at a time
+        const uint32_t idesc = instr_desc_bf16(BM, F_CHUNK);
+        uint32_t cg = 0;
+        bool ok = true;
+        for (uint32_t ti = 0; ok; ++ti) {
+            const uint32_t sl = ti % TR;
+            ok = mbar_wait_warp(smem_u32(&tile_full[sl]), (ti / TR) & 1u, p.status);
+            if (!ok) break;
+            const int n_rows = tdesc[sl].n_rows;
+            __syncwarp();
+            if (n_rows < 0) break;
+            if (elect_one()) mbar_arrive(smem_u32(&tile_empty[sl]));
+            ok = mbar_wait_warp(smem_u32(&h_full), ti & 1u, p.status);
+            for (int c = 0; c < fp.n_chunks && ok; ++c, ++cg) {
+                const uint32_t slot = cg & 1u, use = cg >> 1;
+                ok = mbar_wait_warp(smem_u32(&w2_full[slot]), use & 1u, p.status) &&
+                     mbar_wait_warp(smem_u32(&dn_empty[slot]), (use & 1u) ^ 1u, p.status);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                if (elect_one()) {
+                    for (int k = 0; k < p.gs / UMMA_K; ++k) {
+                        const int j = k >> 2;
+                        const uint64_t koff = (uint64_t)(((k & 3) * UMMA_K * 2) >> 4);
+                        const uint64_t da = smem_desc_sw128(smem_u32(hs + (size_t)j * A_BYTES)) + koff;
+                        const uint64_t db = smem_desc_sw128(smem_u32(w2s + (size_t)(slot * fp.kb2 + j) * A_BYTES)) + koff;
+                        umma_bf16(tmem_base + 256u + slot * 128u, da, db, idesc, k > 0 ? 1u : 0u);
+                    }
+                    umma_commit(smem_u32(&w2_empty[slot]));
+                    umma_commit(smem_u32(&dn_full[slot]));
+                    if (c == fp.n_chunks - 1) umma_commit(smem_u32(&h_empty));      // the H tile may be rewritten
+                }
+                __syncwarp();
+            }
+        }
+    } else if (warp == F_W2) {
+        if (lane == 0) {
+            uint32_t cg = 0;
+            bool ok = true;
+            for (uint32_t ti = 0; ok; ++ti) {
+                const uint32_t sl = ti % TR;
+                ok = mbar_wait(smem_u32(&tile_full[sl]), (ti / TR) & 1u, p.status);
+                if (!ok) break;
+                const int n_rows = tdesc[sl].n_rows, G = tdesc[sl].group;
+                if (n_rows < 0) break;
+                mbar_arrive(smem_u32(&tile_empty[sl]));
+                for (int c = 0; c < fp.n_chunks && ok; ++c, ++cg) {
+                    const uint32_t slot = cg & 1u, use = cg >> 1;
+                    ok = mbar_wait(smem_u32(&w2_empty[slot]), (use & 1u) ^ 1u, p.status);
+                    if (!ok) break;
+                    const uint32_t full = smem_u32(&w2_full[slot]);
+                    mbar_expect_tx(full, (uint32_t)(fp.kb2 * A_BYTES));
+                    for (int j = 0; j < fp.kb2; ++j)
+                        tma_load_2d(smem_u32(w2s + (size_t)(slot * fp.kb2 + j) * A_BYTES), &tm_w2, G * p.gs + j * BK, c * F_CHUNK, full);
+                }
+            }
+        }
+    } else if (warp >= F_GATHER0 && warp < F_EPI1_0) {
+        // ---- gather warps: as in the up-projection kernel
+        const int gw = warp - F_GATHER0, tid_g = gw * 32 + lane;
+        const int chunk = tid_g & 7, rbase = tid_g >> 3;
+        const uint32_t swz = (uint32_t)(((chunk ^ (rbase & 7)) << 4) + (rbase & 7) * 128 + (rbase >> 3) * 1024);
+        uint32_t it = 0;
+        bool ok = true;
+        for (uint32_t ti = 0; ok; ++ti) {
+            const uint32_t sl = ti % TR;
+            ok = mbar_wait_warp(smem_u32(&tile_full[sl]), (ti / TR) & 1u, p.status);
+            if (!ok) break;
+            const int start = tdesc[sl].start, n_rows = tdesc[sl].n_rows, G = tdesc[sl].group;
+            if (n_rows < 0) break;
+            const __nv_bfloat16 *src[PASSES];
+#pragma unroll
+            for (int j = 0; j < PASSES; ++j) {
+                const int r = rbase + ROWS_PER_PASS * j;
+                src[j] = r < n_rows ? p.x + (size_t)fifo[(uint32_t)(start + r) % FIFO_CAP] * p.d + chunk * 8 : nullptr;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&tile_empty[sl]));
+            for (int kb = 0; kb < nkb; ++kb, ++it) {
+                const uint32_t s = it % (uint32_t)p.stages, round = it / (uint32_t)p.stages;
+                ok = mbar_wait_warp(smem_u32(&bar_empty[s]), (round & 1u) ^ 1u, p.status);
+                if (!ok) break;
+                const uint32_t stage = smem_u32(smem + (size_t)s * p.stage_bytes), full = smem_u32(&bar_full[s]);
+                if (gw == 0 && elect_one()) {
+                    mbar_expect_tx(full, (uint32_t)(p.stage_bytes - A_BYTES));
+                    tma_load_2d(stage + A_BYTES, &tm_w1, kb * BK, G * p.gs, full);
+                }
+                const bool in_k = kb * BK + chunk * 8 < p.d;
+#pragma unroll
+                for (int j = 0; j < PASSES; ++j) {
+                    const bool live_row = in_k && src[j] != nullptr;
+                    cp_async16(stage + swz + (uint32_t)(j * ROWS_PER_PASS * 128), live_row ? src[j] + kb * BK : p.x, live_row ? 16u : 0u);
+                }
+                cp_async_arrive(full);
+            }
+        }
+        cp_async_wait_all();
+    } else if (warp >= F_EPI1_0 && warp < F_EPI2_0) {
+        // ---- epilogue 1: up accumulator -> bias, activation, selection bits -> bf16 H tile (swizzled K-major A operand)
+        const int quad = warp & 3, row = quad * 32 + lane;
+        const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+        const int n_units = p.gs >> 4;
+        const bool halves = (p.s & 7) == 0;
+        bool ok = true;
+        for (uint32_t ti = 0; ok; ++ti) {
+            const uint32_t sl = ti % TR;
+            ok = mbar_wait_warp(smem_u32(&tile_full[sl]), (ti / TR) & 1u, p.status);
+            if (!ok) break;
+            const int start = tdesc[sl].start, n_rows = tdesc[sl].n_rows, G = tdesc[sl].group;
+            if (n_rows < 0) break;
+            const bool valid = row < n_rows;
+            const uint32_t tok = valid ? fifo[(uint32_t)(start + row) % FIFO_CAP] : 0u;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&tile_empty[sl]));
+            const int e0 = G * p.g;
+            const uint32_t bits = valid ? __ldg(p.mask + (size_t)tok * p.W + (e0 >> 5)) >> (e0 & 31) : 0u;     // rows past the end keep nothing
+            const __nv_bfloat16 *brow = p.b1 ? p.b1 + (size_t)G * p.gs : nullptr;
+            const uint32_t ub = ti & 1u, use = ti >> 1;
+            ok = mbar_wait_warp(smem_u32(&up_full[ub]), use & 1u, p.status) &&
+                 mbar_wait_warp(smem_u32(&h_empty), (ti & 1u) ^ 1u, p.status);          // the previous tile's down projection has read H
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t tbase = tmem_base + ub * 128u + lane_base;
+            for (int u = 0; u < n_units; ++u) {
+                const int c0 = u * 16;
+                uint32_t ra[16];
+                tmem_ld16_issue(tbase + (uint32_t)c0, ra);
+                float bias[16];
+                if (brow) {
+                    float b8[8];
+                    d2d_load8(brow + c0, b8);
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) bias[q] = b8[q];
+                    d2d_load8(brow + c0 + 8, b8);
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) bias[8 + q] = b8[q];
+                } else {
+#pragma unroll
+                    for (int q = 0; q < 16; ++q) bias[q] = 0.0f;
+                }
+                uint32_t keep;
+                if (halves) {
+                    const uint32_t e_lo = __umulhi((uint32_t)c0, p.inv_s), e_hi = __umulhi((uint32_t)(c0 + 8), p.inv_s);
+                    keep = ((bits >> e_lo) & 1u ? 0x00ffu : 0u) | ((bits >> e_hi) & 1u ? 0xff00u : 0u);
+                } else {
+                    keep = 0u;
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) keep |= ((bits >> __umulhi((uint32_t)(c0 + j), p.inv_s)) & 1u) << j;
+                }
+                tmem_ld_wait();
+                uint32_t pk[8];
+#pragma unroll
+                for (int j = 0; j < 16; j += 2) {
+                    const uint64_t z = add2(pack2(__uint_as_float(ra[j]), __uint_as_float(ra[j + 1])), pack2(bias[j], bias[j + 1]));
+                    float v0, v1;
+                    unpack2(fast_act2<ACT>(z), v0, v1);
+                    const __nv_bfloat162 t2 = __floats2bfloat162_rn(v0, v1);
+                    uint32_t wv = *reinterpret_cast<const uint32_t *>(&t2);
+                    wv = (keep >> j) & 1u ? wv : (wv & 0xffff0000u);
+                    wv = (keep >> (j + 1)) & 1u ? wv : (wv & 0x0000ffffu);
+                    pk[j >> 1] = wv;
+                }
+                const int kb = c0 >> 6, ch = (c0 & 63) >> 3;
+                uint8_t *rowp = hs + (size_t)kb * A_BYTES + (size_t)row * 128;
+                *reinterpret_cast<uint4 *>(rowp + ((ch ^ (row & 7)) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                *reinterpret_cast<uint4 *>(rowp + (((ch + 1) ^ (row & 7)) << 4)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+            }
+            // the accumulator is drained, the H tile is written: hand both on
+            fence_async_smem();
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(smem_u32(&up_empty[ub]));
+                mbar_arrive(smem_u32(&h_full));
+            }
+        }
+    } else {
+        // ---- epilogue 2: down accumulator -> staged rows -> row-contiguous vector reductions into y32 at the tokens' rows.
+        // The four warps meet at named barriers, so every wait is done by one thread and its outcome shared.
+        const int quad = warp & 3, row = quad * 32 + lane, wq = warp - F_EPI2_0;
+        const uint32_t lane_base = (uint32_t)(quad * 32) << 16;
+        const bool leader = warp == F_EPI2_0 && lane == 0;
+        uint32_t cg = 0;
+        for (uint32_t ti = 0;; ++ti) {
+            const uint32_t sl = ti % TR;
+            if (leader) {
+                const bool got = mbar_wait(smem_u32(&tile_full[sl]), (ti / TR) & 1u, p.status);
+                e2_ok = got ? 1 : 0;
+                e2_rows = got ? tdesc[sl].n_rows : -1;
+            }
+            asm volatile("bar.sync 2, 128;" ::: "memory");
+            const int n_rows = e2_rows;
+            if (!e2_ok || n_rows < 0) break;
+            const int start = tdesc[sl].start;
+            if (row < n_rows) tok_s[row] = (int)fifo[(uint32_t)(start + row) % FIFO_CAP];
+            asm volatile("bar.sync 2, 128;" ::: "memory");
+            if (leader) mbar_arrive(smem_u32(&tile_empty[sl]));
+            bool ok = true;
+            for (int c = 0; c < fp.n_chunks; ++c, ++cg) {
+                const uint32_t slot = cg & 1u, use = cg >> 1;
+                if (leader) e2_ok = mbar_wait(smem_u32(&dn_full[slot]), use & 1u, p.status) ? 1 : 0;
+                asm volatile("bar.sync 2, 128;" ::: "memory");
+                ok = e2_ok != 0;
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll
+                for (int hlf = 0; hlf < F_CHUNK / 64; ++hlf) {
+                    uint32_t ra[4][16];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) tmem_ld16_issue(tmem_base + 256u + slot * 128u + lane_base + (uint32_t)(hlf * 64 + u * 16), ra[u]);
+                    tmem_ld_wait();
+                    if (row < n_rows) {
+                        uint4 *o = reinterpret_cast<uint4 *>(stg + (size_t)row * F_STG_ROW);
+#pragma unroll
+                        for (int u = 0; u < 4; ++u)
+#pragma unroll
+                            for (int j = 0; j < 16; j += 4) o[u * 4 + (j >> 2)] = make_uint4(ra[u][j], ra[u][j + 1], ra[u][j + 2], ra[u][j + 3]);
+                    }
+                    asm volatile("bar.sync 2, 128;" ::: "memory");
+                    const int col = c * F_CHUNK + hlf * 64 + (lane & 15) * 4;
+                    for (int r = 2 * wq + (lane >> 4); r < n_rows; r += 8) {
+                        const float4 v = *reinterpret_cast<const float4 *>(stg + (size_t)r * F_STG_ROW + (lane & 15) * 16);
+                        if (col < p.d)
+                            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(fp.y32 + (size_t)tok_s[r] * p.d + col), "f"(v.x),
+                                         "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+                    }
+                    asm volatile("bar.sync 2, 128;" ::: "memory");
+                }
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&dn_empty[slot]));
+            }
+            if (!ok) break;
+        }
+    }
+
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == F_MMA_UP) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+}
+
+// y32[t, :] = b2 before the fused kernel, y = bf16(y32) after it; both follow the fused kernel's dispatch rule
+__global__ void __launch_bounds__(256)
+y32_fill_kernel(float *__restrict__ y32, const __nv_bfloat16 *__restrict__ b2, long long total, int d, const int32_t *n_sel,
+                long long n_sel_min, long long n_sel_max)
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (n_sel) {
+        const long long n = (long long)__ldcg(n_sel);
+        if (!(n > n_sel_min && n <= n_sel_max)) return;
+    }
+    for (long long i = ((long long)blockIdx.x * 256 + threadIdx.x) * 4; i < total; i += (long long)gridDim.x * 1024) {
+        const int n = (int)(i % d);
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (b2) v = make_float4(__bfloat162float(b2[n]), __bfloat162float(b2[n + 1]), __bfloat162float(b2[n + 2]), __bfloat162float(b2[n + 3]));
+        *reinterpret_cast<float4 *>(y32 + i) = v;
+    }
+}
+
+__global__ void __launch_bounds__(256)
+y32_convert_kernel(const float *__restrict__ y32, __nv_bfloat16 *__restrict__ y, long long total, const int32_t *n_sel, long long n_sel_min,
+                   long long n_sel_max)
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (n_sel) {
+        const long long n = (long long)__ldcg(n_sel);
+        if (!(n > n_sel_min && n <= n_sel_max)) return;
+    }
+    for (long long i = ((long long)blockIdx.x * 256 + threadIdx.x) * 4; i < total; i += (long long)gridDim.x * 1024) {
+        const float4 v = __ldcs(reinterpret_cast<const float4 *>(y32 + i));
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+        uint2 o;
+        o.x = *reinterpret_cast<const uint32_t *>(&lo);
+        o.y = *reinterpret_cast<const uint32_t *>(&hi);
+        *reinterpret_cast<uint2 *>(y + i) = o;
+    }
+}
+
 bool ensure_attr(const void *kern, bool (&done)[64])
 {
     int dev = 0;
@@ -636,7 +1029,7 @@ d2d_status launch(const d2d_gather_args &a, cudaStream_t st)
     const int b_rows = GATED ? 2 * gs : gs;
     GatherParams p = {};
     p.x = (const __nv_bfloat16 *)a.x; p.mask = a.mask; p.b1 = (const __nv_bfloat16 *)a.b1; p.H = (__nv_bfloat16 *)a.H;
-    p.status = a.status; p.ctr = a.ctr; p.n_sel = a.n_sel; p.n_sel_max = a.n_sel_max;
+    p.status = a.status; p.ctr = a.ctr; p.n_sel = a.n_sel; p.n_sel_min = a.n_sel_min; p.n_sel_max = a.n_sel_max;
     p.T = a.T; p.d = a.d; p.d_ff = a.d_ff; p.W = (a.n_experts + 31) / 32;
     p.g = a.g; p.s = a.s; p.gs = gs; p.n_groups = a.n_experts / a.g;
     p.inv_s = (uint32_t)((0x100000000ull + (unsigned long long)a.s - 1) / (unsigned long long)a.s);
@@ -722,7 +1115,7 @@ bool d2d_moe_down_masked_supports(const d2d_layer_desc &D)
 }
 
 d2d_status d2d_moe_down_masked(const d2d_layer_desc &D, const void *H, const uint32_t *mask, const void *w2, const void *b2, void *y, int T,
-                               int32_t *status, cudaStream_t st, const int32_t *n_sel, long long n_sel_max)
+                               int32_t *status, cudaStream_t st, const int32_t *n_sel, long long n_sel_min, long long n_sel_max)
 {
     if (T <= 0) return D2D_OK;
     if (!d2d_moe_down_masked_supports(D)) return D2D_ERR_UNSUPPORTED;
@@ -741,7 +1134,7 @@ d2d_status d2d_moe_down_masked(const d2d_layer_desc &D, const void *H, const uin
     p.T = T; p.d = D.d; p.d_ff = D.d_ff; p.W = (D.n_experts + 31) / 32; p.s = D.expert_size;
     p.inv_s = (uint32_t)((0x100000000ull + (unsigned long long)D.expert_size - 1) / (unsigned long long)D.expert_size);
     p.bn = bn;
-    p.n_sel = n_sel; p.n_sel_max = n_sel_max;
+    p.n_sel = n_sel; p.n_sel_min = n_sel_min; p.n_sel_max = n_sel_max;
     p.stage_bytes = A_BYTES + bn * 128;
     const int stages = (192 * 1024) / p.stage_bytes;
     p.stages = stages > MAX_STAGES ? MAX_STAGES : stages;
@@ -770,4 +1163,92 @@ d2d_status d2d_moe_down_masked(const d2d_layer_desc &D, const void *H, const uin
     const cudaError_t err = cudaLaunchKernelEx(&cfg, moe_down_masked_kernel, tw2, p);
     D2D_LAUNCHED(1);
     return err == cudaSuccess && cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
+}
+
+int d2d_gather_ffn_group_for(const d2d_layer_desc &D)
+{
+    // the float32 accumulator [T, d] takes the place of H [T, d_ff] bf16 in the caller's workspace
+    if (D.gated || !d2d_moe_down_masked_supports(D) || D.d % 8 || D.d < 128 || D.d > 128 * 32 || D.d_ff < 2 * D.d) return 0;
+    for (int g = 32; g >= 1; g >>= 1) {
+        const int gs = g * D.expert_size;
+        if (D.n_experts % g == 0 && 32 % g == 0 && gs % 16 == 0 && gs >= 16 && gs <= 128) return g;
+    }
+    return 0;
+}
+
+template <int ACT>
+static d2d_status launch_ffn(const d2d_gather_args &a, float *y32, void *y, const void *w2, const void *b2, cudaStream_t st)
+{
+    const int gs = a.g * a.s;
+    FfnParams fp = {};
+    GatherParams &p = fp.g;
+    p.x = (const __nv_bfloat16 *)a.x; p.mask = a.mask; p.b1 = (const __nv_bfloat16 *)a.b1; p.H = nullptr;
+    p.status = a.status; p.ctr = a.ctr; p.n_sel = a.n_sel; p.n_sel_min = a.n_sel_min; p.n_sel_max = a.n_sel_max;
+    p.T = a.T; p.d = a.d; p.d_ff = a.d_ff; p.W = (a.n_experts + 31) / 32;
+    p.g = a.g; p.s = a.s; p.gs = gs; p.n_groups = a.n_experts / a.g;
+    p.inv_s = (uint32_t)((0x100000000ull + (unsigned long long)a.s - 1) / (unsigned long long)a.s);
+    p.stage_bytes = A_BYTES + gs * 128;
+    fp.y32 = y32;
+    fp.n_chunks = d2d_cdiv(a.d, F_CHUNK);
+    fp.kb2 = d2d_cdiv(gs, BK);
+    const size_t fixed = (size_t)3 * fp.kb2 * A_BYTES + 128 * F_STG_ROW + FIFO_CAP * 4 + 1024;
+    int stages = (int)((216 * 1024 - fixed) / p.stage_bytes);
+    p.stages = stages > MAX_STAGES ? MAX_STAGES : stages;
+    if (p.stages < 2) return D2D_ERR_UNSUPPORTED;
+    const size_t smem = (size_t)p.stages * p.stage_bytes + fixed;
+    p.window = p.n_groups;                                    // plain layers: all weights of these shapes fit in L2
+    const long long group_bytes = (long long)gs * a.d * 4;    // W1 rows and W2 columns of a group
+    long long window = (48ll << 20) / (group_bytes > 0 ? group_bytes : 1);
+    p.window = (int)(window < 4 ? 4 : window > p.n_groups ? p.n_groups : window);
+    if (p.window > p.n_groups) p.window = p.n_groups;
+    const long long want = (long long)a.T * p.n_groups / (8ll * d2d_tc_sm_count());
+    p.sub = want >= 1024 ? 1024 : want >= 512 ? 512 : 256;
+    CUtensorMap tw1, tw2;
+    if (!d2d_tc_make_map(&tw1, a.w1, a.d_ff, a.d, gs) || !d2d_tc_make_map(&tw2, w2, a.d, a.d_ff, 128)) return D2D_ERR_CUDA;
+    auto kern = moe_gather_ffn_kernel<ACT>;
+    static bool attr_set[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return D2D_ERR_CUDA;
+    if (!__atomic_load_n(&attr_set[dev], __ATOMIC_ACQUIRE)) {
+        if (cudaFuncSetAttribute((const void *)kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 217 * 1024) != cudaSuccess) return D2D_ERR_CUDA;
+        __atomic_store_n(&attr_set[dev], true, __ATOMIC_RELEASE);
+    }
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = d2d_tc_pdl_enabled() ? 1 : 0;
+    const long long total = (long long)a.T * a.d;
+    const int blocks = (int)((total / 4 + 255) / 256);
+    const int sms = d2d_tc_sm_count();
+    cfg.gridDim = dim3(blocks < 4 * sms ? blocks : 4 * sms, 1, 1);
+    cfg.blockDim = dim3(256, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cudaError_t err = cudaLaunchKernelEx(&cfg, y32_fill_kernel, y32, (const __nv_bfloat16 *)b2, total, a.d, a.n_sel, a.n_sel_min, a.n_sel_max);
+    if (err == cudaSuccess) {
+        cudaLaunchConfig_t kc = cfg;
+        kc.gridDim = dim3(sms, 1, 1);
+        kc.blockDim = dim3(F_NTHREADS, 1, 1);
+        kc.dynamicSmemBytes = smem;
+        err = cudaLaunchKernelEx(&kc, kern, tw1, tw2, fp);
+    }
+    if (err == cudaSuccess)
+        err = cudaLaunchKernelEx(&cfg, y32_convert_kernel, (const float *)y32, (__nv_bfloat16 *)y, total, a.n_sel, a.n_sel_min, a.n_sel_max);
+    D2D_LAUNCHED(3);
+    return err == cudaSuccess && cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
+}
+
+d2d_status d2d_moe_gather_ffn(const d2d_gather_args &a, float *y32, void *y, const void *w2, const void *b2, cudaStream_t st)
+{
+    if (a.T <= 0) return D2D_OK;
+    if (a.w_gate || a.g < 1 || a.g > 32 || a.g * a.s > 128 || a.n_experts > 2048) return D2D_ERR_UNSUPPORTED;
+    switch (a.act) {
+    case D2D_ACT_RELU: return launch_ffn<D2D_ACT_RELU>(a, y32, y, w2, b2, st);
+    case D2D_ACT_GELU_ERF: return launch_ffn<D2D_ACT_GELU_ERF>(a, y32, y, w2, b2, st);
+    case D2D_ACT_GELU_TANH: return launch_ffn<D2D_ACT_GELU_TANH>(a, y32, y, w2, b2, st);
+    case D2D_ACT_SILU: return launch_ffn<D2D_ACT_SILU>(a, y32, y, w2, b2, st);
+    }
+    return D2D_ERR_INVALID_ARG;
 }

@@ -19,11 +19,12 @@ struct d2d_gather_args {
     int32_t *status;         // device status word (D2D_ERR_TIMEOUT)
     int *ctr;                // n_experts / g + 1 device ints, zero before the first launch; the kernel leaves them at zero
     // Density-adaptive dispatch without a host synchronisation: when n_sel is given, the kernel reads the number of
-    // selected pairs of this batch from it and returns at once if it exceeds n_sel_max (the caller launches the
-    // masked dense up projection with the complementary rule; LLONG_MAX = always run).  The kernel also sizes its
-    // work distribution from that density.  NULL = always run, distribution sized for dense selections.
+    // selected pairs of this batch from it and works only if n_sel_min < n_sel <= n_sel_max, returning at once
+    // otherwise (the caller launches the other paths with the complementary rules; -1 and LLONG_MAX = always run).
+    // The kernel also sizes its work distribution from that density.  NULL = always run, distribution sized for
+    // dense selections.
     const int32_t *n_sel;
-    long long n_sel_max;
+    long long n_sel_min, n_sel_max;
 };
 
 // Experts per group for this layer shape: `want` if it is usable (0 = pick the default), 0 if the gathered path
@@ -36,6 +37,15 @@ d2d_status d2d_moe_gather_up(const d2d_gather_args &a, cudaStream_t st);
 // whose (token, expert) pair is kept.  Follows d2d_moe_gather_up (which writes only those cells) and is equally valid
 // after the masked dense up projection.  w2: [d, d_ff] bf16 as given; requires d % 16 == 0 and s % 8 == 0.
 bool d2d_moe_down_masked_supports(const d2d_layer_desc &D);
-// n_sel / n_sel_max: as in d2d_gather_args (the kernel returns at once when *n_sel > n_sel_max; NULL = always run).
+// n_sel / n_sel_min / n_sel_max: as in d2d_gather_args (NULL = always run).
 d2d_status d2d_moe_down_masked(const d2d_layer_desc &D, const void *H, const uint32_t *mask, const void *w2, const void *b2, void *y, int T,
-                               int32_t *status, cudaStream_t st, const int32_t *n_sel = nullptr, long long n_sel_max = 0);
+                               int32_t *status, cudaStream_t st, const int32_t *n_sel = nullptr, long long n_sel_min = -1,
+                               long long n_sel_max = 0);
+
+// Fused gathered expert step of plain (not gated) layers: up projection, activation, down projection and the
+// scatter-add of the partial outputs per (group, tile of the tokens that keep it), see moe_gather.cu.  a.H is unused,
+// a.g must come from d2d_gather_ffn_group_for (groups of at most 128 neurons).  y32: [T, d] float32 scratch (caller's),
+// filled with b2, accumulated into with vector reductions and converted to y [T, d] bf16: three launches, all
+// following the dispatch rule in `a`.
+int d2d_gather_ffn_group_for(const d2d_layer_desc &D);
+d2d_status d2d_moe_gather_ffn(const d2d_gather_args &a, float *y32, void *y, const void *w2, const void *b2, cudaStream_t st);

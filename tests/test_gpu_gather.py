@@ -224,3 +224,57 @@ def test_decode_batch_with_truncated_lists_stays_inside_its_buffers(api):
     assert bool((guard == -7).all())
     assert torch.isfinite(y.float()).all()
     layer.close()
+
+
+# (workload, tokens, experts per group or 0 = default, d or 0 = the workload's, densities)
+FUSED_CASES = [
+    ("bert", 700, 0, 0, (0.0, 0.03, 0.3, 1.0)),     # s = 24, g = 4: 96-column groups, two H k-blocks, the second half full
+    ("bert", 1024, 2, 0, (0.2,)),                   # 48-column groups: one H k-block
+    ("bert", 333, 0, 464, (0.15,)),                 # d = 464: ragged last k-block of the up projection, ragged last output chunk
+    ("vit", 900, 0, 0, (0.05, 0.5)),                # s = 16, g = 8
+    ("vit", 600, 1, 0, (0.1,)),                     # one expert per group: 16-column groups
+    ("paper", 1500, 0, 0, (0.02, 0.4)),             # s = 128, g = 1
+    ("gpt2_attn", 520, 0, 0, (0.1,)),               # d_ff = 2 d: the accumulator fills the whole of H's place
+]
+
+
+@pytest.mark.parametrize("name,T,g,d,ps", FUSED_CASES)
+def test_fused_gathered_step_equals_oracle(api, name, T, g, d, ps):
+    """The fused kernel (up projection, activation, down projection and merge per group and tile of the tokens that
+    keep it; Listing 1 with the atomic merge of App. C) forced through d2d_layer_set_expert_path: y against the
+    oracle on the same mask, twice in a row (the counters reset themselves, the accumulator is re-filled), with the
+    workspace poisoned before each call."""
+    import dataclasses
+    cfg = wl.with_tokens(wl.CONFIGS[name], T)
+    if d:
+        cfg = dataclasses.replace(cfg, d=d)
+    w, x = wl.make_weights(cfg), wl.make_tokens(cfg)
+    layer = api.Layer.from_config(cfg, w)
+    layer.set_expert_path("fused", group=g)
+    path, gg, _ = layer.get_expert_path()
+    assert path == "fused" and gg >= 1 and gg * cfg.s <= 128 and (g == 0 or gg == g)
+    xd = api.to_device(x, cfg.dtype)
+    act = oracle.ACT_BY_NAME[cfg.act]
+    ws = layer.workspace(T)                                    # the buffer the binding passes to every call
+    for p in ps:
+        G = _structured_mask(cfg, T, p, seed=29) if 0.0 < p < 1.0 else np.full((T, cfg.E), int(p), np.uint8)
+        r = _routing(api, G, cfg.E)
+        y_ref = oracle.moe_ffn(x, w["w1"], w["b1"], w["w_gate"], w["w2"], w["b2"], act, G)
+        for rep in range(2):
+            ws.fill_(0xc1)                                     # float32 0xc1c1c1c1 = -24.2: a stale accumulator would show
+            y = torch.full((T, cfg.d), float("nan"), dtype=torch.bfloat16, device="cuda")
+            layer.moe_ffn_fwd(xd, r, y=y)
+            torch.cuda.synchronize()
+            assert r.status == 0
+            yg = y.float().cpu().numpy()
+            assert np.isfinite(yg).all()
+            assert _rel_err(yg, y_ref) <= TOL_Y, (name, p, rep, _rel_err(yg, y_ref))
+            assert _per_token_err(yg, y_ref) <= 4 * TOL_Y, (name, p, rep, _per_token_err(yg, y_ref))
+        # a token that keeps nothing gets b2 exactly (the accumulator's fill, converted)
+        if 0.0 < p < 1.0:
+            b2 = torch.from_numpy(np.asarray(w["b2"], np.float32)).to(torch.bfloat16).float().numpy() if w["b2"] is not None else 0.0
+            assert np.array_equal(yg[T // 3], np.broadcast_to(b2, (cfg.d,)))
+    # gated layers and groups of more than 128 neurons are refused
+    with pytest.raises(RuntimeError):
+        layer.set_expert_path("fused", group=64)
+    layer.close()
