@@ -156,6 +156,17 @@ D2D_API d2d_status d2d_layer_destroy(d2d_layer *layer);
  *                    and each group runs a contraction over the tokens that keep
  *                    one of its experts (the grouped form of Listing 1): time
  *                    proportional to the number of kept (token, group) pairs.
+ *   D2D_PATH_FUSED   (plain layers, groups of at most 128 neurons) one kernel per
+ *                    (group, tile of the tokens that keep it): up projection,
+ *                    activation, down projection with the group's columns of W2,
+ *                    and the partial outputs added to a float32 accumulator [T, d]
+ *                    with vector reductions (the atomic merge of App. C); the
+ *                    accumulator lives where H would in the workspace, is filled
+ *                    with b2 before and converted to y after.  H never exists and
+ *                    the whole step is proportional to the kept pairs; the merge
+ *                    bounds it, so it wins only at low densities.  The order of
+ *                    the float32 additions is not fixed: y may differ from run to
+ *                    run in the last bits.
  *   D2D_PATH_AUTO    (default) decided per call on the device from the number of
  *                    selected pairs of that batch: gathered when
  *                    n_sel <= rho_max * T * E, dense otherwise.  Both pairs of
@@ -170,9 +181,17 @@ D2D_API d2d_status d2d_layer_destroy(d2d_layer *layer);
  * gated layers).  rho_max: crossover density of D2D_PATH_AUTO, negative =
  * library default for the shape.  Returns D2D_ERR_UNSUPPORTED when the shape
  * cannot take the gathered path (fp32 layers, expert sizes that are not a
- * multiple of 8) and it, or a group, was asked for. */
+ * multiple of 8) and it, or a group, was asked for.
+ * With D2D_PATH_FUSED `group` sets the fused kernel's group (0 = the widest of
+ * at most 128 neurons) and rho_max is ignored.  Under D2D_PATH_AUTO the fused
+ * kernel is a third range below the gathered pair: it runs while
+ * n_sel <= fused_rho_max * T * E (d2d_layer_set_fused_rho_max: negative =
+ * library default for the shape, 0 = never; D2D_ERR_UNSUPPORTED for a positive
+ * value on a shape the fused kernel cannot take: gated, fp32, d_ff < 2 d,
+ * d < 128 or d > 4096). */
 typedef enum { D2D_PATH_AUTO = 0, D2D_PATH_DENSE = 1, D2D_PATH_GATHER = 2, D2D_PATH_FUSED = 3 } d2d_expert_path;
 D2D_API d2d_status d2d_layer_set_expert_path(d2d_layer *layer, d2d_expert_path path, int32_t group, double rho_max);
+D2D_API d2d_status d2d_layer_set_fused_rho_max(d2d_layer *layer, double rho_max);
 /* Current setting; any output pointer may be NULL.  *group is 0 when the shape
  * cannot take the gathered path. */
 D2D_API d2d_status d2d_layer_get_expert_path(const d2d_layer *layer, int32_t *path, int32_t *group, double *rho_max);

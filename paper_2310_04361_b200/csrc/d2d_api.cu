@@ -111,6 +111,16 @@ static double default_gather_rho_max(const d2d_layer_desc &D, int g)
     return 1.0 - pow(1.0 - u_max, 1.0 / g);
 }
 
+// Density up to which the fused gathered kernel beats both pairs.  Its merge moves 4 d bytes of vector reductions per
+// kept (token, group) pair through each SM's path to L2, next to the token and weight rows coming in, and its float32
+// accumulator is written once and read once more than the other paths' output: measured on B200 (d = 768, 128-neuron
+// groups, 50432 tokens) it wins while at most about 6% of the (token, group) pairs are kept.
+static double default_fused_rho_max(int g)
+{
+    if (g <= 0) return 0.0;
+    return 1.0 - pow(1.0 - 0.06, 1.0 / g);
+}
+
 // Expert step of bf16 batches above the decode sizes, on the tensor cores.
 //   up projection    two kernels that compute the same H = G * A(x W1^T + b1):
 //     masked dense   one GEMM over all of d_ff, the selection applied as a mask in the epilogue; its time does not
@@ -137,7 +147,7 @@ static d2d_status launch_tc_experts(const d2d_layer *L, const void *x, int T, co
     // that this is noise.  Below that the fixed costs of the gathered kernel leave it nothing to win anyway.
     const double up_flop = 2.0 * (double)T * D.d * D.d_ff * (D.gated ? 2.0 : 1.0);
     if (path == D2D_PATH_AUTO && (up_flop < 1e11 || !n_sel)) path = D2D_PATH_DENSE;
-    const long long n_sel_max = (long long)(L->gather_rho_max * (double)T * (double)D.n_experts);
+    long long n_sel_max = (long long)(L->gather_rho_max * (double)T * (double)D.n_experts);
     d2d_status rc;
     // Fused gathered step (plain layers): up projection, activation, down projection and the merge in one kernel whose
     // time is proportional to the kept (token, group) pairs; the float32 accumulator takes the place of H.
@@ -148,8 +158,9 @@ static d2d_status launch_tc_experts(const d2d_layer *L, const void *x, int T, co
         fa.T = T; fa.d = D.d; fa.d_ff = D.d_ff; fa.n_experts = D.n_experts; fa.s = D.expert_size; fa.g = L->fused_group;
         fa.act = D.act; fa.status = r->status; fa.ctr = L->gather_ctr;
         if (path == D2D_PATH_AUTO) {
+            // three ranges of n_sel: (.., fused] fused kernel, (fused, max] gathered pair, (max, ..) dense pair
             n_sel_fused = (long long)(L->fused_rho_max * (double)T * (double)D.n_experts);
-            if (n_sel_fused > n_sel_max) n_sel_fused = n_sel_max;
+            if (n_sel_max < n_sel_fused) n_sel_max = n_sel_fused;
             fa.n_sel = n_sel; fa.n_sel_min = -1; fa.n_sel_max = n_sel_fused;
         }
         rc = d2d_moe_gather_ffn(fa, (float *)ws, y, L->w2, L->b2, st);
@@ -263,7 +274,7 @@ d2d_status d2d_layer_create(const d2d_layer_desc *desc, const d2d_weights *w, vo
     L->gather_rho_max = default_gather_rho_max(D, L->gather_group);
     L->expert_path = D2D_PATH_AUTO;
     L->fused_group = d2d_gather_ffn_group_for(D);
-    L->fused_rho_max = 0.0;
+    L->fused_rho_max = default_fused_rho_max(L->fused_group);
     L->gather_ctr_words = D.n_experts + 64;               // enough for any group size: E / g counters + the exit ticket
     const size_t ctr_off = total;
     total += d2d_align_up((size_t)L->gather_ctr_words * sizeof(int), 256);
@@ -375,6 +386,14 @@ d2d_status d2d_layer_set_expert_path(d2d_layer *layer, d2d_expert_path path, int
     layer->gather_group = g;
     layer->expert_path = path;
     layer->gather_rho_max = rho_max >= 0.0 ? (rho_max > 1.0 ? 1.0 : rho_max) : default_gather_rho_max(layer->desc, g);
+    return D2D_OK;
+}
+
+d2d_status d2d_layer_set_fused_rho_max(d2d_layer *layer, double rho_max)
+{
+    if (!layer) return D2D_ERR_INVALID_ARG;
+    if (layer->fused_group <= 0) return rho_max > 0.0 ? D2D_ERR_UNSUPPORTED : D2D_OK;
+    layer->fused_rho_max = rho_max >= 0.0 ? (rho_max > 1.0 ? 1.0 : rho_max) : default_fused_rho_max(layer->fused_group);
     return D2D_OK;
 }
 

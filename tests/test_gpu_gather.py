@@ -166,8 +166,13 @@ def test_device_side_choice_at_full_size(api, name, tau):
     if name == "llama":
         sample = sample[:: 2]                                  # the oracle needs about 0.1 s per Llama-sized token
     ref = None
-    for rho_max in (0.0, 1.0):
+    # (crossover of the gathered pair, upper end of the fused kernel's range): dense pair, gathered pair, fused kernel,
+    # and the defaults
+    settings = [(0.0, 0.0), (1.0, 0.0), (-1.0, -1.0)] + ([] if cfg.gated else [(0.0, 1.0)])
+    for rho_max, fused_max in settings:
         layer.set_expert_path("auto", rho_max=rho_max)
+        if not cfg.gated:
+            layer.set_fused_rho_max(fused_max)
         r = layer.new_routing(T)
         y = torch.full((T, cfg.d), float("nan"), dtype=torch.bfloat16, device="cuda")
         for rep in range(2):
@@ -181,8 +186,12 @@ def test_device_side_choice_at_full_size(api, name, tau):
         assert np.array_equal(G, ref[0])
         yg = y.float().cpu().numpy()
         assert np.isfinite(yg).all()
-        assert _rel_err(yg[sample], ref[1]) <= TOL_Y, (rho_max, _rel_err(yg[sample], ref[1]))
+        assert _rel_err(yg[sample], ref[1]) <= TOL_Y, (rho_max, fused_max, _rel_err(yg[sample], ref[1]))
         assert _per_token_err(yg[sample], ref[1]) <= 4 * TOL_Y
+    if cfg.gated:                                              # the fused kernel takes plain layers only
+        with pytest.raises(api.D2DError) as e:
+            layer.set_fused_rho_max(0.5)
+        assert api.STATUS_NAMES[e.value.code] == "UNSUPPORTED"
     layer.close()
 
 
@@ -275,6 +284,6 @@ def test_fused_gathered_step_equals_oracle(api, name, T, g, d, ps):
             b2 = torch.from_numpy(np.asarray(w["b2"], np.float32)).to(torch.bfloat16).float().numpy() if w["b2"] is not None else 0.0
             assert np.array_equal(yg[T // 3], np.broadcast_to(b2, (cfg.d,)))
     # gated layers and groups of more than 128 neurons are refused
-    with pytest.raises(RuntimeError):
+    with pytest.raises(api.D2DError):
         layer.set_expert_path("fused", group=64)
     layer.close()
