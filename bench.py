@@ -8,7 +8,7 @@ neurons, 8192 tokens) at tau = 0.4; the other configurations are timed in the sa
 reported in `per_config` of the same JSON line.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload llama] [--tau 0.4]
-                    [--tokens T] [--bernoulli p] [--path auto|dense|gather] [--experts-per-group g]
+                    [--tokens T] [--bernoulli p] [--path auto|dense|gather|fused] [--experts-per-group g]
                     [--sweep] [--no-per-config] [--no-cpu-baseline] [--no-graph] [--group N]
     python bench.py --impl reference ...      # times the CPU oracle on the host cores
 
@@ -48,7 +48,8 @@ PER_CONFIG = [
     ("gpt2_ffn", 1, 0.5, None), ("gpt2_ffn", 8, 0.5, None), ("gpt2_ffn", 64, 0.5, None),
     ("gpt2_attn", 1, 0.5, None), ("gpt2_attn", 64, 0.5, None),
     ("llama", None, 0.6, None),
-    ("paper", None, None, 0.1), ("paper", None, None, 0.3), ("paper", None, None, 0.5),
+    ("paper", None, None, 0.02), ("paper", None, None, 0.05), ("paper", None, None, 0.1), ("paper", None, None, 0.3),
+    ("paper", None, None, 0.5),
 ]
 
 
@@ -64,7 +65,7 @@ def parse_args():
     p.add_argument("--bernoulli", type=float, default=None,
                    help="override the gating decisions with Bernoulli(p) samples (the latency protocol of Sec. 4.4): "
                         "the timed step is then the expert step d2d_moe_ffn_fwd on that mask")
-    p.add_argument("--path", default="auto", choices=["auto", "dense", "gather"],
+    p.add_argument("--path", default="auto", choices=["auto", "dense", "gather", "fused"],
                    help="which up projection the tensor-core expert step uses (d2d_layer_set_expert_path)")
     p.add_argument("--experts-per-group", type=int, default=0, help="group size of the gathered path (0 = default)")
     p.add_argument("--sweep", action="store_true", help="also time the workload's whole tau grid")
@@ -514,7 +515,7 @@ def run_ours(args):
             # themselves apply (n_sel against the layer's crossover); each is also timed on its own
             path, group, rho_max = layer.get_expert_path()
             up_flop = 2.0 * T * cfg.d * cfg.d_ff * (2 if cfg.gated else 1)
-            gathered = path == "gather" or (path == "auto" and group > 0 and up_flop >= 1e11 and n_sel <= rho_max * T * cfg.E)
+            gathered = path in ("gather", "fused") or (path == "auto" and group > 0 and up_flop >= 1e11 and n_sel <= rho_max * T * cfg.E)
             H = torch.empty((T, cfg.d_ff), dtype=torch.bfloat16, device=dev)
             t_up_dense = h.time(lambda: layer.expert_up_fwd(x, routing, H=H), sub)["median"]
             t_up_gather = h.time(lambda: layer.expert_up_gather_fwd(x, routing, H=H), sub)["median"] if group > 0 else None
@@ -539,6 +540,17 @@ def run_ours(args):
                         "kernel_ms": t_up, "up_dense_ms": t_up_dense, "up_gather_ms": t_up_gather, "down_dense_ms": t_down,
                         "down_masked_ms": t_down_masked, "expert_path": path, "experts_per_group": group, "rho_crossover": rho_max,
                         "expert_step_frac": f_experts / (t_ffn * 1e-3) / 1e12 / peaks["bf16_tflops"]}
+            fgroup, frho = layer.get_fused()
+            if path == "fused" or (path == "auto" and fgroup > 0 and up_flop >= 1e11 and n_sel <= frho * T * cfg.E):
+                group = fgroup
+                # one kernel does the whole expert step: its FLOPs are those of both projections over the kept pairs
+                gmask = oracle.unpack_mask(routing.mask_u32(), cfg.E).reshape(T, cfg.E // group, group).max(-1)
+                f_exec = 2.0 * cfg.n_mat * cfg.d * cfg.s * group * float(gmask.sum())
+                roofline.update({"kernel": "moe_gather_ffn_kernel (d2d_moe_ffn_fwd, fused path; includes the accumulator's fill and conversion)",
+                                 "achieved": f_experts / (t_ffn * 1e-3) / 1e12, "frac": f_experts / (t_ffn * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                                 "algorithmic_flops_per_launch": f_experts, "executed_flops_per_launch": f_exec,
+                                 "executed_frac": f_exec / (t_ffn * 1e-3) / 1e12 / peaks["bf16_tflops"], "kernel_ms": t_ffn,
+                                 "merge_bytes_per_launch": 4.0 * cfg.d * float(gmask.sum()), "traffic": None})
             del H
 
         dense = dense_comparators(h, api, torch, cfg, weights, layer, x, y, sub)

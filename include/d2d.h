@@ -192,6 +192,9 @@ D2D_API d2d_status d2d_layer_destroy(d2d_layer *layer);
 typedef enum { D2D_PATH_AUTO = 0, D2D_PATH_DENSE = 1, D2D_PATH_GATHER = 2, D2D_PATH_FUSED = 3 } d2d_expert_path;
 D2D_API d2d_status d2d_layer_set_expert_path(d2d_layer *layer, d2d_expert_path path, int32_t group, double rho_max);
 D2D_API d2d_status d2d_layer_set_fused_rho_max(d2d_layer *layer, double rho_max);
+/* The fused kernel's group (0: the shape cannot take it) and the upper end of
+ * its range under D2D_PATH_AUTO; either output pointer may be NULL. */
+D2D_API d2d_status d2d_layer_get_fused(const d2d_layer *layer, int32_t *group, double *rho_max);
 /* Current setting; any output pointer may be NULL.  *group is 0 when the shape
  * cannot take the gathered path. */
 D2D_API d2d_status d2d_layer_get_expert_path(const d2d_layer *layer, int32_t *path, int32_t *group, double *rho_max);

@@ -397,6 +397,14 @@ d2d_status d2d_layer_set_fused_rho_max(d2d_layer *layer, double rho_max)
     return D2D_OK;
 }
 
+d2d_status d2d_layer_get_fused(const d2d_layer *layer, int32_t *group, double *rho_max)
+{
+    if (!layer) return D2D_ERR_INVALID_ARG;
+    if (group) *group = layer->fused_group;
+    if (rho_max) *rho_max = layer->fused_rho_max;
+    return D2D_OK;
+}
+
 d2d_status d2d_layer_get_expert_path(const d2d_layer *layer, int32_t *path, int32_t *group, double *rho_max)
 {
     if (!layer) return D2D_ERR_INVALID_ARG;
