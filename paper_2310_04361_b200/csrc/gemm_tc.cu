@@ -655,19 +655,21 @@ d2d_status launch(const d2d_gemm_args &g, cudaStream_t st)
     return err == cudaSuccess && cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
 }
 
-// Tile width that wastes the fewest SM-rounds: tiles / (rounds * workers), wider tiles preferred on ties
-// (fewer re-reads of A, fewer per-tile overheads).
+// Tile width with the least modelled time: rounds over the SMs x the time of one 64-deep k-block of a 128 x bn tile.
+// That time is not proportional to bn: every k-block brings 16 KB of A and bn / 8 KB of B into the SM, and the SM's
+// path from L2 is what a 128-row tile saturates, so a narrow tile pays almost as much as a wide one for fewer columns.
+// Measured on B200 (K = 11008, T = 4096 and 8192): 0.40 us per k-block at bn = 256, 0.31 us at bn = 128, i.e. about
+// 0.13 us + 0.7 ns per row of A and B staged.  Wider tiles win ties.
 int pick_bn(int M, int N, int tile_m, int workers, const int *cands, int n_cands, int batch = 1)
 {
     int best = cands[0];
-    double best_eff = -1.0;
+    double best_cost = 1e300;
     for (int i = 0; i < n_cands; ++i) {
         const int bn = cands[i];
         const long tiles = (long)d2d_cdiv(N, bn) * d2d_cdiv(M, tile_m) * batch;
         const long rounds = (tiles + workers - 1) / workers;
-        const double useful = (double)N / ((double)d2d_cdiv(N, bn) * bn);       // ragged last column tile
-        const double eff = useful * (double)tiles / (double)(rounds * workers) * (bn >= 128 ? 1.0 : 0.85);
-        if (eff > best_eff + 1e-9) { best_eff = eff; best = bn; }
+        const double cost = (double)rounds * (0.13 + 0.0007 * (double)(tile_m + bn));
+        if (cost < best_cost - 1e-9) { best_cost = cost; best = bn; }
     }
     return best;
 }
