@@ -107,7 +107,10 @@ static double default_gather_rho_max(const d2d_layer_desc &D, int g)
 {
     if (g <= 0) return -1.0;
     const int n_mma = g * D.expert_size * (D.gated ? 2 : 1);
-    const double u_max = n_mma >= 256 ? 0.60 : n_mma >= 192 ? 0.30 : n_mma >= 128 ? 0.25 : 0.15;
+    double u_max = n_mma >= 256 ? 0.60 : n_mma >= 192 ? 0.30 : n_mma >= 128 ? 0.25 : 0.15;
+    // wide layers keep the TMA-fed dense down projection behind the gathered kernel (unkept cells of H zero-filled)
+    // instead of the slower selection-applying one: measured on the Llama shape, the gathered pair wins up to u = 0.7
+    if (D.d >= 2048) u_max += 0.10;
     return 1.0 - pow(1.0 - u_max, 1.0 / g);
 }
 
@@ -180,25 +183,33 @@ static d2d_status launch_tc_experts(const d2d_layer *L, const void *x, int T, co
         rc = d2d_gemm_tc(up, st);
         if (rc != D2D_OK) return rc;
     }
+    // Wide layers: the cells the gathered kernel leaves alone are zero-filled, so that the TMA-fed dense down projection
+    // can follow whichever up projection ran; otherwise the down projection that applies the selection while it stages
+    // H follows the gathered kernel.
+    const bool zero_fill = path != D2D_PATH_DENSE && D.d >= 2048;
     if (path != D2D_PATH_DENSE) {
+        const long long hi = path == D2D_PATH_AUTO ? n_sel_max : LLONG_MAX;
+        if (zero_fill) {
+            rc = d2d_moe_zero_unkept(ws, r->mask, T, D.d_ff, D.n_experts, D.expert_size, L->gather_group, n_sel, n_sel_fused, hi, st);
+            if (rc != D2D_OK) return rc;
+        }
         d2d_gather_args ga = {};
         ga.x = x; ga.w1 = L->w1; ga.w_gate = D.gated ? L->w_gate : nullptr; ga.b1 = L->b1; ga.mask = r->mask; ga.H = ws;
         ga.T = T; ga.d = D.d; ga.d_ff = D.d_ff; ga.n_experts = D.n_experts; ga.s = D.expert_size; ga.g = L->gather_group;
         ga.act = D.act; ga.status = r->status; ga.ctr = L->gather_ctr;
-        ga.n_sel = n_sel; ga.n_sel_min = n_sel_fused; ga.n_sel_max = path == D2D_PATH_AUTO ? n_sel_max : LLONG_MAX;
+        ga.n_sel = n_sel; ga.n_sel_min = n_sel_fused; ga.n_sel_max = hi;
         rc = d2d_moe_gather_up(ga, st);
         if (rc != D2D_OK) return rc;
     }
-    // The gathered kernel writes only the kept cells of H, so whenever it may have run the down projection is the one
-    // that applies the selection while it stages H (it is valid after the masked dense up projection as well).
-    // With the automatic choice both down projections are enqueued as well, each with the rule of its up projection.
-    if (path != D2D_PATH_DENSE) {
+    if (path != D2D_PATH_DENSE && !zero_fill) {
         rc = d2d_moe_down_masked(D, ws, r->mask, L->w2, L->b2, y, T, r->status, st, path == D2D_PATH_AUTO ? n_sel : nullptr, n_sel_fused, n_sel_max);
         if (rc != D2D_OK || path == D2D_PATH_GATHER) return rc;
     }
     d2d_gemm_args dn = {};
     dn.a = ws; dn.b = L->w2; dn.bias = L->b2; dn.out = y;
-    dn.n_sel = path == D2D_PATH_AUTO ? n_sel : nullptr; dn.n_sel_max = n_sel_max;
+    // after a zero fill this kernel serves the gathered range too: it only has to stay out of the fused kernel's range
+    dn.n_sel = path == D2D_PATH_AUTO && (!zero_fill || n_sel_fused >= 0) ? n_sel : nullptr;
+    dn.n_sel_max = zero_fill ? n_sel_fused : n_sel_max;
     dn.M = T; dn.N = D.d; dn.K = D.d_ff; dn.epilogue = D2D_EPI_BIAS_BF16; dn.status = r->status;
     // decode-sized batches: split K over the SMs, partial sums in the float32 scratch behind H
     dn.k_splits = d2d_gemm_tc_splits(T, D.d, D.d_ff);

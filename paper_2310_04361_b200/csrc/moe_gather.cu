@@ -1165,6 +1165,57 @@ d2d_status d2d_moe_down_masked(const d2d_layer_desc &D, const void *H, const uin
     return err == cudaSuccess && cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
 }
 
+// Zero for the cells of H that the gathered up projection leaves alone: (token, group) pairs without a kept expert.
+// With them H is fully defined and the plain TMA-fed dense down projection can follow (10-20 % faster than the one
+// that applies the selection while it stages H); the price is (1 - u) T d_ff 2 bytes of stores at memory bandwidth,
+// which pays for wide layers (the down projection's time grows with d, the fill's does not).
+// One thread per 16-byte chunk: consecutive lanes write consecutive chunks of a token's row.
+__global__ void __launch_bounds__(256)
+h_zero_unkept_kernel(__nv_bfloat16 *__restrict__ H, const uint32_t *__restrict__ mask, int T, int W, int d_ff, int g, uint32_t inv_gs,
+                     const int32_t *n_sel, long long n_sel_min, long long n_sel_max)
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (n_sel) {
+        const long long n = (long long)__ldcg(n_sel);
+        if (!(n > n_sel_min && n <= n_sel_max)) return;
+    }
+    const int chunks = d_ff >> 3;
+    const uint32_t gm = g >= 32 ? 0xffffffffu : (1u << g) - 1u;
+    const long long total = (long long)T * chunks;
+    for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < total; i += (long long)gridDim.x * 256) {
+        const int t = (int)(i / chunks), c = (int)(i - (long long)t * chunks);
+        const int e0 = (int)__umulhi((uint32_t)(c * 8), inv_gs) * g;              // first expert of the chunk's group
+        const uint32_t bits = (__ldg(mask + (size_t)t * W + (e0 >> 5)) >> (e0 & 31)) & gm;
+        if (bits == 0u) *reinterpret_cast<uint4 *>(H + (size_t)t * d_ff + (size_t)c * 8) = make_uint4(0u, 0u, 0u, 0u);
+    }
+}
+
+d2d_status d2d_moe_zero_unkept(void *H, const uint32_t *mask, int T, int d_ff, int n_experts, int s, int g, const int32_t *n_sel,
+                               long long n_sel_min, long long n_sel_max, cudaStream_t st)
+{
+    if (T <= 0) return D2D_OK;
+    const int gs = g * s;
+    if (g < 1 || g > 32 || 32 % g || n_experts % g || gs % 8 || d_ff % 8) return D2D_ERR_UNSUPPORTED;
+    const uint32_t inv_gs = (uint32_t)((0x100000000ull + (unsigned long long)gs - 1) / (unsigned long long)gs);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = d2d_tc_pdl_enabled() ? 1 : 0;
+    const long long total = (long long)T * (d_ff / 8);
+    const long long blocks = (total + 255) / 256;
+    const int cap = 16 * d2d_tc_sm_count();
+    cfg.gridDim = dim3((unsigned)(blocks < cap ? blocks : cap), 1, 1);
+    cfg.blockDim = dim3(256, 1, 1);
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, h_zero_unkept_kernel, (__nv_bfloat16 *)H, mask, T, (n_experts + 31) / 32, d_ff, g, inv_gs,
+                                               n_sel, n_sel_min, n_sel_max);
+    D2D_LAUNCHED(1);
+    return err == cudaSuccess && cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
+}
+
 int d2d_gather_ffn_group_for(const d2d_layer_desc &D)
 {
     // the float32 accumulator [T, d] takes the place of H [T, d_ff] bf16 in the caller's workspace

@@ -49,3 +49,8 @@ d2d_status d2d_moe_down_masked(const d2d_layer_desc &D, const void *H, const uin
 // following the dispatch rule in `a`.
 int d2d_gather_ffn_group_for(const d2d_layer_desc &D);
 d2d_status d2d_moe_gather_ffn(const d2d_gather_args &a, float *y32, void *y, const void *w2, const void *b2, cudaStream_t st);
+
+// Writes zero to the cells of H [T, d_ff] bf16 of (token, group) pairs without a kept expert: what the gathered up
+// projection (groups of g experts) does not write.  Afterwards H is fully defined.  Follows the dispatch rule.
+d2d_status d2d_moe_zero_unkept(void *H, const uint32_t *mask, int T, int d_ff, int n_experts, int s, int g, const int32_t *n_sel,
+                               long long n_sel_min, long long n_sel_max, cudaStream_t st);
