@@ -604,6 +604,10 @@ d2d_status d2d_layer_fwd(const d2d_layer *layer, const void *x, int32_t T, float
         }
         if (!lists) return D2D_ERR_INVALID_ARG;               // the expert kernels of this shape walk the per-expert lists
         rc = d2d_launch_select(nullptr, T, E, tau, 0, routing, base + w.sel_off, st, 1);
+    } else if (T > 8 && d2d_layer_token_fused_supports(layer->desc, T, lists)) {
+        // small float32 problems: router, rule, experts and lists in one launch
+        if (cudaMemsetAsync(routing->status, 0, sizeof(int32_t), st) != cudaSuccess) return D2D_ERR_CUDA;
+        return d2d_layer_token_fused(layer, x, T, tau, y, R_out, routing, lists, layer->tickets + 52, st);
     } else if (!lists) {
         return D2D_ERR_INVALID_ARG;                           // every other path builds (and its expert kernels use) the lists
     } else if (d2d_small_router_supports(layer->desc, T)) {

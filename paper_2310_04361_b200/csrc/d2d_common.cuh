@@ -33,7 +33,8 @@ struct d2d_layer {
     // layer-owned "last CTA" tickets of the decode kernels used by d2d_layer_fwd (zero at creation, reset by the kernel
     // that used them): word 0 decode router, word 16 decode experts, word 32 tile counter of the up projection, words
     // 40 / 41 sum of k and exit ticket of the fused router, word 44 the number of selected pairs the fused router
-    // publishes for the density-adaptive dispatch of the expert step.  Like the side stream, they make concurrent
+    // publishes for the density-adaptive dispatch of the expert step, word 52 exit ticket of the one-launch layer
+    // kernel of small float32 problems.  Like the side stream, they make concurrent
     // d2d_layer_fwd calls on ONE layer object from several streams unsafe; use one layer object per stream for that.
     // A call that ended in D2D_ERR_TIMEOUT may leave them non-zero: d2d_layer_reset_counters clears them.
     unsigned int *tickets;
@@ -101,6 +102,12 @@ d2d_status d2d_launch_moe_ffn(const d2d_layer *L, const void *x, int T, const d2
                               void *ws, size_t ws_bytes, cudaStream_t st, int *up_counter = nullptr, int small_fused = 0,
                               const int32_t *n_sel = nullptr);
 size_t d2d_moe_ffn_ws_bytes(const d2d_layer *L, int T);
+
+// layer_token_fused.cu: the whole layer of a small float32 problem in one launch (router, rule, experts, lists).
+// ticket: a zeroed layer-owned word (left at zero).  The status word must be zero (or hold an earlier error) at launch.
+bool d2d_layer_token_fused_supports(const d2d_layer_desc &D, int T, bool lists);
+d2d_status d2d_layer_token_fused(const d2d_layer *L, const void *x, int T, float tau, void *y, float *R_out, const d2d_routing *r,
+                                 bool lists, unsigned int *ticket, cudaStream_t st);
 
 // small-batch (T <= 64) kernels
 bool d2d_small_select_supports(int T, int E);

@@ -1,0 +1,224 @@
+// The whole layer of a SMALL problem in one launch (Sec. 3.2-3.4): router, dynamic-k rule, kept experts, combine.
+//
+// One CTA per token.  The token row sits in shared memory as float32; the warps compute the router's hidden units
+// (one warp per unit: a d-long dot product reduced by shuffles, bias + ReLU), then the expert scores (one warp per
+// expert, absolute value, Sec. 3.3), warp 0 takes the row maximum, the threshold tau * max as ONE float32 product and
+// the mask words (Eq. 4), and the CTA then runs the token's kept experts exactly like the token-major expert kernel
+// (moe_ffn_token.cu): a fixed summation order, no atomics, y written once with b2 added once.  When the caller wants
+// the per-expert lists (Listing 1), the CTA that finishes last (a ticket) builds them from the mask words of all
+// tokens with the single-CTA selection routine, so that no further launch follows.
+//
+// This is the path of float32 layers whose whole forward pass is a few MFLOP: there the chain of separate router,
+// selection and expert kernels (eight launches) is nothing but launch latency.  Arithmetic is exact float32 FMA.
+#include "d2d_common.cuh"
+#include "small_select.cuh"
+
+namespace {
+
+constexpr int NT = 256;
+constexpr int NWARP = NT / 32;
+constexpr int MAX_S = 128;          // largest expert size staged in shared memory
+constexpr int MAX_COLS = 16;        // output columns per thread: d <= NT * MAX_COLS
+
+struct FusedArgs {
+    const void *x, *w_r1, *b_r1, *w_r2, *b_r2, *w1, *b1, *w_gate, *w2t, *b2;
+    void *y;
+    float *R_out;                   // [T, E] or NULL
+    d2d_routing r;                  // mask, k, status required; lists optional as a set
+    unsigned int *ticket;           // zero at launch, left at zero
+    int T, d, d_h, E, s, W, lists;
+    float tau;
+};
+
+template <typename T, int ACT, bool GATED>
+__global__ void __launch_bounds__(NT)
+layer_token_fused_kernel(const FusedArgs a)
+{
+    extern __shared__ float smem[];
+    float *xs = smem;                                   // [d]
+    float *us = xs + a.d;                               // [d_h]
+    float *Rs = us + a.d_h;                             // [E]
+    float *hs = Rs + a.E;                               // [2][MAX_S]
+    uint32_t *words = reinterpret_cast<uint32_t *>(hs + 2 * MAX_S);      // [W] this token's mask words
+    uint32_t *smask = words + a.W;                      // [T * W] all tokens' words (last CTA, lists only)
+    __shared__ int is_last;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int t = blockIdx.x, d = a.d, s = a.s;
+    const T *x = (const T *)a.x;
+
+    for (int c = tid; c < d; c += NT) xs[c] = d2d_to_float<T>(x[(size_t)t * d + c]);
+    __syncthreads();
+    // ---- router hidden layer: u = ReLU(W_r1 x + b_r1)
+    for (int j = warp; j < a.d_h; j += NWARP) {
+        const T *row = (const T *)a.w_r1 + (size_t)j * d;
+        float v = 0.0f;
+        for (int c = lane * 8; c < d; c += 256) {
+            float wv[8];
+            d2d_load8(row + c, wv);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v = fmaf(wv[i], xs[c + i], v);
+        }
+        v = d2d_warp_sum(v);
+        if (lane == 0) us[j] = fmaxf(v + (a.b_r1 ? d2d_to_float<T>(((const T *)a.b_r1)[j]) : 0.0f), 0.0f);
+    }
+    __syncthreads();
+    // ---- router output layer: R = |W_r2 u + b_r2|
+    for (int e = warp; e < a.E; e += NWARP) {
+        const T *row = (const T *)a.w_r2 + (size_t)e * a.d_h;
+        float v = 0.0f;
+        for (int c = lane * 8; c < a.d_h; c += 256) {
+            float wv[8];
+            d2d_load8(row + c, wv);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v = fmaf(wv[i], us[c + i], v);
+        }
+        v = d2d_warp_sum(v);
+        if (lane == 0) Rs[e] = fabsf(v + (a.b_r2 ? d2d_to_float<T>(((const T *)a.b_r2)[e]) : 0.0f));
+    }
+    __syncthreads();
+    // ---- dynamic-k rule (Eq. 4): keep expert i iff R_i >= tau * max_j R_j, the product rounded once to float32
+    if (warp == 0) {
+        float m = -INFINITY;
+        bool bad = false;
+        for (int i = lane; i < a.E; i += 32) {
+            const float v = Rs[i];
+            bad |= !d2d_small::finite_f32(v);
+            m = v > m ? v : m;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float other = __shfl_xor_sync(0xffffffffu, m, o);
+            m = other > m ? other : m;
+        }
+        bad = __any_sync(0xffffffffu, bad);
+        const float thr = __fmul_rn(a.tau, m);
+        int kt = 0;
+        for (int w = 0; w < a.W; ++w) {
+            const int i = w * 32 + lane;
+            const bool keep = i < a.E && (bad || Rs[i] >= thr);
+            const uint32_t word = __ballot_sync(0xffffffffu, keep);
+            if (lane == 0) {
+                words[w] = word;
+                a.r.mask[(size_t)t * a.W + w] = word;
+            }
+            kt += __popc(word);
+        }
+        if (lane == 0) {
+            a.r.k[t] = kt;
+            if (bad) atomicMax(a.r.status, (int32_t)D2D_ERR_NONFINITE);
+        }
+    } else if (a.R_out) {
+        for (int i = tid - 32; i < a.E; i += NT - 32) a.R_out[(size_t)t * a.E + i] = Rs[i];
+    }
+    __syncthreads();
+    // ---- kept experts: up projection + activation (one warp per neuron), down projection (columns per thread)
+    float acc[MAX_COLS];
+#pragma unroll
+    for (int i = 0; i < MAX_COLS; ++i) acc[i] = 0.0f;
+    int buf = 0;
+    for (int w = 0; w < a.W; ++w) {
+        uint32_t word = words[w];
+        while (word) {
+            const int e = w * 32 + __ffs(word) - 1;
+            word &= word - 1;
+            float *h = hs + buf * MAX_S;
+            for (int nl = warp; nl < s; nl += NWARP) {
+                const size_t n = (size_t)e * s + nl;
+                const T *wrow = (const T *)a.w1 + n * d;
+                const T *grow = GATED ? (const T *)a.w_gate + n * d : nullptr;
+                float up = 0.0f, gate = 0.0f;
+                for (int c = lane * 8; c < d; c += 256) {
+                    float wv[8];
+                    d2d_load8(wrow + c, wv);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) up = fmaf(wv[i], xs[c + i], up);
+                    if (GATED) {
+                        d2d_load8(grow + c, wv);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) gate = fmaf(wv[i], xs[c + i], gate);
+                    }
+                }
+                up = d2d_warp_sum(up);
+                if (GATED) gate = d2d_warp_sum(gate);
+                if (lane == 0) {
+                    if (a.b1) up += d2d_to_float<T>(((const T *)a.b1)[n]);
+                    h[nl] = GATED ? d2d_activate<ACT>(gate) * up : d2d_activate<ACT>(up);
+                }
+            }
+            __syncthreads();
+            for (int nl = 0; nl < s; ++nl) {
+                const float hv = h[nl];
+                const T *row = (const T *)a.w2t + ((size_t)e * s + nl) * d;
+#pragma unroll
+                for (int i = 0; i < MAX_COLS; ++i) {
+                    const int c = tid + NT * i;
+                    if (c < d) acc[i] = fmaf(hv, d2d_to_float<T>(__ldg(row + c)), acc[i]);
+                }
+            }
+            buf ^= 1;              // the next expert writes the other buffer: one barrier per expert
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < MAX_COLS; ++i) {
+        const int c = tid + NT * i;
+        if (c < d) ((T *)a.y)[(size_t)t * d + c] = d2d_from_float<T>(acc[i] + (a.b2 ? d2d_to_float<T>(((const T *)a.b2)[c]) : 0.0f));
+    }
+    if (!a.lists) return;
+    // ---- per-expert lists: the CTA that finishes last builds them from everybody's mask words
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const unsigned int done = atomicAdd(a.ticket, 1u);
+        is_last = done == gridDim.x - 1;
+        if (is_last) *a.ticket = 0u;
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    d2d_small::select_cta(nullptr, a.T, a.E, a.W, a.tau, a.r.mask, a.r.k, a.r.counts, a.r.offsets, a.r.perm, a.r.tok_off, a.r.tok_exp,
+                          a.r.n_sel, a.r.status, a.r.perm_capacity, 1, smask);
+}
+
+template <typename T, int ACT>
+d2d_status launch_act(const FusedArgs &a, bool gated, size_t smem, cudaStream_t st)
+{
+    if (gated)
+        layer_token_fused_kernel<T, ACT, true><<<a.T, NT, smem, st>>>(a);
+    else
+        layer_token_fused_kernel<T, ACT, false><<<a.T, NT, smem, st>>>(a);
+    D2D_LAUNCHED(1);
+    return cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
+}
+
+}  // namespace
+
+// Small float32 problems only: the router's weights are read once per token out of L2 here, which is fine for a few
+// hundred KB and wasteful beyond.
+bool d2d_layer_token_fused_supports(const d2d_layer_desc &D, int T, bool lists)
+{
+    const int W = (D.n_experts + 31) / 32;
+    if (D.dtype != D2D_F32 || T < 1 || D.d > NT * MAX_COLS || D.expert_size > MAX_S || D.d % 8 || D.d_h % 8) return false;
+    if ((size_t)D.d * D.d_h + (size_t)D.d_h * D.n_experts > 65536) return false;
+    if (lists && (T > d2d_small::MAX_T || (size_t)T * W * 4 > 24 * 1024)) return false;
+    return (size_t)(D.d + D.d_h + D.n_experts + 2 * MAX_S + W) * 4 + (size_t)T * W * 4 <= 44 * 1024;
+}
+
+d2d_status d2d_layer_token_fused(const d2d_layer *L, const void *x, int T, float tau, void *y, float *R_out, const d2d_routing *r,
+                                 bool lists, unsigned int *ticket, cudaStream_t st)
+{
+    const d2d_layer_desc &D = L->desc;
+    FusedArgs a = {};
+    a.x = x; a.w_r1 = L->w_r1; a.b_r1 = L->b_r1; a.w_r2 = L->w_r2; a.b_r2 = L->b_r2;
+    a.w1 = L->w1; a.b1 = L->b1; a.w_gate = L->w_gate; a.w2t = L->w2t; a.b2 = L->b2;
+    a.y = y; a.R_out = R_out; a.r = *r; a.ticket = ticket;
+    a.T = T; a.d = D.d; a.d_h = D.d_h; a.E = D.n_experts; a.s = D.expert_size; a.W = (D.n_experts + 31) / 32; a.lists = lists ? 1 : 0;
+    a.tau = tau;
+    const size_t smem = (size_t)(D.d + D.d_h + D.n_experts + 2 * MAX_S + a.W) * 4 + (lists ? (size_t)T * a.W * 4 : 0);
+    switch (D.act) {
+    case D2D_ACT_RELU: return launch_act<float, D2D_ACT_RELU>(a, D.gated != 0, smem, st);
+    case D2D_ACT_GELU_ERF: return launch_act<float, D2D_ACT_GELU_ERF>(a, D.gated != 0, smem, st);
+    case D2D_ACT_GELU_TANH: return launch_act<float, D2D_ACT_GELU_TANH>(a, D.gated != 0, smem, st);
+    case D2D_ACT_SILU: return launch_act<float, D2D_ACT_SILU>(a, D.gated != 0, smem, st);
+    }
+    return D2D_ERR_INVALID_ARG;
+}

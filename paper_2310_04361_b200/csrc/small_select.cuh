@@ -1,4 +1,4 @@
-// Selection for a small batch (T <= 64) done by ONE CTA: row max, threshold, mask words, k, per-expert counts,
+// Selection for a small batch (T <= MAX_T; the stand-alone kernel takes up to 64 tokens) done by ONE CTA: row max, threshold, mask words, k, per-expert counts,
 // offsets, token lists and the token-major dual.  Shared by the stand-alone selection kernel and by the
 // small-batch router kernel, whose last CTA selects right after it has written the scores (one launch less
 // on the decode path).  Dynamic-k rule: Sec. 3.4, Eq. 4 (keep expert i of token t when R[t,i] >= tau * max_j R[t,j]).
@@ -9,6 +9,7 @@
 namespace d2d_small {
 
 constexpr unsigned FULL = 0xffffffffu;
+constexpr int MAX_T = 256;          // tokens select_cta can take (per-token k staged in shared memory)
 
 __device__ __forceinline__ bool finite_f32(float v) { return (__float_as_uint(v) & 0x7f800000u) != 0x7f800000u; }
 
@@ -22,7 +23,7 @@ __device__ __forceinline__ void select_cta(const float *R, int T, int E, int W, 
 {
     __shared__ int warp_sums[32];
     __shared__ int chunk_total;
-    __shared__ int sk[64];
+    __shared__ int sk[MAX_T];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int nthreads = blockDim.x, nwarps = nthreads >> 5;
     if (threadIdx.x == 0 && !keep_status) *status = 0;
@@ -114,9 +115,8 @@ __device__ __forceinline__ void select_cta(const float *R, int T, int E, int W, 
         *n_sel = carry;
         if ((long long)carry > capacity) atomicMax(status, (int32_t)D2D_ERR_CAPACITY);
     }
-    // token-major dual: T <= 64, one thread per token
-    if (tok_off && tok_exp && threadIdx.x < T) {
-        const int t = threadIdx.x;
+    // token-major dual: one thread per token
+    for (int t = threadIdx.x; tok_off && tok_exp && t < T; t += nthreads) {
         long long base = 0;
         for (int u = 0; u < t; ++u) base += sk[u];
         tok_off[t] = (int32_t)base;

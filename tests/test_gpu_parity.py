@@ -621,3 +621,45 @@ def test_argument_errors(api):
     rc = api._lib.d2d_layer_fwd(layer.handle, api._ptr(xd), x.shape[0], ctypes.c_float(0.5), api._ptr(torch.empty_like(xd)),
                                 None, ctypes.byref(r.struct), api._ptr(small), small.numel(), api._stream())
     assert rc == 3
+
+
+SMALL_F32_CASES = [(9, "relu", False, True), (128, "relu", False, True), (256, "gelu_erf", False, True), (100, "silu", True, True),
+                   (300, "gelu_tanh", False, False), (77, "relu", False, False)]
+
+
+@pytest.mark.parametrize("T,act,gated,lists", SMALL_F32_CASES)
+def test_small_fp32_layer_runs_in_one_launch(api, T, act, gated, lists):
+    """Small float32 problems: router, dynamic-k rule (Eq. 4), kept experts and the per-expert lists (Listing 1) come
+    out of ONE kernel launch.  Everything is compared with the oracle: scores, the rule applied to the library's own
+    scores, k, the lists derived from the library's mask, and y on that mask; with every activation and the gated form."""
+    import dataclasses
+    cfg = dataclasses.replace(wl.with_tokens(wl.CONFIGS["tiny"], T), act=act, gated=gated)
+    w, x = wl.make_weights(cfg), wl.make_tokens(cfg)
+    layer = api.Layer.from_config(cfg, w)
+    xd = api.to_device(x, cfg.dtype)
+    tau = 0.5
+    ref = oracle.layer(x, w, oracle.ACT_BY_NAME[cfg.act], tau)
+    for rep in range(2):                                       # twice: the exit ticket resets itself
+        r = layer.new_routing(T, lists=lists)
+        R_out = _poison(torch.empty((T, cfg.E), dtype=torch.float32, device="cuda"))
+        y = _poison(torch.empty((T, cfg.d), dtype=torch.float32, device="cuda"))
+        torch.cuda.synchronize()
+        l0 = api.launch_count()
+        layer.layer_fwd(xd, tau, y=y, R_out=R_out, routing=r)
+        assert api.launch_count() - l0 == 1
+        torch.cuda.synchronize()
+        assert r.status == 0
+        R = R_out.cpu().numpy()
+        assert _rel_err(R, ref["R"]) <= TOL_R["f32"]
+        G = oracle.unpack_mask(r.mask_u32(), cfg.E)
+        G_self, k_self, _ = oracle.select(R, tau)
+        assert np.array_equal(G, G_self) and np.array_equal(r.k[:T].cpu().numpy(), k_self)
+        if lists:
+            meta = oracle.metadata(G)
+            assert r.n_sel == meta["n_sel"]
+            assert np.array_equal(r.counts.cpu().numpy(), meta["counts"])
+            assert np.array_equal(r.offsets.cpu().numpy(), meta["offsets"])
+            assert np.array_equal(r.perm[: meta["n_sel"]].cpu().numpy(), meta["perm"])
+        y_self = oracle.moe_ffn(x, w["w1"], w["b1"], w["w_gate"], w["w2"], w["b2"], oracle.ACT_BY_NAME[cfg.act], G)
+        assert _rel_err(y.cpu().numpy(), y_self) <= TOL_Y["f32"]
+    layer.close()
