@@ -65,6 +65,7 @@ struct GatherParams {
     int stages, stage_bytes;
     int window;                      // groups the CTAs work in at the same time (their weight rows stay in L2)
     int sub;                         // tokens per scheduler draw
+    float visit_tiles;               // full tiles a group visit should yield when the density allows it
 };
 
 struct TileDesc {
@@ -128,7 +129,7 @@ __device__ __forceinline__ void run_scheduler(const GatherParams &p, uint32_t *f
     if (p.n_sel) {
         const float rho = fminf((float)__ldcg(p.n_sel) / ((float)p.T * (float)(Ng * p.g)), 1.0f);
         const float u = fmaxf(1.0f - __expf((float)p.g * log1pf(-fminf(rho, 0.999f))), 1e-6f);
-        const float need = 8.0f * (float)BM * (float)gridDim.x / (u * (float)p.T);
+        const float need = p.visit_tiles * (float)BM * (float)gridDim.x / (u * (float)p.T);
         const int w = need >= (float)Ng ? Ng : (int)need;
         Wn = w > Wn ? w : Wn;
     }
@@ -1041,6 +1042,7 @@ d2d_status launch(const d2d_gather_args &a, cudaStream_t st)
     long long window = (48ll << 20) / (group_bytes > 0 ? group_bytes : 1);
     p.window = (int)(window < 4 ? 4 : window > p.n_groups ? p.n_groups : window);
     if (p.window > p.n_groups) p.window = p.n_groups;
+    p.visit_tiles = 8.0f;
     // tokens per draw: about eight draws per CTA (the CTAs then finish together), 256 .. 1024
     const long long want = (long long)a.T * p.n_groups / (8ll * d2d_tc_sm_count());
     p.sub = want >= 1024 ? 1024 : want >= 512 ? 512 : 256;
@@ -1252,6 +1254,7 @@ static d2d_status launch_ffn(const d2d_gather_args &a, float *y32, void *y, cons
     long long window = (48ll << 20) / (group_bytes > 0 ? group_bytes : 1);
     p.window = (int)(window < 4 ? 4 : window > p.n_groups ? p.n_groups : window);
     if (p.window > p.n_groups) p.window = p.n_groups;
+    p.visit_tiles = 8.0f;
     const long long want = (long long)a.T * p.n_groups / (8ll * d2d_tc_sm_count());
     p.sub = want >= 1024 ? 1024 : want >= 512 ? 512 : 256;
     CUtensorMap tw1, tw2;
