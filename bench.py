@@ -448,7 +448,7 @@ def measure_config(h, api, torch, wl, name, tokens, tau, bern, steps, peaks, pat
            "k": k_histogram(torch, routing, T, cfg.E),
            "step": "d2d_moe_ffn_fwd on the override mask" if bern is not None else "d2d_layer_fwd",
            "ms_median": t["median"], "ms_min": t["min"], "tokens_per_s": T / (t["median"] * 1e-3),
-           "expert_step_ms": t_ffn, "launches_per_step": launches, "expert_path": layer.get_expert_path()[0] if cfg.dtype == "bf16" else "fp32",
+           "expert_step_ms": t_ffn, "launches_per_step": launches, "expert_path": (layer.expert_path_for(T, n_sel) if T > 4 else "decode kernels") if cfg.dtype == "bf16" else "fp32",
            "dense": dense, "speedup_vs_torch_dense": dense["speedup"],
            "speedup_vs_library_dense": dense["speedup_vs_library_dense"], "roofline": roof}
     layer.close()
@@ -549,8 +549,8 @@ def run_ours(args):
             # dominant kernel = the expert up projection; which of its two forms the step ran is the rule the kernels
             # themselves apply (n_sel against the layer's crossover); each is also timed on its own
             path, group, rho_max = layer.get_expert_path()
-            up_flop = 2.0 * T * cfg.d * cfg.d_ff * (2 if cfg.gated else 1)
-            gathered = path in ("gather", "fused") or (path == "auto" and group > 0 and up_flop >= 1e11 and n_sel <= rho_max * T * cfg.E)
+            taken = layer.expert_path_for(T, n_sel)            # the rule the kernels evaluate on the device
+            gathered = taken in ("gather", "fused")
             H = torch.empty((T, cfg.d_ff), dtype=torch.bfloat16, device=dev)
             t_up_dense = h.time(lambda: layer.expert_up_fwd(x, routing, H=H), sub)["median"]
             t_up_gather = h.time(lambda: layer.expert_up_gather_fwd(x, routing, H=H), sub)["median"] if group > 0 else None
@@ -573,10 +573,10 @@ def run_ours(args):
                         "executed_flops_per_launch": f_up_exec,
                         "executed_frac": f_up_exec / (t_up * 1e-3) / 1e12 / peaks["bf16_tflops"],
                         "kernel_ms": t_up, "up_dense_ms": t_up_dense, "up_gather_ms": t_up_gather, "down_dense_ms": t_down,
-                        "down_masked_ms": t_down_masked, "expert_path": path, "experts_per_group": group, "rho_crossover": rho_max,
+                        "down_masked_ms": t_down_masked, "expert_path": path, "path_taken": taken, "experts_per_group": group,
                         "expert_step_frac": f_experts / (t_ffn * 1e-3) / 1e12 / peaks["bf16_tflops"]}
             fgroup, frho = layer.get_fused()
-            if path == "fused" or (path == "auto" and fgroup > 0 and up_flop >= 1e11 and n_sel <= frho * T * cfg.E):
+            if taken == "fused":
                 group = fgroup
                 # one kernel does the whole expert step: its FLOPs are those of both projections over the kept pairs
                 gmask = oracle.unpack_mask(routing.mask_u32(), cfg.E).reshape(T, cfg.E // group, group).max(-1)

@@ -196,8 +196,15 @@ D2D_API d2d_status d2d_layer_set_fused_rho_max(d2d_layer *layer, double rho_max)
  * its range under D2D_PATH_AUTO; either output pointer may be NULL. */
 D2D_API d2d_status d2d_layer_get_fused(const d2d_layer *layer, int32_t *group, double *rho_max);
 /* Current setting; any output pointer may be NULL.  *group is 0 when the shape
- * cannot take the gathered path. */
+ * cannot take the gathered path, *rho_max is negative while the library default
+ * is in force: that default depends on the batch size of each call (the
+ * gathered kernels have a fixed cost that a small batch cannot amortise). */
 D2D_API d2d_status d2d_layer_get_expert_path(const d2d_layer *layer, int32_t *path, int32_t *group, double *rho_max);
+/* Which form of the expert step (D2D_PATH_DENSE, _GATHER or _FUSED) a call
+ * with T tokens and n_sel selected pairs takes under the layer's current
+ * setting: the rule the kernels evaluate on the device, evaluated on the host
+ * (for bf16 batches above the decode sizes; reporting and tests). */
+D2D_API d2d_status d2d_layer_expert_path_for(const d2d_layer *layer, int32_t T, int64_t n_sel, int32_t *path);
 
 /* Clears the layer-owned device counters (the "last CTA" tickets, the tile and
  * sub-chunk counters of the expert kernels).  They reset themselves when a

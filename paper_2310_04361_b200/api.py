@@ -28,7 +28,7 @@ D2D_F32, D2D_BF16 = 0, 1
 ACTS = {"relu": 0, "gelu_erf": 1, "gelu_tanh": 2, "silu": 3}
 PATHS = {"auto": 0, "dense": 1, "gather": 2, "fused": 3}
 EXPORTS = ["d2d_status_str", "d2d_launch_count", "d2d_layer_create", "d2d_layer_destroy", "d2d_workspace_bytes",
-           "d2d_layer_set_expert_path", "d2d_layer_set_fused_rho_max", "d2d_layer_get_fused", "d2d_layer_get_expert_path", "d2d_layer_reset_counters", "d2d_expert_up_gather_fwd", "d2d_expert_down_masked_fwd", "d2d_test_inject_fault",
+           "d2d_layer_set_expert_path", "d2d_layer_set_fused_rho_max", "d2d_layer_get_fused", "d2d_layer_expert_path_for", "d2d_layer_get_expert_path", "d2d_layer_reset_counters", "d2d_expert_up_gather_fwd", "d2d_expert_down_masked_fwd", "d2d_test_inject_fault",
            "d2d_select_workspace_bytes", "d2d_router_fwd", "d2d_select_dynk", "d2d_select_dynk_static", "d2d_select_topk",
            "d2d_routing_from_mask", "d2d_moe_ffn_fwd", "d2d_expert_up_fwd", "d2d_expert_down_fwd", "d2d_layer_fwd", "d2d_layer_fwd_host_workspace_bytes",
            "d2d_layer_fwd_host", "d2d_group_create", "d2d_group_destroy", "d2d_group_workspace_bytes", "d2d_group_fwd"]
@@ -71,6 +71,7 @@ _lib.d2d_expert_down_masked_fwd.argtypes = [c_void_p, c_void_p, c_int32, POINTER
 _lib.d2d_layer_set_expert_path.argtypes = [c_void_p, c_int, c_int32, ctypes.c_double]
 _lib.d2d_layer_set_fused_rho_max.argtypes = [c_void_p, ctypes.c_double]
 _lib.d2d_layer_get_fused.argtypes = [c_void_p, POINTER(c_int32), POINTER(ctypes.c_double)]
+_lib.d2d_layer_expert_path_for.argtypes = [c_void_p, c_int32, ctypes.c_int64, POINTER(c_int32)]
 _lib.d2d_layer_get_expert_path.argtypes = [c_void_p, POINTER(c_int32), POINTER(c_int32), POINTER(ctypes.c_double)]
 _lib.d2d_layer_reset_counters.argtypes = [c_void_p, c_void_p]
 _lib.d2d_test_inject_fault.argtypes = [c_int32]
@@ -227,6 +228,12 @@ class Layer:
     def set_fused_rho_max(self, rho_max: float = -1.0) -> None:
         """Density up to which "auto" takes the fused gathered kernel (negative = default, 0 = never)."""
         _check(_lib.d2d_layer_set_fused_rho_max(self.handle, float(rho_max)), "d2d_layer_set_fused_rho_max")
+
+    def expert_path_for(self, T: int, n_sel: int) -> str:
+        """The form of the expert step a call with T tokens and n_sel selected pairs takes ("dense" | "gather" | "fused")."""
+        path = c_int32()
+        _check(_lib.d2d_layer_expert_path_for(self.handle, int(T), int(n_sel), ctypes.byref(path)), "d2d_layer_expert_path_for")
+        return {v: k for k, v in PATHS.items()}[path.value]
 
     def get_fused(self):
         group, rho = c_int32(), ctypes.c_double()

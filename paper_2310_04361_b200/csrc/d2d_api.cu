@@ -97,20 +97,30 @@ size_t d2d_moe_ffn_ws_bytes(const d2d_layer *L, int T)
     return need;
 }
 
-// Density up to which the gathered up projection (followed by the down projection that applies the selection while it
-// stages H) beats the masked dense pair for this shape: the default crossover of the automatic choice.  Measured on
-// B200: the gathered kernel is bound by the rate at which token rows can be copied into the A stages (about the same
-// time per 128 x 64 tile of gathered rows whatever the MMA width), so its cost relative to the dense kernel is about
-// (256 / MMA columns) per gathered row, plus a fixed part (scanning the mask, one ragged tile per group visit); it wins
-// while the fraction of (token, group) pairs u = 1 - (1 - rho)^g stays below the value tabulated here.
-static double default_gather_rho_max(const d2d_layer_desc &D, int g)
+// Density up to which the gathered pair beats the masked dense pair for this shape and batch size: the default
+// crossover of the automatic choice.  Measured on B200: the gathered kernel is bound by the rate at which token rows
+// can be copied into the A stages (about the same time per 128 x 64 tile of gathered rows whatever the MMA width), so
+// with full-width groups a gathered row costs about 1.2 x a dense one, and the kernel has a fixed part (the scan of the
+// mask, a ragged tile per group visit) worth about five tiles per CTA.  Against a dense up projection of
+// T / 128 x Nd tiles (Nd = 256-column tiles across d_ff) on S SMs that fixed part is T0 = 5 * 128 * 1.2 * S / Nd
+// tokens' worth of dense time, so the pair wins while the fraction of kept (token, group) pairs
+//     u = 1 - (1 - rho)^g  <  U - T0 / T,
+// U = 0.85 for 256 MMA columns (less for narrower groups, 0.05 less where the slower selection-applying down
+// projection follows instead of a zero fill and the TMA-fed one).  Checked against measured crossovers: Llama-shaped
+// layer u = 0.70 at 8192 tokens, 0.55 at 4096; paper's latency shape 0.6-0.75 at 50432 tokens; ViT-shaped 0.5 at
+// 25216; never for the BERT-shaped layer at 4096 tokens.
+int d2d_tc_sm_count();      // gemm_tc.cu
+
+static double default_gather_rho_max(const d2d_layer_desc &D, int g, int T)
 {
-    if (g <= 0) return -1.0;
+    if (g <= 0 || T <= 0) return -1.0;
     const int n_mma = g * D.expert_size * (D.gated ? 2 : 1);
-    double u_max = n_mma >= 256 ? 0.60 : n_mma >= 192 ? 0.30 : n_mma >= 128 ? 0.25 : 0.15;
-    // wide layers keep the TMA-fed dense down projection behind the gathered kernel (unkept cells of H zero-filled)
-    // instead of the slower selection-applying one: measured on the Llama shape, the gathered pair wins up to u = 0.7
-    if (D.d >= 2048) u_max += 0.10;
+    double U = n_mma >= 256 ? 0.85 : n_mma >= 192 ? 0.64 : n_mma >= 128 ? 0.43 : 0.25;
+    if (D.d < 2048) U -= 0.05;
+    const double nd = ceil((double)D.d_ff * (D.gated ? 2.0 : 1.0) / 256.0);
+    const double T0 = 5.0 * 128.0 * 1.2 * (double)d2d_tc_sm_count() / nd;
+    const double u_max = U - T0 / (double)T;
+    if (u_max <= 0.0) return 0.0;
     return 1.0 - pow(1.0 - u_max, 1.0 / g);
 }
 
@@ -150,7 +160,8 @@ static d2d_status launch_tc_experts(const d2d_layer *L, const void *x, int T, co
     // that this is noise.  Below that the fixed costs of the gathered kernel leave it nothing to win anyway.
     const double up_flop = 2.0 * (double)T * D.d * D.d_ff * (D.gated ? 2.0 : 1.0);
     if (path == D2D_PATH_AUTO && (up_flop < 1e11 || !n_sel)) path = D2D_PATH_DENSE;
-    long long n_sel_max = (long long)(L->gather_rho_max * (double)T * (double)D.n_experts);
+    const double rho_max = L->gather_rho_max >= 0.0 ? L->gather_rho_max : default_gather_rho_max(D, L->gather_group, T);
+    long long n_sel_max = (long long)(rho_max * (double)T * (double)D.n_experts);
     d2d_status rc;
     // Fused gathered step (plain layers): up projection, activation, down projection and the merge in one kernel whose
     // time is proportional to the kept (token, group) pairs; the float32 accumulator takes the place of H.
@@ -282,7 +293,7 @@ d2d_status d2d_layer_create(const d2d_layer_desc *desc, const d2d_weights *w, vo
     };
     size_t total = 256;                                   // the ticket words (see d2d_layer::tickets)
     L->gather_group = d2d_gather_group_for(D, 0);
-    L->gather_rho_max = default_gather_rho_max(D, L->gather_group);
+    L->gather_rho_max = -1.0;                             // the default for the shape and the batch size of each call
     L->expert_path = D2D_PATH_AUTO;
     L->fused_group = d2d_gather_ffn_group_for(D);
     L->fused_rho_max = default_fused_rho_max(L->fused_group);
@@ -396,7 +407,7 @@ d2d_status d2d_layer_set_expert_path(d2d_layer *layer, d2d_expert_path path, int
     if (g <= 0 && (path == D2D_PATH_GATHER || group > 0)) return D2D_ERR_UNSUPPORTED;
     layer->gather_group = g;
     layer->expert_path = path;
-    layer->gather_rho_max = rho_max >= 0.0 ? (rho_max > 1.0 ? 1.0 : rho_max) : default_gather_rho_max(layer->desc, g);
+    layer->gather_rho_max = rho_max >= 0.0 ? (rho_max > 1.0 ? 1.0 : rho_max) : -1.0;
     return D2D_OK;
 }
 
@@ -405,6 +416,26 @@ d2d_status d2d_layer_set_fused_rho_max(d2d_layer *layer, double rho_max)
     if (!layer) return D2D_ERR_INVALID_ARG;
     if (layer->fused_group <= 0) return rho_max > 0.0 ? D2D_ERR_UNSUPPORTED : D2D_OK;
     layer->fused_rho_max = rho_max >= 0.0 ? (rho_max > 1.0 ? 1.0 : rho_max) : default_fused_rho_max(layer->fused_group);
+    return D2D_OK;
+}
+
+d2d_status d2d_layer_expert_path_for(const d2d_layer *layer, int32_t T, int64_t n_sel, int32_t *path)
+{
+    if (!layer || !path || T <= 0 || n_sel < 0) return D2D_ERR_INVALID_ARG;
+    const d2d_layer_desc &D = layer->desc;
+    int p = layer->expert_path;
+    if (p == D2D_PATH_FUSED && layer->fused_group <= 0) return D2D_ERR_UNSUPPORTED;
+    if (p != D2D_PATH_FUSED && layer->gather_group <= 0) p = D2D_PATH_DENSE;
+    if (p == D2D_PATH_AUTO) {
+        const double up_flop = 2.0 * (double)T * D.d * D.d_ff * (D.gated ? 2.0 : 1.0);
+        const double pairs = (double)T * (double)D.n_experts;
+        const double rho_max = layer->gather_rho_max >= 0.0 ? layer->gather_rho_max : default_gather_rho_max(D, layer->gather_group, T);
+        if (up_flop < 1e11) p = D2D_PATH_DENSE;
+        else if (layer->fused_group > 0 && layer->fused_rho_max > 0.0 && n_sel <= (long long)(layer->fused_rho_max * pairs)) p = D2D_PATH_FUSED;
+        else if (n_sel <= (long long)(rho_max * pairs) || (layer->fused_group > 0 && n_sel <= (long long)(layer->fused_rho_max * pairs))) p = D2D_PATH_GATHER;
+        else p = D2D_PATH_DENSE;
+    }
+    *path = p;
     return D2D_OK;
 }
 

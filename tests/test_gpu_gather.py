@@ -208,6 +208,18 @@ def test_expert_path_settings_and_errors(api):
     layer.reset_counters()
     torch.cuda.synchronize()
     layer.close()
+    # the host-side copy of the rule the kernels evaluate: small batches stay dense at any density, large ones go from
+    # the fused kernel (plain layers) through the gathered pair to the dense pair as the density grows
+    paper = wl.CONFIGS["paper"]
+    lp = api.Layer.from_config(paper, wl.make_weights(paper))
+    pairs = paper.T * paper.E
+    taken = [lp.expert_path_for(paper.T, int(rho * pairs)) for rho in (0.01, 0.05, 0.1, 0.3, 0.6, 1.0)]
+    assert taken == ["fused", "fused", "gather", "gather", "dense", "dense"]
+    assert all(lp.expert_path_for(2048, int(rho * 2048 * paper.E)) == "dense" for rho in (0.01, 0.3, 1.0))
+    for forced in ("dense", "gather", "fused"):
+        lp.set_expert_path(forced)
+        assert lp.expert_path_for(paper.T, pairs // 2) == forced
+    lp.close()
     tiny = wl.CONFIGS["tiny"]                                  # fp32 layers have no tensor-core expert path
     lt = api.Layer.from_config(tiny, wl.make_weights(tiny))
     assert lt.get_expert_path()[1] == 0
