@@ -3,8 +3,10 @@
 // One CTA per token.  The token row sits in shared memory as float32; the warps compute the router's hidden units
 // (one warp per unit: a d-long dot product reduced by shuffles, bias + ReLU), then the expert scores (one warp per
 // expert, absolute value, Sec. 3.3), warp 0 takes the row maximum, the threshold tau * max as ONE float32 product and
-// the mask words (Eq. 4), and the CTA then runs the token's kept experts exactly like the token-major expert kernel
-// (moe_ffn_token.cu): a fixed summation order, no atomics, y written once with b2 added once.  When the caller wants
+// the mask words (Eq. 4), and the CTA then runs the token's kept experts: all their hidden neurons in one pass (one
+// warp per neuron), then the down projection with the neurons split over thread groups; a fixed summation order, no
+// atomics, y written once with b2 added once.  Loops over weights are unrolled so that their loads are in flight
+// together: at this size the kernel's time is a chain of memory latencies, not arithmetic.  When the caller wants
 // the per-expert lists (Listing 1), the CTA that finishes last (a ticket) builds them from the mask words of all
 // tokens with the single-CTA selection routine, so that no further launch follows.
 //
@@ -17,8 +19,8 @@ namespace {
 
 constexpr int NT = 256;
 constexpr int NWARP = NT / 32;
-constexpr int MAX_S = 128;          // largest expert size staged in shared memory
-constexpr int MAX_COLS = 16;        // output columns per thread: d <= NT * MAX_COLS
+constexpr int MAX_H = 2048;         // hidden neurons of one token's kept experts staged in shared memory: d_ff <= MAX_H
+constexpr int MAX_COLS = 4;         // output columns per thread: d <= NT * MAX_COLS
 
 struct FusedArgs {
     const void *x, *w_r1, *b_r1, *w_r2, *b_r2, *w1, *b1, *w_gate, *w2t, *b2;
@@ -26,7 +28,7 @@ struct FusedArgs {
     float *R_out;                   // [T, E] or NULL
     d2d_routing r;                  // mask, k, status required; lists optional as a set
     unsigned int *ticket;           // zero at launch, left at zero
-    int T, d, d_h, E, s, W, lists;
+    int T, d, d_h, d_ff, E, s, W, lists;
     float tau;
 };
 
@@ -38,9 +40,11 @@ layer_token_fused_kernel(const FusedArgs a)
     float *xs = smem;                                   // [d]
     float *us = xs + a.d;                               // [d_h]
     float *Rs = us + a.d_h;                             // [E]
-    float *hs = Rs + a.E;                               // [2][MAX_S]
-    uint32_t *words = reinterpret_cast<uint32_t *>(hs + 2 * MAX_S);      // [W] this token's mask words
+    float *hs = Rs + a.E;                               // [d_ff] hidden activations of the kept experts, [groups * d] partial sums
+    int *kept = reinterpret_cast<int *>(hs + max(a.d_ff, NT * MAX_COLS));     // [E] kept experts of this token, ascending
+    uint32_t *words = reinterpret_cast<uint32_t *>(kept + a.E);               // [W] this token's mask words
     uint32_t *smask = words + a.W;                      // [T * W] all tokens' words (last CTA, lists only)
+    __shared__ int n_kept;
     __shared__ int is_last;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int t = blockIdx.x, d = a.d, s = a.s;
@@ -49,6 +53,7 @@ layer_token_fused_kernel(const FusedArgs a)
     for (int c = tid; c < d; c += NT) xs[c] = d2d_to_float<T>(x[(size_t)t * d + c]);
     __syncthreads();
     // ---- router hidden layer: u = ReLU(W_r1 x + b_r1)
+#pragma unroll 4
     for (int j = warp; j < a.d_h; j += NWARP) {
         const T *row = (const T *)a.w_r1 + (size_t)j * d;
         float v = 0.0f;
@@ -63,6 +68,7 @@ layer_token_fused_kernel(const FusedArgs a)
     }
     __syncthreads();
     // ---- router output layer: R = |W_r2 u + b_r2|
+#pragma unroll 2
     for (int e = warp; e < a.E; e += NWARP) {
         const T *row = (const T *)a.w_r2 + (size_t)e * a.d_h;
         float v = 0.0f;
@@ -103,65 +109,82 @@ layer_token_fused_kernel(const FusedArgs a)
             }
             kt += __popc(word);
         }
+        int pos = 0;
+        for (int w = 0; w < a.W; ++w) {                        // the kept experts in ascending order
+            const uint32_t word = words[w];
+            if ((word >> lane) & 1u) kept[pos + __popc(word & ((1u << lane) - 1u))] = w * 32 + lane;
+            pos += __popc(word);
+        }
         if (lane == 0) {
             a.r.k[t] = kt;
+            n_kept = kt;
             if (bad) atomicMax(a.r.status, (int32_t)D2D_ERR_NONFINITE);
         }
     } else if (a.R_out) {
         for (int i = tid - 32; i < a.E; i += NT - 32) a.R_out[(size_t)t * a.E + i] = Rs[i];
     }
     __syncthreads();
-    // ---- kept experts: up projection + activation (one warp per neuron), down projection (columns per thread)
+    // ---- kept experts, up projection + activation: one warp per hidden neuron over all kept experts at once
+    const int n_hidden = n_kept * s;
+#pragma unroll 2
+    for (int idx = warp; idx < n_hidden; idx += NWARP) {
+        const size_t n = (size_t)kept[idx / s] * s + idx % s;
+        const T *wrow = (const T *)a.w1 + n * d;
+        const T *grow = GATED ? (const T *)a.w_gate + n * d : nullptr;
+        float up = 0.0f, gate = 0.0f;
+        for (int c = lane * 8; c < d; c += 256) {
+            float wv[8];
+            d2d_load8(wrow + c, wv);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) up = fmaf(wv[i], xs[c + i], up);
+            if (GATED) {
+                d2d_load8(grow + c, wv);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) gate = fmaf(wv[i], xs[c + i], gate);
+            }
+        }
+        up = d2d_warp_sum(up);
+        if (GATED) gate = d2d_warp_sum(gate);
+        if (lane == 0) {
+            if (a.b1) up += d2d_to_float<T>(((const T *)a.b1)[n]);
+            hs[idx] = GATED ? d2d_activate<ACT>(gate) * up : d2d_activate<ACT>(up);
+        }
+    }
+    __syncthreads();
+    // ---- down projection: a thread owns output columns; when d is smaller than the CTA the hidden neurons are split
+    // over NT / d thread groups whose partial sums meet in shared memory.  Fixed order: deterministic.
+    const int groups = d < NT ? NT / d : 1;
+    const int grp = d < NT ? tid / d : 0, col0 = d < NT ? tid % d : tid;
     float acc[MAX_COLS];
 #pragma unroll
     for (int i = 0; i < MAX_COLS; ++i) acc[i] = 0.0f;
-    int buf = 0;
-    for (int w = 0; w < a.W; ++w) {
-        uint32_t word = words[w];
-        while (word) {
-            const int e = w * 32 + __ffs(word) - 1;
-            word &= word - 1;
-            float *h = hs + buf * MAX_S;
-            for (int nl = warp; nl < s; nl += NWARP) {
-                const size_t n = (size_t)e * s + nl;
-                const T *wrow = (const T *)a.w1 + n * d;
-                const T *grow = GATED ? (const T *)a.w_gate + n * d : nullptr;
-                float up = 0.0f, gate = 0.0f;
-                for (int c = lane * 8; c < d; c += 256) {
-                    float wv[8];
-                    d2d_load8(wrow + c, wv);
+    if (grp < groups) {
+#pragma unroll 8
+        for (int idx = grp; idx < n_hidden; idx += groups) {
+            const float hv = hs[idx];
+            const T *row = (const T *)a.w2t + ((size_t)kept[idx / s] * s + idx % s) * d;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) up = fmaf(wv[i], xs[c + i], up);
-                    if (GATED) {
-                        d2d_load8(grow + c, wv);
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) gate = fmaf(wv[i], xs[c + i], gate);
-                    }
-                }
-                up = d2d_warp_sum(up);
-                if (GATED) gate = d2d_warp_sum(gate);
-                if (lane == 0) {
-                    if (a.b1) up += d2d_to_float<T>(((const T *)a.b1)[n]);
-                    h[nl] = GATED ? d2d_activate<ACT>(gate) * up : d2d_activate<ACT>(up);
-                }
+            for (int i = 0; i < MAX_COLS; ++i) {
+                const int c = col0 + NT * i;
+                if (c < d) acc[i] = fmaf(hv, d2d_to_float<T>(__ldg(row + c)), acc[i]);
             }
-            __syncthreads();
-            for (int nl = 0; nl < s; ++nl) {
-                const float hv = h[nl];
-                const T *row = (const T *)a.w2t + ((size_t)e * s + nl) * d;
-#pragma unroll
-                for (int i = 0; i < MAX_COLS; ++i) {
-                    const int c = tid + NT * i;
-                    if (c < d) acc[i] = fmaf(hv, d2d_to_float<T>(__ldg(row + c)), acc[i]);
-                }
-            }
-            buf ^= 1;              // the next expert writes the other buffer: one barrier per expert
         }
     }
+    if (groups > 1) {
+        __syncthreads();                                       // every reader of hs is done: reuse it for the partial sums
+        if (grp < groups) hs[grp * d + col0] = acc[0];
+        __syncthreads();
+        if (tid < d) {
+            float v = a.b2 ? d2d_to_float<T>(((const T *)a.b2)[tid]) : 0.0f;
+            for (int q = 0; q < groups; ++q) v += hs[q * d + tid];
+            ((T *)a.y)[(size_t)t * d + tid] = d2d_from_float<T>(v);
+        }
+    } else {
 #pragma unroll
-    for (int i = 0; i < MAX_COLS; ++i) {
-        const int c = tid + NT * i;
-        if (c < d) ((T *)a.y)[(size_t)t * d + c] = d2d_from_float<T>(acc[i] + (a.b2 ? d2d_to_float<T>(((const T *)a.b2)[c]) : 0.0f));
+        for (int i = 0; i < MAX_COLS; ++i) {
+            const int c = tid + NT * i;
+            if (c < d) ((T *)a.y)[(size_t)t * d + c] = d2d_from_float<T>(acc[i] + (a.b2 ? d2d_to_float<T>(((const T *)a.b2)[c]) : 0.0f));
+        }
     }
     if (!a.lists) return;
     // ---- per-expert lists: the CTA that finishes last builds them from everybody's mask words
@@ -192,15 +215,22 @@ d2d_status launch_act(const FusedArgs &a, bool gated, size_t smem, cudaStream_t 
 
 }  // namespace
 
+static size_t fused_smem_bytes(const d2d_layer_desc &D, int T, bool lists)
+{
+    const int W = (D.n_experts + 31) / 32;
+    const int h = D.d_ff > NT * MAX_COLS ? D.d_ff : NT * MAX_COLS;
+    return (size_t)(D.d + D.d_h + D.n_experts + h + D.n_experts + W) * 4 + (lists ? (size_t)T * W * 4 : 0);
+}
+
 // Small float32 problems only: the router's weights are read once per token out of L2 here, which is fine for a few
 // hundred KB and wasteful beyond.
 bool d2d_layer_token_fused_supports(const d2d_layer_desc &D, int T, bool lists)
 {
     const int W = (D.n_experts + 31) / 32;
-    if (D.dtype != D2D_F32 || T < 1 || D.d > NT * MAX_COLS || D.expert_size > MAX_S || D.d % 8 || D.d_h % 8) return false;
+    if (D.dtype != D2D_F32 || T < 1 || D.d > NT * MAX_COLS || D.d_ff > MAX_H || D.d % 8 || D.d_h % 8) return false;
     if ((size_t)D.d * D.d_h + (size_t)D.d_h * D.n_experts > 65536) return false;
     if (lists && (T > d2d_small::MAX_T || (size_t)T * W * 4 > 24 * 1024)) return false;
-    return (size_t)(D.d + D.d_h + D.n_experts + 2 * MAX_S + W) * 4 + (size_t)T * W * 4 <= 44 * 1024;
+    return fused_smem_bytes(D, T, lists) <= 44 * 1024;
 }
 
 d2d_status d2d_layer_token_fused(const d2d_layer *L, const void *x, int T, float tau, void *y, float *R_out, const d2d_routing *r,
@@ -211,9 +241,9 @@ d2d_status d2d_layer_token_fused(const d2d_layer *L, const void *x, int T, float
     a.x = x; a.w_r1 = L->w_r1; a.b_r1 = L->b_r1; a.w_r2 = L->w_r2; a.b_r2 = L->b_r2;
     a.w1 = L->w1; a.b1 = L->b1; a.w_gate = L->w_gate; a.w2t = L->w2t; a.b2 = L->b2;
     a.y = y; a.R_out = R_out; a.r = *r; a.ticket = ticket;
-    a.T = T; a.d = D.d; a.d_h = D.d_h; a.E = D.n_experts; a.s = D.expert_size; a.W = (D.n_experts + 31) / 32; a.lists = lists ? 1 : 0;
+    a.T = T; a.d = D.d; a.d_h = D.d_h; a.d_ff = D.d_ff; a.E = D.n_experts; a.s = D.expert_size; a.W = (D.n_experts + 31) / 32; a.lists = lists ? 1 : 0;
     a.tau = tau;
-    const size_t smem = (size_t)(D.d + D.d_h + D.n_experts + 2 * MAX_S + a.W) * 4 + (lists ? (size_t)T * a.W * 4 : 0);
+    const size_t smem = fused_smem_bytes(D, T, lists);
     switch (D.act) {
     case D2D_ACT_RELU: return launch_act<float, D2D_ACT_RELU>(a, D.gated != 0, smem, st);
     case D2D_ACT_GELU_ERF: return launch_act<float, D2D_ACT_GELU_ERF>(a, D.gated != 0, smem, st);
