@@ -35,9 +35,12 @@ L2_FLUSH_BYTES = 256 << 20
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from ncu captures of that
 # kernel on that workload (absent: no capture of that combination); keyed by (workload, tokens, kernel).
-# The full-size figure is a one-pass capture of those two counters alone (610.4 MB read + 174.9 MB written).
+# The full-size figures are one-pass captures of those two counters alone: the masked dense up projection reads
+# 610.4 MB and writes 174.9 MB; the gathered one (tau = 0.4) reads 2911.9 MB and writes 107.8 MB (token rows and
+# weight rows together exceed what L2 keeps, so rows are fetched again for many of the groups that use them).
 NCU_TRAFFIC_BYTES = {
     ("llama", 8192, "dense_up"): 610_425_088 + 174_942_464,
+    ("llama", 8192, "gather_up"): 2_911_860_736 + 107_819_520,
 }
 
 # (workload, tokens or None = the workload's own, tau or None, Bernoulli p or None) timed for `per_config`
