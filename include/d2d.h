@@ -172,9 +172,9 @@ D2D_API d2d_status d2d_layer_destroy(d2d_layer *layer);
  *                    n_sel <= rho_max * T * E, dense otherwise.  Both pairs of
  *                    kernels are enqueued and the pair not needed returns at once,
  *                    so there is no host synchronisation.  Batches whose up
- *                    projection is below about 1e11 FLOP (100 us of tensor-core
- *                    time) always take the dense form: the gathered kernel's
- *                    fixed costs leave it nothing to win there, and the dense
+ *                    projection is below 2e11 FLOP (about 150 us of tensor-core
+ *                    time) always take the dense form: the gathered kernels'
+ *                    fixed costs leave them little to win there, and the dense
  *                    kernel then keeps its overlap with the router.
  * group: experts per group, 0 = library default for the shape (a power of two
  * that divides E, group * expert_size a multiple of 16 and at most 256, 128 for

@@ -111,6 +111,8 @@ size_t d2d_moe_ffn_ws_bytes(const d2d_layer *L, int T)
 // 25216; never for the BERT-shaped layer at 4096 tokens.
 int d2d_tc_sm_count();      // gemm_tc.cu
 
+static const double kAutoMinUpFlop = 2e11;      // smallest up projection for which the automatic choice is made
+
 static double default_gather_rho_max(const d2d_layer_desc &D, int g, int T)
 {
     if (g <= 0 || T <= 0) return -1.0;
@@ -155,11 +157,12 @@ static d2d_status launch_tc_experts(const d2d_layer *L, const void *x, int T, co
     const d2d_layer_desc &D = L->desc;
     int path = L->expert_path;
     if (L->gather_group <= 0) path = D2D_PATH_DENSE;
-    // The automatic choice costs two launches that return at once and the overlap of the router with the masked dense
-    // kernel's main loops: only for problems whose up projection takes long enough (about 100 us of tensor-core time)
-    // that this is noise.  Below that the fixed costs of the gathered kernel leave it nothing to win anyway.
+    // The automatic choice costs a few launches that return at once and the overlap of the router with the masked dense
+    // kernel's main loops (measured on the ViT-shaped layer, 1.2e11 FLOP: 241 us against 224 us at every density, while
+    // the gathered paths win there only below rho = 0.03): it is made only for problems whose up projection takes long
+    // enough (2e11 FLOP, about 150 us of tensor-core time) that this is noise.
     const double up_flop = 2.0 * (double)T * D.d * D.d_ff * (D.gated ? 2.0 : 1.0);
-    if (path == D2D_PATH_AUTO && (up_flop < 1e11 || !n_sel)) path = D2D_PATH_DENSE;
+    if (path == D2D_PATH_AUTO && (up_flop < kAutoMinUpFlop || !n_sel)) path = D2D_PATH_DENSE;
     const double rho_max = L->gather_rho_max >= 0.0 ? L->gather_rho_max : default_gather_rho_max(D, L->gather_group, T);
     long long n_sel_max = (long long)(rho_max * (double)T * (double)D.n_experts);
     d2d_status rc;
@@ -430,7 +433,7 @@ d2d_status d2d_layer_expert_path_for(const d2d_layer *layer, int32_t T, int64_t 
         const double up_flop = 2.0 * (double)T * D.d * D.d_ff * (D.gated ? 2.0 : 1.0);
         const double pairs = (double)T * (double)D.n_experts;
         const double rho_max = layer->gather_rho_max >= 0.0 ? layer->gather_rho_max : default_gather_rho_max(D, layer->gather_group, T);
-        if (up_flop < 1e11) p = D2D_PATH_DENSE;
+        if (up_flop < kAutoMinUpFlop) p = D2D_PATH_DENSE;
         else if (layer->fused_group > 0 && layer->fused_rho_max > 0.0 && n_sel <= (long long)(layer->fused_rho_max * pairs)) p = D2D_PATH_FUSED;
         else if (n_sel <= (long long)(rho_max * pairs) || (layer->fused_group > 0 && n_sel <= (long long)(layer->fused_rho_max * pairs))) p = D2D_PATH_GATHER;
         else p = D2D_PATH_DENSE;

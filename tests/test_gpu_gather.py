@@ -148,7 +148,7 @@ def test_layer_fwd_is_the_same_on_both_sides_of_the_dispatch(api, name, T, tau):
     layer.close()
 
 
-@pytest.mark.parametrize("name,tau", [("vit", 0.6), ("llama", 0.6)])
+@pytest.mark.parametrize("name,tau", [("paper", 0.5), ("llama", 0.6)])
 def test_device_side_choice_at_full_size(api, name, tau):
     """Batches large enough for the automatic choice: the crossover is moved to either extreme so that the decision
     taken on the device goes each way (both kernel pairs are enqueued, one returns at once); y is checked against
@@ -181,6 +181,9 @@ def test_device_side_choice_at_full_size(api, name, tau):
             assert r.status == 0
         G = oracle.unpack_mask(r.mask_u32(), cfg.E)
         assert r.n_sel == int(G.sum())
+        if (rho_max, fused_max) != (-1.0, -1.0):               # the host-side copy of the rule agrees with the setting
+            want = "fused" if fused_max == 1.0 else "gather" if rho_max == 1.0 else "dense"
+            assert layer.expert_path_for(T, r.n_sel) == want
         if ref is None:
             ref = (G, oracle.moe_ffn(x[sample], w["w1"], w["b1"], w["w_gate"], w["w2"], w["b2"], act, G[sample]))
         assert np.array_equal(G, ref[0])
