@@ -37,7 +37,7 @@
  *                            the decode kernels (each kept expert's weights read
  *                            once by CUDA cores), larger ones the tensor-core path.
  *   D2D_HOST_CHUNKS=n        1..4: number of pipelined chunks d2d_layer_fwd_host
- *                            cuts a batch into (default: one per 4096 tokens).
+ *                            cuts a batch into, of equal size (default: see there).
  *   D2D_GEMM_BAND=n          row tiles per band of the tile walk of the dense
  *                            kernels when the weight operand exceeds L2 (default:
  *                            about 32 MB of activation rows), 0 = row-major walk.
@@ -352,8 +352,9 @@ D2D_API d2d_status d2d_layer_fwd(const d2d_layer *layer, const void *x, int32_t 
  * ([T,d] of desc.dtype).  The call copies x to the device, runs the layer,
  * copies y back and synchronises `stream`; all device memory it needs comes
  * from `ws` (device, at least d2d_layer_fwd_host_workspace_bytes bytes).
- * Batches of 8192 tokens or more are cut into up to four chunks (of at least
- * 4096 tokens) and pipelined over
+ * Batches of 8192 tokens or more are cut into four chunks of 3/16, 5/16, 5/16
+ * and 3/16 of the tokens (the call then takes about the copy-in of the first
+ * chunk + the layer on all of them + the copy-out of the last) and pipelined over
  * two copy streams the layer owns (copy in / layer / copy out overlap; tokens
  * are independent, so the result is the same); this needs page-locked host
  * buffers to be effective.  Returns the data-dependent status as well

@@ -729,13 +729,25 @@ d2d_status d2d_layer_fwd_host(const d2d_layer *layer, const void *x_host, int32_
     // chunk c+1 to the device (copy-in stream), the layer on chunk c (`stream`) and the copy of chunk c-1 back to the
     // host (copy-out stream) run at the same time; PCIe carries both directions at once.  The routing buffers and the
     // layer workspace are reused chunk after chunk, which is safe because the layer calls are serial on `stream`.
-    // a chunk should still fill the GPU (a 1024-token layer call costs almost as much as a 4096-token one), so
-    // chunks hold at least 4096 tokens
-    int n_chunks = T / 4096;
-    n_chunks = n_chunks < 1 ? 1 : n_chunks > d2d_layer::kHostChunks ? d2d_layer::kHostChunks : n_chunks;
-    if (const char *e = getenv("D2D_HOST_CHUNKS")) {          // 1 .. 4, for tuning
+    // The layer is the slowest of the three legs for the shapes where this matters, so the whole call takes about
+    // (copy-in of the first chunk) + (all layer calls) + (copy-out of the last chunk): the first and the last chunk
+    // are short, the ones in between long (a short chunk costs more per token, so there are few of them).
+    int bounds[d2d_layer::kHostChunks + 1] = {0, T, T, T, T};
+    int n_chunks = 1;
+    if (T >= 8192) {
+        // sizes 3T/16, 5T/16, 5T/16, 3T/16 in multiples of 128 tokens (measured on the Llama-shaped layer, 8192 tokens:
+        // 2.50 ms; T/8, 3T/8, 3T/8, T/8: 2.64; four equal chunks: 2.62; two equal chunks: 3.04)
+        const int a = d2d_cdiv(3 * (T / 16), 128) * 128, b = d2d_cdiv((T - 2 * a) / 2, 128) * 128;
+        bounds[1] = a; bounds[2] = a + b; bounds[3] = T - a > a + b ? T - a : a + b; bounds[4] = T;
+        n_chunks = 4;
+    }
+    if (const char *e = getenv("D2D_HOST_CHUNKS")) {          // 1 .. 4 equal chunks, for tuning
         const int n = atoi(e);
-        if (n >= 1 && n <= d2d_layer::kHostChunks && T >= 128 * n) n_chunks = n;
+        if (n >= 1 && n <= d2d_layer::kHostChunks && T >= 128 * n) {
+            n_chunks = n;
+            const int chunk = d2d_cdiv(d2d_cdiv(T, n), 128) * 128;
+            for (int c = 1; c <= d2d_layer::kHostChunks; ++c) bounds[c] = c * chunk < T && c < n ? c * chunk : T;
+        }
     }
     if (n_chunks == 1) {
         D2D_CUDA_TRY(cudaMemcpyAsync(base + h.x_off, x_host, row_bytes, cudaMemcpyHostToDevice, st));
@@ -746,13 +758,13 @@ d2d_status d2d_layer_fwd_host(const d2d_layer *layer, const void *x_host, int32_
         D2D_CUDA_TRY(cudaStreamSynchronize(st));
         return host_status(r.status, 1);
     }
-    const int chunk = d2d_cdiv(d2d_cdiv(T, n_chunks), 128) * 128;
     // the copies may not start before work already queued on `stream` (which may still use ws) has finished
     D2D_CUDA_TRY(cudaEventRecord(layer->ev_begin, st));
     D2D_CUDA_TRY(cudaStreamWaitEvent(layer->copy_in, layer->ev_begin, 0));
     D2D_CUDA_TRY(cudaStreamWaitEvent(layer->copy_out, layer->ev_begin, 0));
-    for (int c = 0, t0 = 0; t0 < T; ++c, t0 += chunk) {
-        const int tc = T - t0 < chunk ? T - t0 : chunk;
+    for (int c = 0; c < n_chunks; ++c) {
+        const int t0 = bounds[c], tc = bounds[c + 1] - bounds[c];
+        if (tc <= 0) continue;
         D2D_CUDA_TRY(cudaMemcpyAsync(base + h.x_off + (size_t)t0 * tok_bytes, (const char *)x_host + (size_t)t0 * tok_bytes,
                                      (size_t)tc * tok_bytes, cudaMemcpyHostToDevice, layer->copy_in));
         D2D_CUDA_TRY(cudaEventRecord(layer->ev_in[c], layer->copy_in));
@@ -760,9 +772,11 @@ d2d_status d2d_layer_fwd_host(const d2d_layer *layer, const void *x_host, int32_
     d2d_status rc = D2D_OK;
     int32_t *const status0 = r.status;
     int n_used = 0;
-    for (int c = 0, t0 = 0; t0 < T; ++c, t0 += chunk, ++n_used) {
-        const int tc = T - t0 < chunk ? T - t0 : chunk;
-        r.status = status0 + c;                              // one status word per chunk (the layer call clears its own)
+    for (int c = 0; c < n_chunks; ++c) {
+        const int t0 = bounds[c], tc = bounds[c + 1] - bounds[c];
+        if (tc <= 0) continue;
+        r.status = status0 + n_used;                         // one status word per chunk (the layer call clears its own)
+        ++n_used;
         D2D_CUDA_TRY(cudaStreamWaitEvent(st, layer->ev_in[c], 0));
         rc = d2d_layer_fwd(layer, base + h.x_off + (size_t)t0 * tok_bytes, tc, tau, base + h.y_off + (size_t)t0 * tok_bytes,
                            nullptr, &r, base + h.ws_off, h.total - h.ws_off, st);

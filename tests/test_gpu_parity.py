@@ -516,7 +516,7 @@ def test_layer_fwd_host_buffers(api):
 
 
 def test_layer_fwd_host_chunked_pipeline_matches_device_call(api):
-    """8192 tokens or more: the host call runs in pipelined chunks (two here, the second ragged); tokens are
+    """8192 tokens or more: the host call runs in four pipelined chunks (the last one ragged here); tokens are
     independent, so the result equals one device call on the whole batch."""
     T = 8192 + 300
     cfg, w, x, layer = _setup(api, "bert", T)
