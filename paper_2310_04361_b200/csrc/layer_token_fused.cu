@@ -1,10 +1,10 @@
 // The whole layer of a SMALL problem in one launch (Sec. 3.2-3.4): router, dynamic-k rule, kept experts, combine.
 //
 // One CTA per token.  The token row sits in shared memory as float32; the warps compute the router's hidden units
-// (one warp per unit: a d-long dot product reduced by shuffles, bias + ReLU), then the expert scores (one warp per
+// (a sub-warp per unit: a d-long dot product reduced by shuffles, bias + ReLU), then the expert scores (a sub-warp per
 // expert, absolute value, Sec. 3.3), warp 0 takes the row maximum, the threshold tau * max as ONE float32 product and
-// the mask words (Eq. 4), and the CTA then runs the token's kept experts: all their hidden neurons in one pass (one
-// warp per neuron), then the down projection with the neurons split over thread groups; a fixed summation order, no
+// the mask words (Eq. 4), and the CTA then runs the token's kept experts: all their hidden neurons in one pass (a
+// sub-warp per neuron), then the down projection with the neurons split over thread groups; a fixed summation order, no
 // atomics, y written once with b2 added once.  Loops over weights are unrolled so that their loads are in flight
 // together: at this size the kernel's time is a chain of memory latencies, not arithmetic.  When the caller wants
 // the per-expert lists (Listing 1), the CTA that finishes last (a ticket) builds them from the mask words of all
@@ -32,6 +32,31 @@ struct FusedArgs {
     float tau;
 };
 
+// Lanes that share one weight row of `len` elements (8 elements per lane and step): a power of two, at most a warp.
+// Short rows leave room for several rows per warp at a time, which shortens the chain of dependent memory round trips.
+__device__ __forceinline__ int lanes_per_row(int len)
+{
+    int l = 1;
+    while (l < 32 && l * 8 < len) l <<= 1;
+    return l;
+}
+
+// dot(row, vec) for the sub-warp of `lpr` lanes this lane belongs to (every lane of the warp must call it)
+template <typename T>
+__device__ __forceinline__ float subwarp_dot(const T *row, const float *vec, int len, int lpr, int sl, bool valid)
+{
+    float v = 0.0f;
+    if (valid)
+        for (int c = sl * 8; c < len; c += lpr * 8) {
+            float wv[8];
+            d2d_load8(row + c, wv);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v = fmaf(wv[i], vec[c + i], v);
+        }
+    for (int o = lpr >> 1; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
 template <typename T, int ACT, bool GATED>
 __global__ void __launch_bounds__(NT)
 layer_token_fused_kernel(const FusedArgs a)
@@ -53,33 +78,27 @@ layer_token_fused_kernel(const FusedArgs a)
     for (int c = tid; c < d; c += NT) xs[c] = d2d_to_float<T>(x[(size_t)t * d + c]);
     __syncthreads();
     // ---- router hidden layer: u = ReLU(W_r1 x + b_r1)
-#pragma unroll 4
-    for (int j = warp; j < a.d_h; j += NWARP) {
-        const T *row = (const T *)a.w_r1 + (size_t)j * d;
-        float v = 0.0f;
-        for (int c = lane * 8; c < d; c += 256) {
-            float wv[8];
-            d2d_load8(row + c, wv);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) v = fmaf(wv[i], xs[c + i], v);
+    {
+        const int lpr = lanes_per_row(d), rpw = 32 / lpr, sub = lane / lpr, sl = lane % lpr;
+#pragma unroll 2
+        for (int j0 = warp * rpw; j0 < a.d_h; j0 += NWARP * rpw) {
+            const int j = j0 + sub;
+            const bool valid = j < a.d_h;
+            const float v = subwarp_dot((const T *)a.w_r1 + (size_t)(valid ? j : 0) * d, xs, d, lpr, sl, valid);
+            if (valid && sl == 0) us[j] = fmaxf(v + (a.b_r1 ? d2d_to_float<T>(((const T *)a.b_r1)[j]) : 0.0f), 0.0f);
         }
-        v = d2d_warp_sum(v);
-        if (lane == 0) us[j] = fmaxf(v + (a.b_r1 ? d2d_to_float<T>(((const T *)a.b_r1)[j]) : 0.0f), 0.0f);
     }
     __syncthreads();
     // ---- router output layer: R = |W_r2 u + b_r2|
+    {
+        const int lpr = lanes_per_row(a.d_h), rpw = 32 / lpr, sub = lane / lpr, sl = lane % lpr;
 #pragma unroll 2
-    for (int e = warp; e < a.E; e += NWARP) {
-        const T *row = (const T *)a.w_r2 + (size_t)e * a.d_h;
-        float v = 0.0f;
-        for (int c = lane * 8; c < a.d_h; c += 256) {
-            float wv[8];
-            d2d_load8(row + c, wv);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) v = fmaf(wv[i], us[c + i], v);
+        for (int e0 = warp * rpw; e0 < a.E; e0 += NWARP * rpw) {
+            const int e = e0 + sub;
+            const bool valid = e < a.E;
+            const float v = subwarp_dot((const T *)a.w_r2 + (size_t)(valid ? e : 0) * a.d_h, us, a.d_h, lpr, sl, valid);
+            if (valid && sl == 0) Rs[e] = fabsf(v + (a.b_r2 ? d2d_to_float<T>(((const T *)a.b_r2)[e]) : 0.0f));
         }
-        v = d2d_warp_sum(v);
-        if (lane == 0) Rs[e] = fabsf(v + (a.b_r2 ? d2d_to_float<T>(((const T *)a.b_r2)[e]) : 0.0f));
     }
     __syncthreads();
     // ---- dynamic-k rule (Eq. 4): keep expert i iff R_i >= tau * max_j R_j, the product rounded once to float32
@@ -124,30 +143,22 @@ layer_token_fused_kernel(const FusedArgs a)
         for (int i = tid - 32; i < a.E; i += NT - 32) a.R_out[(size_t)t * a.E + i] = Rs[i];
     }
     __syncthreads();
-    // ---- kept experts, up projection + activation: one warp per hidden neuron over all kept experts at once
+    // ---- kept experts, up projection + activation: all hidden neurons of all kept experts in one pass
     const int n_hidden = n_kept * s;
+    {
+        const int lpr = lanes_per_row(d), rpw = 32 / lpr, sub = lane / lpr, sl = lane % lpr;
 #pragma unroll 2
-    for (int idx = warp; idx < n_hidden; idx += NWARP) {
-        const size_t n = (size_t)kept[idx / s] * s + idx % s;
-        const T *wrow = (const T *)a.w1 + n * d;
-        const T *grow = GATED ? (const T *)a.w_gate + n * d : nullptr;
-        float up = 0.0f, gate = 0.0f;
-        for (int c = lane * 8; c < d; c += 256) {
-            float wv[8];
-            d2d_load8(wrow + c, wv);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) up = fmaf(wv[i], xs[c + i], up);
-            if (GATED) {
-                d2d_load8(grow + c, wv);
-#pragma unroll
-                for (int i = 0; i < 8; ++i) gate = fmaf(wv[i], xs[c + i], gate);
+        for (int i0 = warp * rpw; i0 < n_hidden; i0 += NWARP * rpw) {
+            const int idx = i0 + sub;
+            const bool valid = idx < n_hidden;
+            const size_t n = valid ? (size_t)kept[idx / s] * s + idx % s : 0;
+            float up = subwarp_dot((const T *)a.w1 + n * d, xs, d, lpr, sl, valid);
+            float gate = 0.0f;
+            if (GATED) gate = subwarp_dot((const T *)a.w_gate + n * d, xs, d, lpr, sl, valid);
+            if (valid && sl == 0) {
+                if (a.b1) up += d2d_to_float<T>(((const T *)a.b1)[n]);
+                hs[idx] = GATED ? d2d_activate<ACT>(gate) * up : d2d_activate<ACT>(up);
             }
-        }
-        up = d2d_warp_sum(up);
-        if (GATED) gate = d2d_warp_sum(gate);
-        if (lane == 0) {
-            if (a.b1) up += d2d_to_float<T>(((const T *)a.b1)[n]);
-            hs[idx] = GATED ? d2d_activate<ACT>(gate) * up : d2d_activate<ACT>(up);
         }
     }
     __syncthreads();

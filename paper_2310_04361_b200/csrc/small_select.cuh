@@ -68,8 +68,56 @@ __device__ __forceinline__ void select_cta(const float *R, int T, int E, int W, 
     }
     __syncthreads();
 
-    // per-expert counts and the exclusive scan over experts (chunks of blockDim.x experts)
+    // per-expert counts, the exclusive scan over experts and the token lists
     int carry = 0;
+    if (E * 4 <= nthreads) {
+        // few experts: a warp per expert with its lanes over the tokens (ballots keep the lists in ascending order)
+        __shared__ int scnt[256], soff[256];
+        const uint32_t lower = (1u << lane) - 1u;
+        for (int e = warp; e < E; e += nwarps) {
+            int c = 0;
+            for (int t0 = 0; t0 < T; t0 += 32) {
+                const int t = t0 + lane;
+                const bool bit = t < T && ((smask[t * W + (e >> 5)] >> (e & 31)) & 1u);
+                c += __popc(__ballot_sync(FULL, bit));
+            }
+            if (lane == 0) scnt[e] = c;
+        }
+        __syncthreads();
+        if (warp == 0) {
+            int run = 0;
+            for (int e0 = 0; e0 < E; e0 += 32) {
+                const int e = e0 + lane;
+                const int c = e < E ? scnt[e] : 0;
+                int inc = c;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int n = __shfl_up_sync(FULL, inc, o);
+                    if (lane >= o) inc += n;
+                }
+                if (e < E) {
+                    soff[e] = run + inc - c;
+                    counts[e] = c;
+                    offsets[e] = run + inc - c;
+                }
+                run += __shfl_sync(FULL, inc, 31);
+            }
+            if (lane == 0) chunk_total = run;
+        }
+        __syncthreads();
+        carry = chunk_total;
+        for (int e = warp; e < E; e += nwarps) {
+            long long idx = soff[e];
+            for (int t0 = 0; t0 < T; t0 += 32) {
+                const int t = t0 + lane;
+                const bool bit = t < T && ((smask[t * W + (e >> 5)] >> (e & 31)) & 1u);
+                const uint32_t b = __ballot_sync(FULL, bit);
+                const long long at = idx + __popc(b & lower);
+                if (bit && at < capacity) perm[at] = t;
+                idx += __popc(b);
+            }
+        }
+    } else {
     for (int e0 = 0; e0 < E; e0 += nthreads) {
         const int e = e0 + threadIdx.x;
         int c = 0;
@@ -110,24 +158,44 @@ __device__ __forceinline__ void select_cta(const float *R, int T, int E, int W, 
         carry += chunk_total;
         __syncthreads();
     }
+    }
     if (threadIdx.x == 0) {
         offsets[E] = carry;
         *n_sel = carry;
         if ((long long)carry > capacity) atomicMax(status, (int32_t)D2D_ERR_CAPACITY);
     }
-    // token-major dual: one thread per token
-    for (int t = threadIdx.x; tok_off && tok_exp && t < T; t += nthreads) {
-        long long base = 0;
-        for (int u = 0; u < t; ++u) base += sk[u];
-        tok_off[t] = (int32_t)base;
-        if (t == T - 1) tok_off[T] = (int32_t)(base + sk[t]);
-        for (int w = 0; w < W; ++w) {
-            uint32_t word = smask[t * W + w];
-            while (word) {
-                const int b = __ffs(word) - 1;
-                word &= word - 1;
-                if (base < capacity) tok_exp[base] = w * 32 + b;
-                ++base;
+    // token-major dual: exclusive scan of k by warp 0, then one thread per token
+    if (tok_off && tok_exp) {
+        __shared__ int stok[MAX_T];
+        __syncthreads();
+        if (warp == 0) {
+            int run = 0;
+            for (int t0 = 0; t0 < T; t0 += 32) {
+                const int t = t0 + lane;
+                const int c = t < T ? sk[t] : 0;
+                int inc = c;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int n = __shfl_up_sync(FULL, inc, o);
+                    if (lane >= o) inc += n;
+                }
+                if (t < T) stok[t] = run + inc - c;
+                run += __shfl_sync(FULL, inc, 31);
+            }
+        }
+        __syncthreads();
+        for (int t = threadIdx.x; t < T; t += nthreads) {
+            long long base = stok[t];
+            tok_off[t] = (int32_t)base;
+            if (t == T - 1) tok_off[T] = (int32_t)(base + sk[t]);
+            for (int w = 0; w < W; ++w) {
+                uint32_t word = smask[t * W + w];
+                while (word) {
+                    const int b = __ffs(word) - 1;
+                    word &= word - 1;
+                    if (base < capacity) tok_exp[base] = w * 32 + b;
+                    ++base;
+                }
             }
         }
     }
