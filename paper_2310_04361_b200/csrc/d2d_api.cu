@@ -204,8 +204,14 @@ static d2d_status launch_tc_experts(const d2d_layer *L, const void *x, int T, co
     if (path != D2D_PATH_DENSE) {
         const long long hi = path == D2D_PATH_AUTO ? n_sel_max : LLONG_MAX;
         if (zero_fill) {
-            rc = d2d_moe_zero_unkept(ws, r->mask, T, D.d_ff, D.n_experts, D.expert_size, L->gather_group, n_sel, n_sel_fused, hi, st);
+            // on the layer's side stream: the fill and the gathered kernel write disjoint cells, and its small CTAs fit
+            // beside the persistent ones; joined before the down projection
+            if (cudaEventRecord(L->ev_fill_fork, st) != cudaSuccess || cudaStreamWaitEvent(L->side_stream, L->ev_fill_fork, 0) != cudaSuccess)
+                return D2D_ERR_CUDA;
+            rc = d2d_moe_zero_unkept(ws, r->mask, T, D.d_ff, D.n_experts, D.expert_size, L->gather_group, n_sel, n_sel_fused, hi,
+                                     L->side_stream);
             if (rc != D2D_OK) return rc;
+            if (cudaEventRecord(L->ev_fill_join, L->side_stream) != cudaSuccess) return D2D_ERR_CUDA;
         }
         d2d_gather_args ga = {};
         ga.x = x; ga.w1 = L->w1; ga.w_gate = D.gated ? L->w_gate : nullptr; ga.b1 = L->b1; ga.mask = r->mask; ga.H = ws;
@@ -219,6 +225,7 @@ static d2d_status launch_tc_experts(const d2d_layer *L, const void *x, int T, co
         rc = d2d_moe_down_masked(D, ws, r->mask, L->w2, L->b2, y, T, r->status, st, path == D2D_PATH_AUTO ? n_sel : nullptr, n_sel_fused, n_sel_max);
         if (rc != D2D_OK || path == D2D_PATH_GATHER) return rc;
     }
+    if (zero_fill && cudaStreamWaitEvent(st, L->ev_fill_join, 0) != cudaSuccess) return D2D_ERR_CUDA;
     d2d_gemm_args dn = {};
     dn.a = ws; dn.b = L->w2; dn.bias = L->b2; dn.out = y;
     // after a zero fill this kernel serves the gathered range too: it only has to stay out of the fused kernel's range
@@ -350,7 +357,9 @@ d2d_status d2d_layer_create(const d2d_layer_desc *desc, const d2d_weights *w, vo
     if (rc == D2D_OK && cudaStreamSynchronize(st) != cudaSuccess) rc = D2D_ERR_CUDA;
     if (rc == D2D_OK && (cudaStreamCreateWithFlags(&L->side_stream, cudaStreamNonBlocking) != cudaSuccess ||
                          cudaEventCreateWithFlags(&L->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
-                         cudaEventCreateWithFlags(&L->ev_join, cudaEventDisableTiming) != cudaSuccess))
+                         cudaEventCreateWithFlags(&L->ev_join, cudaEventDisableTiming) != cudaSuccess ||
+                         cudaEventCreateWithFlags(&L->ev_fill_fork, cudaEventDisableTiming) != cudaSuccess ||
+                         cudaEventCreateWithFlags(&L->ev_fill_join, cudaEventDisableTiming) != cudaSuccess))
         rc = D2D_ERR_CUDA;
     if (rc == D2D_OK) {
         bool ok = cudaStreamCreateWithFlags(&L->copy_in, cudaStreamNonBlocking) == cudaSuccess &&
@@ -374,6 +383,8 @@ d2d_status d2d_layer_destroy(d2d_layer *layer)
 {
     if (!layer) return D2D_OK;
     if (layer->ev_join) cudaEventDestroy(layer->ev_join);
+    if (layer->ev_fill_fork) cudaEventDestroy(layer->ev_fill_fork);
+    if (layer->ev_fill_join) cudaEventDestroy(layer->ev_fill_join);
     if (layer->ev_fork) cudaEventDestroy(layer->ev_fork);
     if (layer->side_stream) cudaStreamDestroy(layer->side_stream);
     for (int c = 0; c < d2d_layer::kHostChunks; ++c) {

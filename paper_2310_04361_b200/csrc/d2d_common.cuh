@@ -25,6 +25,7 @@ struct d2d_layer {
     // expert GEMMs, which do not read it
     cudaStream_t side_stream;
     cudaEvent_t ev_fork, ev_join;
+    cudaEvent_t ev_fill_fork, ev_fill_join;      // zero fill of H beside the gathered up projection (side stream)
     // d2d_layer_fwd_host: copy-in and copy-out streams and per-chunk events, so that the host -> device copy of one
     // chunk of tokens, the layer on the previous chunk and the device -> host copy of the one before overlap
     static const int kHostChunks = 4;
