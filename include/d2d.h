@@ -335,8 +335,8 @@ D2D_API d2d_status d2d_test_inject_fault(int32_t kind);
  * are outputs): mask, k and status are required; the per-expert lists
  * (counts, offsets, perm, n_sel and the dual) may be NULL as a set, in which
  * case they are not built -- allowed where the expert kernels read only the
- * mask (bf16 batches of 5 or more tokens with d_h = 128 and E <= 256),
- * D2D_ERR_INVALID_ARG elsewhere.  Work is enqueued on `stream`; the per-expert
+ * mask (bf16 batches of more than 64 tokens; from 5 tokens with d_h = 128 and
+ * E <= 256; small float32 problems), D2D_ERR_INVALID_ARG elsewhere.  Work is enqueued on `stream`; the per-expert
  * metadata may be built on a stream the layer owns, joined back into `stream`
  * before the call's last operation, so everything the call writes is ordered
  * before whatever the caller enqueues on `stream` next.  The layer object

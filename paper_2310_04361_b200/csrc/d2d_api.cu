@@ -653,9 +653,7 @@ d2d_status d2d_layer_fwd(const d2d_layer *layer, const void *x, int32_t T, float
         // small float32 problems: router, rule, experts and lists in one launch
         if (cudaMemsetAsync(routing->status, 0, sizeof(int32_t), st) != cudaSuccess) return D2D_ERR_CUDA;
         return d2d_layer_token_fused(layer, x, T, tau, y, R_out, routing, lists, layer->tickets + 52, st);
-    } else if (!lists) {
-        return D2D_ERR_INVALID_ARG;                           // every other path builds (and its expert kernels use) the lists
-    } else if (d2d_small_router_supports(layer->desc, T)) {
+    } else if (lists && d2d_small_router_supports(layer->desc, T)) {
         // decode batches: the router kernel's last CTA selects as well (one launch for router + selection)
         const bool small = use_small_ffn(layer, T);
         float *y32 = (float *)(base + w.ffn_off + 256);
@@ -663,6 +661,27 @@ d2d_status d2d_layer_fwd(const d2d_layer *layer, const void *x, int32_t T, float
                               small ? T * layer->desc.d : 0);
         if (rc != D2D_OK) return rc;
         return d2d_launch_moe_ffn(layer, x, T, routing, y, base + w.ffn_off, w.total - w.ffn_off, st, nullptr, small ? 1 : 0);
+    } else if (use_dense_masked(layer, T) && !use_small_ffn(layer, T) && !d2d_small_select_supports(T, E)) {
+        // router shapes the fused kernel does not take, tensor-core expert step: scores by two GEMMs, then mask, k and
+        // the number of selected pairs by one kernel; the per-expert lists (when wanted) are built on the side stream
+        // while the experts, which read only the mask, run
+        rc = d2d_launch_router(layer, x, T, R, (float *)(base + w.u_off), st);
+        if (rc != D2D_OK) return rc;
+        int32_t *ksum = (int32_t *)(layer->tickets + 40);
+        rc = d2d_launch_dynk_mask(R, T, E, tau, routing, ksum, st);
+        if (rc != D2D_OK) return rc;
+        if (lists) {
+            if (cudaEventRecord(layer->ev_fork, st) != cudaSuccess || cudaStreamWaitEvent(layer->side_stream, layer->ev_fork, 0) != cudaSuccess)
+                return D2D_ERR_CUDA;
+            rc = d2d_launch_select(nullptr, T, E, tau, 0, routing, base + w.sel_off, layer->side_stream, 1);
+            if (rc != D2D_OK) return rc;
+        }
+        rc = d2d_launch_moe_ffn(layer, x, T, routing, y, base + w.ffn_off, w.total - w.ffn_off, st, nullptr, 0, ksum + 4);
+        if (lists && (cudaEventRecord(layer->ev_join, layer->side_stream) != cudaSuccess || cudaStreamWaitEvent(st, layer->ev_join, 0) != cudaSuccess))
+            return D2D_ERR_CUDA;
+        return rc;
+    } else if (!lists) {
+        return D2D_ERR_INVALID_ARG;                           // every other path builds (and its expert kernels use) the lists
     } else {
         rc = d2d_launch_router(layer, x, T, R, (float *)(base + w.u_off), st);
         if (rc != D2D_OK) return rc;

@@ -94,6 +94,7 @@ d2d_status d2d_launch_router(const d2d_layer *L, const void *x, int T, float *R,
 size_t d2d_select_ws_bytes(int T, int E);
 // R == nullptr: the mask is an input.  mask_ready != 0: mask, k and the status word were already written
 // (fused router), only the per-expert metadata is built.
+d2d_status d2d_launch_dynk_mask(const float *R, int T, int E, float tau, const d2d_routing *out, int32_t *ksum, cudaStream_t st);
 d2d_status d2d_launch_select(const float *R, int T, int E, float tau, int topk, const d2d_routing *out,
                              void *ws, cudaStream_t st, int mask_ready = 0);
 

@@ -23,39 +23,59 @@ __device__ __forceinline__ bool is_finite_f32(float v) { return (__float_as_uint
 
 // ---------------------------------------------------------------------------- mask kernels
 
+// ksum (optional): [0] running sum of k over the CTAs, [1] exit ticket (both zero at launch and left at zero), [4]
+// receives the total = number of selected (token, expert) pairs, for the density-adaptive dispatch of the expert step.
 __global__ void __launch_bounds__(256)
 dynk_mask_kernel(const float *__restrict__ R, int T, int E, int W, float tau,
-                 uint32_t *__restrict__ mask, int32_t *__restrict__ k, int32_t *__restrict__ status)
+                 uint32_t *__restrict__ mask, int32_t *__restrict__ k, int32_t *__restrict__ status, int32_t *ksum)
 {
+    __shared__ int block_k;
+    if (ksum) {
+        if (threadIdx.x == 0) block_k = 0;
+        __syncthreads();
+    }
     const int lane = threadIdx.x & 31;
     const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (t >= T) return;
-    const float *row = R + (size_t)t * E;
-    float m = -INFINITY;
-    bool bad = false;
-    for (int i = lane; i < E; i += 32) {
-        const float v = __ldg(row + i);
-        bad |= !is_finite_f32(v);
-        m = v > m ? v : m;
-    }
+    if (t < T) {
+        const float *row = R + (size_t)t * E;
+        float m = -INFINITY;
+        bool bad = false;
+        for (int i = lane; i < E; i += 32) {
+            const float v = __ldg(row + i);
+            bad |= !is_finite_f32(v);
+            m = v > m ? v : m;
+        }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        const float other = __shfl_xor_sync(FULL, m, o);
-        m = other > m ? other : m;
+        for (int o = 16; o > 0; o >>= 1) {
+            const float other = __shfl_xor_sync(FULL, m, o);
+            m = other > m ? other : m;
+        }
+        bad = __any_sync(FULL, bad);
+        const float thr = __fmul_rn(tau, m);     // the one rounding the rule is defined with
+        int kt = 0;
+        for (int w = 0; w < W; ++w) {
+            const int i = w * 32 + lane;
+            const bool keep = (i < E) && (bad || __ldg(row + i) >= thr);
+            const uint32_t word = __ballot_sync(FULL, keep);
+            if (lane == 0) mask[(size_t)t * W + w] = word;
+            kt += __popc(word);
+        }
+        if (lane == 0) {
+            k[t] = kt;
+            if (bad) atomicMax(status, (int32_t)D2D_ERR_NONFINITE);
+            if (ksum) atomicAdd(&block_k, kt);
+        }
     }
-    bad = __any_sync(FULL, bad);
-    const float thr = __fmul_rn(tau, m);     // the one rounding the rule is defined with
-    int kt = 0;
-    for (int w = 0; w < W; ++w) {
-        const int i = w * 32 + lane;
-        const bool keep = (i < E) && (bad || __ldg(row + i) >= thr);
-        const uint32_t word = __ballot_sync(FULL, keep);
-        if (lane == 0) mask[(size_t)t * W + w] = word;
-        kt += __popc(word);
-    }
-    if (lane == 0) {
-        k[t] = kt;
-        if (bad) atomicMax(status, (int32_t)D2D_ERR_NONFINITE);
+    if (!ksum) return;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        atomicAdd(ksum, block_k);
+        __threadfence();
+        if (atomicAdd(ksum + 1, 1) == (int)gridDim.x - 1) {          // the last CTA publishes the total and resets
+            __threadfence();
+            ksum[4] = atomicExch(ksum, 0);
+            ksum[1] = 0;
+        }
     }
 }
 
@@ -335,6 +355,16 @@ size_t d2d_select_ws_bytes(int T, int E)
     return 256 + d2d_align_up(nblk * (size_t)E * sizeof(int32_t), 256);
 }
 
+// Mask, k and status only (Eq. 4), T > 0; the sum of k is published through ksum (see the kernel).  The per-expert
+// lists can be built afterwards, on any stream ordered behind this one, with d2d_launch_select(nullptr, ..., mask_ready = 1).
+d2d_status d2d_launch_dynk_mask(const float *R, int T, int E, float tau, const d2d_routing *out, int32_t *ksum, cudaStream_t st)
+{
+    D2D_CUDA_TRY(cudaMemsetAsync(out->status, 0, sizeof(int32_t), st));
+    dynk_mask_kernel<<<d2d_cdiv(T, 8), 256, 0, st>>>(R, T, E, (E + 31) / 32, tau, out->mask, out->k, out->status, ksum);
+    D2D_LAUNCHED(1);
+    return cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
+}
+
 d2d_status d2d_launch_select(const float *R, int T, int E, float tau, int topk, const d2d_routing *out,
                              void *ws, cudaStream_t st, int mask_ready)
 {
@@ -354,7 +384,7 @@ d2d_status d2d_launch_select(const float *R, int T, int E, float tau, int topk, 
         if (topk > 0)
             topk_mask_kernel<<<grid_tok, 256, 0, st>>>(R, T, E, W, topk, out->mask, out->k, out->status);
         else
-            dynk_mask_kernel<<<grid_tok, 256, 0, st>>>(R, T, E, W, tau, out->mask, out->k, out->status);
+            dynk_mask_kernel<<<grid_tok, 256, 0, st>>>(R, T, E, W, tau, out->mask, out->k, out->status, nullptr);
     } else if (!mask_ready) {
         k_from_mask_kernel<<<d2d_cdiv(T, 256), 256, 0, st>>>(out->mask, T, W, out->k);
     }
