@@ -984,11 +984,21 @@ y32_fill_kernel(float *__restrict__ y32, const __nv_bfloat16 *__restrict__ b2, l
         const long long n = (long long)__ldcg(n_sel);
         if (!(n > n_sel_min && n <= n_sel_max)) return;
     }
-    for (long long i = ((long long)blockIdx.x * 256 + threadIdx.x) * 4; i < total; i += (long long)gridDim.x * 1024) {
-        const int n = (int)(i % d);
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (b2) v = make_float4(__bfloat162float(b2[n]), __bfloat162float(b2[n + 1]), __bfloat162float(b2[n + 2]), __bfloat162float(b2[n + 3]));
-        *reinterpret_cast<float4 *>(y32 + i) = v;
+    // one float4 per thread and step, four steps in flight; the column of a float4 by 32-bit arithmetic
+    const unsigned int q_total = (unsigned int)(total >> 2), q_row = (unsigned int)(d >> 2), stride = gridDim.x * 256u;
+    for (unsigned int q0 = blockIdx.x * 256u + threadIdx.x; q0 < q_total; q0 += 4u * stride) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const unsigned int q = q0 + (unsigned int)u * stride;
+            if (q >= q_total) break;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (b2) {
+                const uint2 w = __ldg(reinterpret_cast<const uint2 *>(b2) + q % q_row);
+                const __nv_bfloat162 lo = *reinterpret_cast<const __nv_bfloat162 *>(&w.x), hi = *reinterpret_cast<const __nv_bfloat162 *>(&w.y);
+                v = make_float4(__low2float(lo), __high2float(lo), __low2float(hi), __high2float(hi));
+            }
+            __stcs(reinterpret_cast<float4 *>(y32) + q, v);
+        }
     }
 }
 
@@ -1002,13 +1012,24 @@ y32_convert_kernel(const float *__restrict__ y32, __nv_bfloat16 *__restrict__ y,
         const long long n = (long long)__ldcg(n_sel);
         if (!(n > n_sel_min && n <= n_sel_max)) return;
     }
-    for (long long i = ((long long)blockIdx.x * 256 + threadIdx.x) * 4; i < total; i += (long long)gridDim.x * 1024) {
-        const float4 v = __ldcs(reinterpret_cast<const float4 *>(y32 + i));
-        const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
-        uint2 o;
-        o.x = *reinterpret_cast<const uint32_t *>(&lo);
-        o.y = *reinterpret_cast<const uint32_t *>(&hi);
-        *reinterpret_cast<uint2 *>(y + i) = o;
+    const unsigned int q_total = (unsigned int)(total >> 2), stride = gridDim.x * 256u;
+    for (unsigned int q0 = blockIdx.x * 256u + threadIdx.x; q0 < q_total; q0 += 4u * stride) {
+        float4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const unsigned int q = q0 + (unsigned int)u * stride;
+            if (q < q_total) v[u] = __ldcs(reinterpret_cast<const float4 *>(y32) + q);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const unsigned int q = q0 + (unsigned int)u * stride;
+            if (q >= q_total) break;
+            const __nv_bfloat162 lo = __floats2bfloat162_rn(v[u].x, v[u].y), hi = __floats2bfloat162_rn(v[u].z, v[u].w);
+            uint2 o;
+            o.x = *reinterpret_cast<const uint32_t *>(&lo);
+            o.y = *reinterpret_cast<const uint32_t *>(&hi);
+            reinterpret_cast<uint2 *>(y)[q] = o;
+        }
     }
 }
 
@@ -1277,7 +1298,8 @@ static d2d_status launch_ffn(const d2d_gather_args &a, float *y32, void *y, cons
     const long long total = (long long)a.T * a.d;
     const int blocks = (int)((total / 4 + 255) / 256);
     const int sms = d2d_tc_sm_count();
-    cfg.gridDim = dim3(blocks < 4 * sms ? blocks : 4 * sms, 1, 1);
+    if (total / 4 >= (1ll << 31)) return D2D_ERR_UNSUPPORTED;
+    cfg.gridDim = dim3(blocks < 8 * sms ? blocks : 8 * sms, 1, 1);
     cfg.blockDim = dim3(256, 1, 1);
     cfg.dynamicSmemBytes = 0;
     cudaError_t err = cudaLaunchKernelEx(&cfg, y32_fill_kernel, y32, (const __nv_bfloat16 *)b2, total, a.d, a.n_sel, a.n_sel_min, a.n_sel_max);
