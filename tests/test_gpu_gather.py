@@ -36,6 +36,15 @@ def _per_token_err(got, ref):
     return float((np.abs(got - ref).max(1) / np.maximum(np.abs(ref).max(1), 1e-30)).max())
 
 
+def _config(name):
+    """Workload by name; "wide" is a plain GELU layer with d = 2048 (the only plain shape here on which the gathered path
+    zero-fills H and keeps the TMA-fed down projection, and on which all three ranges of the automatic choice exist)."""
+    if name == "wide":
+        import dataclasses
+        return dataclasses.replace(wl.CONFIGS["bert"], name="wide", d=2048, d_ff=4096, T=12288, seed=9)
+    return wl.CONFIGS[name]
+
+
 def _routing(api, G, E):
     return api.routing_from_mask(torch.from_numpy(oracle.pack_mask(G).view(np.int32)).cuda(), E)
 
@@ -105,14 +114,14 @@ def test_gathered_up_projection_equals_masked_dense_and_oracle(api, name, T, g, 
     layer.close()
 
 
-PATH_CASES = [("bert", 1000, 0.5), ("bert", 640, 0.9), ("vit", 1500, 0.6), ("paper", 1500, 0.3), ("llama", 520, 0.6)]
+PATH_CASES = [("bert", 1000, 0.5), ("bert", 640, 0.9), ("vit", 1500, 0.6), ("paper", 1500, 0.3), ("llama", 520, 0.6), ("wide", 700, 0.5)]
 
 
 @pytest.mark.parametrize("name,T,tau", PATH_CASES)
 def test_layer_fwd_is_the_same_on_both_sides_of_the_dispatch(api, name, T, tau):
     """d2d_layer_fwd and d2d_moe_ffn_fwd with the up projection forced dense, forced gathered, and chosen on the
     device with the crossover moved to either extreme: identical masks, y equal to the oracle's on that mask."""
-    cfg = wl.with_tokens(wl.CONFIGS[name], T)
+    cfg = wl.with_tokens(_config(name), T)
     w, x = wl.make_weights(cfg), wl.make_tokens(cfg)
     layer = api.Layer.from_config(cfg, w)
     xd = api.to_device(x, cfg.dtype)
@@ -146,12 +155,12 @@ def test_layer_fwd_is_the_same_on_both_sides_of_the_dispatch(api, name, T, tau):
     layer.close()
 
 
-@pytest.mark.parametrize("name,tau", [("paper", 0.5), ("llama", 0.6)])
+@pytest.mark.parametrize("name,tau", [("paper", 0.5), ("llama", 0.6), ("wide", 0.5)])
 def test_device_side_choice_at_full_size(api, name, tau):
     """Batches large enough for the automatic choice: the crossover is moved to either extreme so that the decision
     taken on the device goes each way (both kernel pairs are enqueued, one returns at once); y is checked against
     the oracle on sampled tokens, at least one from every 128-token row tile."""
-    cfg = wl.CONFIGS[name]
+    cfg = _config(name)
     w, x = wl.make_weights(cfg), wl.make_tokens(cfg)
     layer = api.Layer.from_config(cfg, w)
     xd = api.to_device(x, cfg.dtype)
@@ -161,7 +170,7 @@ def test_device_side_choice_at_full_size(api, name, tau):
     tiles = np.arange(0, T, 128)
     sample = np.unique(np.concatenate([tiles + rng.integers(0, 128, tiles.shape), [0, T - 1]]))
     sample = sample[sample < T]
-    if name == "llama":
+    if name in ("llama", "wide"):
         sample = sample[:: 2]                                  # the oracle needs about 0.1 s per Llama-sized token
     ref = None
     # (crossover of the gathered pair, upper end of the fused kernel's range): dense pair, gathered pair, fused kernel,
