@@ -183,3 +183,61 @@ def layer(x, wts: dict, act: int, tau: float) -> dict:
     meta = metadata(G)
     y = moe_ffn(x, wts["w1"], wts.get("b1"), wts.get("w_gate"), wts["w2"], wts.get("b2"), act, G)
     return {"R": R, "G": G, "k": k, "nonfinite": bad, "y": y, **meta}
+
+
+# ---------------------------------------------------------------------------------------------------------
+# Low-precision expert weights (the paper's App. C runs the expert kernels on narrower number formats): an
+# expert's weights as 8-bit floating point (1 sign, 4 exponent, 3 mantissa bits, bias 7, no infinities: the
+# "e4m3" format) with ONE power-of-two scale per expert and matrix.  Written out from the format's definition:
+# the 127 finite non-negative values are tabulated and a weight goes to the nearest one, ties to the code with
+# an even mantissa bit, values beyond the largest finite one (448) to 448.
+
+def e4m3_values() -> np.ndarray:
+    """The value of every non-negative finite code 0x00 .. 0x7e (code 0x7f is NaN), ascending."""
+    v = np.empty(127, dtype=np.float64)
+    for code in range(127):
+        e, m = code >> 3, code & 7
+        v[code] = (m / 8.0) * 2.0 ** -6 if e == 0 else (1.0 + m / 8.0) * 2.0 ** (e - 7)
+    return v
+
+
+def e4m3_encode(a) -> np.ndarray:
+    """Codes (uint8, sign in bit 7) of the e4m3 values nearest to `a` (float array, finite): round to nearest,
+    ties to even, saturating at +-448."""
+    a = np.asarray(a, dtype=np.float64)
+    vals = e4m3_values()
+    mag = np.minimum(np.abs(a), vals[-1])
+    hi = np.searchsorted(vals, mag, side="left")              # first code whose value is >= mag
+    hi = np.minimum(hi, 126)
+    lo = np.maximum(hi - 1, 0)
+    d_lo, d_hi = mag - vals[lo], vals[hi] - mag
+    take_hi = (d_hi < d_lo) | ((d_hi == d_lo) & (hi % 2 == 0))
+    code = np.where(take_hi, hi, lo).astype(np.uint8)
+    return code | (np.signbit(a).astype(np.uint8) << 7)
+
+
+def e4m3_decode(code) -> np.ndarray:
+    code = np.asarray(code, dtype=np.uint8)
+    v = e4m3_values()[np.minimum(code & 0x7F, 126)]
+    return np.where(code & 0x80, -v, v)
+
+
+def quantize_experts_e4m3(w_rows, n_experts: int):
+    """w_rows: [n_experts * s, d] float, expert e owns rows [e*s, (e+1)*s) (W1 or W_gate as given; for W2 pass its
+    transpose).  Per expert: scale 2^k with the smallest integer k for which max|w| / 2^k <= 448 (k = 0 for an
+    all-zero expert), codes = e4m3_encode(w / 2^k).  Returns (codes uint8 [n_experts*s, d], k int32 [n_experts],
+    dequantised float32 [n_experts*s, d] = decode(codes) * 2^k, exactly representable in bfloat16)."""
+    w = np.asarray(w_rows, dtype=np.float64)
+    rows, d = w.shape
+    s = rows // n_experts
+    blocks = w.reshape(n_experts, s * d)
+    amax = np.abs(blocks).max(axis=1)
+    k = np.zeros(n_experts, dtype=np.int32)
+    nz = amax > 0
+    # smallest k with amax <= 448 * 2^k: frexp gives amax / 448 = f * 2^p with f in [0.5, 1), so k = p unless f == 0.5
+    f, p = np.frexp(amax[nz] / 448.0)
+    k[nz] = np.where(f == 0.5, p - 1, p)
+    scale = np.ldexp(1.0, k)[:, None]
+    codes = e4m3_encode(blocks / scale)
+    deq = (e4m3_decode(codes) * scale).astype(np.float32)
+    return codes.reshape(rows, d), k, deq.reshape(rows, d)

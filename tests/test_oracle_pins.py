@@ -348,3 +348,68 @@ def test_cost_ratio_closed_form(d_m, e, n, d_h):
         assert math.isclose(ratio, closed, rel_tol=1e-12)
     if d_m == 6 * d_h and n == 128:       # the paper's setting d_m = 6 d_h, e = 4
         assert math.isclose((c_router) / c_dense, 0.024305555555555556, rel_tol=1e-12)
+
+
+# ---------------------------------------------------------------- 8-bit expert weights (App. C: narrower formats)
+
+def test_e4m3_table_against_the_format_and_a_library_cast():
+    """The 127 finite values: smallest subnormal 2^-9, smallest normal 2^-6, largest 448, eight codes per binade with
+    a spacing that doubles from binade to binade; and code for code what torch's float8_e4m3fn holds."""
+    v = oracle.e4m3_values()
+    assert len(v) == 127 and v[0] == 0.0 and v[1] == 2.0 ** -9 and v[8] == 2.0 ** -6 and v[126] == 448.0
+    assert (np.diff(v) > 0).all()
+    steps = np.diff(v)
+    assert (steps[:15] == 2.0 ** -9).all()                           # subnormals and the first binade share one step
+    for b in range(2, 15):                                           # binade b starts at code 8 b
+        assert (steps[8 * b: 8 * b + 7] == 2.0 ** (b - 10)).all()
+    lib = torch.arange(256, dtype=torch.uint8).view(torch.float8_e4m3fn).float().numpy()
+    codes = np.arange(256, dtype=np.uint8)
+    finite = (codes & 0x7F) != 0x7F
+    assert np.array_equal(oracle.e4m3_decode(codes[finite]), lib[finite].astype(np.float64))
+
+
+def test_e4m3_rounding_is_to_nearest_with_ties_to_even_and_saturates():
+    # hand-placed ties: halfway between two neighbours the code with an even mantissa bit wins
+    x = np.array([2.0 ** -10, 3 * 2.0 ** -10, 1.0625, 1.1875, 17.0, 19.0, -17.0, 432.0])
+    assert oracle.e4m3_encode(x).tolist() == [0, 2, 56, 58, 88, 90, 0x80 | 88, 126]
+    # just off the tie the nearer neighbour wins
+    assert oracle.e4m3_encode(np.array([1.0625 + 1e-9, 1.0625 - 1e-9])).tolist() == [57, 56]
+    # beyond the largest finite value: saturation, never the NaN code
+    assert oracle.e4m3_encode(np.array([449.0, 1e9, -1e9])).tolist() == [126, 126, 0x80 | 126]
+    # every representable value encodes to itself
+    codes = np.array([c for c in range(256) if (c & 0x7F) != 0x7F and c != 0x80], dtype=np.uint8)
+    assert np.array_equal(oracle.e4m3_encode(oracle.e4m3_decode(codes)), codes)
+    # a library cast agrees on random in-range values (torch rounds to nearest even as well)
+    rng = np.random.default_rng(5)
+    r = (rng.standard_normal(20000) * np.exp(rng.uniform(-8, 5, 20000))).astype(np.float32)
+    r = r[np.abs(r) <= 448.0]
+    lib = torch.from_numpy(r).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    ours = oracle.e4m3_encode(r)
+    zero = (ours & 0x7F) == 0                                        # the sign of a value rounded to zero is free
+    assert np.array_equal(ours[~zero], lib[~zero]) and ((lib[zero] & 0x7F) == 0).all()
+
+
+def test_expert_scales_are_the_smallest_power_of_two_that_fits():
+    rng = np.random.default_rng(8)
+    E, s, d = 6, 8, 32
+    w = (rng.standard_normal((E * s, d)) * 0.02).astype(np.float32)
+    w[2 * s: 3 * s] = 0.0                                            # an all-zero expert
+    w[3 * s: 4 * s] *= 0.0
+    w[3 * s, 0] = 448.0 * 2.0 ** -9                                  # an expert whose maximum sits exactly on the boundary
+    w[4 * s: 5 * s] *= 1e3
+    codes, k, deq = oracle.quantize_experts_e4m3(w, E)
+    assert k[2] == 0 and not codes[2 * s: 3 * s].any()
+    assert k[3] == -9 and codes[3 * s, 0] == 126
+    for e in range(E):
+        blk = np.abs(w[e * s: (e + 1) * s].astype(np.float64))
+        if blk.max() > 0:
+            assert blk.max() <= 448.0 * 2.0 ** int(k[e]) < 2 * blk.max()        # fits, and half the scale would not
+        # error of a normal value: half a mantissa step, 2^-4 relative; below the smallest normal: 2^(k - 10) absolute
+        err = np.abs(deq[e * s: (e + 1) * s].astype(np.float64) - w[e * s: (e + 1) * s])
+        assert (err <= np.maximum(blk * 2.0 ** -4, 2.0 ** (int(k[e]) - 10))).all()
+    # the dequantised weights are bfloat16 values: a layer can hold them in its bf16 copies without further rounding
+    assert torch.equal(torch.from_numpy(deq).to(torch.bfloat16).float(), torch.from_numpy(deq))
+    # scaling an expert by a power of two moves its exponent and leaves its codes alone
+    w2 = w.copy(); w2[: s] *= 4.0
+    codes2, k2, _ = oracle.quantize_experts_e4m3(w2, E)
+    assert k2[0] == k[0] + 2 and np.array_equal(codes2[: s], codes[: s])
