@@ -144,6 +144,25 @@ D2D_API uint64_t d2d_launch_count(void);
  * pointers.  On failure *out is NULL. */
 D2D_API d2d_status d2d_layer_create(const d2d_layer_desc *desc, const d2d_weights *w, void *stream, d2d_layer **out);
 
+/* The same layer with 8-bit expert weights (App. C runs the expert kernels on
+ * narrower number formats).  Every expert's slice of W1, W_gate and W2 is
+ * rounded to 8-bit floating point codes (e4m3: 1 sign, 4 exponent, 3 mantissa
+ * bits, bias 7, largest value 448; round to nearest, ties to even, saturating)
+ * with ONE power-of-two scale 2^k per expert and matrix, k the smallest integer
+ * for which the slice's largest magnitude fits (0 for an all-zero slice).  The
+ * layer then computes with the rounded weights value(code) * 2^k on every path
+ * (they are exactly bf16 values, kept in the packed bf16 copies); the decode
+ * kernels read the codes, half the bytes per kept expert.  Router weights and
+ * biases are not touched.  bf16 layers with d and expert_size * d multiples of
+ * 16 only (D2D_ERR_UNSUPPORTED otherwise).  Costs d_ff * d bytes per matrix on
+ * top of d2d_layer_create. */
+D2D_API d2d_status d2d_layer_create_fp8(const d2d_layer_desc *desc, const d2d_weights *w, void *stream, d2d_layer **out);
+/* Copies the codes (device uint8 [d_ff, d]; an expert = expert_size contiguous
+ * rows; which = 2: of W2 transposed) and/or the exponents k (device int32 [E])
+ * of which = 0: W1, 1: W_gate, 2: W2.  Either output may be NULL.
+ * D2D_ERR_UNSUPPORTED for a layer without 8-bit weights (or without W_gate). */
+D2D_API d2d_status d2d_layer_get_fp8(const d2d_layer *layer, int32_t which, uint8_t *codes, int32_t *exps, void *stream);
+
 /* Frees the handle and its device copies.  NULL is a no-op. */
 D2D_API d2d_status d2d_layer_destroy(d2d_layer *layer);
 

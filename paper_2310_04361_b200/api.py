@@ -27,7 +27,7 @@ STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "WORKSPACE", 4: 
 D2D_F32, D2D_BF16 = 0, 1
 ACTS = {"relu": 0, "gelu_erf": 1, "gelu_tanh": 2, "silu": 3}
 PATHS = {"auto": 0, "dense": 1, "gather": 2, "fused": 3}
-EXPORTS = ["d2d_status_str", "d2d_launch_count", "d2d_layer_create", "d2d_layer_destroy", "d2d_workspace_bytes",
+EXPORTS = ["d2d_status_str", "d2d_launch_count", "d2d_layer_create", "d2d_layer_create_fp8", "d2d_layer_get_fp8", "d2d_layer_destroy", "d2d_workspace_bytes",
            "d2d_layer_set_expert_path", "d2d_layer_set_fused_rho_max", "d2d_layer_get_fused", "d2d_layer_expert_path_for", "d2d_layer_get_expert_path", "d2d_layer_reset_counters", "d2d_expert_up_gather_fwd", "d2d_expert_down_masked_fwd", "d2d_test_inject_fault",
            "d2d_select_workspace_bytes", "d2d_router_fwd", "d2d_select_dynk", "d2d_select_dynk_static", "d2d_select_topk",
            "d2d_routing_from_mask", "d2d_moe_ffn_fwd", "d2d_expert_up_fwd", "d2d_expert_down_fwd", "d2d_layer_fwd", "d2d_layer_fwd_host_workspace_bytes",
@@ -54,6 +54,8 @@ _lib.d2d_launch_count.argtypes = []
 _lib.d2d_status_str.restype = c_char_p
 _lib.d2d_status_str.argtypes = [c_int]
 _lib.d2d_layer_create.argtypes = [POINTER(LayerDesc), POINTER(Weights), c_void_p, POINTER(c_void_p)]
+_lib.d2d_layer_create_fp8.argtypes = [POINTER(LayerDesc), POINTER(Weights), c_void_p, POINTER(c_void_p)]
+_lib.d2d_layer_get_fp8.argtypes = [c_void_p, c_int32, c_void_p, c_void_p, c_void_p]
 _lib.d2d_layer_destroy.argtypes = [c_void_p]
 _lib.d2d_workspace_bytes.restype = c_size_t
 _lib.d2d_workspace_bytes.argtypes = [c_void_p, c_int32]
@@ -169,7 +171,7 @@ class Layer:
     """One D2DMoE layer: packed device weights plus the calls of the C ABI."""
 
     def __init__(self, d: int, d_ff: int, n_experts: int, d_h: int, dtype: str, act: str, gated: bool,
-                 weights: dict, device="cuda:0"):
+                 weights: dict, device="cuda:0", fp8_experts: bool = False):
         self.device = torch.device(device)
         self.dtype_name = dtype
         self.tdtype = torch_dtype(dtype)
@@ -186,14 +188,24 @@ class Layer:
         w = Weights(**{n: (dev[n].data_ptr() if n in dev else None) for n, _ in Weights._fields_})
         handle = c_void_p()
         with torch.cuda.device(self.device):
-            _check(_lib.d2d_layer_create(ctypes.byref(self.desc), ctypes.byref(w), _stream(), ctypes.byref(handle)),
-                   "d2d_layer_create")
+            create = _lib.d2d_layer_create_fp8 if fp8_experts else _lib.d2d_layer_create
+            _check(create(ctypes.byref(self.desc), ctypes.byref(w), _stream(), ctypes.byref(handle)),
+                   "d2d_layer_create_fp8" if fp8_experts else "d2d_layer_create")
         self.handle = handle
+        self.fp8_experts = bool(fp8_experts)
         self._ws = None
 
     @classmethod
-    def from_config(cls, cfg, weights: dict, device="cuda:0") -> "Layer":
-        return cls(cfg.d, cfg.d_ff, cfg.E, cfg.d_h, cfg.dtype, cfg.act, cfg.gated, weights, device)
+    def from_config(cls, cfg, weights: dict, device="cuda:0", fp8_experts: bool = False) -> "Layer":
+        return cls(cfg.d, cfg.d_ff, cfg.E, cfg.d_h, cfg.dtype, cfg.act, cfg.gated, weights, device, fp8_experts)
+
+    def get_fp8(self, which: str):
+        """Codes (uint8 [d_ff, d]; "w2": of the transposed W2) and scale exponents (int32 [E]) of "w1" | "w_gate" | "w2"."""
+        codes = torch.empty((self.d_ff, self.d), dtype=torch.uint8, device=self.device)
+        exps = torch.empty((self.E,), dtype=torch.int32, device=self.device)
+        _check(_lib.d2d_layer_get_fp8(self.handle, {"w1": 0, "w_gate": 1, "w2": 2}[which], _ptr(codes), _ptr(exps), _stream()),
+               "d2d_layer_get_fp8")
+        return codes, exps
 
     def close(self):
         if getattr(self, "handle", None):

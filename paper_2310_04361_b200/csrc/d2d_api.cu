@@ -267,6 +267,27 @@ const char *d2d_status_str(d2d_status s)
     return "unknown status";
 }
 
+// Gated bf16 layers: W1 and W_gate once more, interleaved in blocks of 128 rows (the gated up projection fetches both
+// tiles with one TMA box).  Built from the layer's own packed copies (again after they were replaced by dequantised values).
+static d2d_status build_gate_cat(d2d_layer *L, cudaStream_t st)
+{
+    const d2d_layer_desc &D = L->desc;
+    const int cat_block = 128;
+    const size_t cat_rows = (size_t)2 * cat_block * d2d_cdiv(D.d_ff, cat_block);
+    const size_t row_b = (size_t)D.d * L->elem;
+    char *cat = (char *)L->w1g;
+    if (cudaMemsetAsync(cat, 0, cat_rows * row_b, st) != cudaSuccess) return D2D_ERR_CUDA;
+    for (int r0 = 0, b = 0; r0 < D.d_ff; r0 += cat_block, ++b) {
+        const size_t rows = (size_t)(D.d_ff - r0 < cat_block ? D.d_ff - r0 : cat_block);
+        char *dst = cat + (size_t)b * 2 * cat_block * row_b;
+        if (cudaMemcpyAsync(dst, (const char *)L->w1 + (size_t)r0 * row_b, rows * row_b, cudaMemcpyDeviceToDevice, st) != cudaSuccess ||
+            cudaMemcpyAsync(dst + (size_t)cat_block * row_b, (const char *)L->w_gate + (size_t)r0 * row_b, rows * row_b,
+                            cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+            return D2D_ERR_CUDA;
+    }
+    return D2D_OK;
+}
+
 d2d_status d2d_layer_create(const d2d_layer_desc *desc, const d2d_weights *w, void *stream, d2d_layer **out)
 {
     if (out) *out = nullptr;
@@ -342,18 +363,8 @@ d2d_status d2d_layer_create(const d2d_layer_desc *desc, const d2d_weights *w, vo
         if (rc != D2D_OK) break;
     }
     if (rc == D2D_OK && want_cat) {
-        char *cat = (char *)L->slab + cat_off;
-        const size_t row_b = (size_t)D.d * el;
-        if (cudaMemsetAsync(cat, 0, cat_rows * row_b, st) != cudaSuccess) rc = D2D_ERR_CUDA;
-        for (int r0 = 0, b = 0; r0 < D.d_ff && rc == D2D_OK; r0 += cat_block, ++b) {
-            const size_t rows = (size_t)(D.d_ff - r0 < cat_block ? D.d_ff - r0 : cat_block);
-            char *dst = cat + (size_t)b * 2 * cat_block * row_b;
-            if (cudaMemcpyAsync(dst, (const char *)w->w1 + (size_t)r0 * row_b, rows * row_b, cudaMemcpyDeviceToDevice, st) != cudaSuccess ||
-                cudaMemcpyAsync(dst + (size_t)cat_block * row_b, (const char *)w->w_gate + (size_t)r0 * row_b, rows * row_b,
-                                cudaMemcpyDeviceToDevice, st) != cudaSuccess)
-                rc = D2D_ERR_CUDA;
-        }
-        L->w1g = cat;
+        L->w1g = (char *)L->slab + cat_off;
+        rc = build_gate_cat(L, st);
     }
     if (rc == D2D_OK && cudaStreamSynchronize(st) != cudaSuccess) rc = D2D_ERR_CUDA;
     if (rc == D2D_OK && (cudaStreamCreateWithFlags(&L->side_stream, cudaStreamNonBlocking) != cudaSuccess ||
@@ -396,9 +407,59 @@ d2d_status d2d_layer_destroy(d2d_layer *layer)
     if (layer->ev_end) cudaEventDestroy(layer->ev_end);
     if (layer->copy_in) cudaStreamDestroy(layer->copy_in);
     if (layer->copy_out) cudaStreamDestroy(layer->copy_out);
+    if (layer->q_slab) cudaFree(layer->q_slab);
     cudaError_t e = cudaFree(layer->slab);
     delete layer;
     return e == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
+}
+
+d2d_status d2d_layer_create_fp8(const d2d_layer_desc *desc, const d2d_weights *w, void *stream, d2d_layer **out)
+{
+    if (out) *out = nullptr;
+    if (!desc || desc->dtype != D2D_BF16) return D2D_ERR_UNSUPPORTED;
+    if (desc->d % 16 || ((int64_t)desc->expert_size * desc->d) % 16) return D2D_ERR_UNSUPPORTED;   // 16-byte pieces of codes
+    d2d_layer *L = nullptr;
+    d2d_status rc = d2d_layer_create(desc, w, stream, &L);
+    if (rc != D2D_OK) return rc;
+    const d2d_layer_desc &D = L->desc;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t n_w = (size_t)D.d_ff * D.d, n_mat = D.gated ? 3 : 2;
+    const size_t codes_b = d2d_align_up(n_w, 256), exps_b = d2d_align_up((size_t)D.n_experts * sizeof(int32_t), 256);
+    if (cudaMalloc(&L->q_slab, n_mat * (codes_b + exps_b)) != cudaSuccess) {
+        d2d_layer_destroy(L);
+        return D2D_ERR_CUDA;
+    }
+    char *q = (char *)L->q_slab;
+    L->q_w1 = (uint8_t *)q; L->q_k1 = (int32_t *)(q + codes_b); q += codes_b + exps_b;
+    L->q_w2t = (uint8_t *)q; L->q_k2 = (int32_t *)(q + codes_b); q += codes_b + exps_b;
+    if (D.gated) { L->q_wg = (uint8_t *)q; L->q_kg = (int32_t *)(q + codes_b); }
+    const int per = D.expert_size * D.d;
+    // the packed bf16 copies are replaced by the dequantised values, so every path of the layer computes with them
+    rc = d2d_quantize_experts_e4m3(L->w1, L->q_w1, L->q_k1, D.n_experts, per, st);
+    if (rc == D2D_OK) rc = d2d_quantize_experts_e4m3(L->w2t, L->q_w2t, L->q_k2, D.n_experts, per, st);
+    if (rc == D2D_OK && D.gated) rc = d2d_quantize_experts_e4m3(L->w_gate, L->q_wg, L->q_kg, D.n_experts, per, st);
+    if (rc == D2D_OK) rc = d2d_launch_transpose(L->w2t, L->w2, D.d_ff, D.d, L->elem, st);      // W2 [d, d_ff] from the transposed copy
+    if (rc == D2D_OK && L->w1g) rc = build_gate_cat(L, st);
+    if (rc == D2D_OK && cudaStreamSynchronize(st) != cudaSuccess) rc = D2D_ERR_CUDA;
+    if (rc != D2D_OK) {
+        d2d_layer_destroy(L);
+        return rc;
+    }
+    *out = L;
+    return D2D_OK;
+}
+
+d2d_status d2d_layer_get_fp8(const d2d_layer *layer, int32_t which, uint8_t *codes, int32_t *exps, void *stream)
+{
+    if (!layer || which < 0 || which > 2 || (!codes && !exps)) return D2D_ERR_INVALID_ARG;
+    const uint8_t *c = which == 0 ? layer->q_w1 : which == 1 ? layer->q_wg : layer->q_w2t;
+    const int32_t *k = which == 0 ? layer->q_k1 : which == 1 ? layer->q_kg : layer->q_k2;
+    if (!c || !k) return D2D_ERR_UNSUPPORTED;
+    const d2d_layer_desc &D = layer->desc;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (codes && cudaMemcpyAsync(codes, c, (size_t)D.d_ff * D.d, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return D2D_ERR_CUDA;
+    if (exps && cudaMemcpyAsync(exps, k, (size_t)D.n_experts * sizeof(int32_t), cudaMemcpyDeviceToDevice, st) != cudaSuccess) return D2D_ERR_CUDA;
+    return D2D_OK;
 }
 
 d2d_status d2d_layer_set_expert_path(d2d_layer *layer, d2d_expert_path path, int32_t group, double rho_max)

@@ -26,6 +26,11 @@ struct d2d_layer {
     cudaStream_t side_stream;
     cudaEvent_t ev_fork, ev_join;
     cudaEvent_t ev_fill_fork, ev_fill_join;      // zero fill of H beside the gathered up projection (side stream)
+    // 8-bit expert weights (d2d_layer_create_fp8): e4m3 codes [d_ff, d] of W1, W_gate and the transposed W2, one scale
+    // exponent per expert and matrix; NULL for ordinary layers.  w1, w_gate, w2, w2t, w1g then hold the dequantised values.
+    void *q_slab;
+    uint8_t *q_w1, *q_wg, *q_w2t;
+    int32_t *q_k1, *q_kg, *q_k2;
     // d2d_layer_fwd_host: copy-in and copy-out streams and per-chunk events, so that the host -> device copy of one
     // chunk of tokens, the layer on the previous chunk and the device -> host copy of the one before overlap
     static const int kHostChunks = 4;
@@ -139,6 +144,10 @@ d2d_status d2d_small_ffn(const d2d_layer *L, const void *x, int T, const d2d_rou
                          int fused = 0);
 
 d2d_status d2d_launch_transpose(const void *src, void *dst, int rows, int cols, size_t elem, cudaStream_t st);
+
+// quant_fp8.cu: per-expert e4m3 codes + power-of-two scale exponents of n_experts slices of per_expert bf16 weights;
+// the weights are replaced in place by their dequantised values (exactly bf16)
+d2d_status d2d_quantize_experts_e4m3(void *w, uint8_t *codes, int32_t *exps, int n_experts, int per_expert, cudaStream_t st);
 
 // ---- device helpers ------------------------------------------------------------------------
 

@@ -12,6 +12,9 @@
 //                         once (only experts some token kept do any work), the expert's tokens are
 //                         handled 8 at a time, partial output rows go to a float32 accumulator with
 //                         16-byte vector reductions; the last CTA adds b2 and writes y
+#include <cuda_fp8.h>
+#include <type_traits>
+
 #include "d2d_common.cuh"
 #include "small_select.cuh"
 
@@ -53,9 +56,23 @@ __device__ __forceinline__ void lds8(const __nv_bfloat16 *p, float (&o)[8])
     }
 }
 
+// 8 consecutive 8-bit floating point codes (e4m3) as floats; the expert's power-of-two scale is applied by the caller
+__device__ __forceinline__ void lds8(const uint8_t *p, float (&o)[8])
+{
+    const uint2 raw = *reinterpret_cast<const uint2 *>(p);
+    const uint32_t w[2] = {raw.x, raw.y};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const __half2_raw h = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)((w[i >> 1] >> ((i & 1) * 16)) & 0xffffu), __NV_E4M3);
+        const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&h));
+        o[2 * i] = f.x;
+        o[2 * i + 1] = f.y;
+    }
+}
+
 // One warp: dot products of a weight row with up to TBLK token rows, all operands in shared memory.
-template <typename TT, int TBLK>
-__device__ __forceinline__ void warp_row_dots(const TT *wrow, const TT *xs, int d, int lane, float (&acc)[TBLK])
+template <typename WT, typename TT, int TBLK>
+__device__ __forceinline__ void warp_row_dots(const WT *wrow, const TT *xs, int d, int lane, float (&acc)[TBLK])
 {
 #pragma unroll
     for (int i = 0; i < TBLK; ++i) acc[i] = 0.0f;
@@ -162,7 +179,7 @@ small_router_kernel(const TT *__restrict__ x, int T, int d, int d_h, int E, int 
         __syncthreads();
         if (warp < rows) {
             float acc[TBLK];
-            warp_row_dots<TT, TBLK>(w1s + (size_t)warp * d, xs, d, lane, acc);
+            warp_row_dots<TT, TT, TBLK>(w1s + (size_t)warp * d, xs, d, lane, acc);
             if (lane == 0) {
                 const float bj = b_r1 ? d2d_to_float<TT>(b_r1[j0 + warp]) : 0.0f;
 #pragma unroll
@@ -226,26 +243,31 @@ __device__ __forceinline__ void red_add_v4(float *addr, float a, float b, float 
 // dynamic shared memory: [ W1 rows: rc*d | W_gate rows: rc*d (gated) | W2T rows: rc*d | token block: TBLK*d | h: TBLK*rc floats ]
 // rc = neurons handled per pass (the whole expert when its slices fit).
 struct SmallFfnLayer {
-    const void *w1, *b1, *w_gate, *w2t, *b2;
+    const void *w1, *b1, *w_gate, *w2t, *b2;   // Q8 kernels: w1, w_gate, w2t are e4m3 codes [d_ff, d]
     const int32_t *offsets, *perm;
     float *y32;
     unsigned int *ticket;
     void *y;
     long long capacity;      // entries the caller's perm buffer holds: a list truncated by D2D_ERR_CAPACITY is never read past it
+    const int32_t *k1, *kg, *k2;      // Q8 kernels: per-expert exponents of the scales 2^k of W1, W_gate, W2
 };
 struct SmallFfnArgs {
     SmallFfnLayer l[D2D_MAX_GROUP];
 };
 
-template <typename TT, int ACT, bool GATED, int TBLK>
+// Q8: the expert weights are 8-bit floating point codes (e4m3) with one power-of-two scale per expert and matrix
+// (App. C runs the expert kernels on narrower formats): half the bytes per kept expert; the codes are widened when they
+// are used and the scale, a power of two, is applied to the finished sums (exactly what scaling every weight would give).
+template <typename TT, int ACT, bool GATED, int TBLK, bool Q8>
 __global__ void __launch_bounds__(NT)
 small_ffn_kernel(const TT *__restrict__ x, int T, int d, int s, int rc, const __grid_constant__ SmallFfnArgs args)
 {
+    using WT = typename std::conditional<Q8, uint8_t, TT>::type;
     const SmallFfnLayer &P = args.l[blockIdx.y];
-    const TT *__restrict__ w1 = static_cast<const TT *>(P.w1);
+    const WT *__restrict__ w1 = static_cast<const WT *>(P.w1);
     const TT *__restrict__ b1 = static_cast<const TT *>(P.b1);
-    const TT *__restrict__ w_gate = static_cast<const TT *>(P.w_gate);
-    const TT *__restrict__ w2t = static_cast<const TT *>(P.w2t);
+    const WT *__restrict__ w_gate = static_cast<const WT *>(P.w_gate);
+    const WT *__restrict__ w2t = static_cast<const WT *>(P.w2t);
     const TT *__restrict__ b2 = static_cast<const TT *>(P.b2);
     const int32_t *__restrict__ offsets = P.offsets;
     const int32_t *__restrict__ perm = P.perm;
@@ -253,15 +275,16 @@ small_ffn_kernel(const TT *__restrict__ x, int T, int d, int s, int rc, const __
     unsigned int *__restrict__ ticket = P.ticket;
     TT *__restrict__ y = static_cast<TT *>(P.y);
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    TT *w1s = reinterpret_cast<TT *>(smem_raw);
-    TT *wgs = w1s + (size_t)rc * d;
-    TT *w2s = wgs + (GATED ? (size_t)rc * d : 0);
-    TT *xs = w2s + (size_t)rc * d;
+    WT *w1s = reinterpret_cast<WT *>(smem_raw);
+    WT *wgs = w1s + (size_t)rc * d;
+    WT *w2s = wgs + (GATED ? (size_t)rc * d : 0);
+    TT *xs = reinterpret_cast<TT *>(w2s + (size_t)rc * d);
     float *hs = reinterpret_cast<float *>(xs + (size_t)TBLK * d);
     __shared__ unsigned int my_ticket;
     __shared__ int stok[TBLK];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int e = blockIdx.x;
+    const float sc1 = Q8 ? ldexpf(1.0f, P.k1[e]) : 1.0f, scg = Q8 && GATED ? ldexpf(1.0f, P.kg[e]) : 1.0f, sc2 = Q8 ? ldexpf(1.0f, P.k2[e]) : 1.0f;
     // perm may have been truncated at `capacity` entries (the selection then reported D2D_ERR_CAPACITY): stay inside it
     const long long cap = P.capacity;
     const int end = (long long)offsets[e + 1] < cap ? offsets[e + 1] : (int)cap;
@@ -272,9 +295,9 @@ small_ffn_kernel(const TT *__restrict__ x, int T, int d, int s, int rc, const __
             const int rows = s - r0 < rc ? s - r0 : rc;
             const size_t n0 = (size_t)e * s + r0;
             __syncthreads();                                      // readers of the previous pass are done
-            cta_copy_async(w1s, w1 + n0 * d, (size_t)rows * d * sizeof(TT));
-            if (GATED) cta_copy_async(wgs, w_gate + n0 * d, (size_t)rows * d * sizeof(TT));
-            cta_copy_async(w2s, w2t + n0 * d, (size_t)rows * d * sizeof(TT));
+            cta_copy_async(w1s, w1 + n0 * d, (size_t)rows * d * sizeof(WT));
+            if (GATED) cta_copy_async(wgs, w_gate + n0 * d, (size_t)rows * d * sizeof(WT));
+            cta_copy_async(w2s, w2t + n0 * d, (size_t)rows * d * sizeof(WT));
             cp_async_commit();
             for (int p0 = beg; p0 < end; p0 += TBLK) {
                 const int ntok = end - p0 < TBLK ? end - p0 : TBLK;
@@ -293,14 +316,14 @@ small_ffn_kernel(const TT *__restrict__ x, int T, int d, int s, int rc, const __
                 // ---- up projection + activation: one warp per neuron
                 for (int nl = warp; nl < rows; nl += NT / 32) {
                     float up[TBLK], gate[TBLK];
-                    warp_row_dots<TT, TBLK>(w1s + (size_t)nl * d, xs, d, lane, up);
-                    if (GATED) warp_row_dots<TT, TBLK>(wgs + (size_t)nl * d, xs, d, lane, gate);
+                    warp_row_dots<WT, TT, TBLK>(w1s + (size_t)nl * d, xs, d, lane, up);
+                    if (GATED) warp_row_dots<WT, TT, TBLK>(wgs + (size_t)nl * d, xs, d, lane, gate);
                     if (lane == 0) {
                         const float bn = b1 ? d2d_to_float<TT>(b1[n0 + nl]) : 0.0f;
 #pragma unroll
                         for (int i = 0; i < TBLK; ++i) {
-                            const float z = up[i] + bn;
-                            hs[i * rc + nl] = GATED ? d2d_activate<ACT>(gate[i]) * z : d2d_activate<ACT>(z);
+                            const float z = up[i] * sc1 + bn;
+                            hs[i * rc + nl] = GATED ? d2d_activate<ACT>(gate[i] * scg) * z : d2d_activate<ACT>(z);
                         }
                     }
                 }
@@ -311,9 +334,16 @@ small_ffn_kernel(const TT *__restrict__ x, int T, int d, int s, int rc, const __
 #pragma unroll
                     for (int i = 0; i < TBLK; ++i) acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.0f;
                     for (int nl = 0; nl < rows; ++nl) {
-                        const TT *wp = w2s + (size_t)nl * d + c;
+                        const WT *wp = w2s + (size_t)nl * d + c;
                         float w0, w1v, w2v, w3;
-                        if (sizeof(TT) == 2) {
+                        if (Q8) {
+                            const uint32_t raw = *reinterpret_cast<const uint32_t *>(wp);
+                            const __half2_raw lo = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)(raw & 0xffffu), __NV_E4M3);
+                            const __half2_raw hi = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)(raw >> 16), __NV_E4M3);
+                            const float2 a = __half22float2(*reinterpret_cast<const __half2 *>(&lo));
+                            const float2 b = __half22float2(*reinterpret_cast<const __half2 *>(&hi));
+                            w0 = a.x; w1v = a.y; w2v = b.x; w3 = b.y;
+                        } else if (sizeof(TT) == 2) {
                             const uint2 raw = *reinterpret_cast<const uint2 *>(wp);
                             w0 = __uint_as_float(raw.x << 16); w1v = __uint_as_float(raw.x & 0xffff0000u);
                             w2v = __uint_as_float(raw.y << 16); w3 = __uint_as_float(raw.y & 0xffff0000u);
@@ -332,7 +362,8 @@ small_ffn_kernel(const TT *__restrict__ x, int T, int d, int s, int rc, const __
                     }
 #pragma unroll
                     for (int i = 0; i < TBLK; ++i)
-                        if (i < ntok) red_add_v4(y32 + (size_t)stok[i] * d + c, acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+                        if (i < ntok)
+                            red_add_v4(y32 + (size_t)stok[i] * d + c, acc[i][0] * sc2, acc[i][1] * sc2, acc[i][2] * sc2, acc[i][3] * sc2);
                 }
             }
         }
@@ -358,12 +389,13 @@ small_ffn_kernel(const TT *__restrict__ x, int T, int d, int s, int rc, const __
 constexpr size_t kSmemLimit = 200 * 1024;
 
 // neurons per pass so that the slices, one token block and the hidden values fit in shared memory
-int rows_per_pass(const d2d_layer_desc &D, size_t elem, int tb = MAX_TBLK)
+int rows_per_pass(const d2d_layer_desc &D, size_t elem, int tb = MAX_TBLK, size_t welem = 0)
 {
+    if (welem == 0) welem = elem;                              // weights stored like the activations unless stated
     const size_t n_mat = D.gated ? 3 : 2;
     const size_t fixed = (size_t)tb * D.d * elem;
     for (int rc = D.expert_size; rc >= 1; rc = (rc + 1) / 2) {
-        const size_t need = n_mat * rc * D.d * elem + fixed + (size_t)tb * rc * 4;
+        const size_t need = n_mat * rc * D.d * welem + fixed + (size_t)tb * rc * 4;
         if (need <= kSmemLimit) return rc;
         if (rc == 1) break;
     }
@@ -374,13 +406,14 @@ int rows_per_pass(const d2d_layer_desc &D, size_t elem, int tb = MAX_TBLK)
 // still costs its share of the dot products)
 int token_block(int T) { return T <= 1 ? 1 : T <= 2 ? 2 : T <= 4 ? 4 : 8; }
 
-template <typename TT, int ACT, bool GATED, int TBLK>
-d2d_status launch_ffn_tb(const d2d_layer_desc &D, int n_layers, const SmallFfnArgs &args, const void *x, int T, cudaStream_t st)
+template <typename TT, int ACT, bool GATED, int TBLK, bool Q8>
+d2d_status launch_ffn_q(const d2d_layer_desc &D, int n_layers, const SmallFfnArgs &args, const void *x, int T, cudaStream_t st)
 {
-    const int rc = rows_per_pass(D, sizeof(TT), TBLK);
+    const size_t welem = Q8 ? 1 : sizeof(TT);
+    const int rc = rows_per_pass(D, sizeof(TT), TBLK, welem);
     if (rc <= 0) return D2D_ERR_UNSUPPORTED;
-    const size_t smem = (size_t)(GATED ? 3 : 2) * rc * D.d * sizeof(TT) + (size_t)TBLK * D.d * sizeof(TT) + (size_t)TBLK * rc * 4;
-    auto kern = small_ffn_kernel<TT, ACT, GATED, TBLK>;
+    const size_t smem = (size_t)(GATED ? 3 : 2) * rc * D.d * welem + (size_t)TBLK * D.d * sizeof(TT) + (size_t)TBLK * rc * 4;
+    auto kern = small_ffn_kernel<TT, ACT, GATED, TBLK, Q8>;
     static size_t attr_smem = 0;
     if (smem > attr_smem) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess) return D2D_ERR_CUDA;
@@ -389,6 +422,15 @@ d2d_status launch_ffn_tb(const d2d_layer_desc &D, int n_layers, const SmallFfnAr
     kern<<<dim3(D.n_experts, n_layers), NT, smem, st>>>((const TT *)x, T, D.d, D.expert_size, rc, args);
     D2D_LAUNCHED(1);
     return cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
+}
+
+template <typename TT, int ACT, bool GATED, int TBLK>
+d2d_status launch_ffn_tb(const d2d_layer_desc &D, int n_layers, const SmallFfnArgs &args, const void *x, int T, cudaStream_t st)
+{
+    // 8-bit weights: bf16 layers only (one layer per launch: every layer of the launch must hold codes)
+    if (std::is_same<TT, __nv_bfloat16>::value && n_layers == 1 && args.l[0].k1 != nullptr)
+        return launch_ffn_q<TT, ACT, GATED, TBLK, std::is_same<TT, __nv_bfloat16>::value>(D, n_layers, args, x, T, st);
+    return launch_ffn_q<TT, ACT, GATED, TBLK, false>(D, n_layers, args, x, T, st);
 }
 
 template <typename TT, int ACT, bool GATED>
@@ -529,6 +571,10 @@ d2d_status d2d_small_ffn(const d2d_layer *L, const void *x, int T, const d2d_rou
     if (!fused) D2D_CUDA_TRY(cudaMemsetAsync(ws, 0, 256 + (size_t)T * L->desc.d * 4, st));
     SmallFfnArgs a = {};
     a.l[0] = {L->w1, L->b1, L->w_gate, L->w2t, L->b2, r->offsets, r->perm, y32, ticket, y, (long long)r->perm_capacity};
+    if (L->q_w1 && L->desc.d % 16 == 0) {                     // 8-bit expert weights: the kernel reads the codes
+        a.l[0].w1 = L->q_w1; a.l[0].w_gate = L->q_wg; a.l[0].w2t = L->q_w2t;
+        a.l[0].k1 = L->q_k1; a.l[0].kg = L->q_kg; a.l[0].k2 = L->q_k2;
+    }
     if (L->desc.dtype == D2D_F32) return launch_ffn_dtype<float>(L->desc, 1, a, x, T, st);
     return launch_ffn_dtype<__nv_bfloat16>(L->desc, 1, a, x, T, st);
 }
