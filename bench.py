@@ -51,6 +51,8 @@ PER_CONFIG = [
     ("gpt2_ffn", 1, 0.5, None), ("gpt2_ffn", 8, 0.5, None), ("gpt2_ffn", 64, 0.5, None),
     ("gpt2_attn", 1, 0.5, None), ("gpt2_attn", 64, 0.5, None),
     ("llama", None, 0.6, None),
+    # decode on the Llama shape, where the kept experts' bytes set the time: bf16 weights, then 8-bit (e4m3) weights
+    ("llama", 1, 0.2, None), ("llama", 1, 0.2, None, True), ("llama", 2, 0.2, None), ("llama", 2, 0.2, None, True),
     ("paper", None, None, 0.02), ("paper", None, None, 0.05), ("paper", None, None, 0.1), ("paper", None, None, 0.3),
     ("paper", None, None, 0.5),
 ]
@@ -396,7 +398,7 @@ def k_histogram(torch, routing, T, E):
             "p99": float(torch.quantile(k, 0.99).item()), "max": int(k.max().item()), "experts_used": used}
 
 
-def measure_config(h, api, torch, wl, name, tokens, tau, bern, steps, peaks, path="auto", group=0, full=False, rank=0):
+def measure_config(h, api, torch, wl, name, tokens, tau, bern, steps, peaks, path="auto", group=0, full=False, rank=0, fp8=False):
     """One configuration: layer time, kept fraction, k histogram, dense comparators, roofline fraction of the expert step."""
     import numpy as np
     import oracle
@@ -407,7 +409,7 @@ def measure_config(h, api, torch, wl, name, tokens, tau, bern, steps, peaks, pat
     dev = h.dev
     weights = wl.make_weights(cfg)
     x_np = wl.make_tokens(cfg, stream=rank)
-    layer = api.Layer.from_config(cfg, weights, device=dev)
+    layer = api.Layer.from_config(cfg, weights, device=dev, fp8_experts=fp8)
     if cfg.dtype == "bf16" and (path != "auto" or group):
         layer.set_expert_path(path, group)
     x = api.to_device(x_np, cfg.dtype, dev)
@@ -442,16 +444,17 @@ def measure_config(h, api, torch, wl, name, tokens, tau, bern, steps, peaks, pat
     elem = 2 if cfg.dtype == "bf16" else 4
     n_used = int((routing.counts > 0).sum().item())
     if T <= 64 or cfg.dtype == "f32":
-        touched = n_used * (cfg.n_mat * cfg.s * cfg.d + cfg.s) * elem + 2 * T * cfg.d * elem + cfg.d * elem
+        welem = 1 if fp8 else elem                           # 8-bit expert weights: one byte per weight
+        touched = n_used * (cfg.n_mat * cfg.s * cfg.d * welem + cfg.s * elem) + 2 * T * cfg.d * elem + cfg.d * elem
         roof = {"bound": "hbm", "frac": touched / (t_ffn * 1e-3) / 1e9 / peaks["hbm_gbs"], "of": "touched expert bytes / expert-step time / HBM peak"}
     else:
         roof = {"bound": "tensor", "frac": f_experts / (t_ffn * 1e-3) / 1e12 / peaks["bf16_tflops"],
                 "of": "algorithmic expert FLOP / expert-step time / bf16 peak"}
-    out = {"workload": cfg.name, "tokens": T, "tau": tau, "bernoulli_p": bern, "rho": rho, "pruned_flop_fraction": 1 - rho,
+    out = {"workload": cfg.name, "tokens": T, "tau": tau, "bernoulli_p": bern, "expert_weights": "e4m3 + 2^k per expert" if fp8 else cfg.dtype, "rho": rho, "pruned_flop_fraction": 1 - rho,
            "k": k_histogram(torch, routing, T, cfg.E),
            "step": "d2d_moe_ffn_fwd on the override mask" if bern is not None else "d2d_layer_fwd",
            "ms_median": t["median"], "ms_min": t["min"], "tokens_per_s": T / (t["median"] * 1e-3),
-           "expert_step_ms": t_ffn, "launches_per_step": launches, "expert_path": (layer.expert_path_for(T, n_sel) if T > 4 else "decode kernels") if cfg.dtype == "bf16" else "fp32",
+           "expert_step_ms": t_ffn, "launches_per_step": launches, "expert_path": (layer.expert_path_for(T, n_sel) if launches > 2 else "decode kernels") if cfg.dtype == "bf16" else "fp32",
            "dense": dense, "speedup_vs_torch_dense": dense["speedup"],
            "speedup_vs_library_dense": dense["speedup_vs_library_dense"], "roofline": roof}
     layer.close()
@@ -544,7 +547,7 @@ def run_ours(args):
             # decode regime: the expert kernel is bound by HBM traffic on the touched expert slices
             touched = n_used * (cfg.n_mat * cfg.s * cfg.d + cfg.s) * elem + 2 * T * cfg.d * elem + cfg.d * elem
             achieved = touched / (t_ffn * 1e-3) / 1e9
-            roofline = {"bound": "hbm", "kernel": "moe_ffn_fwd (small_ffn_kernel)" if T <= 4 else "moe_ffn_fwd", "achieved": achieved,
+            roofline = {"bound": "hbm", "kernel": "moe_ffn_fwd (small_ffn_kernel)" if launches_per_step <= 2 else "moe_ffn_fwd", "achieved": achieved,
                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None,
                         "peak_source": f"{peaks['source']} HBM copy", "algorithmic_bytes_per_launch": touched,
                         "experts_touched": n_used, "kernel_ms": t_ffn}
@@ -666,9 +669,9 @@ def run_ours(args):
         per_config = None
         if not args.no_per_config:
             per_config = []
-            for name, tokens, tau, bern in PER_CONFIG:
+            for name, tokens, tau, bern, *rest in PER_CONFIG:
                 try:
-                    per_config.append(measure_config(h, api, torch, wl, name, tokens, tau, bern, 20, peaks))
+                    per_config.append(measure_config(h, api, torch, wl, name, tokens, tau, bern, 20, peaks, fp8=bool(rest and rest[0])))
                 except Exception as e:      # a configuration that fails must not take the headline down with it
                     per_config.append({"workload": name, "tokens": tokens, "tau": tau, "bernoulli_p": bern, "error": repr(e)})
                 torch.cuda.empty_cache()

@@ -33,9 +33,11 @@
  *
  * Environment variables (tuning aids, read once per process; results never
  * depend on them)
- *   D2D_DECODE_MAX_TOKENS=n  0..8, default 4: bf16 batches of up to n tokens take
- *                            the decode kernels (each kept expert's weights read
- *                            once by CUDA cores), larger ones the tensor-core path.
+ *   D2D_DECODE_MAX_TOKENS=n  0..8: bf16 batches of up to n tokens take the decode
+ *                            kernels (each kept expert's weights read once by CUDA
+ *                            cores), larger ones the tensor-core path.  Default: 4
+ *                            tokens, 2 for layers with more than 256 KB of weights
+ *                            per expert.
  *   D2D_HOST_CHUNKS=n        1..4: number of pipelined chunks d2d_layer_fwd_host
  *                            cuts a batch into, of equal size (default: see there).
  *   D2D_GEMM_BAND=n          row tiles per band of the tile walk of the dense

@@ -59,28 +59,32 @@ ws_layout layout_for(const d2d_layer *L, int T)
 
 }  // namespace
 
-// Measured on the GPT-2-medium-shaped FFN (us per layer call, decode kernels / tensor-core path): T = 3: 31 / 39,
-// T = 4: 33 / 39, T = 5: 41 / 40, T = 8: 43 / 39.
-int d2d_decode_max_tokens()
+// Up to this many tokens a bf16 layer takes the decode kernels.  Measured (us per layer call, decode kernels /
+// tensor-core path): GPT-2-medium-shaped FFN (64 KB of weights per expert) T = 3: 31 / 39, T = 4: 33 / 39, T = 5:
+// 41 / 40, T = 8: 43 / 39; Llama-shaped layer (786 KB per expert) T = 1: 84 / 129, T = 2: 108 / 133, T = 3: 221 / 133,
+// T = 4: 229 / 127.  So 4 tokens for small experts, 2 for large ones; D2D_DECODE_MAX_TOKENS overrides both.
+int d2d_decode_max_tokens(const d2d_layer_desc &D)
 {
     static const int v = [] {
         const char *e = getenv("D2D_DECODE_MAX_TOKENS");
-        const int n = e ? atoi(e) : 4;
-        return n < 0 ? 0 : n > 8 ? 8 : n;
+        const int n = e ? atoi(e) : -1;
+        return n > 8 ? 8 : n;
     }();
-    return v;
+    if (v >= 0) return v;
+    const size_t expert_bytes = (size_t)(D.gated ? 3 : 2) * D.expert_size * D.d * 2;
+    return expert_bytes > ((size_t)256 << 10) ? 2 : 4;
 }
 
 static bool use_dense_masked(const d2d_layer *L, int T)
 {
-    return L->desc.dtype == D2D_BF16 && T > d2d_decode_max_tokens() && L->desc.d_ff % 8 == 0 && d2d_gemm_tc_available();
+    return L->desc.dtype == D2D_BF16 && T > d2d_decode_max_tokens(L->desc) && L->desc.d_ff % 8 == 0 && d2d_gemm_tc_available();
 }
 
 // Up to this many tokens the expert-per-CTA kernel (each kept expert's slice read once) is used.
 
 static bool use_small_ffn(const d2d_layer *L, int T)
 {
-    const int lim = L->desc.dtype == D2D_BF16 ? d2d_decode_max_tokens() : 8;      // fp32 layers have no tensor-core path
+    const int lim = L->desc.dtype == D2D_BF16 ? d2d_decode_max_tokens(L->desc) : 8;      // fp32 layers have no tensor-core path
     return T <= lim && d2d_small_ffn_supports(L->desc);
 }
 
@@ -89,7 +93,7 @@ size_t d2d_moe_ffn_ws_bytes(const d2d_layer *L, int T)
     size_t need = 256;
     if (use_small_ffn(L, T)) need = d2d_small_ffn_ws_bytes(L, T);
     // hidden activations H [T, d_ff] bf16 of the dense-masked path
-    if (L->desc.dtype == D2D_BF16 && T > d2d_decode_max_tokens()) {
+    if (L->desc.dtype == D2D_BF16 && T > d2d_decode_max_tokens(L->desc)) {
         size_t h = d2d_align_up((size_t)T * L->desc.d_ff * 2, 256);
         if (d2d_gemm_tc_splits(T, L->desc.d, L->desc.d_ff) > 1) h += d2d_align_up((size_t)T * L->desc.d * 4, 256);   // split-K partial sums
         if (h > need) need = h;

@@ -87,7 +87,7 @@ extern unsigned long long d2d_launch_counter;
 
 // Largest batch served by the decode kernels (cp.async CUDA-core kernels, two launches per layer call); larger bf16
 // batches take the tensor-core path.  4 by default, D2D_DECODE_MAX_TOKENS=n (0 .. 8) overrides it for tuning.
-int d2d_decode_max_tokens();
+int d2d_decode_max_tokens(const d2d_layer_desc &D);
 
 static inline size_t d2d_align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 static inline int d2d_cdiv(int a, int b) { return (a + b - 1) / b; }

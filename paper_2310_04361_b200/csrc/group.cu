@@ -179,7 +179,7 @@ d2d_status d2d_group_fwd(const d2d_group *g, const void *x, int32_t T, float tau
     char *base = (char *)ws;
 
     // ---- decode batches: two launches for the whole group
-    if (d2d_small_router_supports(D, T) && d2d_small_ffn_supports(D) && T <= (D.dtype == D2D_BF16 ? d2d_decode_max_tokens() : 8)) {
+    if (d2d_small_router_supports(D, T) && d2d_small_ffn_supports(D) && T <= (D.dtype == D2D_BF16 ? d2d_decode_max_tokens(D) : 8)) {
         float *R[D2D_MAX_GROUP], *u[D2D_MAX_GROUP], *y32[D2D_MAX_GROUP];
         for (int l = 0; l < n; ++l) {
             R[l] = (float *)(base + w.r_off + (size_t)l * w.r_each);

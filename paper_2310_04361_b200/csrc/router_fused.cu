@@ -389,7 +389,7 @@ d2d_status launch(const d2d_layer_desc &D, const d2d_router_weights &w, int n_la
 bool d2d_router_fused_supports(const d2d_layer_desc &D, int T)
 {
     // d_h = 128 (the paper's router width) and E <= 256: operand ring, u and W_r2 then fit in shared memory together
-    return D.dtype == D2D_BF16 && T > d2d_decode_max_tokens() && D.d_h == 128 && D.n_experts <= 256 && D.d % 8 == 0 && d2d_gemm_tc_available();
+    return D.dtype == D2D_BF16 && T > d2d_decode_max_tokens(D) && D.d_h == 128 && D.n_experts <= 256 && D.d % 8 == 0 && d2d_gemm_tc_available();
 }
 
 // R may be NULL when only the mask is wanted; mask / k / status are used when do_mask != 0.

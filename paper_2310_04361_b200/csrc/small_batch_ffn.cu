@@ -515,7 +515,7 @@ size_t d2d_small_router_ws_bytes(const d2d_layer *L, int T) { return 256 + d2d_a
 bool d2d_small_router_supports(const d2d_layer_desc &D, int T)
 {
     const size_t elem = D.dtype == D2D_F32 ? 4 : 2;
-    return T >= 1 && T <= (D.dtype == D2D_BF16 ? d2d_decode_max_tokens() : 8) && D.d % 8 == 0 && D.d_h % 8 == 0 &&
+    return T >= 1 && T <= (D.dtype == D2D_BF16 ? d2d_decode_max_tokens(D) : 8) && D.d % 8 == 0 && D.d_h % 8 == 0 &&
            (size_t)(8 + MAX_TBLK) * D.d * elem + (size_t)T * D.d_h * 4 + (size_t)T * ((D.n_experts + 31) / 32) * 4 <= kSmemLimit;
 }
 
