@@ -8,7 +8,7 @@ neurons, 8192 tokens) at tau = 0.4; the other configurations are timed in the sa
 reported in `per_config` of the same JSON line.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload llama] [--tau 0.4]
-                    [--tokens T] [--bernoulli p] [--path auto|dense|gather|fused] [--experts-per-group g]
+                    [--tokens T] [--bernoulli p] [--path auto|dense|gather|fused] [--experts-per-group g] [--fp8-experts]
                     [--sweep] [--no-per-config] [--no-cpu-baseline] [--no-graph] [--group N]
     python bench.py --impl reference ...      # times the CPU oracle on the host cores
 
@@ -73,6 +73,8 @@ def parse_args():
     p.add_argument("--path", default="auto", choices=["auto", "dense", "gather", "fused"],
                    help="which up projection the tensor-core expert step uses (d2d_layer_set_expert_path)")
     p.add_argument("--experts-per-group", type=int, default=0, help="group size of the gathered path (0 = default)")
+    p.add_argument("--fp8-experts", action="store_true",
+                   help="expert weights as 8-bit e4m3 codes with one power-of-two scale per expert (d2d_layer_create_fp8)")
     p.add_argument("--sweep", action="store_true", help="also time the workload's whole tau grid")
     p.add_argument("--no-per-config", action="store_true", help="skip the other configurations")
     p.add_argument("--no-cpu-baseline", action="store_true")
@@ -481,7 +483,7 @@ def run_ours(args):
     peaks = measured_peaks()
 
     m = measure_config(h, api, torch, wl, args.workload, args.tokens, args.tau, args.bernoulli, args.steps, peaks,
-                       path=args.path, group=args.experts_per_group, full=True, rank=rank)
+                       path=args.path, group=args.experts_per_group, full=True, rank=rank, fp8=args.fp8_experts)
     cfg, layer, weights, x, x_np, y, routing, step = (m[k] for k in ("cfg", "layer", "weights", "x", "x_np", "y", "routing", "step"))
     T = cfg.T
     launches_per_step = m["launches"]
@@ -545,7 +547,8 @@ def run_ours(args):
         n_used = int((routing.counts > 0).sum().item())
         if T <= 64 or cfg.dtype == "f32":
             # decode regime: the expert kernel is bound by HBM traffic on the touched expert slices
-            touched = n_used * (cfg.n_mat * cfg.s * cfg.d + cfg.s) * elem + 2 * T * cfg.d * elem + cfg.d * elem
+            welem = 1 if args.fp8_experts else elem           # 8-bit expert weights: one byte per weight
+            touched = n_used * (cfg.n_mat * cfg.s * cfg.d * welem + cfg.s * elem) + 2 * T * cfg.d * elem + cfg.d * elem
             achieved = touched / (t_ffn * 1e-3) / 1e9
             roofline = {"bound": "hbm", "kernel": "moe_ffn_fwd (small_ffn_kernel)" if launches_per_step <= 2 else "moe_ffn_fwd", "achieved": achieved,
                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None,
@@ -680,7 +683,7 @@ def run_ours(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": total_ms / args.steps, "ms_median": st_layer["median"], "ms_min": st_layer["min"],
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": cfg.dtype, "data": "synthetic",
+            "dtype": cfg.dtype + (" (expert weights e4m3 + 2^k per expert)" if args.fp8_experts else ""), "data": "synthetic",
             "config": config_dict(cfg, args.tau, args.bernoulli),
             "run": {"tokens_per_gpu": T, "rho": rho, "pruned_flop_fraction": 1 - rho, "k": khist,
                     "step": "d2d_moe_ffn_fwd on the override mask" if args.bernoulli is not None else "d2d_layer_fwd",
