@@ -8,7 +8,7 @@
 //                         shared memory, one warp per unit forms u[t, j]; every CTA also prefetches
 //                         W_r2, and the CTA that finishes last (ticket) computes layer 2 from it and,
 //                         when asked to, the dynamic-k selection and its metadata as well (no second launch)
-//   small_ffn_kernel      one CTA per expert: its W1 / W_gate / W2 slices are read from HBM exactly
+//   small_ffn_kernel      one CTA per expert (several for experts too large for one pass): the W1 / W_gate / W2 slices are read from HBM exactly
 //                         once (only experts some token kept do any work), the expert's tokens are
 //                         handled 8 at a time, partial output rows go to a float32 accumulator with
 //                         16-byte vector reductions; the last CTA adds b2 and writes y
@@ -260,7 +260,7 @@ struct SmallFfnArgs {
 // are used and the scale, a power of two, is applied to the finished sums (exactly what scaling every weight would give).
 template <typename TT, int ACT, bool GATED, int TBLK, bool Q8>
 __global__ void __launch_bounds__(NT)
-small_ffn_kernel(const TT *__restrict__ x, int T, int d, int s, int rc, const __grid_constant__ SmallFfnArgs args)
+small_ffn_kernel(const TT *__restrict__ x, int T, int d, int s, int rc, int splits, const __grid_constant__ SmallFfnArgs args)
 {
     using WT = typename std::conditional<Q8, uint8_t, TT>::type;
     const SmallFfnLayer &P = args.l[blockIdx.y];
@@ -283,7 +283,10 @@ small_ffn_kernel(const TT *__restrict__ x, int T, int d, int s, int rc, const __
     __shared__ unsigned int my_ticket;
     __shared__ int stok[TBLK];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int e = blockIdx.x;
+    // an expert too large for one pass is shared by `splits` CTAs, each with its own range of neurons (one pass of rc
+    // neurons when splits = ceil(s / rc)): the kept experts then fill the machine instead of a fraction of its SMs
+    const int e = blockIdx.x / splits, part = blockIdx.x - e * splits;
+    const int span = ((s + splits - 1) / splits + rc - 1) / rc * rc, r_begin = part * span, r_end = r_begin + span < s ? r_begin + span : s;
     const float sc1 = Q8 ? ldexpf(1.0f, P.k1[e]) : 1.0f, scg = Q8 && GATED ? ldexpf(1.0f, P.kg[e]) : 1.0f, sc2 = Q8 ? ldexpf(1.0f, P.k2[e]) : 1.0f;
     // perm may have been truncated at `capacity` entries (the selection then reported D2D_ERR_CAPACITY): stay inside it
     const long long cap = P.capacity;
@@ -291,8 +294,8 @@ small_ffn_kernel(const TT *__restrict__ x, int T, int d, int s, int rc, const __
     const int beg = offsets[e] < end ? offsets[e] : end;
 
     if (beg < end) {
-        for (int r0 = 0; r0 < s; r0 += rc) {
-            const int rows = s - r0 < rc ? s - r0 : rc;
+        for (int r0 = r_begin; r0 < r_end; r0 += rc) {
+            const int rows = r_end - r0 < rc ? r_end - r0 : rc;
             const size_t n0 = (size_t)e * s + r0;
             __syncthreads();                                      // readers of the previous pass are done
             cta_copy_async(w1s, w1 + n0 * d, (size_t)rows * d * sizeof(WT));
@@ -419,7 +422,9 @@ d2d_status launch_ffn_q(const d2d_layer_desc &D, int n_layers, const SmallFfnArg
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess) return D2D_ERR_CUDA;
         attr_smem = kSmemLimit;
     }
-    kern<<<dim3(D.n_experts, n_layers), NT, smem, st>>>((const TT *)x, T, D.d, D.expert_size, rc, args);
+    // one pass per CTA for experts that need several; experts that fit in one pass keep one CTA each
+    const int splits = d2d_cdiv(D.expert_size, rc);
+    kern<<<dim3(D.n_experts * splits, n_layers), NT, smem, st>>>((const TT *)x, T, D.d, D.expert_size, rc, splits, args);
     D2D_LAUNCHED(1);
     return cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
 }
