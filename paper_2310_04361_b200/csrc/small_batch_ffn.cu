@@ -422,8 +422,9 @@ d2d_status launch_ffn_q(const d2d_layer_desc &D, int n_layers, const SmallFfnArg
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit) != cudaSuccess) return D2D_ERR_CUDA;
         attr_smem = kSmemLimit;
     }
-    // one pass per CTA for experts that need several; experts that fit in one pass keep one CTA each
-    const int splits = d2d_cdiv(D.expert_size, rc);
+    // a single token: one pass per CTA for experts that need several (measured on the Llama-shaped layer: 86 -> 82 us at
+    // one token, but 108 -> 117 us at two, where every extra CTA stages the token rows and merges its partial sums again)
+    const int splits = T == 1 ? d2d_cdiv(D.expert_size, rc) : 1;
     kern<<<dim3(D.n_experts * splits, n_layers), NT, smem, st>>>((const TT *)x, T, D.d, D.expert_size, rc, splits, args);
     D2D_LAUNCHED(1);
     return cudaGetLastError() == cudaSuccess ? D2D_OK : D2D_ERR_CUDA;
