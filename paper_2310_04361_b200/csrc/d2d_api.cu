@@ -109,9 +109,8 @@ size_t d2d_moe_ffn_ws_bytes(const d2d_layer *L, int T)
 // T / 128 x Nd tiles (Nd = 256-column tiles across d_ff) on S SMs that fixed part is T0 = 5 * 128 * 1.2 * S / Nd
 // tokens' worth of dense time, so the pair wins while the fraction of kept (token, group) pairs
 //     u = 1 - (1 - rho)^g  <  U - T0 / T,
-// U = 0.85 for 256 MMA columns (less for narrower groups, 0.05 less where the slower selection-applying down
-// projection follows instead of a zero fill and the TMA-fed one).  Checked against measured crossovers: Llama-shaped
-// layer u = 0.70 at 8192 tokens, 0.55 at 4096; paper's latency shape 0.6-0.75 at 50432 tokens; ViT-shaped 0.5 at
+// U = 0.85 for 256 MMA columns (less for narrower groups).  Checked against measured crossovers: Llama-shaped
+// layer u = 0.70 at 8192 tokens, 0.55 at 4096; paper's latency shape 0.7 at 50432 tokens (357 against 374 us at rho = 0.4, 387 against 381 us at 0.5); ViT-shaped 0.5 at
 // 25216; never for the BERT-shaped layer at 4096 tokens.
 int d2d_tc_sm_count();      // gemm_tc.cu
 
@@ -122,7 +121,6 @@ static double default_gather_rho_max(const d2d_layer_desc &D, int g, int T)
     if (g <= 0 || T <= 0) return -1.0;
     const int n_mma = g * D.expert_size * (D.gated ? 2 : 1);
     double U = n_mma >= 256 ? 0.85 : n_mma >= 192 ? 0.64 : n_mma >= 128 ? 0.43 : 0.25;
-    if (D.d < 2048) U -= 0.05;
     const double nd = ceil((double)D.d_ff * (D.gated ? 2.0 : 1.0) / 256.0);
     const double T0 = 5.0 * 128.0 * 1.2 * (double)d2d_tc_sm_count() / nd;
     const double u_max = U - T0 / (double)T;
